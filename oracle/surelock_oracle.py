@@ -1,0 +1,308 @@
+"""SureLock locked forward and sure test: the CPU oracle.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain fp64 statement of what
+one SureLock decoding step computes.  Only the test-suite, the smoke check and
+the benchmark's CPU-baseline leg may import it; the CUDA product path never does,
+and this module imports nothing from the CUDA package (numpy only).
+
+Every function cites the passage of the paper it follows
+("Stopping Computation for Converged Tokens in Masked Diffusion-LM Decoding").
+Arithmetic is float64 throughout; inputs that the GPU receives rounded to bf16 or
+fp32 are handed in already rounded and are widened here.  A matrix product is a
+single library call (numpy ``@`` / ``einsum``); nothing is blocked, fused or
+reordered beyond what the paper's Algorithm 1 states.
+
+Readings taken where the paper leaves a choice open (each also listed in the
+design notes of the repository):
+  * the active set is "not locked" (Algorithm 1, line 6), not "unmasked and not
+    locked" (Sec. 2.1 prose): masked positions must be computed to be predicted;
+  * block structure (the paper says only LN / Proj / Attn / FFN): pre-norm
+    residual block, RMSNorm, no biases, rotary embedding in rotate-half pairing
+    applied with the ORIGINAL position index, keys cached after the rotation,
+    softmax scale 1/sqrt(d_h), no attention mask, SwiGLU FFN with three matrices
+    (the paper's 6*d*d_ff FLOP term), untied output projection;
+  * KL(p_t || p_{t-1}) in nats from log-softmax; the test is D <= eps; a row
+    without a previous posterior has D = +inf (Algorithm 1, line 19);
+  * the lock test reads the mask state the forward pass saw (the state passed
+    to this step), so a row can lock only after a step that was fed its token;
+  * the optional confidence-percentile gate (Algorithm 1, line 21) is off.
+
+Parity pins (tests that run without a GPU) tie this file to closed forms, printed
+values of the paper's Table 2, library routines of a different library (torch
+fp64), and a pure-Python brute force.  Nothing here is unpinned except sampler
+trajectories of trained models, which need the paper's weights and datasets.
+"""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+F64 = np.float64
+
+
+@dataclasses.dataclass
+class ModelCfg:
+    """Shape of the masked-diffusion transformer (paper Sec. 2.3 symbols L, d, H, d_h, d_ff)."""
+    n_layers: int
+    d_model: int
+    n_heads: int
+    head_dim: int
+    d_ff: int
+    vocab: int
+    rms_eps: float = 1e-5
+    rope_theta: float = 10000.0
+
+
+# --------------------------------------------------------------------------
+# Algorithm 1, line 6: active / locked split
+# --------------------------------------------------------------------------
+def active_set(lock: np.ndarray):
+    """A_t = {i : lock_i = 0} per sequence, ascending (Algorithm 1, line 6).
+
+    lock: [B][N] of 0/1.  Returns (active_idx, row_offsets): flat indices b*N+i of
+    the unlocked positions in ascending order, and row_offsets[b] = number of
+    active rows of sequences 0..b-1 (length B+1, last entry = M).
+    """
+    lock = np.asarray(lock)
+    B, N = lock.shape
+    idx: List[int] = []
+    offs = [0]
+    for b in range(B):
+        for i in range(N):
+            if lock[b, i] == 0:
+                idx.append(b * N + i)
+        offs.append(len(idx))
+    return np.asarray(idx, dtype=np.int32), np.asarray(offs, dtype=np.int32)
+
+
+# --------------------------------------------------------------------------
+# Row-wise building blocks of the transformer block (Algorithm 1, lines 10-12)
+# --------------------------------------------------------------------------
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """"LN" of Algorithm 1 line 10, read as RMSNorm: x / sqrt(mean(x^2) + eps) * g."""
+    x = np.asarray(x, F64)
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * np.asarray(g, F64)
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary position embedding, rotate-half pairing (j, j + d_h/2).
+
+    x: [m][H][d_h]; pos: [m] ORIGINAL sequence positions i (not packed rows).
+    Pair j is rotated by the angle pos * theta**(-2j/d_h).
+    """
+    x = np.asarray(x, F64)
+    m, H, dh = x.shape
+    half = dh // 2
+    j = np.arange(half, dtype=F64)
+    inv_freq = np.asarray(theta, F64) ** (-2.0 * j / dh)          # [half]
+    ang = np.asarray(pos, F64)[:, None] * inv_freq[None, :]       # [m][half]
+    c = np.cos(ang)[:, None, :]
+    s = np.sin(ang)[:, None, :]
+    lo, hi = x[..., :half], x[..., half:]
+    out = np.empty_like(x)
+    out[..., :half] = lo * c - hi * s
+    out[..., half:] = hi * c + lo * s
+    return out
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    x = np.asarray(x, F64)
+    return x / (1.0 + np.exp(-x))
+
+
+def attention_rows(q: np.ndarray, K: np.ndarray, V: np.ndarray) -> np.ndarray:
+    """Attn(Q[A_t], K^all, V^all) of Algorithm 1 line 12 for ONE sequence.
+
+    q: [m][H][d_h] queries of the active rows; K, V: [N][H][d_h], every position
+    of the sequence (fresh rows for active positions, frozen rows for locked
+    ones).  Bidirectional: every query sees all N keys.  Returns [m][H*d_h].
+    """
+    q = np.asarray(q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    m, H, dh = q.shape
+    s = np.einsum("mhd,nhd->hmn", q, K) / np.sqrt(F64(dh))
+    s = s - s.max(axis=-1, keepdims=True)
+    a = np.exp(s)
+    a = a / a.sum(axis=-1, keepdims=True)
+    o = np.einsum("hmn,nhd->mhd", a, V)
+    return o.reshape(m, H * dh)
+
+
+def log_softmax(z: np.ndarray) -> np.ndarray:
+    """log p = z - logsumexp(z) along the vocabulary (Algorithm 1, line 15)."""
+    z = np.asarray(z, F64)
+    zmax = z.max(axis=-1, keepdims=True)
+    lse = zmax + np.log(np.exp(z - zmax).sum(axis=-1, keepdims=True))
+    return z - lse
+
+
+def kl_rows(logp: np.ndarray, logp_prev: np.ndarray) -> np.ndarray:
+    """D = KL(p_t || p_{t-1}) = sum_v p_t(v) (log p_t(v) - log p_{t-1}(v)), nats (Sec. 2.2)."""
+    logp = np.asarray(logp, F64)
+    logp_prev = np.asarray(logp_prev, F64)
+    return np.sum(np.exp(logp) * (logp - logp_prev), axis=-1)
+
+
+def kl_from_logits(z: np.ndarray, z_prev: np.ndarray) -> np.ndarray:
+    """Step-wise KL of the posteriors given raw (temperature-1) logits of both steps."""
+    return kl_rows(log_softmax(z), log_softmax(z_prev))
+
+
+def posterior_stats(z: np.ndarray):
+    """(conf, argmax) with conf = max_v p(v) = 1 - u (Algorithm 1 line 18); lowest index on ties."""
+    logp = log_softmax(z)
+    am = np.argmax(logp, axis=-1)
+    conf = np.exp(np.take_along_axis(logp, am[..., None], axis=-1))[..., 0]
+    return conf, am.astype(np.int32)
+
+
+def sure_test(D: np.ndarray, masked: np.ndarray, kl_eps: float) -> np.ndarray:
+    """F_t = {i in A_t, unmasked : D_i <= eps} (Algorithm 1, lines 20 and 23, gate off). NaN never locks."""
+    D = np.asarray(D, F64)
+    return (np.asarray(masked) == 0) & (D <= kl_eps)
+
+
+# --------------------------------------------------------------------------
+# Algorithmic FLOPs (Sec. 2.3)
+# --------------------------------------------------------------------------
+def flops_base_step(cfg: ModelCfg, B: int, N: int, n_kv_heads: Optional[int] = None) -> int:
+    """F^t_base of Sec. 2.3: GEMM-only FLOPs of one full-recompute step of a batch."""
+    L, d, H, dh, dff = cfg.n_layers, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.d_ff
+    Hkv = H if n_kv_heads is None else n_kv_heads
+    return L * (4 * B * H * N * N * dh + 2 * B * N * d * d + 2 * B * N * d * d
+                + 4 * B * N * d * Hkv * dh + 6 * B * N * d * dff)
+
+
+def flops_prop_step(cfg: ModelCfg, B: int, N: int, M: int) -> float:
+    """F^t_prop = (M / (B N)) F^t_base (Sec. 2.3, SureLock paragraph)."""
+    return flops_base_step(cfg, B, N) * (M / (B * N))
+
+
+# --------------------------------------------------------------------------
+# One transformer block on the active rows (Algorithm 1, lines 10-13)
+# --------------------------------------------------------------------------
+def qkv_rows(cfg: ModelCfg, lw: Dict[str, np.ndarray], x: np.ndarray, pos: np.ndarray):
+    """Proj_{Q,K,V}(LN(x[A_t])) with the rotation applied to q and k (line 10).
+
+    x: [m][d] block input of active rows; pos: [m] their sequence positions.
+    Weight matrices are stored [out][in].  Returns q, k, v as [m][H][d_h].
+    """
+    H, dh = cfg.n_heads, cfg.head_dim
+    h = rmsnorm(x, lw["attn_norm_g"], cfg.rms_eps)
+    m = h.shape[0]
+    q = (h @ np.asarray(lw["wq"], F64).T).reshape(m, H, dh)
+    k = (h @ np.asarray(lw["wk"], F64).T).reshape(m, H, dh)
+    v = (h @ np.asarray(lw["wv"], F64).T).reshape(m, H, dh)
+    return rope(q, pos, cfg.rope_theta), rope(k, pos, cfg.rope_theta), v
+
+
+def ffn_rows(cfg: ModelCfg, lw: Dict[str, np.ndarray], x: np.ndarray) -> np.ndarray:
+    """x + W_d( silu(W_g h) * (W_u h) ), h = RMSNorm(x): the FFN sub-block on active rows (line 12)."""
+    h = rmsnorm(x, lw["ffn_norm_g"], cfg.rms_eps)
+    a = silu(h @ np.asarray(lw["w_gate"], F64).T) * (h @ np.asarray(lw["w_up"], F64).T)
+    return np.asarray(x, F64) + a @ np.asarray(lw["w_down"], F64).T
+
+
+def layer_rows(cfg: ModelCfg, lw: Dict[str, np.ndarray], x: np.ndarray, pos: np.ndarray,
+               Kc: np.ndarray, Vc: np.ndarray) -> np.ndarray:
+    """One block for the active rows of ONE sequence (Algorithm 1, lines 10-13).
+
+    x: [m][d]; pos: [m] ascending positions of those rows; Kc, Vc: [N][H][d_h]
+    this layer's cache of the sequence, updated IN PLACE at the active positions
+    (line 11: fresh K/V for A_t, cached K/V for L_t) before attention reads all N
+    rows.  Locked rows are not touched (line 13: they pass through).
+    """
+    x = np.asarray(x, F64)
+    q, k, v = qkv_rows(cfg, lw, x, pos)
+    Kc[pos] = k
+    Vc[pos] = v
+    o = attention_rows(q, Kc, Vc)
+    x = x + o @ np.asarray(lw["wo"], F64).T
+    return ffn_rows(cfg, lw, x)
+
+
+def layer_flops(cfg: ModelCfg, m: int, N: int) -> int:
+    """GEMM FLOPs layer_rows() performs for m active rows against N keys (same terms as Sec. 2.3)."""
+    d, H, dh, dff = cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.d_ff
+    return 4 * H * m * N * dh + 2 * m * d * d + 2 * m * d * d + 4 * m * d * H * dh + 6 * m * d * dff
+
+
+# --------------------------------------------------------------------------
+# Sampler-visible state and one full step (Algorithm 1, lines 6-24)
+# --------------------------------------------------------------------------
+class OracleState:
+    """lock-independent state of Algorithm 1 lines 1-2: per-layer K/V caches and p_{t-1}.
+
+    K, V: [L][B][N][H][d_h] float64.  prev_logp: [B][N][V] float64 with
+    prev_valid [B][N]; an invalid row stands for "p_{t-1} = None".
+    """
+
+    def __init__(self, cfg: ModelCfg, B: int, N: int):
+        self.cfg, self.B, self.N = cfg, B, N
+        shp = (cfg.n_layers, B, N, cfg.n_heads, cfg.head_dim)
+        self.K = np.zeros(shp, F64)
+        self.V = np.zeros(shp, F64)
+        self.prev_logp = np.zeros((B, N, cfg.vocab), F64)
+        self.prev_valid = np.zeros((B, N), bool)
+        self.flops = 0
+
+    def reset(self):
+        self.prev_valid[:] = False
+        self.flops = 0
+
+
+def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.ndarray,
+         lock: np.ndarray, kl_eps: float, logits_round=None):
+    """One SureLock step (Algorithm 1, lines 6-15 and 18-24; line 16 belongs to the caller).
+
+    weights: {"tok_emb": [V][d], "lm_head": [V][d], "final_norm_g": [d],
+              "layers": [ {attn_norm_g, wq, wk, wv, wo, ffn_norm_g, w_gate, w_up, w_down} ]}.
+    tokens [B][N] int; mask_state [B][N] (1 = masked); lock [B][N] (1 = locked),
+    NOT modified.  logits_round: optional callable applied to the logits before
+    the posterior is formed (lets a test reproduce the storage precision of the
+    logits, e.g. rounding to bf16); None = no rounding.
+
+    Returns dict: active_idx, row_offsets, hidden [M][d] (x^{(L+1)}), logits
+    [M][V], kl [M], conf [M], argmax [M], new_lock [B][N], flops (GEMM FLOPs of
+    the L blocks, the quantity Sec. 2.3 counts).
+    """
+    cfg, B, N = state.cfg, state.B, state.N
+    tokens = np.asarray(tokens)
+    idx, offs = active_set(lock)
+    M = len(idx)
+    emb = np.asarray(weights["tok_emb"])
+    hidden = np.zeros((M, cfg.d_model), F64)
+    flops = 0
+    for b in range(B):
+        r0, r1 = int(offs[b]), int(offs[b + 1])
+        if r1 == r0:
+            continue
+        pos = (idx[r0:r1] - b * N).astype(np.int64)
+        x = np.asarray(emb[tokens[b, pos]], F64)                  # line 7
+        for l, lw in enumerate(weights["layers"]):                # lines 9-14
+            x = layer_rows(cfg, lw, x, pos, state.K[l, b], state.V[l, b])
+            flops += layer_flops(cfg, r1 - r0, N)
+        hidden[r0:r1] = x
+    hn = rmsnorm(hidden, weights["final_norm_g"], cfg.rms_eps)
+    logits = hn @ np.asarray(weights["lm_head"], F64).T           # line 15
+    if logits_round is not None:
+        logits = np.asarray(logits_round(logits), F64)
+    logp = log_softmax(logits)
+    conf, am = posterior_stats(logits)                            # line 18
+    bb, ii = idx // N, idx % N
+    D = np.full(M, np.inf, F64)                                   # line 19
+    has_prev = state.prev_valid[bb, ii]
+    if has_prev.any():
+        D[has_prev] = kl_rows(logp[has_prev], state.prev_logp[bb[has_prev], ii[has_prev]])
+    lockable = sure_test(D, np.asarray(mask_state)[bb, ii], kl_eps)  # lines 20, 23
+    new_lock = np.array(lock, dtype=np.uint8, copy=True)
+    new_lock[bb[lockable], ii[lockable]] = 1                      # line 24
+    state.prev_logp[bb, ii] = logp                                # locked rows keep p_{t*}
+    state.prev_valid[bb, ii] = True
+    state.flops += flops
+    return dict(active_idx=idx, row_offsets=offs, hidden=hidden, logits=logits, kl=D,
+                conf=conf, argmax=am, new_lock=new_lock, flops=flops)
