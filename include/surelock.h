@@ -1,0 +1,206 @@
+/*
+ * surelock.h -- C ABI of the SureLock locked-forward hot path for NVIDIA B200 (sm_100a).
+ *
+ * SureLock ("Stopping Computation for Converged Tokens in Masked Diffusion-LM Decoding",
+ * Algorithm 1) decodes a masked-diffusion LM while recomputing, at every step, only the M
+ * positions of an N-token sequence that are not yet locked.  This library is one such step:
+ * compaction of the active rows, RMSNorm / RoPE / QKV on those rows, scatter of their fresh
+ * K/V into an N-length per-layer cache whose locked rows stay frozen, M x N bidirectional
+ * attention, SwiGLU FFN and LM head on the M rows, and a fused softmax that computes each
+ * active row's step-wise KL, applies the lock test and updates the lock mask.
+ *
+ * General rules
+ *  - Every function returns 0 (SL_OK) or a negative surelock_status; nothing throws or exits.
+ *  - "dev" pointers are CUDA device pointers, "host" pointers ordinary host memory.
+ *  - Work is enqueued on the cudaStream_t passed (as void*) at init or to the call; calls do
+ *    not synchronise with the host unless stated.
+ *  - A device-side problem (a bounded wait that ran out, an index out of range) sets a sticky
+ *    status word that surelock_status_poll() returns; kernels never trap.
+ *  - There is no CPU fallback: every step of the path runs in the library's CUDA kernels.
+ */
+#ifndef SURELOCK_H
+#define SURELOCK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SL_OK = 0,
+  SL_EINVAL = -1,       /* null pointer, size out of range, negative or NaN threshold ...      */
+  SL_ENOMEM = -2,       /* device allocation failed at init                                    */
+  SL_ECUDA = -3,        /* a CUDA runtime call failed (sticky CUDA error)                      */
+  SL_EDEVICE = -4,      /* a kernel reported a problem through the status word                 */
+  SL_EUNSUPPORTED = -5  /* shape not supported by the kernels (e.g. head_dim not 64 or 128)    */
+} surelock_status;
+
+enum { SL_BF16 = 0, SL_FP32 = 1 };   /* storage type of weights, activations, caches and logits; accumulation is fp32 */
+
+typedef struct surelock_ctx surelock_ctx;   /* opaque: owns caches, workspaces and previous logits */
+
+/* Shape of the transformer (symbols of Sec. 2.3: L, d, H, d_h, H_kv, d_ff, vocabulary).
+ * n_kv_heads must equal n_heads.  vocab may be 0: then there is no LM head and only
+ * surelock_layer_step() can be used.  head_dim must be 64 or 128 and even. */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, n_kv_heads, d_ff, vocab;
+  int32_t dtype;                 /* SL_BF16 or SL_FP32 */
+  float rms_eps, rope_theta;
+  int32_t mask_token_id;         /* informational; the caller writes it into `tokens` */
+} surelock_model_cfg;
+
+/* Weights: dev pointers, BORROWED (must outlive the ctx), element type cfg.dtype, every matrix row-major
+ * [out_features][in_features].  The per-layer members are host arrays of n_layers dev pointers.
+ * tok_emb [vocab][d], lm_head [vocab][d], norm gains [d], wq/wk/wv [H*d_h][d], wo [d][H*d_h],
+ * w_gate/w_up [d_ff][d], w_down [d][d_ff].  With vocab == 0, tok_emb/lm_head/final_norm_g may be NULL. */
+typedef struct {
+  const void *tok_emb, *lm_head, *final_norm_g;
+  const void *const *attn_norm_g, *const *wq, *const *wk, *const *wv, *const *wo;
+  const void *const *ffn_norm_g, *const *w_gate, *const *w_up, *const *w_down;
+} surelock_weights;
+
+/* Results of a step: dev pointers into ctx-owned buffers, valid until the next step/reset/destroy.
+ * Rows are PACKED: row r belongs to flat position active_idx[r] = b*N + i. */
+typedef struct {
+  const int32_t *active_idx;     /* [M] ascending flat positions of the unlocked rows (Algorithm 1 line 6)     */
+  const int32_t *row_offsets;    /* [B+1] packed-row offset of each sequence; row_offsets[B] = M              */
+  const int32_t *n_active;       /* [1] M                                                                      */
+  const void *logits;            /* [M][vocab], cfg.dtype (Algorithm 1 line 15, before the softmax)            */
+  const float *hidden;           /* [M][d] fp32, output of the last block (before the final norm)              */
+  const float *kl;               /* [M] D = KL(p_t || p_{t-1}) in nats, +inf without a previous posterior      */
+  const float *conf;             /* [M] max_v p_t(v) = 1 - u (Algorithm 1 line 18)                             */
+  const int32_t *argmax;         /* [M] argmax_v p_t(v), lowest index on ties                                  */
+} surelock_step_out;
+
+/* ---- context ------------------------------------------------------------------------------------------- */
+
+/* Allocate a context for sequences of exactly N tokens in batches of exactly `batch` sequences
+ * (Algorithm 1 lines 1-2: lock-independent state = per-layer K/V caches and previous posteriors).
+ * Allocates (cudaMalloc, on the current device) the K/V cache [L][2][B*N][H*d_h], packed workspaces for
+ * M = B*N rows, two logit buffers [B*N][vocab] and index arrays; builds a rotary table.  The first call in a
+ * process also raises kernel shared-memory limits.  Not asynchronous.  `cuda_stream` (a cudaStream_t, may be 0)
+ * is the stream every later call of this ctx enqueues on. */
+int surelock_init(surelock_ctx **out, const surelock_model_cfg *cfg, const surelock_weights *w,
+                  int N, int batch, void *cuda_stream);
+
+/* Forget the previous posteriors (p_{t-1} = None, so the next step's KL is +inf for every row: Algorithm 1
+ * line 19) and clear the device status word.  Cache contents are kept (a caller may have pre-filled them). */
+int surelock_reset(surelock_ctx *ctx);
+
+/* One SureLock step (Algorithm 1 lines 6-15 and 18-24; the unmasking policy of line 16 is the caller's).
+ *   tokens      dev int32 [B][N]   current sequence (mask positions hold the mask token id)
+ *   mask_state  dev uint8 [B][N]   1 = masked.  The state the forward pass sees; a row can lock only if 0.
+ *   lock_mask   dev uint8 [B][N]   in: locks entering the step (1 = locked; such rows are neither recomputed
+ *                                  nor rewritten in the cache); out: rows passing D <= kl_eps are set to 1.
+ *                                  Locking a row whose cache entries were never written is the caller's error.
+ *   kl_eps      threshold eps >= 0 (not NaN)
+ *   out         host struct filled with dev pointers (may be NULL)
+ * Asynchronous; performs no allocation and no host synchronisation. */
+int surelock_step(surelock_ctx *ctx, const int32_t *tokens, const uint8_t *mask_state, uint8_t *lock_mask,
+                  float kl_eps, surelock_step_out *out);
+
+/* The same step for callers whose buffers live in HOST memory: copies tokens, mask_state and lock_mask to
+ * ctx-owned device staging, runs surelock_step, copies back lock_mask (updated, [B][N]) and, for the M active
+ * rows, kl / conf / argmax / active_idx (each array must have room for B*N entries; any may be NULL), stores
+ * M in *n_active and synchronises the stream.  For best speed pass page-locked host memory. */
+int surelock_step_host(surelock_ctx *ctx, const int32_t *tokens, const uint8_t *mask_state, uint8_t *lock_mask,
+                       float kl_eps, int32_t *n_active, int32_t *active_idx, float *kl, float *conf,
+                       int32_t *argmax);
+
+/* One transformer block on the active rows (Algorithm 1 lines 6 and 10-13 for a single layer): compaction,
+ * RMSNorm, QKV + RoPE, K/V scatter into this layer's cache, M x N attention, O-projection + residual,
+ * RMSNorm, SwiGLU FFN + residual.
+ *   hidden_in   dev [B][N][d] cfg.dtype; only rows of unlocked positions are read
+ *   lock_mask   dev uint8 [B][N], read only
+ *   hidden_out  dev fp32 [M][d] packed (room for B*N rows)
+ *   out         host struct (may be NULL): active_idx, row_offsets, n_active are filled, the rest NULL
+ * Asynchronous. */
+int surelock_layer_step(surelock_ctx *ctx, int layer, const void *hidden_in, const uint8_t *lock_mask,
+                        float *hidden_out, surelock_step_out *out);
+
+/* Synchronise the ctx stream and report: *device_status = 0, or the code a kernel stored (see SL_DEV_* in
+ * the source) ; returns SL_EDEVICE if non-zero, SL_ECUDA if the stream reported a CUDA error. */
+int surelock_status_poll(surelock_ctx *ctx, int *device_status);
+
+/* K/V cache of one layer (Algorithm 1 line 11: K^all / V^all): dev pointers to [B*N][H][d_h] arrays of
+ * cfg.dtype, token-major (row b*N+i holds all heads of position i of sequence b, keys stored AFTER the rotary
+ * embedding).  row_stride_elems = H*d_h.  For pre-filling and for parity checks. */
+int surelock_kv_cache(surelock_ctx *ctx, int layer, void **k, void **v, size_t *row_stride_elems);
+
+/* Previous-step logits (the stored form of p_{t-1}, Algorithm 1 line 2): *buf = dev [rows][vocab] cfg.dtype,
+ * packed as the PREVIOUS step packed them; *row_of_pos = dev int32 [B*N], row of each flat position in *buf
+ * or -1 when the position has no previous posterior.  Writing both lets a caller seed p_{t-1}. */
+int surelock_prev_logits(surelock_ctx *ctx, void **buf, int32_t **row_of_pos);
+
+/* Tuning / test switches.  "gemm_impl": 0 = tensor-core GEMM and attention when the shape allows (default),
+ * 1 = force the CUDA-core kernels.  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
+ * (after a caller seeded them), 0 forgets them.  Unknown names return SL_EINVAL. */
+int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
+
+/* Number of kernels the last surelock_step / surelock_layer_step call launched (host-side count). */
+int surelock_last_launch_count(surelock_ctx *ctx);
+
+void surelock_destroy(surelock_ctx *ctx);
+const char *surelock_strerror(int status);
+
+/* ---- single stages (same kernels the step uses; for stage-wise parity and for timing them alone) -------- */
+
+/* Bytes of zero-initialisable scratch surelock_compact needs for `total` flags. */
+size_t surelock_compact_scratch_bytes(int64_t total);
+
+/* Active-row compaction (Algorithm 1 line 6): A_t = { i : lock_i = 0 } for B sequences of N flags.
+ *   lock_mask  dev uint8 [B*N]
+ *   active_idx dev int32 [>= number of zeros]  ascending flat positions b*N+i
+ *   row_offsets dev int32 [B+1]                exclusive per-sequence offsets, [B] = M
+ *   n_active   dev int32 [1]                   M
+ *   row_of_pos dev int32 [B*N] or NULL         packed row of each position, -1 for locked positions
+ *   scratch    dev, surelock_compact_scratch_bytes(B*N) bytes; cleared by this call (cudaMemsetAsync)
+ *   dev_status dev int32 [1] or NULL           set non-zero if a bounded wait ran out
+ * B*N < 2^31.  Asynchronous on `stream`. */
+int surelock_compact(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
+                     int32_t *n_active, int32_t *row_of_pos, void *scratch, int32_t *dev_status, void *stream);
+
+/* K/V cache scatter (Algorithm 1 line 11, K^all[A_t] <- K[A_t]): cache row active_idx[r] <- packed row r, for
+ * r < *n_active; other cache rows are not touched.  k, v: dev [M][row_elems]; k_cache, v_cache: dev
+ * [B*N][row_elems]; dtype SL_BF16 or SL_FP32; row_elems*sizeof(elem) must be a multiple of 16. */
+int surelock_kv_scatter(const void *k, const void *v, const int32_t *active_idx, const int32_t *n_active,
+                        int max_rows, int row_elems, void *k_cache, void *v_cache, int dtype, void *stream);
+
+/* Fused softmax + step-wise KL + confidence + argmax + lock test + lock update (Algorithm 1 lines 15, 18-20,
+ * 23-24 with the confidence gate off), for rows r < *n_active:
+ *   p = softmax(logits[r]); conf[r] = max p; argmax[r]; pr = prev_row[...]:
+ *   kl[r] = sum_v p(v) (log p(v) - log q(v)) with q = softmax(prev_logits[pr]), or +inf when pr < 0;
+ *   if mask_state[pos] == 0 and kl[r] <= kl_eps: lock_mask[pos] = 1      (pos = active_idx[r])
+ *   logits      dev [M][vocab] dtype        prev_logits dev [*][vocab] dtype
+ *   row_of_pos_prev dev int32 [B*N]: row of position pos in prev_logits, or -1 (NULL: row r pairs with row r)
+ *   prev_lse    dev fp32 [rows of prev_logits] log-sum-exp of each previous row as an earlier call's lse_out
+ *               produced it, or NULL: then it is recomputed here from prev_logits
+ *   active_idx  dev int32 [M] (NULL: pos = r)      mask_state dev uint8 [B*N]     lock_mask dev uint8 [B*N]
+ *   kl, conf dev fp32 [M]; argmax dev int32 [M]; lse_out dev fp32 [M] or NULL (log-sum-exp of logits[r]).
+ * vocab*sizeof(elem) must be a multiple of 16.  prev_logits == NULL means "no previous posterior at all". */
+int surelock_softmax_kl_sure(const void *logits, const void *prev_logits, const int32_t *row_of_pos_prev,
+                             const float *prev_lse, const int32_t *active_idx, const int32_t *n_active, int max_rows,
+                             int vocab, int dtype, const uint8_t *mask_state, uint8_t *lock_mask, float kl_eps,
+                             float *kl, float *conf, int32_t *argmax, float *lse_out, void *stream);
+
+/* Dense contraction on packed rows, C[r][n] = sum_k A[r][k] * W[n][k] for r < *n_active (the projections of
+ * Algorithm 1 lines 10, 12, 15; FLOP terms of Sec. 2.3).  A: dev [M][K]; W: dev [n_out][K]; C: dev [M][n_out];
+ * A, W, C of `dtype`; fp32 accumulation.  impl: 0 = best available (tcgen05 tensor cores for SL_BF16 when the
+ * shape allows), 1 = force the CUDA-core kernel.  dev_status as for surelock_compact. */
+int surelock_gemm(const void *A, const void *W, void *C, const int32_t *n_active, int max_rows, int n_out, int K,
+                  int dtype, int impl, int32_t *dev_status, void *stream);
+
+/* M x N bidirectional attention of the packed queries against the whole cache (Algorithm 1 line 12; Sec. 2.1:
+ * "variable-length attention against the full key/value tables"): for packed row r at flat position
+ * active_idx[r] = b*N+i and every head h, o[r][h] = softmax_j(q[r][h] . K[b*N+j][h] / sqrt(d_h)) V[b*N+j][h],
+ * j = 0..N-1.  q, o: dev [M][H][d_h]; k_cache, v_cache: dev [B*N][H][d_h]; all of `dtype`. */
+int surelock_attention(const void *q, const void *k_cache, const void *v_cache, const int32_t *active_idx,
+                       const int32_t *row_offsets, const int32_t *n_active, int max_rows, int B, int N, int H,
+                       int head_dim, void *o, int dtype, int impl, int32_t *dev_status, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SURELOCK_H */

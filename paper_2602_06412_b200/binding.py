@@ -1,0 +1,258 @@
+"""Thin ctypes binding over the C ABI of include/surelock.h: argument marshalling only.
+
+Function names match the C entry points.  Tensors are torch CUDA tensors used as
+device memory; their `data_ptr()` is what crosses the boundary.  Outputs that the
+library owns are exposed as zero-copy torch views of the library's buffers.
+There is no fallback: if the shared library is missing, `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libsurelock.so")
+SL_BF16, SL_FP32 = 0, 1
+_lib = None
+
+
+class SurelockError(RuntimeError):
+    pass
+
+
+class _ModelCfg(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "n_kv_heads", "d_ff", "vocab",
+                                         "dtype")] + [("rms_eps", C.c_float), ("rope_theta", C.c_float),
+                                                      ("mask_token_id", C.c_int32)]
+
+
+class _Weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("tok_emb", "lm_head", "final_norm_g")] + \
+               [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm_g", "wq", "wk", "wv", "wo", "ffn_norm_g", "w_gate",
+                                                     "w_up", "w_down")]
+
+
+class _StepOut(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("active_idx", "row_offsets", "n_active", "logits", "hidden", "kl", "conf",
+                                          "argmax")]
+
+
+def lib() -> C.CDLL:
+    """Load libsurelock.so (built in-tree by `paper_2602_06412_b200.build`); raises if it is not there."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise SurelockError(f"{LIB_PATH} not built: run `python -m paper_2602_06412_b200.build` "
+                            "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, f32, sz = C.c_void_p, C.c_int, C.c_float, C.c_size_t
+    sig = {
+        "surelock_init": (i32, [C.POINTER(vp), C.POINTER(_ModelCfg), C.POINTER(_Weights), i32, i32, vp]),
+        "surelock_reset": (i32, [vp]),
+        "surelock_step": (i32, [vp, vp, vp, vp, f32, C.POINTER(_StepOut)]),
+        "surelock_step_host": (i32, [vp, vp, vp, vp, f32, vp, vp, vp, vp, vp]),
+        "surelock_layer_step": (i32, [vp, i32, vp, vp, vp, C.POINTER(_StepOut)]),
+        "surelock_status_poll": (i32, [vp, C.POINTER(i32)]),
+        "surelock_kv_cache": (i32, [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(sz)]),
+        "surelock_prev_logits": (i32, [vp, C.POINTER(vp), C.POINTER(vp)]),
+        "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
+        "surelock_last_launch_count": (i32, [vp]),
+        "surelock_destroy": (None, [vp]),
+        "surelock_strerror": (C.c_char_p, [i32]),
+        "surelock_compact_scratch_bytes": (sz, [C.c_int64]),
+        "surelock_compact": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "surelock_kv_scatter": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]),
+        "surelock_softmax_kl_sure": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, f32, vp, vp, vp, vp, vp]),
+        "surelock_gemm": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]),
+        "surelock_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32, vp, vp]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(L, name)
+        f.restype, f.argtypes = res, args
+    _lib = L
+    return L
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise SurelockError(f"{what}: {lib().surelock_strerror(rc).decode()} ({rc})")
+
+
+def _p(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors crossing the C ABI must be contiguous"
+    return t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return SL_BF16
+    if t.dtype == torch.float32:
+        return SL_FP32
+    raise SurelockError(f"unsupported dtype {t.dtype}")
+
+
+class _DevArray:
+    def __init__(self, ptr, shape, typestr):
+        self.__cuda_array_interface__ = dict(data=(ptr, False), shape=tuple(shape), typestr=typestr, version=2,
+                                             strides=None)
+
+
+def device_view(ptr: int, shape, dtype: torch.dtype) -> torch.Tensor:
+    """Zero-copy torch view of library-owned device memory."""
+    ts = {torch.int32: "<i4", torch.float32: "<f4", torch.uint8: "|u1", torch.bfloat16: "<i2"}[dtype]
+    t = torch.as_tensor(_DevArray(ptr, shape, ts), device="cuda")
+    return t.view(torch.bfloat16) if dtype == torch.bfloat16 else t
+
+
+class StepOut:
+    """Views of a step's packed outputs; every array has room for B*N rows, the first M = n_active are valid."""
+
+    def __init__(self, raw: _StepOut, R: int, B: int, d: int, V: int, tdtype):
+        self.active_idx = device_view(raw.active_idx, (R,), torch.int32)
+        self.row_offsets = device_view(raw.row_offsets, (B + 1,), torch.int32)
+        self.n_active = device_view(raw.n_active, (1,), torch.int32)
+        self.hidden = device_view(raw.hidden, (R, d), torch.float32) if raw.hidden else None
+        self.logits = device_view(raw.logits, (R, V), tdtype) if raw.logits and V > 0 else None
+        self.kl = device_view(raw.kl, (R,), torch.float32) if raw.kl else None
+        self.conf = device_view(raw.conf, (R,), torch.float32) if raw.conf else None
+        self.argmax = device_view(raw.argmax, (R,), torch.int32) if raw.argmax else None
+
+    def M(self) -> int:
+        return int(self.n_active.item())
+
+
+class Ctx:
+    def __init__(self, handle, cfg, N, B, tdtype, keep):
+        self.handle, self.cfg, self.N, self.B, self.tdtype, self._keep = handle, cfg, N, B, tdtype, keep
+
+    def __del__(self):
+        try:
+            surelock_destroy(self)
+        except Exception:
+            pass
+
+
+def surelock_init(cfg: Dict, weights: Dict, N: int, batch: int) -> Ctx:
+    """cfg: dict with the model shape; weights: dict of CUDA tensors (layout of inputs.make_weights)."""
+    layers = weights["layers"]
+    tdtype = layers[0]["wq"].dtype
+    mc = _ModelCfg(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["head_dim"], cfg["n_heads"], cfg["d_ff"],
+                   cfg["vocab"], _dt(layers[0]["wq"]), cfg["rms_eps"], cfg["rope_theta"], max(cfg["vocab"] - 1, 0))
+    w = _Weights()
+    keep = []
+    for name in ("tok_emb", "lm_head", "final_norm_g"):
+        setattr(w, name, _p(weights.get(name)) if cfg["vocab"] > 0 else None)
+    for name in ("attn_norm_g", "wq", "wk", "wv", "wo", "ffn_norm_g", "w_gate", "w_up", "w_down"):
+        arr = (C.c_void_p * len(layers))(*[_p(lw[name]) for lw in layers])
+        keep.append(arr)
+        setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
+    h = C.c_void_p()
+    _check(lib().surelock_init(C.byref(h), C.byref(mc), C.byref(w), N, batch, _stream()), "surelock_init")
+    return Ctx(h, dict(cfg), N, batch, tdtype, (keep, weights))
+
+
+def surelock_destroy(ctx: Ctx):
+    if ctx.handle:
+        lib().surelock_destroy(ctx.handle)
+        ctx.handle = None
+
+
+def surelock_reset(ctx: Ctx):
+    _check(lib().surelock_reset(ctx.handle), "surelock_reset")
+
+
+def surelock_step(ctx: Ctx, tokens, mask_state, lock_mask, kl_eps: float) -> StepOut:
+    raw = _StepOut()
+    _check(lib().surelock_step(ctx.handle, _p(tokens), _p(mask_state), _p(lock_mask), kl_eps, C.byref(raw)),
+           "surelock_step")
+    return StepOut(raw, ctx.N * ctx.B, ctx.B, ctx.cfg["d_model"], ctx.cfg["vocab"], ctx.tdtype)
+
+
+def surelock_step_host(ctx: Ctx, tokens, mask_state, lock_mask, kl_eps: float, n_active, active_idx=None, kl=None,
+                       conf=None, argmax=None):
+    """All tensors are HOST (CPU, ideally pinned) tensors; lock_mask is updated in place."""
+    _check(lib().surelock_step_host(ctx.handle, _p(tokens), _p(mask_state), _p(lock_mask), kl_eps, _p(n_active),
+                                    _p(active_idx), _p(kl), _p(conf), _p(argmax)), "surelock_step_host")
+
+
+def surelock_layer_step(ctx: Ctx, layer: int, hidden_in, lock_mask, hidden_out) -> StepOut:
+    raw = _StepOut()
+    _check(lib().surelock_layer_step(ctx.handle, layer, _p(hidden_in), _p(lock_mask), _p(hidden_out), C.byref(raw)),
+           "surelock_layer_step")
+    return StepOut(raw, ctx.N * ctx.B, ctx.B, ctx.cfg["d_model"], 0, ctx.tdtype)
+
+
+def surelock_status_poll(ctx: Ctx) -> int:
+    s = C.c_int(0)
+    rc = lib().surelock_status_poll(ctx.handle, C.byref(s))
+    if rc not in (0, -4):
+        _check(rc, "surelock_status_poll")
+    return s.value
+
+
+def surelock_kv_cache(ctx: Ctx, layer: int):
+    k, v, stride = C.c_void_p(), C.c_void_p(), C.c_size_t()
+    _check(lib().surelock_kv_cache(ctx.handle, layer, C.byref(k), C.byref(v), C.byref(stride)), "surelock_kv_cache")
+    shape = (ctx.B * ctx.N, ctx.cfg["n_heads"], ctx.cfg["head_dim"])
+    return device_view(k.value, shape, ctx.tdtype), device_view(v.value, shape, ctx.tdtype)
+
+
+def surelock_prev_logits(ctx: Ctx):
+    buf, rop = C.c_void_p(), C.c_void_p()
+    _check(lib().surelock_prev_logits(ctx.handle, C.byref(buf), C.byref(rop)), "surelock_prev_logits")
+    R = ctx.B * ctx.N
+    return device_view(buf.value, (R, ctx.cfg["vocab"]), ctx.tdtype), device_view(rop.value, (R,), torch.int32)
+
+
+def surelock_set_option(ctx: Ctx, name: str, value: int):
+    _check(lib().surelock_set_option(ctx.handle, name.encode(), value), "surelock_set_option")
+
+
+def surelock_last_launch_count(ctx: Ctx) -> int:
+    return lib().surelock_last_launch_count(ctx.handle)
+
+
+# ---- single stages -----------------------------------------------------------------------------------------
+def surelock_compact_scratch_bytes(total: int) -> int:
+    return lib().surelock_compact_scratch_bytes(total)
+
+
+def surelock_compact(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos, scratch, dev_status=None):
+    _check(lib().surelock_compact(_p(lock_mask), B, N, _p(active_idx), _p(row_offsets), _p(n_active), _p(row_of_pos),
+                                  _p(scratch), _p(dev_status), _stream()), "surelock_compact")
+
+
+def surelock_kv_scatter(k, v, active_idx, n_active, k_cache, v_cache):
+    _check(lib().surelock_kv_scatter(_p(k), _p(v), _p(active_idx), _p(n_active), k.shape[0], k[0].numel(), _p(k_cache),
+                                     _p(v_cache), _dt(k), _stream()), "surelock_kv_scatter")
+
+
+def surelock_softmax_kl_sure(logits, prev_logits, row_of_pos_prev, prev_lse, active_idx, n_active, mask_state,
+                             lock_mask, kl_eps: float, kl, conf, argmax, lse_out=None):
+    _check(lib().surelock_softmax_kl_sure(_p(logits), _p(prev_logits), _p(row_of_pos_prev), _p(prev_lse),
+                                          _p(active_idx), _p(n_active), logits.shape[0], logits.shape[1], _dt(logits),
+                                          _p(mask_state), _p(lock_mask), kl_eps, _p(kl), _p(conf), _p(argmax),
+                                          _p(lse_out), _stream()), "surelock_softmax_kl_sure")
+
+
+def surelock_gemm(A, W, Cout, n_active, impl: int = 0, dev_status=None):
+    _check(lib().surelock_gemm(_p(A), _p(W), _p(Cout), _p(n_active), A.shape[0], W.shape[0], A.shape[1], _dt(A), impl,
+                               _p(dev_status), _stream()), "surelock_gemm")
+
+
+def surelock_attention(q, k_cache, v_cache, active_idx, row_offsets, n_active, B: int, N: int, o, impl: int = 0,
+                       dev_status=None):
+    H, dh = q.shape[1], q.shape[2]
+    _check(lib().surelock_attention(_p(q), _p(k_cache), _p(v_cache), _p(active_idx), _p(row_offsets), _p(n_active),
+                                    q.shape[0], B, N, H, dh, _p(o), _dt(q), impl, _p(dev_status), _stream()),
+           "surelock_attention")

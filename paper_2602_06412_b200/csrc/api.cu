@@ -1,0 +1,375 @@
+// C ABI of the SureLock step: context, per-step launch sequence, accessors (see include/surelock.h).
+// The step is a fixed sequence of kernel launches on one stream; the number of active rows M lives in device
+// memory and every kernel reads it there, so nothing in surelock_step waits for the GPU.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace sl;
+
+struct surelock_ctx {
+  surelock_model_cfg cfg;
+  int N = 0, B = 0, R = 0;            // R = B*N = capacity in packed rows
+  size_t esz = 2;
+  cudaStream_t st = nullptr;
+  const void *tok_emb = nullptr, *lm_head = nullptr, *final_norm_g = nullptr;
+  std::vector<const void*> attn_norm_g, wq, wk, wv, wo, ffn_norm_g, w_gate, w_up, w_down;
+  std::vector<void*> allocs;
+  char* kv = nullptr;                 // [L][2][R][H*dh]
+  float* x = nullptr;                 // residual stream, fp32 [R][d]
+  void *h = nullptr, *q = nullptr, *k = nullptr, *v = nullptr, *attn = nullptr, *act = nullptr;
+  void* logits[2] = {nullptr, nullptr};
+  float* lse[2] = {nullptr, nullptr};
+  int32_t* row_of_pos[2] = {nullptr, nullptr};
+  int32_t *idx = nullptr, *row_offsets = nullptr, *n_active = nullptr, *status = nullptr, *argmax = nullptr;
+  float *kl = nullptr, *conf = nullptr;
+  void* scratch = nullptr;
+  float2* rope = nullptr;
+  int32_t* st_tokens = nullptr;       // device staging for surelock_step_host
+  uint8_t *st_mask = nullptr, *st_lock = nullptr;
+  int cur = 0;
+  bool have_prev = false;
+  int launches = 0;
+  int gemm_impl = 0;                  // 0 = tensor cores when possible, 1 = CUDA cores
+
+  size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
+  void* kcache(int l) const { return kv + (size_t)(2 * l) * kv_layer_bytes(); }
+  void* vcache(int l) const { return kv + (size_t)(2 * l + 1) * kv_layer_bytes(); }
+};
+
+#define SL_TRY(expr)            \
+  do {                          \
+    int rc__ = (expr);          \
+    if (rc__ != SL_OK) return rc__; \
+  } while (0)
+
+template <typename P>
+static int dev_alloc(surelock_ctx* c, P** p, size_t bytes) {
+  void* q = nullptr;
+  if (bytes == 0) bytes = 16;
+  if (cudaMalloc(&q, bytes) != cudaSuccess) {
+    cudaGetLastError();
+    return SL_ENOMEM;
+  }
+  c->allocs.push_back(q);
+  *p = reinterpret_cast<P*>(q);
+  return SL_OK;
+}
+
+namespace sl {
+int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
+                   int n_out, int K, int epilogue, int32_t* status, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
+}
+
+static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
+  ++c->launches;
+  if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
+    const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->st);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
+  return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
+}
+
+// Algorithm 1 lines 10-13 for one layer on the packed rows in x (fp32 [M][d], updated in place).
+static int run_layer(surelock_ctx* c, int l, float* x) {
+  const surelock_model_cfg& g = c->cfg;
+  const int d = g.d_model, hd = g.n_heads * g.head_dim;
+  SL_TRY(launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
+  ++c->launches;
+  SL_TRY(gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
+  SL_TRY(gemm(c, c->h, c->wk[l], nullptr, c->k, hd, d, EPI_STORE));
+  SL_TRY(gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
+  SL_TRY(launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
+  SL_TRY(launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
+  SL_TRY(launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads,
+                               g.head_dim, c->attn, g.dtype, c->st));
+  c->launches += 3;
+  SL_TRY(gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
+  SL_TRY(launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
+  ++c->launches;
+  SL_TRY(gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
+  SL_TRY(gemm(c, c->act, c->w_down[l], nullptr, x, d, g.d_ff, EPI_RESIDUAL));
+  return SL_OK;
+}
+
+extern "C" {
+
+int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surelock_weights* w, int N, int batch,
+                  void* cuda_stream) {
+  if (!out || !cfg || !w || N <= 0 || batch <= 0) return SL_EINVAL;
+  *out = nullptr;
+  if (cfg->n_layers <= 0 || cfg->d_model <= 0 || cfg->n_heads <= 0 || cfg->d_ff <= 0 || cfg->vocab < 0)
+    return SL_EINVAL;
+  if (cfg->dtype != SL_BF16 && cfg->dtype != SL_FP32) return SL_EINVAL;
+  if (cfg->n_kv_heads != cfg->n_heads) return SL_EUNSUPPORTED;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return SL_EUNSUPPORTED;
+  if (cfg->d_model % 8 || cfg->d_ff % 8 || cfg->vocab % 8) return SL_EUNSUPPORTED;
+  if ((long long)N * batch >= (1ll << 31)) return SL_EINVAL;
+  if (!w->attn_norm_g || !w->wq || !w->wk || !w->wv || !w->wo || !w->ffn_norm_g || !w->w_gate || !w->w_up ||
+      !w->w_down)
+    return SL_EINVAL;
+  if (cfg->vocab > 0 && (!w->tok_emb || !w->lm_head || !w->final_norm_g)) return SL_EINVAL;
+  for (int l = 0; l < cfg->n_layers; ++l)
+    if (!w->attn_norm_g[l] || !w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->ffn_norm_g[l] ||
+        !w->w_gate[l] || !w->w_up[l] || !w->w_down[l])
+      return SL_EINVAL;
+
+  surelock_ctx* c = new (std::nothrow) surelock_ctx();
+  if (!c) return SL_ENOMEM;
+  c->cfg = *cfg;
+  c->N = N;
+  c->B = batch;
+  c->R = N * batch;
+  c->esz = cfg->dtype == SL_BF16 ? 2 : 4;
+  c->st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  c->tok_emb = w->tok_emb;
+  c->lm_head = w->lm_head;
+  c->final_norm_g = w->final_norm_g;
+  const int L = cfg->n_layers;
+  c->attn_norm_g.assign(w->attn_norm_g, w->attn_norm_g + L);
+  c->wq.assign(w->wq, w->wq + L);
+  c->wk.assign(w->wk, w->wk + L);
+  c->wv.assign(w->wv, w->wv + L);
+  c->wo.assign(w->wo, w->wo + L);
+  c->ffn_norm_g.assign(w->ffn_norm_g, w->ffn_norm_g + L);
+  c->w_gate.assign(w->w_gate, w->w_gate + L);
+  c->w_up.assign(w->w_up, w->w_up + L);
+  c->w_down.assign(w->w_down, w->w_down + L);
+
+  const size_t R = c->R, d = cfg->d_model, hd = (size_t)cfg->n_heads * cfg->head_dim, F = cfg->d_ff, V = cfg->vocab;
+  const size_t e = c->esz;
+  int rc = SL_OK;
+#define A_(p, bytes) if (rc == SL_OK) rc = dev_alloc(c, &(p), (bytes))
+  A_(c->kv, 2 * (size_t)L * R * hd * e);
+  A_(c->x, R * d * 4);
+  A_(c->h, R * d * e);
+  A_(c->q, R * hd * e);
+  A_(c->k, R * hd * e);
+  A_(c->v, R * hd * e);
+  A_(c->attn, R * hd * e);
+  A_(c->act, R * F * e);
+  for (int i = 0; i < 2; ++i) {
+    A_(c->logits[i], R * V * e);
+    A_(c->lse[i], R * 4);
+    A_(c->row_of_pos[i], R * 4);
+  }
+  A_(c->idx, R * 4);
+  A_(c->row_offsets, ((size_t)batch + 1) * 4);
+  A_(c->n_active, 16);
+  A_(c->status, 16);
+  A_(c->argmax, R * 4);
+  A_(c->kl, R * 4);
+  A_(c->conf, R * 4);
+  A_(c->scratch, compact_scratch_bytes((int64_t)R));
+  A_(c->rope, (size_t)N * (cfg->head_dim / 2) * sizeof(float2));
+  A_(c->st_tokens, R * 4);
+  A_(c->st_mask, R);
+  A_(c->st_lock, R);
+#undef A_
+  if (rc == SL_OK && cudaMemsetAsync(c->kv, 0, 2 * (size_t)L * R * hd * e, c->st) != cudaSuccess) rc = SL_ECUDA;
+  if (rc == SL_OK) rc = build_rope_table(c->rope, N, cfg->head_dim, cfg->rope_theta, c->st);
+  if (rc == SL_OK) rc = surelock_reset(c);
+  if (rc == SL_OK && cudaStreamSynchronize(c->st) != cudaSuccess) rc = SL_ECUDA;
+  if (rc != SL_OK) {
+    surelock_destroy(c);
+    return rc;
+  }
+  *out = c;
+  return SL_OK;
+}
+
+int surelock_reset(surelock_ctx* c) {
+  if (!c) return SL_EINVAL;
+  c->have_prev = false;
+  c->cur = 0;
+  for (int i = 0; i < 2; ++i) SL_CUDA_TRY(cudaMemsetAsync(c->row_of_pos[i], 0xff, (size_t)c->R * 4, c->st));
+  SL_CUDA_TRY(cudaMemsetAsync(c->status, 0, 16, c->st));
+  SL_CUDA_TRY(cudaMemsetAsync(c->n_active, 0, 16, c->st));
+  return SL_OK;
+}
+
+int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps,
+                  surelock_step_out* out) {
+  if (!c || !tokens || !mask_state || !lock_mask) return SL_EINVAL;
+  if (!(kl_eps >= 0.f)) return SL_EINVAL;   // also rejects NaN
+  if (c->cfg.vocab <= 0) return SL_EUNSUPPORTED;
+  const surelock_model_cfg& g = c->cfg;
+  c->launches = 0;
+  const int cur = c->cur, prv = cur ^ 1;
+  SL_TRY(launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur], c->scratch,
+                        c->status, c->st));
+  SL_TRY(launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype,
+                            c->status, c->st));
+  c->launches += 2;
+  for (int l = 0; l < g.n_layers; ++l) SL_TRY(run_layer(c, l, c->x));
+  SL_TRY(launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
+  ++c->launches;
+  SL_TRY(gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
+  SL_TRY(launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
+                                c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state, lock_mask,
+                                kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st));
+  ++c->launches;
+  if (out) {
+    out->active_idx = c->idx;
+    out->row_offsets = c->row_offsets;
+    out->n_active = c->n_active;
+    out->logits = c->logits[cur];
+    out->hidden = c->x;
+    out->kl = c->kl;
+    out->conf = c->conf;
+    out->argmax = c->argmax;
+  }
+  c->cur = prv;
+  c->have_prev = true;
+  return SL_OK;
+}
+
+int surelock_step_host(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_state, uint8_t* lock_mask,
+                       float kl_eps, int32_t* n_active, int32_t* active_idx, float* kl, float* conf, int32_t* argmax) {
+  if (!c || !tokens || !mask_state || !lock_mask || !n_active) return SL_EINVAL;
+  const size_t R = c->R;
+  SL_CUDA_TRY(cudaMemcpyAsync(c->st_tokens, tokens, R * 4, cudaMemcpyHostToDevice, c->st));
+  SL_CUDA_TRY(cudaMemcpyAsync(c->st_mask, mask_state, R, cudaMemcpyHostToDevice, c->st));
+  SL_CUDA_TRY(cudaMemcpyAsync(c->st_lock, lock_mask, R, cudaMemcpyHostToDevice, c->st));
+  SL_TRY(surelock_step(c, c->st_tokens, c->st_mask, c->st_lock, kl_eps, nullptr));
+  SL_CUDA_TRY(cudaMemcpyAsync(lock_mask, c->st_lock, R, cudaMemcpyDeviceToHost, c->st));
+  SL_CUDA_TRY(cudaMemcpyAsync(n_active, c->n_active, 4, cudaMemcpyDeviceToHost, c->st));
+  if (active_idx) SL_CUDA_TRY(cudaMemcpyAsync(active_idx, c->idx, R * 4, cudaMemcpyDeviceToHost, c->st));
+  if (kl) SL_CUDA_TRY(cudaMemcpyAsync(kl, c->kl, R * 4, cudaMemcpyDeviceToHost, c->st));
+  if (conf) SL_CUDA_TRY(cudaMemcpyAsync(conf, c->conf, R * 4, cudaMemcpyDeviceToHost, c->st));
+  if (argmax) SL_CUDA_TRY(cudaMemcpyAsync(argmax, c->argmax, R * 4, cudaMemcpyDeviceToHost, c->st));
+  SL_CUDA_TRY(cudaStreamSynchronize(c->st));
+  return SL_OK;
+}
+
+int surelock_layer_step(surelock_ctx* c, int layer, const void* hidden_in, const uint8_t* lock_mask, float* hidden_out,
+                        surelock_step_out* out) {
+  if (!c || !hidden_in || !lock_mask || !hidden_out) return SL_EINVAL;
+  if (layer < 0 || layer >= c->cfg.n_layers) return SL_EINVAL;
+  const surelock_model_cfg& g = c->cfg;
+  c->launches = 0;
+  SL_TRY(launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, nullptr, c->scratch, c->status,
+                        c->st));
+  SL_TRY(launch_gather_rows(hidden_in, nullptr, c->idx, c->n_active, c->R, g.d_model, c->R, hidden_out, g.dtype,
+                            c->status, c->st));
+  c->launches += 2;
+  SL_TRY(run_layer(c, layer, hidden_out));
+  if (out) {
+    memset(out, 0, sizeof(*out));
+    out->active_idx = c->idx;
+    out->row_offsets = c->row_offsets;
+    out->n_active = c->n_active;
+    out->hidden = hidden_out;
+  }
+  return SL_OK;
+}
+
+int surelock_status_poll(surelock_ctx* c, int* device_status) {
+  if (!c) return SL_EINVAL;
+  int32_t s = 0;
+  if (cudaStreamSynchronize(c->st) != cudaSuccess) return SL_ECUDA;
+  if (cudaMemcpy(&s, c->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return SL_ECUDA;
+  if (device_status) *device_status = s;
+  return s ? SL_EDEVICE : SL_OK;
+}
+
+int surelock_kv_cache(surelock_ctx* c, int layer, void** k, void** v, size_t* row_stride_elems) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers) return SL_EINVAL;
+  if (k) *k = c->kcache(layer);
+  if (v) *v = c->vcache(layer);
+  if (row_stride_elems) *row_stride_elems = (size_t)c->cfg.n_heads * c->cfg.head_dim;
+  return SL_OK;
+}
+
+int surelock_prev_logits(surelock_ctx* c, void** buf, int32_t** row_of_pos) {
+  if (!c) return SL_EINVAL;
+  // the buffer the NEXT step reads as "previous" is the one the last step wrote
+  const int prv = c->cur ^ 1;
+  if (buf) *buf = c->logits[prv];
+  if (row_of_pos) *row_of_pos = c->row_of_pos[prv];
+  return SL_OK;
+}
+
+int surelock_set_option(surelock_ctx* c, const char* name, int value) {
+  if (!c || !name) return SL_EINVAL;
+  if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
+  if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
+  return SL_EINVAL;
+}
+
+int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
+
+void surelock_destroy(surelock_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->st);
+  for (void* p : c->allocs) cudaFree(p);
+  delete c;
+}
+
+const char* surelock_strerror(int s) {
+  switch (s) {
+    case SL_OK: return "ok";
+    case SL_EINVAL: return "invalid argument";
+    case SL_ENOMEM: return "device allocation failed";
+    case SL_ECUDA: return "CUDA runtime error";
+    case SL_EDEVICE: return "a kernel reported an error through the status word";
+    case SL_EUNSUPPORTED: return "shape or type not supported";
+    default: return "unknown status";
+  }
+}
+
+// ---- single stages ------------------------------------------------------------------------------------------
+
+size_t surelock_compact_scratch_bytes(int64_t total) { return compact_scratch_bytes(total); }
+
+int surelock_compact(const uint8_t* lock_mask, int B, int N, int32_t* active_idx, int32_t* row_offsets, int32_t* n_active,
+                     int32_t* row_of_pos, void* scratch, int32_t* dev_status, void* stream) {
+  return launch_compact(lock_mask, B, N, active_idx, row_offsets, n_active, row_of_pos, scratch, dev_status,
+                        (cudaStream_t)stream);
+}
+
+int surelock_kv_scatter(const void* k, const void* v, const int32_t* active_idx, const int32_t* n_active, int max_rows,
+                        int row_elems, void* k_cache, void* v_cache, int dtype, void* stream) {
+  if (!k || !v || !active_idx || !n_active || !k_cache || !v_cache || max_rows < 0 || row_elems <= 0) return SL_EINVAL;
+  if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
+  return launch_kv_scatter(k, v, active_idx, n_active, max_rows, row_elems, k_cache, v_cache, dtype, (cudaStream_t)stream);
+}
+
+int surelock_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
+                             const float* prev_lse, const int32_t* active_idx, const int32_t* n_active, int max_rows,
+                             int vocab, int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
+                             float* conf, int32_t* argmax, float* lse_out, void* stream) {
+  if (!logits || !n_active || !mask_state || !lock_mask || !kl || !conf || !argmax || max_rows < 0) return SL_EINVAL;
+  if (!(kl_eps >= 0.f)) return SL_EINVAL;
+  if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
+  return launch_softmax_kl_sure(logits, prev_logits, row_of_pos_prev, prev_lse, active_idx, n_active, max_rows, vocab,
+                                dtype, mask_state, lock_mask, kl_eps, kl, conf, argmax, lse_out, (cudaStream_t)stream);
+}
+
+int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active, int max_rows, int n_out, int K,
+                  int dtype, int impl, int32_t* dev_status, void* stream) {
+  if (!A || !W || !C || !n_active || max_rows < 0 || n_out <= 0 || K <= 0) return SL_EINVAL;
+  if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
+  if (dtype == SL_BF16 && impl == 0) {
+    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, (cudaStream_t)stream);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
+  return launch_gemm_simt(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, (cudaStream_t)stream);
+}
+
+int surelock_attention(const void* q, const void* k_cache, const void* v_cache, const int32_t* active_idx,
+                       const int32_t* row_offsets, const int32_t* n_active, int max_rows, int B, int N, int H,
+                       int head_dim, void* o, int dtype, int impl, int32_t* dev_status, void* stream) {
+  if (!q || !k_cache || !v_cache || !active_idx || !n_active || !o || max_rows < 0 || B <= 0 || N <= 0 || H <= 0)
+    return SL_EINVAL;
+  if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
+  (void)row_offsets; (void)impl; (void)dev_status;
+  return launch_attention_simt(q, k_cache, v_cache, active_idx, n_active, max_rows, N, H, head_dim, o, dtype,
+                               (cudaStream_t)stream);
+}
+
+}  // extern "C"

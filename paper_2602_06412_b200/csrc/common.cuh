@@ -1,0 +1,84 @@
+// Shared declarations of the SureLock CUDA library (internal; the public interface is include/surelock.h).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "surelock.h"
+
+// Device status codes stored (first writer wins) in the ctx status word.
+enum {
+  SL_DEV_OK = 0,
+  SL_DEV_COMPACT_TIMEOUT = 1,   // decoupled look-back of the compaction gave up waiting for a predecessor chunk
+  SL_DEV_GEMM_TIMEOUT = 2,      // an mbarrier wait in the tcgen05 GEMM ran out
+  SL_DEV_ATTN_TIMEOUT = 3,      // an mbarrier wait in the tcgen05 attention ran out
+  SL_DEV_BAD_INDEX = 4          // an index read from device memory was out of range and was skipped
+};
+
+#define SL_CUDA_TRY(expr)                       \
+  do {                                          \
+    cudaError_t e__ = (expr);                   \
+    if (e__ != cudaSuccess) return SL_ECUDA;    \
+  } while (0)
+
+namespace sl {
+
+typedef __nv_bfloat16 bf16;
+
+__device__ __forceinline__ float to_f(float v) { return v; }
+__device__ __forceinline__ float to_f(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f(float v);
+template <> __device__ __forceinline__ float from_f<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ void set_status(int32_t* status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+inline int sm_count() {
+  static int n = 0;
+  if (!n) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+    if (n <= 0) n = 148;
+  }
+  return n;
+}
+
+// ---- launchers (one per kernel family); all asynchronous on `st`, rows beyond *n_active are not touched ----
+
+size_t compact_scratch_bytes(int64_t total);
+int launch_compact(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
+                   int32_t* row_of_pos, void* scratch, int32_t* status, cudaStream_t st);
+
+// x[r] = table[tokens[idx[r]]] (embedding) or x[r] = src[idx[r]] (tokens == nullptr), widened to fp32
+int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* idx, const int32_t* n_active,
+                       int max_rows, int d, int table_rows, float* x, int dtype, int32_t* status, cudaStream_t st);
+int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_active, int max_rows, int d,
+                   float eps, int dtype, cudaStream_t st);
+int build_rope_table(float2* table, int N, int head_dim, float theta, cudaStream_t st);
+// in-place rotation of q and k [M][H][dh] with position idx[r] % N
+int launch_rope(void* q, void* k, const int32_t* idx, const int32_t* n_active, int max_rows, int N, int H,
+                int head_dim, const float2* table, int dtype, cudaStream_t st);
+int launch_kv_scatter(const void* k, const void* v, const int32_t* idx, const int32_t* n_active, int max_rows,
+                      int row_elems, void* kc, void* vc, int dtype, cudaStream_t st);
+
+enum GemmEpilogue {
+  EPI_STORE = 0,      // C[T] = acc
+  EPI_RESIDUAL = 1,   // Cf32 += acc
+  EPI_SWIGLU = 2      // C[T] = silu(acc(W)) * acc(W2)
+};
+// C = A[M][K] . W[n_out][K]^T on CUDA cores (fp32 FMA); W2 only for EPI_SWIGLU
+int launch_gemm_simt(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
+                     int n_out, int K, int dtype, int epilogue, cudaStream_t st);
+
+int launch_attention_simt(const void* q, const void* kc, const void* vc, const int32_t* idx, const int32_t* n_active,
+                          int max_rows, int N, int H, int head_dim, void* o, int dtype, cudaStream_t st);
+
+int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
+                           const float* prev_lse, const int32_t* idx, const int32_t* n_active, int max_rows, int vocab,
+                           int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
+                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st);
+
+}  // namespace sl

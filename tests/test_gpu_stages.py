@@ -1,0 +1,228 @@
+"""Stage-wise GPU parity: each kernel, called through the C ABI, against the CPU oracle on the same seeded inputs.
+
+Integer and byte work is compared bit for bit; floating point within the stated tolerances:
+hidden states / logits / GEMM and attention outputs 2e-2 max relative error (bf16 path; the fp32 path is held to
+1e-4), KL 1e-3 relative (plus 1e-9 absolute so that "KL of identical posteriors is 0" is testable), lock
+decisions exact except where the oracle's KL lies within 1e-3 relative of the threshold.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import surelock_oracle as O
+from paper_2602_06412_b200 import binding as SL
+from paper_2602_06412_b200 import inputs
+from tests.parity_util import f64, rel_err_rows
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def _compact(lock):
+    B, N = lock.shape
+    d = lock.to(DEV).contiguous()
+    idx = torch.full((B * N,), -7, dtype=torch.int32, device=DEV)
+    offs = torch.full((B + 1,), -7, dtype=torch.int32, device=DEV)
+    n = torch.full((1,), -7, dtype=torch.int32, device=DEV)
+    rop = torch.full((B * N,), -7, dtype=torch.int32, device=DEV)
+    scratch = torch.empty(SL.surelock_compact_scratch_bytes(B * N), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    SL.surelock_compact(d, B, N, idx, offs, n, rop, scratch, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    return idx.cpu().numpy(), offs.cpu().numpy(), int(n.item()), rop.cpu().numpy()
+
+
+def _check_compact(lock):
+    idx, offs, M, rop = _compact(lock)
+    ridx, roffs = O.active_set(lock.numpy())
+    assert M == len(ridx)
+    assert np.array_equal(idx[:M], ridx)
+    assert np.array_equal(offs, roffs)
+    assert np.all(idx[M:] == -7)                                     # nothing written past M
+    want = np.full(lock.numel(), -1, np.int32)
+    want[ridx] = np.arange(M, dtype=np.int32)
+    assert np.array_equal(rop, want)
+
+
+@pytest.mark.parametrize("B,N", [(1, 128), (3, 37), (1, 1), (5, 16), (8, 1536), (4, 4096), (2, 4099), (7, 5)])
+def test_compact_random(B, N):
+    g = torch.Generator().manual_seed(B * 1000 + N)
+    for p in (0.5, 0.05, 0.95):
+        _check_compact((torch.rand((B, N), generator=g) < p).to(torch.uint8))
+
+
+def test_compact_degenerate_masks():
+    for B, N in [(1, 128), (4, 4096), (3, 37)]:
+        _check_compact(torch.zeros((B, N), dtype=torch.uint8))       # nothing locked: M = B*N
+        _check_compact(torch.ones((B, N), dtype=torch.uint8))        # everything locked: M = 0
+        one = torch.ones((B, N), dtype=torch.uint8)
+        one[B - 1, N - 1] = 0
+        _check_compact(one)                                          # single active row, the very last flag
+        one = torch.zeros((B, N), dtype=torch.uint8)
+        one[0, 0] = 1
+        _check_compact(one)
+    # any non-zero byte counts as locked
+    lk = torch.tensor([[0, 2, 0, 255, 0, 1, 0, 0]], dtype=torch.uint8)
+    idx, offs, M, _ = _compact(lk)
+    assert list(idx[:M]) == [0, 2, 4, 6, 7]
+
+
+def test_compact_many_chunks_lookback():
+    B, N = 3, (1 << 20) + 5                                          # 769 chunks of 4096 flags, ragged tail
+    g = torch.Generator().manual_seed(9)
+    lock = (torch.rand((B, N), generator=g) < 0.4).to(torch.uint8)
+    idx, offs, M, rop = _compact(lock)
+    flat = lock.numpy().reshape(-1)
+    ref = np.flatnonzero(flat == 0).astype(np.int32)                 # same definition as oracle.active_set, vectorised
+    small, _ = O.active_set(lock[:, :2000].numpy())                  # and the oracle itself on a slice
+    assert np.array_equal(small, np.concatenate([np.flatnonzero(lock[b, :2000].numpy() == 0) + b * 2000 for b in range(B)]))
+    assert M == len(ref) and np.array_equal(idx[:M], ref)
+    assert list(offs) == [0] + list(np.cumsum((lock.numpy() == 0).sum(1)))
+
+
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+def test_kv_scatter_layout_bit_exact(dtype):
+    B, N, H, dh = 2, 300, 4, 64
+    lock = inputs.random_lock(B, N, [123, 7], 3)
+    idx, _ = O.active_set(lock.numpy())
+    M = len(idx)
+    g = torch.Generator().manual_seed(1)
+    k = torch.randn((B * N, H * dh), generator=g).to(dtype).to(DEV)
+    v = torch.randn((B * N, H * dh), generator=g).to(dtype).to(DEV)
+    kc0 = torch.randn((B * N, H * dh), generator=g).to(dtype).to(DEV)
+    vc0 = torch.randn((B * N, H * dh), generator=g).to(dtype).to(DEV)
+    kc, vc = kc0.clone(), vc0.clone()
+    SL.surelock_kv_scatter(k, v, torch.from_numpy(idx).to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV), kc, vc)
+    torch.cuda.synchronize()
+    want_k, want_v = kc0.clone(), vc0.clone()
+    li = torch.from_numpy(idx).long().to(DEV)
+    want_k[li] = k[:M]
+    want_v[li] = v[:M]
+    as_bits = lambda t: t.view(torch.int16 if dtype == torch.bfloat16 else torch.int32)
+    assert torch.equal(as_bits(kc), as_bits(want_k)) and torch.equal(as_bits(vc), as_bits(want_v))
+
+
+def _kl_case(rows, V, dtype, seed, eps=1e-3, use_lse=False):
+    cur, prev, mask = inputs.kl_logit_pairs(rows, V, seed, dtype=dtype)
+    rop = torch.arange(rows, dtype=torch.int32)
+    rop[rows // 3] = -1                                              # one row without a previous posterior
+    perm = torch.randperm(rows, generator=torch.Generator().manual_seed(seed))
+    prev_shuf = torch.empty_like(prev)                               # previous rows live at other packed rows
+    prev_shuf[perm] = prev
+    rop_pos = torch.where(rop >= 0, perm.to(torch.int32), rop)
+    pos = torch.arange(rows, dtype=torch.int32)
+    lock = torch.zeros(rows, dtype=torch.uint8)
+    d = lambda t: t.to(DEV)
+    kl = torch.empty(rows, dtype=torch.float32, device=DEV)
+    conf = torch.empty_like(kl)
+    am = torch.empty(rows, dtype=torch.int32, device=DEV)
+    lse = torch.empty_like(kl)
+    lock_d = d(lock)
+    n = torch.tensor([rows], dtype=torch.int32, device=DEV)
+    prev_lse = None
+    if use_lse:                                                      # produce lse of the previous rows with the kernel itself
+        pl = torch.empty_like(kl)
+        SL.surelock_softmax_kl_sure(d(prev_shuf), None, None, None, None, n, d(torch.ones(rows, dtype=torch.uint8)),
+                                    torch.zeros(rows, dtype=torch.uint8, device=DEV), 0.0, kl.clone(), conf.clone(),
+                                    am.clone(), pl)
+        prev_lse = pl
+    SL.surelock_softmax_kl_sure(d(cur), d(prev_shuf), d(rop_pos), prev_lse, d(pos), n, d(mask), lock_d, eps, kl, conf, am, lse)
+    torch.cuda.synchronize()
+    z, y = f64(cur), f64(prev)
+    ref_kl = O.kl_from_logits(z, y)
+    ref_kl[rows // 3] = np.inf
+    ref_conf, ref_am = O.posterior_stats(z)
+    got_kl = kl.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(ref_kl)
+    assert np.all(np.isinf(got_kl[~fin]))
+    err = np.abs(got_kl[fin] - ref_kl[fin])
+    assert np.all(err <= 1e-3 * ref_kl[fin] + 1e-9), (err.max(), ref_kl[fin][np.argmax(err / (ref_kl[fin] + 1e-30))])
+    same = (np.arange(rows) % 20) == 7
+    same[rows // 3] = False
+    assert np.all(got_kl[same] == 0.0)                               # identical posteriors: exactly 0
+    assert np.array_equal(am.cpu().numpy(), ref_am)
+    np.testing.assert_allclose(conf.cpu().numpy(), ref_conf, rtol=2e-5)
+    np.testing.assert_allclose(lse.cpu().numpy(), (z - O.log_softmax(z))[:, 0], rtol=0, atol=2e-5)
+    want = O.sure_test(ref_kl, mask.numpy(), eps)
+    near = fin & (np.abs(ref_kl - eps) <= 1e-3 * eps)
+    got = lock_d.cpu().numpy().astype(bool)
+    assert np.array_equal(got[~near], want[~near])
+    assert not got[mask.numpy() == 1].any()
+    return got_kl, ref_kl
+
+
+def test_softmax_kl_sure_llada_vocab_bf16():
+    got, ref = _kl_case(96, 126464, torch.bfloat16, 5)
+    fin = np.isfinite(ref) & (ref > 0)
+    assert ref[fin].min() < 1e-5 and ref[fin].max() > 1e-2           # the case really spans the threshold range
+
+
+def test_softmax_kl_sure_with_kept_lse():
+    _kl_case(40, 126464, torch.bfloat16, 6, use_lse=True)
+
+
+def test_softmax_kl_sure_small_vocab_fp32_and_bf16():
+    _kl_case(33, 2048, torch.float32, 7)
+    _kl_case(33, 2048, torch.bfloat16, 8)
+    _kl_case(5, 8, torch.bfloat16, 9)                                # a single 128-bit vector per row
+    _kl_case(600, 512, torch.float32, 10, eps=5e-5)                  # more rows than CTAs
+
+
+def test_softmax_kl_sure_first_step_and_empty():
+    rows, V = 12, 2048
+    cur, prev, mask = inputs.kl_logit_pairs(rows, V, 3, dtype=torch.float32)
+    kl = torch.full((rows,), -1.0, device=DEV)
+    conf = torch.full((rows,), -1.0, device=DEV)
+    am = torch.full((rows,), -1, dtype=torch.int32, device=DEV)
+    lock = torch.zeros(rows, dtype=torch.uint8, device=DEV)
+    n = torch.tensor([rows], dtype=torch.int32, device=DEV)
+    # no previous posterior at all: D = inf, nothing locks (first step)
+    SL.surelock_softmax_kl_sure(cur.to(DEV), None, None, None, None, n, torch.zeros(rows, dtype=torch.uint8, device=DEV),
+                                lock, 1e9, kl, conf, am)
+    torch.cuda.synchronize()
+    assert torch.isinf(kl).all() and not lock.any()
+    # M = 0: outputs untouched
+    kl.fill_(-1.0)
+    SL.surelock_softmax_kl_sure(cur.to(DEV), prev.to(DEV), None, None, None, torch.zeros(1, dtype=torch.int32, device=DEV),
+                                mask.to(DEV), lock, 1e-3, kl, conf, am)
+    torch.cuda.synchronize()
+    assert (kl == -1.0).all()
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
+@pytest.mark.parametrize("M,n_out,K", [(70, 200, 132), (1, 64, 64), (257, 96, 1024)])
+def test_gemm_cuda_cores(dtype, tol, M, n_out, K):
+    if dtype == torch.bfloat16:
+        n_out, K = (n_out + 7) // 8 * 8, (K + 7) // 8 * 8
+    g = torch.Generator().manual_seed(M + K)
+    A = torch.randn((M + 5, K), generator=g).to(dtype)
+    W = (torch.randn((n_out, K), generator=g) * 0.05).to(dtype)
+    out = torch.full((M + 5, n_out), 3.0, dtype=dtype, device=DEV)
+    SL.surelock_gemm(A.to(DEV), W.to(DEV), out, torch.tensor([M], dtype=torch.int32, device=DEV), impl=1)
+    torch.cuda.synchronize()
+    ref = f64(A[:M]) @ f64(W).T
+    assert rel_err_rows(f64(out[:M]), ref) < tol
+    assert (out[M:] == 3.0).all()                                    # rows beyond M untouched
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
+@pytest.mark.parametrize("B,N,H,dh,n_act", [(2, 77, 3, 64, [20, 77]), (1, 200, 2, 128, [9]), (3, 33, 1, 64, [0, 33, 1])])
+def test_attention_cuda_cores(dtype, tol, B, N, H, dh, n_act):
+    lock = inputs.random_lock(B, N, n_act, 11)
+    idx, offs = O.active_set(lock.numpy())
+    M = len(idx)
+    g = torch.Generator().manual_seed(N)
+    q = torch.randn((B * N, H, dh), generator=g).to(dtype)
+    Kc = torch.randn((B * N, H, dh), generator=g).to(dtype)
+    Vc = torch.randn((B * N, H, dh), generator=g).to(dtype)
+    o = torch.zeros((B * N, H, dh), dtype=dtype, device=DEV)
+    SL.surelock_attention(q.to(DEV), Kc.to(DEV), Vc.to(DEV), torch.from_numpy(idx).to(DEV) if M else torch.zeros(1, dtype=torch.int32, device=DEV),
+                          torch.from_numpy(offs).to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV), B, N, o, impl=1)
+    torch.cuda.synchronize()
+    for b in range(B):
+        r0, r1 = offs[b], offs[b + 1]
+        if r1 == r0:
+            continue
+        ref = O.attention_rows(f64(q[r0:r1]), f64(Kc[b * N:(b + 1) * N]), f64(Vc[b * N:(b + 1) * N]))
+        assert rel_err_rows(f64(o[r0:r1]).reshape(r1 - r0, -1), ref) < tol

@@ -1,0 +1,172 @@
+"""Whole-step GPU parity against the CPU oracle: the tiny fp32 model (free running, sampler loop, natural and
+forced lock schedules), a bf16 model through the same step, the single-layer call at LLaDA-8B layer shape, the
+host-buffer entry point, and the invariants of the cache (locked rows' bytes never change)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import surelock_oracle as O
+from paper_2602_06412_b200 import binding as SL
+from paper_2602_06412_b200 import inputs
+from tests.parity_util import f64, rel_err_rows, to_dev
+from tests.stepper import run_side_by_side
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def test_tiny_fp32_sampler_natural_locks():
+    cfg = inputs.model_shape("tiny")
+    log = []
+    trace, ctx, st = run_side_by_side(cfg, torch.float32, B=1, N=128, n_prompt=64, steps=64, kl_eps=1e-3, seed=1,
+                                      tol_logits=1e-4, check_kl_free_running=True, log=log)
+    assert trace[0] == 128 and trace[1] == 128          # D_1 = inf: nothing can lock before the second step
+    assert min(trace) < 128                             # and SureLock does shrink the active set afterwards
+    assert all(a >= b for a, b in zip(trace, trace[1:]))
+
+
+def test_tiny_fp32_forced_lock_schedule_and_peaked_posteriors():
+    cfg = inputs.model_shape("tiny")
+    # larger weights give peaked, moving posteriors: KL spreads on both sides of the threshold
+    trace, ctx, st = run_side_by_side(cfg, torch.float32, B=2, N=96, n_prompt=40, steps=24, kl_eps=1e-3, seed=2,
+                                      tol_logits=2e-4, std=0.08, forced_p=0.25, check_kl_free_running=True,
+                                      kl_floor=1e-8)
+    assert trace[-1] < trace[0]
+
+
+def test_tiny_bf16_step():
+    cfg = inputs.model_shape("tiny")
+    run_side_by_side(cfg, torch.bfloat16, B=2, N=128, n_prompt=64, steps=10, kl_eps=1e-3, seed=3, tol_logits=2e-2,
+                     std=0.05, forced_p=0.2)
+
+
+def test_bf16_head_dim_128_ragged_batch():
+    cfg = inputs.model_shape("tiny", d_model=512, n_heads=4, head_dim=128, d_ff=1536, vocab=4096, n_layers=3)
+    run_side_by_side(cfg, torch.bfloat16, B=3, N=200, n_prompt=90, steps=8, kl_eps=1e-3, seed=4, tol_logits=2e-2,
+                     std=0.04, forced_p=0.3)
+
+
+def test_locked_rows_cache_bytes_never_change_and_active_rows_are_rewritten():
+    cfg = inputs.model_shape("tiny")
+    w = inputs.make_weights(cfg, 5, dtype=torch.bfloat16, std=0.05)
+    B, N = 2, 128
+    ctx = SL.surelock_init(cfg, to_dev(w), N, B)
+    tokens, mask = inputs.make_tokens(B, N, 64, cfg["vocab"], 5)
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, 0.0)
+    snap = [[t.clone() for t in SL.surelock_kv_cache(ctx, l)] for l in range(cfg["n_layers"])]
+    lock2 = inputs.random_lock(B, N, [50, 3], 6).to(DEV)
+    tok2 = tokens.clone()
+    tok2[:, 64:80] = 7
+    SL.surelock_step(ctx, tok2.to(DEV), mask.to(DEV), lock2.clone(), 0.0)
+    torch.cuda.synchronize()
+    locked = lock2.reshape(-1).bool()
+    for l in range(cfg["n_layers"]):
+        k, v = SL.surelock_kv_cache(ctx, l)
+        for new, old in ((k, snap[l][0]), (v, snap[l][1])):
+            assert torch.equal(new[locked].view(torch.int16), old[locked].view(torch.int16))
+        changed = (k.view(torch.int16) != snap[l][0].view(torch.int16)).flatten(1).any(1)
+        assert not (changed & locked).any()
+        if l > 0:                                       # deeper layers see the new tokens through attention
+            assert (changed & ~locked).sum() >= (~locked).sum() // 2
+    assert SL.surelock_status_poll(ctx) == 0
+
+
+def test_step_is_deterministic_and_host_entry_point_matches():
+    cfg = inputs.model_shape("tiny")
+    w = to_dev(inputs.make_weights(cfg, 7, dtype=torch.bfloat16, std=0.05))
+    B, N = 2, 128
+    tokens, mask = inputs.make_tokens(B, N, 64, cfg["vocab"], 7)
+    results = []
+    for use_host in (False, False, True):
+        ctx = SL.surelock_init(cfg, w, N, B)
+        lock = torch.zeros((B, N), dtype=torch.uint8)
+        outs = []
+        for t in range(3):
+            if use_host:
+                tk, mk, lk = tokens.clone().pin_memory(), mask.clone().pin_memory(), lock.clone().pin_memory()
+                n = torch.zeros(1, dtype=torch.int32).pin_memory()
+                R = B * N
+                ai = torch.zeros(R, dtype=torch.int32).pin_memory()
+                kl, cf = torch.zeros(R).pin_memory(), torch.zeros(R).pin_memory()
+                am = torch.zeros(R, dtype=torch.int32).pin_memory()
+                SL.surelock_step_host(ctx, tk, mk, lk, 1e-3, n, ai, kl, cf, am)
+                M = int(n.item())
+                outs.append((M, ai[:M].clone(), kl[:M].clone(), cf[:M].clone(), am[:M].clone(), lk.clone()))
+                lock = lk.clone()
+            else:
+                ld = lock.to(DEV)
+                o = SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), ld, 1e-3)
+                M = o.M()
+                outs.append((M, o.active_idx[:M].cpu(), o.kl[:M].cpu(), o.conf[:M].cpu(), o.argmax[:M].cpu(), ld.cpu()))
+                lock = ld.cpu()
+        assert SL.surelock_status_poll(ctx) == 0
+        results.append(outs)
+    for a, b in ((results[0], results[1]), (results[0], results[2])):
+        for sa, sb in zip(a, b):
+            assert sa[0] == sb[0]
+            for x, y in zip(sa[1:], sb[1:]):
+                assert torch.equal(x, y)                # bitwise: same inputs, same outputs, device or host buffers
+
+
+def test_argument_errors_are_reported_not_fatal():
+    cfg = inputs.model_shape("tiny")
+    w = to_dev(inputs.make_weights(cfg, 8, dtype=torch.float32))
+    ctx = SL.surelock_init(cfg, w, 32, 1)
+    tokens, mask = inputs.make_tokens(1, 32, 16, cfg["vocab"], 8)
+    lock = torch.zeros((1, 32), dtype=torch.uint8, device=DEV)
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, float("nan"))
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, -1.0)
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_step(ctx, None, mask.to(DEV), lock, 1e-3)
+    bad = dict(cfg, head_dim=48, n_heads=4)
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_init(bad, w, 32, 1)
+    # an out-of-range token is skipped and reported through the status word; the context stays usable
+    tk = tokens.clone()
+    tk[0, 3] = cfg["vocab"] + 5
+    SL.surelock_step(ctx, tk.to(DEV), mask.to(DEV), lock, 1e-3)
+    assert SL.surelock_status_poll(ctx) == 4
+    SL.surelock_reset(ctx)
+    SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, 1e-3)
+    assert SL.surelock_status_poll(ctx) == 0
+
+
+@pytest.mark.parametrize("M_list", [[1024, 256, 32]])
+def test_single_layer_llada_shape(M_list):
+    """Single LLaDA-8B-shaped layer, N=1024: cache pre-filled by one full pass, then seeded random active subsets."""
+    cfg = inputs.model_shape("llada8b", n_layers=1, vocab=0)
+    oc = O.ModelCfg(**cfg)
+    N, d = 1024, cfg["d_model"]
+    lw = inputs.make_layer_weights(cfg, 0, 21, dtype=torch.bfloat16)
+    w = dict(layers=[lw])
+    wn = inputs.weights_to_numpy(w)["layers"][0]
+    ctx = SL.surelock_init(cfg, to_dev(w), N, 1)
+    H0 = inputs.hidden_states(N, d, 1)
+    H1 = inputs.hidden_states(N, d, 2)
+    out_buf = torch.zeros((N, d), dtype=torch.float32, device=DEV)
+    Kc = np.zeros((N, cfg["n_heads"], cfg["head_dim"]))
+    Vc = np.zeros_like(Kc)
+    for M in M_list:
+        if M == N:
+            lock = torch.zeros((1, N), dtype=torch.uint8)
+            Hin = H0
+        else:
+            lock = inputs.random_lock(1, N, [M], 100 + M)
+            Hin = H1
+        o = SL.surelock_layer_step(ctx, 0, Hin.to(DEV), lock.to(DEV), out_buf)
+        assert SL.surelock_status_poll(ctx) == 0
+        idx, _ = O.active_set(lock.numpy())
+        assert o.M() == M and np.array_equal(o.active_idx[:M].cpu().numpy(), idx)
+        # the oracle's cache holds the GPU's (bf16) cache before this pass: stage-wise, teacher-forced
+        kg, vg = SL.surelock_kv_cache(ctx, 0)
+        ref = O.layer_rows(oc, wn, f64(Hin[idx]), idx.astype(np.int64), Kc, Vc)
+        e = rel_err_rows(f64(out_buf[:M]), ref)
+        assert e < 2e-2, (M, e)
+        ek = rel_err_rows(f64(kg).reshape(N, -1), Kc.reshape(N, -1))
+        ev = rel_err_rows(f64(vg).reshape(N, -1), Vc.reshape(N, -1))
+        assert ek < 2e-2 and ev < 2e-2, (M, ek, ev)
+        Kc[:] = f64(kg)
+        Vc[:] = f64(vg)
