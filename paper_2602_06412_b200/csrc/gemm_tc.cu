@@ -1,6 +1,405 @@
+// Tensor-core GEMM for the packed active rows on sm_100a: C[r][n] = sum_k A[r][k] W[n][k], bf16 in, fp32 accumulate
+// (the Q/K/V, output, SwiGLU and LM-head contractions of Algorithm 1 lines 10, 12 and 15).
+//
+// Persistent, warp-specialised CTAs, one per SM:
+//   warp 0   TMA producer: cp.async.bulk.tensor loads of a 128x64 A tile and two 128x64 W tiles per stage into
+//            128-byte-swizzled shared memory, completion counted on an mbarrier (no multicast);
+//   warp 1   allocates tensor memory and issues tcgen05.mma (128 x BN x 16, cta_group::1) from one thread, operands
+//            described by shared-memory matrix descriptors; tcgen05.commit hands smem stages back to the producer
+//            and finished accumulators to the epilogue;
+//   warps 2-5 epilogue: tcgen05.ld the fp32 accumulator (one row per thread), apply the fused operation
+//            (store bf16 | add into the fp32 residual stream | silu(gate)*up) and write with 128-bit stores.
+// Two accumulators live in tensor memory so the epilogue of tile i overlaps the main loop of tile i+1.
+// The number of rows M is read from device memory: tiles whose first row is >= M are never scheduled, TMA zero-fills
+// rows beyond the allocation, and the epilogue stores only rows < M.  Every mbarrier wait is bounded: when it runs out
+// the CTA records SL_DEV_GEMM_TIMEOUT, all roles leave their loops, tensor memory is freed and the kernel returns.
+#include <cuda.h>
+
+#include <mutex>
+#include <unordered_map>
+
 #include "common.cuh"
+
 namespace sl {
-int launch_gemm_tc(const void*, const void*, const void*, void*, const int32_t*, int, int, int, int, int32_t*, cudaStream_t) {
-  return SL_EUNSUPPORTED;
+
+constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+constexpr unsigned long long TC_WAIT_CYCLES = 4000000000ull;   // ~2 s at 2 GHz
+
+// ----------------------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the wait ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = clock64();
+  unsigned spins = 0;
+  while (!mbar_try(bar, parity)) {
+    if ((++spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > TC_WAIT_CYCLES) {
+        *abort_flag = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile in shared memory, rows of 128 bytes (64 bf16), 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  return (uint64_t)((addr >> 4) & 0x3fffu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// bf16 x bf16 -> fp32, A and B K-major, M = 128, N = n
+__host__ __device__ constexpr uint32_t idesc_bf16(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// ----------------------------------------------------------------------------------------------- kernel
+template <int EPI, int BN, int STAGES>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmB1, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
+               int n_out, int K, int32_t* status) {
+  constexpr int A_BYTES = TC_BM * TC_BK * 2;              // 16 KB
+  constexpr int B_BYTES = BN * TC_BK * 2;                 // 32 KB (two 128-row halves)
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int OUT_BN = EPI == EPI_SWIGLU ? BN / 2 : BN; // output columns per tile
+  constexpr uint32_t TMEM_COLS = 2 * BN;                  // two accumulators
+  static_assert(TMEM_COLS == 512 || TMEM_COLS == 256, "tensor memory allocation must be a power of two");
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  // bars: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar(a), 1);
+      mbar_init(acce_bar(a), 4);
+    }
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int M = *n_active;
+  const int m_tiles = (M + TC_BM - 1) / TC_BM;
+  const int n_tiles = (n_out + OUT_BN - 1) / OUT_BN;
+  const int total = m_tiles * n_tiles;
+  const int num_kb = (K + TC_BK - 1) / TC_BK;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * OUT_BN;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
+          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(stage));
+          if (EPI == EPI_SWIGLU) {
+            tma_load_2d(sb, &tmB0, kb * TC_BK, n0, full_bar(stage));
+            tma_load_2d(sb + B_BYTES / 2, &tmB1, kb * TC_BK, n0, full_bar(stage));
+          } else {
+#pragma unroll
+            for (int hb = 0; hb < BN / 128; ++hb)
+              tma_load_2d(sb + hb * (B_BYTES / (BN / 128)), &tmB0, kb * TC_BK, n0 + hb * 128, full_bar(stage));
+          }
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc = idesc_bf16(BN);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t use = (uint32_t)(it >> 1);
+        if (!(ok = mbar_wait(acce_bar(acc), (use & 1) ^ 1, s_abort))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, s_abort))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
+          const uint64_t adesc = smem_desc_sw128(sa), bdesc = smem_desc_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)   // 16 bf16 = 32 bytes along K inside the 128-byte swizzle row
+            tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+          tc_commit(empty_bar(stage));
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) tc_commit(accf_bar(acc));
+      }
+    }
+  } else {
+    const int quarter = warp & 3;             // tensor-memory lanes 32*quarter .. 32*quarter+31
+    bool ok = true;
+    int it = 0;
+    for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+      const int acc = it & 1;
+      const uint32_t use = (uint32_t)(it >> 1);
+      const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * OUT_BN;
+      ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+      for (int c0 = 0; c0 < OUT_BN; c0 += 32) {
+        uint32_t v[32];
+        tc_ld32(taddr + c0, v);
+        if (EPI == EPI_SWIGLU) {
+          uint32_t u[32];
+          tc_ld32(taddr + OUT_BN + c0, u);
+          tc_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const float g = __uint_as_float(v[j]);
+            v[j] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
+          }
+        } else {
+          tc_wait_ld();
+        }
+        const int col = n0 + c0;
+        if (row < M && col < n_out) {
+          if (EPI == EPI_RESIDUAL) {
+            float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
+            if (col + 32 <= n_out) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                float4 o = *reinterpret_cast<float4*>(dst + j);
+                o.x += __uint_as_float(v[j]); o.y += __uint_as_float(v[j + 1]);
+                o.z += __uint_as_float(v[j + 2]); o.w += __uint_as_float(v[j + 3]);
+                *reinterpret_cast<float4*>(dst + j) = o;
+              }
+            } else {
+              for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] += __uint_as_float(v[j]);
+            }
+          } else {
+            bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
+            if (col + 32 <= n_out) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 o;
+                o.x = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
+                o.y = pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                o.z = pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
+                o.w = pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
+                *reinterpret_cast<uint4*>(dst + j) = o;
+              }
+            } else {
+              for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce_bar(acc));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_GEMM_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+// ----------------------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+struct MapKey {
+  const void* ptr;
+  long long rows, cols;
+  int box_rows;
+  bool operator==(const MapKey& o) const { return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    return std::hash<const void*>()(k.ptr) ^ (std::hash<long long>()(k.rows) * 31) ^ (std::hash<long long>()(k.cols) * 131) ^
+           (size_t)k.box_rows;
+  }
+};
+
+// 2-D bf16 row-major [rows][cols] tensor, box = box_rows x 64 elements, 128-byte swizzle, zero fill out of bounds
+static int get_map(const void* ptr, long long rows, long long cols, int box_rows, CUtensorMap* out) {
+  static std::mutex mu;
+  static std::unordered_map<MapKey, CUtensorMap, MapKeyHash> cache;
+  const MapKey key{ptr, rows, cols, box_rows};
+  std::lock_guard<std::mutex> g(mu);
+  auto it = cache.find(key);
+  if (it != cache.end()) {
+    *out = it->second;
+    return SL_OK;
+  }
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return SL_ECUDA;
+  CUtensorMap m;
+  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)TC_BK, (cuuint32_t)box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return SL_ECUDA;
+  if (cache.size() > 4096) cache.clear();
+  cache.emplace(key, m);
+  *out = m;
+  return SL_OK;
+}
+
+template <int EPI, int BN, int STAGES>
+static int launch_cfg(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, void* C, const int32_t* n_active,
+                      int max_rows, int n_out, int K, int32_t* status, cudaStream_t st) {
+  constexpr int SMEM = STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024 + 256;
+  static bool attr_set = false;
+  if (!attr_set) {
+    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+    attr_set = true;
+  }
+  constexpr int OUT_BN = EPI == EPI_SWIGLU ? BN / 2 : BN;
+  const long long tiles = (long long)((max_rows + TC_BM - 1) / TC_BM) * ((n_out + OUT_BN - 1) / OUT_BN);
+  int grid = sm_count();
+  if (tiles < grid) grid = (int)tiles;
+  if (grid < 1) grid = 1;
+  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b0, b1, C, n_active, n_out, K, status);
+  SL_CUDA_TRY(cudaGetLastError());
+  return SL_OK;
+}
+
+int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
+                   int n_out, int K, int epilogue, int32_t* status, cudaStream_t st) {
+  // TMA needs 16-byte aligned bases and row strides; the epilogue's 128-bit stores need n_out % 8 == 0
+  if (K % 8 || n_out % 8 || max_rows < 1) return SL_EUNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(W2) |
+       reinterpret_cast<uintptr_t>(C)) & 15)
+    return SL_EUNSUPPORTED;
+  if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
+  CUtensorMap a, b0, b1;
+  {
+    int rc = get_map(A, max_rows, K, TC_BM, &a);
+    if (rc != SL_OK) return rc;
+    rc = get_map(W, n_out, K, 128, &b0);
+    if (rc != SL_OK) return rc;
+    b1 = b0;
+    if (W2) {
+      rc = get_map(W2, n_out, K, 128, &b1);
+      if (rc != SL_OK) return rc;
+    }
+  }
+  switch (epilogue) {
+    case EPI_STORE: return launch_cfg<EPI_STORE, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
+    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
+    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
+    default: return SL_EINVAL;
+  }
+}
+
 }  // namespace sl

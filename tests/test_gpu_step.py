@@ -36,13 +36,13 @@ def test_tiny_fp32_forced_lock_schedule_and_peaked_posteriors():
 
 def test_tiny_bf16_step():
     cfg = inputs.model_shape("tiny")
-    run_side_by_side(cfg, torch.bfloat16, B=2, N=128, n_prompt=64, steps=10, kl_eps=1e-3, seed=3, tol_logits=2e-2,
+    run_side_by_side(cfg, torch.bfloat16, B=2, N=128, n_prompt=64, steps=10, kl_eps=1e-3, seed=3, tol_logits=5e-2,
                      std=0.05, forced_p=0.2)
 
 
 def test_bf16_head_dim_128_ragged_batch():
     cfg = inputs.model_shape("tiny", d_model=512, n_heads=4, head_dim=128, d_ff=1536, vocab=4096, n_layers=3)
-    run_side_by_side(cfg, torch.bfloat16, B=3, N=200, n_prompt=90, steps=8, kl_eps=1e-3, seed=4, tol_logits=2e-2,
+    run_side_by_side(cfg, torch.bfloat16, B=3, N=200, n_prompt=90, steps=8, kl_eps=1e-3, seed=4, tol_logits=5e-2,
                      std=0.04, forced_p=0.3)
 
 
