@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the SureLock locked-forward step on B200.
+
+One "step" = one pass of the whole hot path (compaction, embedding gather, L transformer blocks on the active
+rows with K/V scatter and M x N attention, LM head, fused softmax-KL-lock) over one batch of synthetic
+LLaDA-8B-shaped input.  Prints ONE JSON line (rank 0).  `value` is active tokens/s = packed active rows M
+processed per second, inputs resident in HBM; `e2e` is the same through the host-buffer entry point with the
+host<->device copies inside the timed region.  `sweep` repeats the measurement over M/N.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c3|c5|tiny] [--ratio 0.5]
+                    [--ratios 1,0.5,0.25,0.125,0.05] [--impl ours|reference]
+
+With --impl reference the CPU oracle is timed on the host cores on a bounded sample of the same workload.
+For N > 1 (torchrun) every rank runs an independent replica of the workload (the path shards by sequence with
+no exchange step): weak scaling, no collective on the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_06412_b200 import inputs  # noqa: E402
+
+WORKLOADS = {
+    # name: (model shape, batch, N, prompt length, lock pattern)
+    "c3": ("llada8b", 1, 512, 256, "random"),
+    "c4": ("llada8b", 8, 1536, 512, "random"),
+    "c5": ("llada8b", 4, 4096, 3584, "contiguous_plus_random"),
+    "tiny": ("tiny", 1, 128, 64, "random"),
+}
+FALLBACK_PEAKS = dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def n_active_per_seq(B, N, ratio, seed):
+    """Ragged per-sequence active counts around ratio*N (+-30 %, seeded); all N when ratio == 1."""
+    if ratio >= 1.0:
+        return [N] * B
+    g = torch.Generator().manual_seed(seed)
+    u = torch.rand(B, generator=g) * 2 - 1
+    return [int(min(N, max(1, round(N * ratio * (1 + 0.3 * float(x)))))) for x in u]
+
+
+def gemm_flops_per_row(cfg):
+    d, F, V, L = cfg["d_model"], cfg["d_ff"], cfg["vocab"], cfg["n_layers"]
+    hd = cfg["n_heads"] * cfg["head_dim"]
+    return L * (2 * d * 3 * hd + 2 * hd * d + 2 * d * 2 * F + 2 * F * d) + 2 * d * V
+
+
+def weight_bytes(cfg, esz=2):
+    d, F, V, L = cfg["d_model"], cfg["d_ff"], cfg["vocab"], cfg["n_layers"]
+    hd = cfg["n_heads"] * cfg["head_dim"]
+    return esz * (L * (3 * hd * d + hd * d + 3 * d * F) + d * V)
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.th.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], 0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = max(mx, float(r[1]))
+                for n, v in zip(names, r[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=mx or None, reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+# ----------------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(cfg, B, N, rows=128, head_rows=32):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: ONE of the L blocks on `rows`
+    active rows of one sequence against an N-row cache, plus final norm + LM head + softmax/KL/lock test on
+    `head_rows` rows; the block time is scaled by L.  Returns (tokens_per_s, seconds, threads, description)."""
+    from oracle import surelock_oracle as O
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        threads = os.cpu_count() or 1
+    oc = O.ModelCfg(**cfg)
+    lw = {k: v.float().numpy() for k, v in inputs.make_layer_weights(cfg, 0, 1).items()}
+    g = np.random.default_rng(0)
+    d, H, dh, V = cfg["d_model"], cfg["n_heads"], cfg["head_dim"], cfg["vocab"]
+    x = g.standard_normal((rows, d))
+    pos = np.sort(g.choice(N, size=rows, replace=False))
+    Kc, Vc = g.standard_normal((N, H, dh)), g.standard_normal((N, H, dh))
+    t0 = time.perf_counter()
+    O.layer_rows(oc, lw, x, pos, Kc, Vc)
+    t_layer = time.perf_counter() - t0
+    head = inputs._normal((V, d), 0.02, 3, torch.bfloat16, "cpu").float().numpy()
+    xh = g.standard_normal((head_rows, d))
+    zprev = g.standard_normal((head_rows, V)) * 3
+    t0 = time.perf_counter()
+    z = O.rmsnorm(xh, np.ones(d), cfg["rms_eps"]) @ np.asarray(head, np.float64).T
+    O.posterior_stats(z)
+    O.sure_test(O.kl_from_logits(z, zprev), np.zeros(head_rows), 1e-3)
+    t_head = time.perf_counter() - t0
+    per_row = cfg["n_layers"] * t_layer / rows + t_head / head_rows
+    desc = (f"1 of {cfg['n_layers']} blocks on {rows} active rows of one N={N} sequence (x{cfg['n_layers']}) + LM head/"
+            f"softmax-KL on {head_rows} rows; extrapolated per row")
+    return 1.0 / per_row, t_layer + t_head, threads, desc
+
+
+def run_reference(args, cfgname, B, N):
+    cfg = inputs.model_shape(cfgname)
+    vals, secs = [], 0.0
+    for _ in range(max(1, min(args.steps, 3))):
+        v, s, threads, desc = oracle_sample(cfg, B, N, rows=64, head_rows=16)
+        vals.append(v); secs += s
+    v = float(np.median(vals))
+    return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
+            "steps": len(vals), "warmup": 0, "ms_per_step": 1e3 * secs / len(vals), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "batch": B, "seq_len": N, "note": "CPU oracle, bounded sample per step"},
+            "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+            "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+# ----------------------------------------------------------------------------------------------------- GPU leg
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
+    ap.add_argument("--ratio", type=float, default=0.5, help="active fraction M/N of the headline measurement")
+    ap.add_argument("--ratios", default="1,0.5,0.25,0.125,0.05", help="M/N sweep ('' = none)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    cfgname, B, N, n_prompt, pattern = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args, cfgname, B, N)), flush=True)
+        return 0
+
+    from paper_2602_06412_b200 import binding as SL
+    SL.lib()                                       # fail loudly if the CUDA library is missing
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    args.warmup = max(args.warmup, 3)
+    cfg = inputs.model_shape(cfgname)
+    dtype = torch.bfloat16 if cfgname != "tiny" else torch.float32
+    seed = 1234 + rank
+    w = inputs.make_weights(cfg, seed, dtype=dtype, device=dev)
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], seed)
+    tokens_d, mask_d = tokens.to(dev), mask.to(dev)
+    R = B * N
+    lock_d = torch.zeros((B, N), dtype=torch.uint8, device=dev)
+
+    def lock_pattern(ratio):
+        na = n_active_per_seq(B, N, ratio, seed * 31 + int(ratio * 1000))
+        f = inputs.contiguous_plus_random_lock if pattern == "contiguous_plus_random" else inputs.random_lock
+        return f(B, N, na, seed), sum(na)
+
+    # pre-fill: one full step (nothing locked) writes every cache row and the first "previous" logits
+    SL.surelock_step(ctx, tokens_d, mask_d, lock_d, 1e-3)
+    torch.cuda.synchronize()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    def timed(ratio, steps, warmup, sampler=None):
+        lock0, M = lock_pattern(ratio)
+        lock0 = lock0.to(dev)
+        for _ in range(warmup):
+            lock_d.copy_(lock0)
+            out = SL.surelock_step(ctx, tokens_d, mask_d, lock_d, 1e-3)
+        barrier()
+        assert out.M() == M, (out.M(), M)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = 0
+        if sampler:
+            sampler.__enter__()
+        e0.record()
+        for _ in range(steps):
+            lock_d.copy_(lock0)                    # the sure test locks converged rows; restore so M stays fixed
+            SL.surelock_step(ctx, tokens_d, mask_d, lock_d, 1e-3)
+            launches += SL.surelock_last_launch_count(ctx)
+        e1.record()
+        barrier()
+        if sampler:
+            sampler.__exit__()
+        ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], device=dev)
+            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+            ms = float(t.item())
+        return M, ms, launches, lock0
+
+    pk, pk_kind = peaks()
+    sampler = ClockSampler(local)
+    M, ms, launches, lock0 = timed(args.ratio, args.steps, args.warmup, sampler)
+    clocks = sampler.summary()
+    value = world * M / (ms * 1e-3)
+
+    # per-kernel-class breakdown of the same step (separate pass: events around every launch)
+    SL.surelock_set_option(ctx, "time_kernels", 1)
+    acc = {}
+    for _ in range(2):
+        lock_d.copy_(lock0)
+        SL.surelock_step(ctx, tokens_d, mask_d, lock_d, 1e-3)
+        for k, (t, n) in SL.surelock_kernel_times(ctx).items():
+            a = acc.setdefault(k, [0.0, 0])
+            a[0] += t / 2; a[1] = n
+    SL.surelock_set_option(ctx, "time_kernels", 0)
+    gemm_ms = sum(acc[k][0] for k in acc if k.startswith("gemm"))
+    gemm_launch = sum(acc[k][1] for k in acc if k.startswith("gemm"))
+    flops = M * gemm_flops_per_row(cfg)
+    wbytes = weight_bytes(cfg)
+    ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
+    if M >= ridge:
+        ach = flops / (gemm_ms * 1e-3) / 1e12
+        roof = dict(kernel="gemm_tc (all GEMM launches of the step)", bound="tensor", achieved=ach,
+                    peak=pk["bf16_tflops_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_tflops_sustained"],
+                    traffic=None, peak_kind=f"{pk_kind}, sustained", launches_per_step=gemm_launch,
+                    avg_launch_ms=gemm_ms / max(gemm_launch, 1))
+    else:
+        ach = wbytes / (gemm_ms * 1e-3) / 1e9
+        roof = dict(kernel="gemm_tc (all GEMM launches of the step, weight streaming)", bound="hbm", achieved=ach,
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=None, peak_kind=pk_kind,
+                    launches_per_step=gemm_launch, avg_launch_ms=gemm_ms / max(gemm_launch, 1))
+    total_k = sum(v[0] for v in acc.values())
+    kernels = {k: dict(ms=round(v[0], 4), launches=v[1], share=round(v[0] / total_k, 4)) for k, v in acc.items()}
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    tk, mk = tokens.pin_memory(), mask.pin_memory()
+    lk0 = lock0.cpu()
+    lk = lk0.clone().pin_memory()
+    n_h = torch.zeros(1, dtype=torch.int32).pin_memory()
+    ai = torch.zeros(R, dtype=torch.int32).pin_memory()
+    klh, cfh = torch.zeros(R).pin_memory(), torch.zeros(R).pin_memory()
+    amh = torch.zeros(R, dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        lk.copy_(lk0)
+        SL.surelock_step_host(ctx, tk, mk, lk, 1e-3, n_h, ai, klh, cfh, amh)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        lk.copy_(lk0)
+        SL.surelock_step_host(ctx, tk, mk, lk, 1e-3, n_h, ai, klh, cfh, amh)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = dict(value=world * int(n_h.item()) / (e2e_ms * 1e-3), unit="tokens/s", ms_per_step=e2e_ms,
+               h2d_bytes_per_step=R * 4 + R + R, d2h_bytes_per_step=R + 4 + 4 * R * 4)
+
+    sweep = []
+    if args.ratios:
+        for r in [float(x) for x in args.ratios.split(",") if x]:
+            Ms, mss, _, _ = timed(r, max(2, args.steps // 2), 3)
+            ideal_ms = max(Ms * gemm_flops_per_row(cfg) / (pk["bf16_tflops_sustained"] * 1e12),
+                           wbytes / (pk["hbm_gbs"] * 1e9)) * 1e3
+            sweep.append(dict(ratio=r, M=Ms, ms_per_step=round(mss, 4), tokens_per_s=round(world * Ms / (mss * 1e-3), 1),
+                              gemm_ideal_ms=round(ideal_ms, 4), frac_of_gemm_ideal=round(ideal_ms / mss, 4)))
+
+    status = SL.surelock_status_poll(ctx)
+    line = {
+        "metric": "active_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if dtype == torch.bfloat16 else "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: full {cfgname} stack ({cfg['n_layers']} layers, d={cfg['d_model']}, "
+                               f"vocab={cfg['vocab']}), batch {B}, N={N}, M/N={args.ratio} ragged per sequence (M={M}), "
+                               f"{pattern} lock pattern", "batch": B, "seq_len": N, "active_rows": M,
+                   "l2": "inputs larger than L2 (every step streams all weights, %.1f GB)" % (wbytes / 1e9),
+                   "multi_gpu": "replicas only (one independent batch per rank, no collective)"},
+        "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "roofline": roof, "kernels": kernels, "sweep": sweep,
+        "device_status": status,
+    }
+    if rank == 0 and not args.no_cpu_baseline:
+        v, secs, threads, desc = oracle_sample(cfg, B, N)
+        line["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc,
+                                "seconds": round(secs, 2)}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

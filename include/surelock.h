@@ -135,12 +135,21 @@ int surelock_kv_cache(surelock_ctx *ctx, int layer, void **k, void **v, size_t *
 int surelock_prev_logits(surelock_ctx *ctx, void **buf, int32_t **row_of_pos);
 
 /* Tuning / test switches.  "gemm_impl": 0 = tensor-core GEMM and attention when the shape allows (default),
- * 1 = force the CUDA-core kernels.  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
+ * 1 = force the CUDA-core kernels.  "time_kernels": 1 creates an event pool (once) and brackets every launch of
+ * later steps with CUDA events for surelock_kernel_times().  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
  * (after a caller seeded them), 0 forgets them.  Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
 /* Number of kernels the last surelock_step / surelock_layer_step call launched (host-side count). */
 int surelock_last_launch_count(surelock_ctx *ctx);
+
+/* Per-kernel-class device time of the LAST step, measured with CUDA events on the ctx stream; needs
+ * surelock_set_option(ctx, "time_kernels", 1) before that step (events add a few microseconds per launch, so time
+ * whole steps with the option off).  Synchronises the stream.  ms[i], launches[i] (may be NULL) for class i:
+ * 0 compaction, 1 embedding/row gather, 2 RMSNorm, 3 QKV GEMM, 4 RoPE, 5 K/V scatter, 6 attention, 7 O-proj GEMM,
+ * 8 gate/up GEMM + SwiGLU, 9 down GEMM, 10 LM-head GEMM, 11 softmax-KL-lock.  n_classes >= 12. */
+#define SURELOCK_KERNEL_CLASSES 12
+int surelock_kernel_times(surelock_ctx *ctx, float *ms, int32_t *launches, int n_classes);
 
 void surelock_destroy(surelock_ctx *ctx);
 const char *surelock_strerror(int status);

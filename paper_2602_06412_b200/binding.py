@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         "surelock_prev_logits": (i32, [vp, C.POINTER(vp), C.POINTER(vp)]),
         "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
         "surelock_last_launch_count": (i32, [vp]),
+        "surelock_kernel_times": (i32, [vp, vp, vp, i32]),
         "surelock_destroy": (None, [vp]),
         "surelock_strerror": (C.c_char_p, [i32]),
         "surelock_compact_scratch_bytes": (sz, [C.c_int64]),
@@ -220,6 +221,20 @@ def surelock_set_option(ctx: Ctx, name: str, value: int):
 
 def surelock_last_launch_count(ctx: Ctx) -> int:
     return lib().surelock_last_launch_count(ctx.handle)
+
+
+KERNEL_CLASSES = ("compact", "gather", "rmsnorm", "gemm_qkv", "rope", "kv_scatter", "attention", "gemm_o",
+                  "gemm_gateup", "gemm_down", "gemm_head", "softmax_kl")
+
+
+def surelock_kernel_times(ctx: Ctx):
+    """{class: (ms, launches)} of the last step (needs surelock_set_option(ctx, "time_kernels", 1))."""
+    n = len(KERNEL_CLASSES)
+    ms = (C.c_float * n)()
+    cnt = (C.c_int32 * n)()
+    _check(lib().surelock_kernel_times(ctx.handle, C.cast(ms, C.c_void_p), C.cast(cnt, C.c_void_p), n),
+           "surelock_kernel_times")
+    return {k: (ms[i], cnt[i]) for i, k in enumerate(KERNEL_CLASSES)}
 
 
 # ---- single stages -----------------------------------------------------------------------------------------

@@ -35,6 +35,10 @@ struct surelock_ctx {
   bool have_prev = false;
   int launches = 0;
   int gemm_impl = 0;                  // 0 = tensor cores when possible, 1 = CUDA cores
+  bool timing = false;                // per-kernel-class CUDA-event timing (off by default)
+  std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
+  std::vector<int> ev_cls;            // class of the launch bracketed by events 2i, 2i+1
+  int n_ev = 0;
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
   void* kcache(int l) const { return kv + (size_t)(2 * l) * kv_layer_bytes(); }
@@ -60,13 +64,36 @@ static int dev_alloc(surelock_ctx* c, P** p, size_t bytes) {
   return SL_OK;
 }
 
+// Kernel classes for the timing breakdown (order is part of the C ABI: surelock_kernel_times)
+enum { K_COMPACT = 0, K_GATHER, K_RMSNORM, K_GEMM_QKV, K_ROPE, K_SCATTER, K_ATTN, K_GEMM_O, K_GEMM_GATEUP, K_GEMM_DOWN,
+       K_GEMM_HEAD, K_SOFTMAX_KL, K_NUM };
+
+static inline void tick(surelock_ctx* c, int cls) {
+  if (c->timing && c->n_ev + 2 <= (int)c->ev.size()) {
+    c->ev_cls[c->n_ev / 2] = cls;
+    cudaEventRecord(c->ev[c->n_ev], c->st);
+  }
+}
+static inline void tock(surelock_ctx* c) {
+  if (c->timing && c->n_ev + 2 <= (int)c->ev.size()) {
+    cudaEventRecord(c->ev[c->n_ev + 1], c->st);
+    c->n_ev += 2;
+  }
+  ++c->launches;
+}
+#define SL_K(cls, expr) \
+  do {                  \
+    tick(c, cls);       \
+    SL_TRY(expr);       \
+    tock(c);            \
+  } while (0)
+
 namespace sl {
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
                    int n_out, int K, int epilogue, int32_t* status, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
 }
 
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
-  ++c->launches;
   if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->st);
     if (rc != SL_EUNSUPPORTED) return rc;
@@ -78,21 +105,18 @@ static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, v
 static int run_layer(surelock_ctx* c, int l, float* x) {
   const surelock_model_cfg& g = c->cfg;
   const int d = g.d_model, hd = g.n_heads * g.head_dim;
-  SL_TRY(launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
-  ++c->launches;
-  SL_TRY(gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
-  SL_TRY(gemm(c, c->h, c->wk[l], nullptr, c->k, hd, d, EPI_STORE));
-  SL_TRY(gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
-  SL_TRY(launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
-  SL_TRY(launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
-  SL_TRY(launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads,
-                               g.head_dim, c->attn, g.dtype, c->st));
-  c->launches += 3;
-  SL_TRY(gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
-  SL_TRY(launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
-  ++c->launches;
-  SL_TRY(gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
-  SL_TRY(gemm(c, c->act, c->w_down[l], nullptr, x, d, g.d_ff, EPI_RESIDUAL));
+  SL_K(K_RMSNORM, launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
+  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
+  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wk[l], nullptr, c->k, hd, d, EPI_STORE));
+  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
+  SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
+  SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
+  SL_K(K_ATTN, launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads,
+                                     g.head_dim, c->attn, g.dtype, c->st));
+  SL_K(K_GEMM_O, gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
+  SL_K(K_RMSNORM, launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
+  SL_K(K_GEMM_GATEUP, gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
+  SL_K(K_GEMM_DOWN, gemm(c, c->act, c->w_down[l], nullptr, x, d, g.d_ff, EPI_RESIDUAL));
   return SL_OK;
 }
 
@@ -200,19 +224,17 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   const surelock_model_cfg& g = c->cfg;
   c->launches = 0;
   const int cur = c->cur, prv = cur ^ 1;
-  SL_TRY(launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur], c->scratch,
-                        c->status, c->st));
-  SL_TRY(launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype,
-                            c->status, c->st));
-  c->launches += 2;
+  c->n_ev = 0;
+  SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur],
+                                 c->scratch, c->status, c->st));
+  SL_K(K_GATHER, launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype,
+                                    c->status, c->st));
   for (int l = 0; l < g.n_layers; ++l) SL_TRY(run_layer(c, l, c->x));
-  SL_TRY(launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
-  ++c->launches;
-  SL_TRY(gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
-  SL_TRY(launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
-                                c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state, lock_mask,
-                                kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st));
-  ++c->launches;
+  SL_K(K_RMSNORM, launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
+  SL_K(K_GEMM_HEAD, gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
+  SL_K(K_SOFTMAX_KL, launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
+                                            c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state,
+                                            lock_mask, kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st));
   if (out) {
     out->active_idx = c->idx;
     out->row_offsets = c->row_offsets;
@@ -252,11 +274,11 @@ int surelock_layer_step(surelock_ctx* c, int layer, const void* hidden_in, const
   if (layer < 0 || layer >= c->cfg.n_layers) return SL_EINVAL;
   const surelock_model_cfg& g = c->cfg;
   c->launches = 0;
-  SL_TRY(launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, nullptr, c->scratch, c->status,
-                        c->st));
-  SL_TRY(launch_gather_rows(hidden_in, nullptr, c->idx, c->n_active, c->R, g.d_model, c->R, hidden_out, g.dtype,
-                            c->status, c->st));
-  c->launches += 2;
+  c->n_ev = 0;
+  SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, nullptr, c->scratch,
+                                 c->status, c->st));
+  SL_K(K_GATHER, launch_gather_rows(hidden_in, nullptr, c->idx, c->n_active, c->R, g.d_model, c->R, hidden_out, g.dtype,
+                                    c->status, c->st));
   SL_TRY(run_layer(c, layer, hidden_out));
   if (out) {
     memset(out, 0, sizeof(*out));
@@ -298,14 +320,44 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
+  if (!strcmp(name, "time_kernels")) {
+    if (value && c->ev.empty()) {
+      const int n = 2 * (16 * c->cfg.n_layers + 16);
+      c->ev.resize(n);
+      c->ev_cls.assign(n / 2, 0);
+      for (int i = 0; i < n; ++i)
+        if (cudaEventCreate(&c->ev[i]) != cudaSuccess) return SL_ECUDA;
+    }
+    c->timing = value != 0;
+    c->n_ev = 0;
+    return SL_OK;
+  }
   return SL_EINVAL;
 }
 
 int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
 
+int surelock_kernel_times(surelock_ctx* c, float* ms, int32_t* launches, int n_classes) {
+  if (!c || !ms || n_classes < K_NUM) return SL_EINVAL;
+  for (int i = 0; i < n_classes; ++i) {
+    ms[i] = 0.f;
+    if (launches) launches[i] = 0;
+  }
+  if (!c->timing) return SL_OK;
+  SL_CUDA_TRY(cudaStreamSynchronize(c->st));
+  for (int i = 0; i + 1 < c->n_ev; i += 2) {
+    float t = 0.f;
+    SL_CUDA_TRY(cudaEventElapsedTime(&t, c->ev[i], c->ev[i + 1]));
+    ms[c->ev_cls[i / 2]] += t;
+    if (launches) ++launches[c->ev_cls[i / 2]];
+  }
+  return SL_OK;
+}
+
 void surelock_destroy(surelock_ctx* c) {
   if (!c) return;
   cudaStreamSynchronize(c->st);
+  for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
   for (void* p : c->allocs) cudaFree(p);
   delete c;
 }
