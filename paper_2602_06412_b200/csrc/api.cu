@@ -91,6 +91,19 @@ static inline void tock(surelock_ctx* c) {
 namespace sl {
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
                    int n_out, int K, int epilogue, int32_t* status, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
+int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                        int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
+}
+
+static int attention(surelock_ctx* c, int l) {
+  const surelock_model_cfg& g = c->cfg;
+  if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
+    const int rc = launch_attention_tc(c->q, c->kcache(l), c->vcache(l), c->row_offsets, c->R, c->B, c->N, g.n_heads,
+                                       g.head_dim, c->attn, c->status, c->st);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
+  return launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim,
+                               c->attn, g.dtype, c->st);
 }
 
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
@@ -111,8 +124,7 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   SL_K(K_GEMM_QKV, gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
   SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
   SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
-  SL_K(K_ATTN, launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads,
-                                     g.head_dim, c->attn, g.dtype, c->st));
+  SL_K(K_ATTN, attention(c, l));
   SL_K(K_GEMM_O, gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
   SL_K(K_GEMM_GATEUP, gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
@@ -419,7 +431,11 @@ int surelock_attention(const void* q, const void* k_cache, const void* v_cache, 
   if (!q || !k_cache || !v_cache || !active_idx || !n_active || !o || max_rows < 0 || B <= 0 || N <= 0 || H <= 0)
     return SL_EINVAL;
   if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
-  (void)row_offsets; (void)impl; (void)dev_status;
+  if (dtype == SL_BF16 && impl == 0 && row_offsets) {
+    const int rc = launch_attention_tc(q, k_cache, v_cache, row_offsets, max_rows, B, N, H, head_dim, o, dev_status,
+                                       (cudaStream_t)stream);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
   return launch_attention_simt(q, k_cache, v_cache, active_idx, n_active, max_rows, N, H, head_dim, o, dtype,
                                (cudaStream_t)stream);
 }

@@ -1,0 +1,338 @@
+// Tensor-core M x N attention on sm_100a (Algorithm 1 line 12; Sec. 2.1: the packed queries of the active rows
+// attend to ALL N cached keys/values of their sequence, bidirectional, no mask).
+//
+// Work item = (sequence b, head h, tile of up to 128 consecutive packed rows of that sequence); items never
+// straddle sequences.  Persistent CTAs take items round-robin; the q-tile index runs fastest so CTAs working at the
+// same time read the same K/V head through L2.  Per item the keys are streamed in blocks of 128:
+//   warp 0    TMA producer: Q tile once, then K and V blocks (two stages each), token-major cache rows, 128-byte swizzle;
+//   warp 1    one thread issues S = Q K^T (tcgen05.mma, 128x128xd_h, accumulator in tensor memory, two S buffers so
+//             S of block j+1 is computed while block j is in the softmax) and O += P V (V is the MN-major operand);
+//   warps 2-5 softmax: each thread owns one query row: tcgen05.ld its 128 scores, online max / sum in fp32 with the
+//             1/sqrt(d_h) scale folded into an exp2, P written as bf16 into swizzled shared memory for the second MMA.
+//             O stays in tensor memory; it is rescaled (tcgen05.ld / st) only when a row's running maximum grows by
+//             more than 2^8, so after the first blocks the correction is almost never taken.  The final O / l is
+//             stored as bf16.
+// Keys beyond N in the last block are masked to -inf.  All waits are bounded (SL_DEV_ATTN_TIMEOUT).
+#include "tc_common.cuh"
+
+namespace sl {
+
+constexpr int AT_THREADS = 192;
+constexpr int AT_BQ = 128, AT_BKV = 128;
+constexpr int AT_MAX_B = 1024;
+
+template <int DH>
+__global__ void __launch_bounds__(AT_THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
+                    bf16* __restrict__ o, float scale_log2, int32_t* status) {
+  constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
+  constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
+  constexpr int Q_BYTES = SLABS * SLAB_BYTES;
+  constexpr int KV_BYTES = SLABS * SLAB_BYTES;         // one K or V block of 128 keys
+  constexpr int P_BYTES = 2 * SLAB_BYTES;              // 128 queries x 128 keys, bf16
+  constexpr uint32_t TMEM_COLS = 512;                  // S0 [0,128) S1 [128,256) O [256,256+DH)
+  constexpr uint32_t O_COL = 256;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;
+  uint8_t* sK = sQ + Q_BYTES;                          // 2 stages
+  uint8_t* sV = sK + 2 * KV_BYTES;                     // 2 stages
+  uint8_t* sP = sV + 2 * KV_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
+  // q_full, q_free, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], s_free[2], p_full, p_free, o_free
+  enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
+         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, NUM_BARS };
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  int* s_prefix = reinterpret_cast<int*>(s_tmem + 2);   // [B+1] work-item prefix per sequence
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NUM_BARS; ++i) {
+      uint32_t cnt = 1;
+      if (i == S_FREE || i == S_FREE + 1 || i == O_FREE) cnt = 4;
+      if (i == P_FULL) cnt = 128;
+      mbar_init(bar(i), cnt);
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    int acc = 0;
+    s_prefix[0] = 0;
+    for (int b = 0; b < B; ++b) {
+      const int mb = row_offsets[b + 1] - row_offsets[b];
+      acc += ((mb + AT_BQ - 1) / AT_BQ) * H;
+      s_prefix[b + 1] = acc;
+    }
+  }
+  if (warp == 1) tc_alloc(smem_u32(s_tmem), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int total = s_prefix[B];
+  const int nblk = (N + AT_BKV - 1) / AT_BKV;
+
+  // item -> (b, h, first packed row, rows in tile)
+  auto decode = [&](int w, int& b, int& h, int& row0, int& nrows) {
+    int lo = 0, hi = B;                                 // largest b with prefix[b] <= w
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_prefix[mid] <= w) lo = mid; else hi = mid;
+    }
+    b = lo;
+    const int r0 = row_offsets[b], mb = row_offsets[b + 1] - r0;
+    const int tiles = (mb + AT_BQ - 1) / AT_BQ;
+    const int local = w - s_prefix[b];
+    h = local / tiles;
+    const int qt = local % tiles;
+    row0 = r0 + qt * AT_BQ;
+    nrows = mb - qt * AT_BQ < AT_BQ ? mb - qt * AT_BQ : AT_BQ;
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t kcnt = 0, qcnt = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++qcnt) {
+        int b, h, row0, nrows;
+        decode(w, b, h, row0, nrows);
+        if (!(ok = mbar_wait(bar(Q_FREE), (qcnt & 1) ^ 1, s_abort))) break;
+        mbar_expect_tx(bar(Q_FULL), Q_BYTES);
+#pragma unroll
+        for (int s = 0; s < SLABS; ++s) tma_load_2d(smem_u32(sQ + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0, bar(Q_FULL));
+        for (int j = 0; j < nblk; ++j, ++kcnt) {
+          const int st = kcnt & 1;
+          const uint32_t ph = (kcnt >> 1) & 1;
+          const int key0 = b * N + j * AT_BKV;
+          if (!(ok = mbar_wait(bar(K_FREE + st), ph ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
+#pragma unroll
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sK + st * KV_BYTES + s * SLAB_BYTES), &tmK, h * DH + 64 * s, key0, bar(K_FULL + st));
+          if (!(ok = mbar_wait(bar(V_FREE + st), ph ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(V_FULL + st), KV_BYTES);
+#pragma unroll
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sV + st * KV_BYTES + s * SLAB_BYTES), &tmV, h * DH + 64 * s, key0, bar(V_FULL + st));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_m128(AT_BKV, false);
+      constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
+      uint32_t g = 0, it = 0;
+      bool ok = true;
+      // S(gi) = Q K^T for global block gi into S buffer gi & 1
+      auto issue_s = [&](uint32_t gi) -> bool {
+        const int st = gi & 1;
+        const uint32_t ph = (gi >> 1) & 1;
+        if (!mbar_wait(bar(K_FULL + st), ph, s_abort)) return false;
+        if (!mbar_wait(bar(S_FREE + st), ph ^ 1, s_abort)) return false;
+        tc_fence_after();
+        const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * KV_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
+          tc_mma_bf16(tmem_base + st * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
+        }
+        tc_commit(bar(K_FREE + st));
+        tc_commit(bar(S_FULL + st));
+        return true;
+      };
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+        if (!(ok = mbar_wait(bar(Q_FULL), it & 1, s_abort))) break;
+        if (!(ok = issue_s(g))) break;
+        for (int j = 0; j < nblk && ok; ++j) {
+          const uint32_t gj = g + j;
+          if (j + 1 < nblk) {
+            if (!(ok = issue_s(gj + 1))) break;
+          } else {
+            tc_commit(bar(Q_FREE));                      // every S MMA of this item has been issued
+          }
+          const int st = gj & 1;
+          const uint32_t ph = (gj >> 1) & 1;
+          if (!(ok = mbar_wait(bar(P_FULL), gj & 1, s_abort))) break;
+          if (!(ok = mbar_wait(bar(V_FULL + st), ph, s_abort))) break;
+          if (j == 0 && !(ok = mbar_wait(bar(O_FREE), (it & 1) ^ 1, s_abort))) break;
+          tc_fence_after();
+          const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * KV_BYTES);
+#pragma unroll
+          for (int kk = 0; kk < AT_BKV / 16; ++kk) {
+            const uint64_t ad = smem_desc_k_sw128(pa + (kk >> 2) * SLAB_BYTES + (kk & 3) * 32);
+            const uint64_t bd = smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES);
+            tc_mma_bf16(tmem_base + O_COL, ad, bd, idesc_o, (j | kk) != 0);
+          }
+          tc_commit(bar(V_FREE + st));
+          tc_commit(bar(P_FREE));
+        }
+        g += nblk;
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    const int trow = quarter * 32 + lane;                // query row of this thread inside the tile
+    const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    uint32_t g = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+      int b, h, row0, nrows;
+      decode(w, b, h, row0, nrows);
+      float m_used = 0.f, l = 0.f;
+      for (int j = 0; j < nblk; ++j) {
+        const uint32_t gj = g + j;
+        const int sb = gj & 1;
+        const uint32_t ph = (gj >> 1) & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), ph, s_abort));
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tc_ld32(tmem_base + tlane + sb * 128 + c * 32, s + 32 * c);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(S_FREE + sb));
+        const int nvalid = N - j * AT_BKV;               // keys of this block that exist
+        float mx = -INFINITY;
+#pragma unroll
+        for (int c = 0; c < 128; ++c) {
+          float v = __uint_as_float(s[c]) * scale_log2;
+          if (c >= nvalid) v = -INFINITY;
+          s[c] = __float_as_uint(v);
+          mx = fmaxf(mx, v);
+        }
+        bool need = false;
+        float corr = 1.f;
+        if (j == 0) {
+          m_used = mx;
+        } else if (mx > m_used + 8.f) {
+          need = true;
+          corr = fast_exp2(m_used - mx);
+          m_used = mx;
+          l *= corr;
+        }
+        float sum = 0.f;
+        uint32_t pk[64];
+#pragma unroll
+        for (int c = 0; c < 128; c += 2) {
+          const float p0 = fast_exp2(__uint_as_float(s[c]) - m_used);
+          const float p1 = fast_exp2(__uint_as_float(s[c + 1]) - m_used);
+          sum += p0 + p1;
+          pk[c >> 1] = pack_bf16(p0, p1);
+        }
+        l += sum;
+        if (gj > 0) {
+          ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (gj - 1) & 1, s_abort));   // P V of the previous block done
+          if (!ok) break;
+        }
+        if (j > 0 && __any_sync(0xffffffffu, need)) {
+          tc_fence_after();
+#pragma unroll 1
+          for (int c = 0; c < DH; c += 32) {
+            uint32_t ov[32];
+            tc_ld32(tmem_base + tlane + O_COL + c, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * corr);
+            tc_st32(tmem_base + tlane + O_COL + c, ov);
+          }
+          tc_wait_st();
+        }
+        // P row -> shared memory, 128-byte swizzle: 16-byte chunk c of row r sits at chunk position c ^ (r & 7)
+        {
+          uint8_t* prow = sP + (trow >> 3) * 1024 + (trow & 7) * 128;
+#pragma unroll
+          for (int ch = 0; ch < 16; ++ch) {
+            const int slab = ch >> 3, c = ch & 7;
+            *reinterpret_cast<uint4*>(prow + slab * SLAB_BYTES + ((c ^ (trow & 7)) << 4)) =
+                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+          }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        mbar_arrive(bar(P_FULL));
+      }
+      if (!ok) break;
+      g += nblk;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (g - 1) & 1, s_abort));       // last P V of the item done
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = 1.f / l;
+      bf16* orow = o + ((long long)(row0 + trow) * H + h) * DH;
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 32) {
+        uint32_t ov[32];
+        tc_ld32(tmem_base + tlane + O_COL + c, ov);
+        tc_wait_ld();
+        if (trow < nrows) {
+#pragma unroll
+          for (int k = 0; k < 32; k += 8) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(ov[k]) * inv, __uint_as_float(ov[k + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(ov[k + 2]) * inv, __uint_as_float(ov[k + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(ov[k + 4]) * inv, __uint_as_float(ov[k + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(ov[k + 6]) * inv, __uint_as_float(ov[k + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c + k) = v;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(O_FREE));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_ATTN_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int DH>
+static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
+                     int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
+  constexpr int SLABS = DH / 64;
+  const int smem = 5 * SLABS * 128 * 128 + 2 * 128 * 128 + 1024 + 512 + 4 * (B + 2);
+  static int attr_smem = 0;
+  if (smem > attr_smem) {
+    SL_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_smem = smem;
+  }
+  long long items = (long long)H * ((max_rows + AT_BQ - 1) / AT_BQ + B);
+  int grid = sm_count();
+  if (items < grid) grid = (int)items;
+  if (grid < 1) grid = 1;
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+  attention_tc_kernel<DH><<<grid, AT_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status);
+  SL_CUDA_TRY(cudaGetLastError());
+  return SL_OK;
+}
+
+int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                        int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
+  if ((head_dim != 64 && head_dim != 128) || B > AT_MAX_B || max_rows < 1 || !row_offsets) return SL_EUNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |
+       reinterpret_cast<uintptr_t>(o)) & 15)
+    return SL_EUNSUPPORTED;
+  CUtensorMap tq, tk, tv;
+  const long long cols = (long long)H * head_dim;
+  int rc = get_tensor_map_2d(q, max_rows, cols, 128, &tq);
+  if (rc != SL_OK) return rc;
+  rc = get_tensor_map_2d(kc, (long long)B * N, cols, 128, &tk);
+  if (rc != SL_OK) return rc;
+  rc = get_tensor_map_2d(vc, (long long)B * N, cols, 128, &tv);
+  if (rc != SL_OK) return rc;
+  return head_dim == 128 ? launch_dh<128>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st)
+                         : launch_dh<64>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st);
+}
+
+}  // namespace sl

@@ -244,3 +244,33 @@ def test_attention_cuda_cores(dtype, tol, B, N, H, dh, n_act):
             continue
         ref = O.attention_rows(f64(q[r0:r1]), f64(Kc[b * N:(b + 1) * N]), f64(Vc[b * N:(b + 1) * N]))
         assert rel_err_rows(f64(o[r0:r1]).reshape(r1 - r0, -1), ref) < tol
+
+
+@pytest.mark.parametrize("B,N,H,dh,n_act,qscale", [
+    (2, 77, 3, 64, [20, 77], 1.0), (1, 200, 2, 128, [9], 1.0), (3, 33, 1, 64, [0, 33, 1], 1.0),
+    (2, 300, 2, 128, [300, 150], 1.0), (1, 1536, 4, 128, [700], 1.0), (2, 640, 2, 64, [129, 640], 6.0),
+    (1, 1024, 2, 128, [1024], 8.0)])
+def test_attention_tensor_cores(B, N, H, dh, n_act, qscale):
+    """tcgen05 attention: ragged per-sequence tiles, key counts that are not multiples of the 128-key block, and
+    (qscale > 1) score ranges that make the running maximum move so the lazy rescaling of O is exercised."""
+    lock = inputs.random_lock(B, N, n_act, 12)
+    idx, offs = O.active_set(lock.numpy())
+    M = len(idx)
+    g = torch.Generator().manual_seed(N + dh)
+    q = (torch.randn((B * N, H, dh), generator=g) * qscale).to(torch.bfloat16)
+    Kc = torch.randn((B * N, H, dh), generator=g).to(torch.bfloat16)
+    Vc = torch.randn((B * N, H, dh), generator=g).to(torch.bfloat16)
+    o = torch.full((B * N, H, dh), 5.0, dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    SL.surelock_attention(q.to(DEV), Kc.to(DEV), Vc.to(DEV), torch.from_numpy(idx).to(DEV),
+                          torch.from_numpy(offs).to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV), B, N, o, impl=0,
+                          dev_status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for b in range(B):
+        r0, r1 = offs[b], offs[b + 1]
+        if r1 == r0:
+            continue
+        ref = O.attention_rows(f64(q[r0:r1]), f64(Kc[b * N:(b + 1) * N]), f64(Vc[b * N:(b + 1) * N]))
+        assert rel_err_rows(f64(o[r0:r1]).reshape(r1 - r0, -1), ref) < 2e-2, (b,)
+    assert (o[M:] == 5.0).all()                                      # rows beyond M untouched
