@@ -34,7 +34,8 @@ typedef enum {
   SL_ENOMEM = -2,       /* device allocation failed at init                                    */
   SL_ECUDA = -3,        /* a CUDA runtime call failed (sticky CUDA error)                      */
   SL_EDEVICE = -4,      /* a kernel reported a problem through the status word                 */
-  SL_EUNSUPPORTED = -5  /* shape not supported by the kernels (e.g. head_dim not 64 or 128)    */
+  SL_EUNSUPPORTED = -5, /* shape not supported by the kernels (e.g. head_dim not 64 or 128)    */
+  SL_ELIMIT = -6        /* size beyond the fixed capacity of an allocation-free entry point    */
 } surelock_status;
 
 enum { SL_BF16 = 0, SL_FP32 = 1 };   /* storage type of weights, activations, caches and logits; accumulation is fp32 */
@@ -170,6 +171,30 @@ size_t surelock_compact_scratch_bytes(int64_t total);
  * B*N < 2^31.  Asynchronous on `stream`. */
 int surelock_compact(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
                      int32_t *n_active, int32_t *row_of_pos, void *scratch, int32_t *dev_status, void *stream);
+
+/* Compaction for callers that must not allocate device memory.  (No counterpart in the paper: this is a
+ * packaging variant of surelock_compact, same kernel, same results.)
+ *
+ * Who needs it: code that is handed its input and output buffers but may not call cudaMalloc itself -- a plug-in
+ * running inside someone else's serving process whose memory was all reserved up front by that process's pool
+ * allocator, or a latency-critical loop in which cudaMalloc's implicit device-wide synchronisation is not
+ * acceptable.  Such a caller cannot provide the scratch words surelock_compact asks for, so here they live in a
+ * fixed array that is part of the library image: 32,784 bytes of device memory on every GPU that loads the
+ * library, held until the process exits.  That fixes the capacity: B*N <= 16,777,216 flags (4096 chunks of 4096);
+ * larger inputs are refused with SL_ELIMIT and nothing is launched.
+ *
+ * Arguments and results are exactly those of surelock_compact minus `scratch`.  The call performs no cudaMalloc,
+ * cudaFree or other allocating call; it enqueues one cudaMemsetAsync (the array keeps the previous call's
+ * contents, so the words this call uses are cleared first) and one kernel on `stream`.
+ * The FIRST call on each device also asks the CUDA runtime for the array's device address (with that device
+ * current) and caches it; make that first call outside any stream capture.
+ * All calls on a device share the one array: two calls whose kernels may overlap on the GPU (different streams,
+ * or different host threads) race on it and give wrong results -- serialise them. */
+int surelock_compact_noalloc(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
+                             int32_t *n_active, int32_t *row_of_pos, int32_t *dev_status, void *stream);
+
+/* Capacity of surelock_compact_noalloc in flags (B*N). */
+int64_t surelock_compact_noalloc_max_flags(void);
 
 /* K/V cache scatter (Algorithm 1 line 11, K^all[A_t] <- K[A_t]): cache row active_idx[r] <- packed row r, for
  * r < *n_active; other cache rows are not touched.  k, v: dev [M][row_elems]; k_cache, v_cache: dev

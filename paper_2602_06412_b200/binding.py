@@ -66,6 +66,8 @@ def lib() -> C.CDLL:
         "surelock_strerror": (C.c_char_p, [i32]),
         "surelock_compact_scratch_bytes": (sz, [C.c_int64]),
         "surelock_compact": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "surelock_compact_noalloc": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, vp]),
+        "surelock_compact_noalloc_max_flags": (C.c_int64, []),
         "surelock_kv_scatter": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]),
         "surelock_softmax_kl_sure": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, f32, vp, vp, vp, vp, vp]),
         "surelock_gemm": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]),
@@ -245,6 +247,18 @@ def surelock_compact_scratch_bytes(total: int) -> int:
 def surelock_compact(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos, scratch, dev_status=None):
     _check(lib().surelock_compact(_p(lock_mask), B, N, _p(active_idx), _p(row_offsets), _p(n_active), _p(row_of_pos),
                                   _p(scratch), _p(dev_status), _stream()), "surelock_compact")
+
+
+def surelock_compact_noalloc(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos=None,
+                             dev_status=None):
+    """Compaction without caller scratch and without any device allocation (fixed in-library array; see the header
+    for the capacity and the rule that calls sharing a GPU must not overlap)."""
+    _check(lib().surelock_compact_noalloc(_p(lock_mask), B, N, _p(active_idx), _p(row_offsets), _p(n_active),
+                                          _p(row_of_pos), _p(dev_status), _stream()), "surelock_compact_noalloc")
+
+
+def surelock_compact_noalloc_max_flags() -> int:
+    return lib().surelock_compact_noalloc_max_flags()
 
 
 def surelock_kv_scatter(k, v, active_idx, n_active, k_cache, v_cache):

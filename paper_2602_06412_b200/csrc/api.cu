@@ -382,6 +382,7 @@ const char* surelock_strerror(int s) {
     case SL_ECUDA: return "CUDA runtime error";
     case SL_EDEVICE: return "a kernel reported an error through the status word";
     case SL_EUNSUPPORTED: return "shape or type not supported";
+    case SL_ELIMIT: return "size exceeds the fixed capacity of the allocation-free entry point";
     default: return "unknown status";
   }
 }
@@ -395,6 +396,14 @@ int surelock_compact(const uint8_t* lock_mask, int B, int N, int32_t* active_idx
   return launch_compact(lock_mask, B, N, active_idx, row_offsets, n_active, row_of_pos, scratch, dev_status,
                         (cudaStream_t)stream);
 }
+
+int surelock_compact_noalloc(const uint8_t* lock_mask, int B, int N, int32_t* active_idx, int32_t* row_offsets,
+                             int32_t* n_active, int32_t* row_of_pos, int32_t* dev_status, void* stream) {
+  return launch_compact_noalloc(lock_mask, B, N, active_idx, row_offsets, n_active, row_of_pos, dev_status,
+                                (cudaStream_t)stream);
+}
+
+int64_t surelock_compact_noalloc_max_flags(void) { return compact_noalloc_max_flags(); }
 
 int surelock_kv_scatter(const void* k, const void* v, const int32_t* active_idx, const int32_t* n_active, int max_rows,
                         int row_elems, void* k_cache, void* v_cache, int dtype, void* stream) {

@@ -52,6 +52,10 @@ size_t compact_scratch_bytes(int64_t total);
 int launch_compact(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
                    int32_t* row_of_pos, void* scratch, int32_t* status, cudaStream_t st);
 
+long long compact_noalloc_max_flags();
+int launch_compact_noalloc(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
+                           int32_t* row_of_pos, int32_t* status, cudaStream_t st);
+
 // x[r] = table[tokens[idx[r]]] (embedding) or x[r] = src[idx[r]] (tokens == nullptr), widened to fp32
 int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* idx, const int32_t* n_active,
                        int max_rows, int d, int table_rows, float* x, int dtype, int32_t* status, cudaStream_t st);

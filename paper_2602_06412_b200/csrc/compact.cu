@@ -5,6 +5,8 @@
 // flags (a ticket fixes the chunk order, so a chunk's predecessors have always started), scans it with warp
 // shuffles, and obtains its global offset by decoupled look-back over 64-bit (status,value) words.  The
 // look-back wait is bounded; when it runs out the CTA records SL_DEV_COMPACT_TIMEOUT and returns.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace sl {
@@ -174,6 +176,47 @@ int launch_compact(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row
   if (total >= (1ll << 31)) return SL_EINVAL;
   const int chunks = (int)((total + CP_CHUNK - 1) / CP_CHUNK);
   SL_CUDA_TRY(cudaMemsetAsync(scratch, 0, compact_scratch_bytes(total), st));
+  compact_kernel<<<chunks, CP_THREADS, 0, st>>>(lock, (int)total, N, B, idx, row_offsets, n_active, row_of_pos,
+                                                 reinterpret_cast<CompactScratch*>(scratch), status);
+  SL_CUDA_TRY(cudaGetLastError());
+  return SL_OK;
+}
+
+// ---- allocation-free variant ---------------------------------------------------------------------------------
+// The look-back words live in a fixed array inside the library image instead of caller-provided scratch.
+constexpr long long CP_NOALLOC_MAX_FLAGS = 1ll << 24;                                    // 4096 chunks
+constexpr size_t CP_NOALLOC_BYTES = 16 + 8 * (size_t)(CP_NOALLOC_MAX_FLAGS / CP_CHUNK);  // 32,784 bytes
+static __device__ __align__(256) unsigned char g_compact_scratch[CP_NOALLOC_BYTES];
+
+constexpr int CP_MAX_DEVICES = 64;
+static void* g_scratch_addr[CP_MAX_DEVICES];   // device address of g_compact_scratch, per device, filled on first use
+static std::mutex g_scratch_mu;
+
+long long compact_noalloc_max_flags() { return CP_NOALLOC_MAX_FLAGS; }
+
+int launch_compact_noalloc(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
+                           int32_t* row_of_pos, int32_t* status, cudaStream_t st) {
+  if (!lock || !idx || !row_offsets || !n_active || B <= 0 || N <= 0) return SL_EINVAL;
+  const long long total = (long long)B * N;
+  if (total > CP_NOALLOC_MAX_FLAGS) return SL_ELIMIT;
+  int dev = -1;
+  SL_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= CP_MAX_DEVICES) return SL_EUNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> g(g_scratch_mu);
+    if (!g_scratch_addr[dev]) {
+      // In host code the array's name is only a handle; the address a kernel can use comes from the runtime,
+      // for the device that is current now.
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_compact_scratch) != cudaSuccess || !p) return SL_ECUDA;
+      g_scratch_addr[dev] = p;
+    }
+    scratch = g_scratch_addr[dev];
+  }
+  const int chunks = (int)((total + CP_CHUNK - 1) / CP_CHUNK);
+  // the array keeps the previous call's words: the ticket and this call's chunk words must start at zero
+  SL_CUDA_TRY(cudaMemsetAsync(scratch, 0, 16 + 8 * (size_t)chunks, st));
   compact_kernel<<<chunks, CP_THREADS, 0, st>>>(lock, (int)total, N, B, idx, row_offsets, n_active, row_of_pos,
                                                  reinterpret_cast<CompactScratch*>(scratch), status);
   SL_CUDA_TRY(cudaGetLastError());
