@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         "surelock_prev_logits": (i32, [vp, C.POINTER(vp), C.POINTER(vp)]),
         "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
         "surelock_last_launch_count": (i32, [vp]),
+        "surelock_layer_trace": (i32, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "surelock_kernel_times": (i32, [vp, vp, vp, i32]),
         "surelock_destroy": (None, [vp]),
         "surelock_strerror": (C.c_char_p, [i32]),
@@ -219,6 +220,13 @@ def surelock_prev_logits(ctx: Ctx):
 
 def surelock_set_option(ctx: Ctx, name: str, value: int):
     _check(lib().surelock_set_option(ctx.handle, name.encode(), value), "surelock_set_option")
+
+
+def surelock_layer_trace(ctx: Ctx) -> torch.Tensor:
+    """View [L+1][B*N][d] fp32 of the per-layer residual stream of the last step ("trace_layers" must be on)."""
+    buf, stride = C.c_void_p(), C.c_size_t()
+    _check(lib().surelock_layer_trace(ctx.handle, C.byref(buf), C.byref(stride)), "surelock_layer_trace")
+    return device_view(buf.value, (ctx.cfg["n_layers"] + 1, ctx.B * ctx.N, ctx.cfg["d_model"]), torch.float32)
 
 
 def surelock_last_launch_count(ctx: Ctx) -> int:

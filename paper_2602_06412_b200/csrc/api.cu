@@ -39,6 +39,7 @@ struct surelock_ctx {
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
   std::vector<int> ev_cls;            // class of the launch bracketed by events 2i, 2i+1
   int n_ev = 0;
+  float* trace = nullptr;             // [L+1][R][d] block inputs/outputs of the last step (only when switched on)
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
   void* kcache(int l) const { return kv + (size_t)(2 * l) * kv_layer_bytes(); }
@@ -241,7 +242,14 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
                                  c->scratch, c->status, c->st));
   SL_K(K_GATHER, launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype,
                                     c->status, c->st));
-  for (int l = 0; l < g.n_layers; ++l) SL_TRY(run_layer(c, l, c->x));
+  const size_t xbytes = (size_t)c->R * g.d_model * sizeof(float);
+  if (c->trace) SL_CUDA_TRY(cudaMemcpyAsync(c->trace, c->x, xbytes, cudaMemcpyDeviceToDevice, c->st));
+  for (int l = 0; l < g.n_layers; ++l) {
+    SL_TRY(run_layer(c, l, c->x));
+    if (c->trace)
+      SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(l + 1) * c->R * g.d_model, c->x, xbytes, cudaMemcpyDeviceToDevice,
+                                  c->st));
+  }
   SL_K(K_RMSNORM, launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
   SL_K(K_GEMM_HEAD, gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
   SL_K(K_SOFTMAX_KL, launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
@@ -332,6 +340,15 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
+  if (!strcmp(name, "trace_layers")) {
+    if (value && !c->trace) {
+      const size_t bytes = (size_t)(c->cfg.n_layers + 1) * c->R * c->cfg.d_model * sizeof(float);
+      const int rc = dev_alloc(c, &c->trace, bytes);
+      if (rc != SL_OK) return rc;
+    }
+    if (!value) c->trace = nullptr;   // the buffer stays allocated until destroy; tracing stops
+    return SL_OK;
+  }
   if (!strcmp(name, "time_kernels")) {
     if (value && c->ev.empty()) {
       const int n = 2 * (16 * c->cfg.n_layers + 16);
@@ -345,6 +362,13 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
     return SL_OK;
   }
   return SL_EINVAL;
+}
+
+int surelock_layer_trace(surelock_ctx* c, float** buf, size_t* layer_stride_elems) {
+  if (!c || !buf) return SL_EINVAL;
+  *buf = c->trace;
+  if (layer_stride_elems) *layer_stride_elems = (size_t)c->R * c->cfg.d_model;
+  return c->trace ? SL_OK : SL_EINVAL;
 }
 
 int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
