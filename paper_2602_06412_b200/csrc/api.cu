@@ -92,6 +92,9 @@ static inline void tock(surelock_ctx* c) {
 namespace sl {
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
                    int n_out, int K, int epilogue, int32_t* status, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
+int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
+                       void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
+                       int n_seq, int hd, int dh, int K, int32_t* status, cudaStream_t st);   // gemm_tc.cu
 int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
 }
@@ -120,11 +123,26 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   const surelock_model_cfg& g = c->cfg;
   const int d = g.d_model, hd = g.n_heads * g.head_dim;
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
-  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
-  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wk[l], nullptr, c->k, hd, d, EPI_STORE));
-  SL_K(K_GEMM_QKV, gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
-  SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
-  SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
+  bool fused = false;
+  if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
+    // one launch: Q, K, V projections + RoPE + K/V written straight into the cache rows of the active positions
+    tick(c, K_GEMM_QKV);
+    const int rc = launch_gemm_tc_qkv(c->h, c->wq[l], c->wk[l], c->wv[l], c->q, c->kcache(l), c->vcache(l), c->idx, c->rope,
+                                      c->n_active, c->R, c->N, hd, g.head_dim, d, c->status, c->st);
+    if (rc == SL_OK) {
+      tock(c);
+      fused = true;
+    } else if (rc != SL_EUNSUPPORTED) {
+      return rc;
+    }
+  }
+  if (!fused) {
+    SL_K(K_GEMM_QKV, gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
+    SL_K(K_GEMM_QKV, gemm(c, c->h, c->wk[l], nullptr, c->k, hd, d, EPI_STORE));
+    SL_K(K_GEMM_QKV, gemm(c, c->h, c->wv[l], nullptr, c->v, hd, d, EPI_STORE));
+    SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
+    SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
+  }
   SL_K(K_ATTN, attention(c, l));
   SL_K(K_GEMM_O, gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));

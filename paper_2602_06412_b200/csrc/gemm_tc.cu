@@ -8,7 +8,9 @@
 //            described by shared-memory matrix descriptors; tcgen05.commit hands smem stages back to the producer
 //            and finished accumulators to the epilogue;
 //   warps 2-5 epilogue: tcgen05.ld the fp32 accumulator (one row per thread), apply the fused operation
-//            (store bf16 | add into the fp32 residual stream | silu(gate)*up) and write with 128-bit stores.
+//            (store bf16 | add into the fp32 residual stream | silu(gate)*up | QKV: rotary embedding on q and k with
+//            the row's ORIGINAL position, q stored packed, k and v written straight into the cache row of that
+//            position, which is Algorithm 1 line 11 done in the epilogue) and write with 128-bit stores.
 // Two accumulators live in tensor memory so the epilogue of tile i overlaps the main loop of tile i+1.
 // The number of rows M is read from device memory: tiles whose first row is >= M are never scheduled, TMA zero-fills
 // rows beyond the allocation, and the epilogue stores only rows < M.  Every mbarrier wait is bounded: when it runs out
@@ -21,13 +23,21 @@
 namespace sl {
 
 constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+constexpr int EPI_QKV = 3;   // three weight matrices side by side; epilogue = RoPE + packed q + K/V cache scatter
+
+struct QkvArgs {
+  bf16 *q, *kc, *vc;          // q packed [M][hd]; caches [B*N][hd]
+  const int32_t* idx;         // [M] flat position of each packed row
+  const float2* rope;         // [n_seq][dh/2] (cos, sin)
+  int n_seq, hd, dh;
+};
 
 // ----------------------------------------------------------------------------------------------- kernel
 template <int EPI, int BN, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-               const __grid_constant__ CUtensorMap tmB1, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
-               int n_out, int K, int32_t* status) {
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, void* __restrict__ Cv,
+               const int32_t* __restrict__ n_active, int n_out, int K, int32_t* status, const QkvArgs qkv) {
   constexpr int A_BYTES = TC_BM * TC_BK * 2;              // 16 KB
   constexpr int B_BYTES = BN * TC_BK * 2;                 // 32 KB (two 128-row halves)
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
@@ -88,6 +98,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (EPI == EPI_SWIGLU) {
             tma_load_2d(sb, &tmB0, kb * TC_BK, n0, full_bar(stage));
             tma_load_2d(sb + B_BYTES / 2, &tmB1, kb * TC_BK, n0, full_bar(stage));
+          } else if (EPI == EPI_QKV) {
+            const int src = n0 / qkv.hd, ln0 = n0 - src * qkv.hd;      // a tile never straddles two matrices
+            const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
+#pragma unroll
+            for (int hb = 0; hb < BN / 128; ++hb)
+              tma_load_2d(sb + hb * (B_BYTES / (BN / 128)), mp, kb * TC_BK, ln0 + hb * 128, full_bar(stage));
           } else {
 #pragma unroll
             for (int hb = 0; hb < BN / 128; ++hb)
@@ -138,6 +154,66 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_after();
       const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      if (EPI == EPI_QKV) {
+        const int src = n0 / qkv.hd, ln0 = n0 - src * qkv.hd;
+        const bool live = row < M;
+        const int pos = live ? qkv.idx[row] : 0;
+        bf16* drow = src == 0 ? qkv.q + (long long)row * qkv.hd
+                              : (src == 1 ? qkv.kc : qkv.vc) + (long long)pos * qkv.hd;
+        if (src == 2) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < BN; c0 += 32) {
+            uint32_t v[32];
+            tc_ld32(taddr + c0, v);
+            tc_wait_ld();
+            if (live) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8)
+                *reinterpret_cast<uint4*>(drow + ln0 + c0 + j) =
+                    make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+                               pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
+                               pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
+                               pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+            }
+          }
+        } else {
+          const int half = qkv.dh >> 1;
+          const float2* tr = qkv.rope + (long long)(pos % qkv.n_seq) * half;
+#pragma unroll 1
+          for (int hh = 0; hh < BN; hh += qkv.dh) {            // heads inside this tile
+#pragma unroll 1
+            for (int cc = 0; cc < half; cc += 32) {              // pair (j, j + dh/2), 32 pairs at a time
+              uint32_t lo[32], hi[32];
+              tc_ld32(taddr + hh + cc, lo);
+              tc_ld32(taddr + hh + half + cc, hi);
+              tc_wait_ld();
+              if (live) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  const float2 cs = __ldg(tr + cc + j);
+                  const float a = __uint_as_float(lo[j]), b = __uint_as_float(hi[j]);
+                  lo[j] = __float_as_uint(a * cs.x - b * cs.y);
+                  hi[j] = __float_as_uint(b * cs.x + a * cs.y);
+                }
+                bf16* d0 = drow + ln0 + hh + cc;
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  *reinterpret_cast<uint4*>(d0 + j) =
+                      make_uint4(pack_bf16(__uint_as_float(lo[j]), __uint_as_float(lo[j + 1])),
+                                 pack_bf16(__uint_as_float(lo[j + 2]), __uint_as_float(lo[j + 3])),
+                                 pack_bf16(__uint_as_float(lo[j + 4]), __uint_as_float(lo[j + 5])),
+                                 pack_bf16(__uint_as_float(lo[j + 6]), __uint_as_float(lo[j + 7])));
+                  *reinterpret_cast<uint4*>(d0 + half + j) =
+                      make_uint4(pack_bf16(__uint_as_float(hi[j]), __uint_as_float(hi[j + 1])),
+                                 pack_bf16(__uint_as_float(hi[j + 2]), __uint_as_float(hi[j + 3])),
+                                 pack_bf16(__uint_as_float(hi[j + 4]), __uint_as_float(hi[j + 5])),
+                                 pack_bf16(__uint_as_float(hi[j + 6]), __uint_as_float(hi[j + 7])));
+                }
+              }
+            }
+          }
+        }
+      } else
 #pragma unroll 1
       for (int c0 = 0; c0 < OUT_BN; c0 += 32) {
         uint32_t v[32];
@@ -263,8 +339,9 @@ int get_tensor_map_2d(const void* ptr, long long rows, long long cols, int box_r
 }
 
 template <int EPI, int BN, int STAGES>
-static int launch_cfg(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, void* C, const int32_t* n_active,
-                      int max_rows, int n_out, int K, int32_t* status, cudaStream_t st) {
+static int launch_cfg(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& b2, void* C,
+                      const int32_t* n_active, int max_rows, int n_out, int K, int32_t* status, const QkvArgs& qkv,
+                      cudaStream_t st) {
   constexpr int SMEM = STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024 + 256;
   static bool attr_set = false;
   if (!attr_set) {
@@ -276,7 +353,7 @@ static int launch_cfg(const CUtensorMap& a, const CUtensorMap& b0, const CUtenso
   int grid = sm_count();
   if (tiles < grid) grid = (int)tiles;
   if (grid < 1) grid = 1;
-  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b0, b1, C, n_active, n_out, K, status);
+  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b0, b1, b2, C, n_active, n_out, K, status, qkv);
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }
@@ -302,11 +379,30 @@ int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const 
     }
   }
   switch (epilogue) {
-    case EPI_STORE: return launch_cfg<EPI_STORE, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
-    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
-    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 256, 4>(a, b0, b1, C, n_active, max_rows, n_out, K, status, st);
+    case EPI_STORE: return launch_cfg<EPI_STORE, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
+    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
+    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
     default: return SL_EINVAL;
   }
+}
+
+// Q/K/V projections in one launch with RoPE and the cache scatter in the epilogue (Algorithm 1 lines 10-11).
+int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
+                       void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
+                       int n_seq, int hd, int dh, int K, int32_t* status, cudaStream_t st) {
+  if (K % 8 || hd % 256 || (dh != 64 && dh != 128) || max_rows < 1) return SL_EUNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(Wq) | reinterpret_cast<uintptr_t>(Wk) |
+       reinterpret_cast<uintptr_t>(Wv) | reinterpret_cast<uintptr_t>(q_out) | reinterpret_cast<uintptr_t>(k_cache) |
+       reinterpret_cast<uintptr_t>(v_cache)) & 15)
+    return SL_EUNSUPPORTED;
+  CUtensorMap a, b0, b1, b2;
+  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
+  if (rc == SL_OK) rc = get_tensor_map_2d(Wq, hd, K, 128, &b0);
+  if (rc == SL_OK) rc = get_tensor_map_2d(Wk, hd, K, 128, &b1);
+  if (rc == SL_OK) rc = get_tensor_map_2d(Wv, hd, K, 128, &b2);
+  if (rc != SL_OK) return rc;
+  QkvArgs qa{(bf16*)q_out, (bf16*)k_cache, (bf16*)v_cache, idx, rope, n_seq, hd, dh};
+  return launch_cfg<EPI_QKV, 256, 4>(a, b0, b1, b2, nullptr, n_active, max_rows, 3 * hd, K, status, qa, st);
 }
 
 }  // namespace sl
