@@ -7,7 +7,7 @@
 #include <new>
 #include <vector>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 using namespace sl;
 
@@ -39,6 +39,7 @@ struct surelock_ctx {
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
   std::vector<int> ev_cls;            // class of the launch bracketed by events 2i, 2i+1
   int n_ev = 0;
+  SplitWs split;                      // split-K workspace of the tensor-core GEMM (bf16 only)
   float* trace = nullptr;             // [L+1][R][d] block inputs/outputs of the last step (only when switched on)
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
@@ -91,10 +92,10 @@ static inline void tock(surelock_ctx* c) {
 
 namespace sl {
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
-                   int n_out, int K, int epilogue, int32_t* status, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
+                   int n_out, int K, int epilogue, int32_t* status, const SplitWs& sw, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
 int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
                        void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
-                       int n_seq, int hd, int dh, int K, int32_t* status, cudaStream_t st);   // gemm_tc.cu
+                       int n_seq, int hd, int dh, int K, int32_t* status, const SplitWs& sw, cudaStream_t st);   // gemm_tc.cu
 int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
 }
@@ -112,7 +113,7 @@ static int attention(surelock_ctx* c, int l) {
 
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
   if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
-    const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->st);
+    const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->split, c->st);
     if (rc != SL_EUNSUPPORTED) return rc;
   }
   return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
@@ -128,7 +129,7 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
     // one launch: Q, K, V projections + RoPE + K/V written straight into the cache rows of the active positions
     tick(c, K_GEMM_QKV);
     const int rc = launch_gemm_tc_qkv(c->h, c->wq[l], c->wk[l], c->wv[l], c->q, c->kcache(l), c->vcache(l), c->idx, c->rope,
-                                      c->n_active, c->R, c->N, hd, g.head_dim, d, c->status, c->st);
+                                      c->n_active, c->R, c->N, hd, g.head_dim, d, c->status, c->split, c->st);
     if (rc == SL_OK) {
       tock(c);
       fused = true;
@@ -221,6 +222,13 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
   A_(c->conf, R * 4);
   A_(c->scratch, compact_scratch_bytes((int64_t)R));
   A_(c->rope, (size_t)N * (cfg->head_dim / 2) * sizeof(float2));
+  if (cfg->dtype == SL_BF16) {
+    c->split.tiles = 2 * sm_count();
+    A_(c->split.ws, (size_t)c->split.tiles * SPLIT_TILE_BYTES);
+    A_(c->split.counters, (size_t)c->split.tiles * sizeof(int));
+    if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * sizeof(int), c->st) != cudaSuccess)
+      rc = SL_ECUDA;
+  }
   A_(c->st_tokens, R * 4);
   A_(c->st_mask, R);
   A_(c->st_lock, R);
@@ -470,7 +478,7 @@ int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active
   if (!A || !W || !C || !n_active || max_rows < 0 || n_out <= 0 || K <= 0) return SL_EINVAL;
   if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
   if (dtype == SL_BF16 && impl == 0) {
-    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, (cudaStream_t)stream);
+    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, SplitWs{}, (cudaStream_t)stream);
     if (rc != SL_EUNSUPPORTED) return rc;
   }
   return launch_gemm_simt(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, (cudaStream_t)stream);

@@ -15,6 +15,9 @@
 // The number of rows M is read from device memory: tiles whose first row is >= M are never scheduled, TMA zero-fills
 // rows beyond the allocation, and the epilogue stores only rows < M.  Every mbarrier wait is bounded: when it runs out
 // the CTA records SL_DEV_GEMM_TIMEOUT, all roles leave their loops, tensor memory is freed and the kernel returns.
+#include <stdlib.h>
+#include <string.h>
+
 #include <mutex>
 #include <unordered_map>
 
@@ -33,17 +36,210 @@ struct QkvArgs {
 };
 
 // ----------------------------------------------------------------------------------------------- kernel
-template <int EPI, int BN, int STAGES>
+// Source of accumulator values for the epilogue: tensor memory (one tile computed by this CTA), or the sum of the
+// fp32 partial tiles that the K-splits of a tile left in the workspace (summed in split order: deterministic).
+struct TmemSrc {
+  uint32_t taddr;
+  __device__ __forceinline__ void load(int col, uint32_t* v) const {
+    tc_ld32(taddr + col, v);
+    tc_wait_ld();
+  }
+  __device__ __forceinline__ void load2(int col0, uint32_t* v0, int col1, uint32_t* v1) const {
+    tc_ld32(taddr + col0, v0);
+    tc_ld32(taddr + col1, v1);
+    tc_wait_ld();
+  }
+};
+struct WsSrc {
+  const float* row;       // this thread's row in the partial tile of split 0
+  size_t split_stride;    // floats between consecutive splits of the same tile
+  int S;
+  bool live;
+  __device__ __forceinline__ void load(int col, uint32_t* v) const {
+    float acc[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+    if (live) {
+      int s = 0;
+      for (; s + 2 <= S; s += 2) {                     // two splits in flight; the sum order stays s = 0, 1, 2, ...
+        const float4* p0 = reinterpret_cast<const float4*>(row + (size_t)s * split_stride + col);
+        const float4* p1 = reinterpret_cast<const float4*>(row + (size_t)(s + 1) * split_stride + col);
+        float4 t0[8], t1[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { t0[j] = __ldcg(p0 + j); t1[j] = __ldcg(p1 + j); }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          acc[4 * j] += t0[j].x; acc[4 * j + 1] += t0[j].y; acc[4 * j + 2] += t0[j].z; acc[4 * j + 3] += t0[j].w;
+          acc[4 * j] += t1[j].x; acc[4 * j + 1] += t1[j].y; acc[4 * j + 2] += t1[j].z; acc[4 * j + 3] += t1[j].w;
+        }
+      }
+      for (; s < S; ++s) {
+        const float4* p = reinterpret_cast<const float4*>(row + (size_t)s * split_stride + col);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float4 t = __ldcg(p + j);
+          acc[4 * j] += t.x; acc[4 * j + 1] += t.y; acc[4 * j + 2] += t.z; acc[4 * j + 3] += t.w;
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+  }
+  __device__ __forceinline__ void load2(int col0, uint32_t* v0, int col1, uint32_t* v1) const {
+    load(col0, v0);
+    load(col1, v1);
+  }
+};
+
+__device__ __forceinline__ void store_bf16x32(bf16* dst, const uint32_t* v) {
+#pragma unroll
+  for (int j = 0; j < 32; j += 8)
+    *reinterpret_cast<uint4*>(dst + j) = make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+                                                    pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
+                                                    pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
+                                                    pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+}
+
+// Fused epilogue of one 128 x BN tile for the row this thread owns.
+template <int EPI, typename Src>
+__device__ __forceinline__ void epilogue_row(const Src& src, int bn, int row, int M, int n0, int n_out,
+                                             void* __restrict__ Cv, const QkvArgs& qkv) {
+  const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
+  const bool live = row < M;
+  if (EPI == EPI_QKV) {
+    const int srcm = n0 / qkv.hd, ln0 = n0 - srcm * qkv.hd;
+    const int pos = live ? qkv.idx[row] : 0;
+    bf16* drow = srcm == 0 ? qkv.q + (long long)row * qkv.hd : (srcm == 1 ? qkv.kc : qkv.vc) + (long long)pos * qkv.hd;
+    if (srcm == 2) {
+#pragma unroll 1
+      for (int c0 = 0; c0 < bn; c0 += 32) {
+        uint32_t v[32];
+        src.load(c0, v);
+        if (live) store_bf16x32(drow + ln0 + c0, v);
+      }
+    } else {
+      const int half = qkv.dh >> 1;
+      const float2* tr = qkv.rope + (long long)(pos % qkv.n_seq) * half;
+#pragma unroll 1
+      for (int hh = 0; hh < bn; hh += qkv.dh) {              // heads inside this tile
+#pragma unroll 1
+        for (int cc = 0; cc < half; cc += 32) {                // pairs (j, j + dh/2), 32 at a time
+          uint32_t lo[32], hi[32];
+          src.load2(hh + cc, lo, hh + half + cc, hi);
+          if (live) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float2 cs = __ldg(tr + cc + j);
+              const float a = __uint_as_float(lo[j]), b = __uint_as_float(hi[j]);
+              lo[j] = __float_as_uint(a * cs.x - b * cs.y);
+              hi[j] = __float_as_uint(b * cs.x + a * cs.y);
+            }
+            store_bf16x32(drow + ln0 + hh + cc, lo);
+            store_bf16x32(drow + ln0 + hh + half + cc, hi);
+          }
+        }
+      }
+    }
+    return;
+  }
+#pragma unroll 1
+  for (int c0 = 0; c0 < out_bn; c0 += 32) {
+    uint32_t v[32];
+    if (EPI == EPI_SWIGLU) {
+      uint32_t u[32];
+      src.load2(c0, v, out_bn + c0, u);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) {
+        const float g = __uint_as_float(v[j]);
+        v[j] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
+      }
+    } else {
+      src.load(c0, v);
+    }
+    const int col = n0 + c0;
+    if (live && col < n_out) {
+      if (EPI == EPI_RESIDUAL) {
+        float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
+        if (col + 32 <= n_out) {
+#pragma unroll
+          for (int j = 0; j < 32; j += 4) {
+            float4 o = *reinterpret_cast<float4*>(dst + j);
+            o.x += __uint_as_float(v[j]); o.y += __uint_as_float(v[j + 1]);
+            o.z += __uint_as_float(v[j + 2]); o.w += __uint_as_float(v[j + 3]);
+            *reinterpret_cast<float4*>(dst + j) = o;
+          }
+        } else {
+          for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] += __uint_as_float(v[j]);
+        }
+      } else {
+        bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
+        if (col + 32 <= n_out) {
+          store_bf16x32(dst, v);
+        } else {
+          for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+        }
+      }
+    }
+  }
+}
+
+// Tile width and K-split for this launch, derived on the device from M so that every role of every CTA agrees.
+// Wide tiles (256 weight rows) when there are enough of them to fill the GPU; narrower tiles when M is small; and
+// when even 64-wide tiles are too few (weight-streaming regime, M <= 128 rows and a narrow output), K is split.
+struct TileCfg {
+  int bn, S, kb_per, m_tiles, n_tiles, tiles, total;
+};
+template <int EPI>
+__device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, int grid, bool can_split, int ws_tiles,
+                                                int min_bn) {
+  TileCfg c;
+  c.m_tiles = (M + TC_BM - 1) / TC_BM;
+  c.bn = 256;
+  auto ntiles = [&](int bn) {
+    const int ob = EPI == EPI_SWIGLU ? bn >> 1 : bn;
+    return (n_out + ob - 1) / ob;
+  };
+  while (c.bn > min_bn && c.m_tiles * ntiles(c.bn) < grid) c.bn >>= 1;
+  c.n_tiles = ntiles(c.bn);
+  c.tiles = c.m_tiles * c.n_tiles;
+  c.S = 1;
+  if (can_split && c.tiles > 0 && c.tiles < grid) {
+    // pick the split whose items fill whole rounds of the grid best; prefer fewer splits on near ties
+    float best = (float)c.tiles / (float)grid;
+    int smax = num_kb / 4;
+    if (smax > 8) smax = 8;
+    if (smax > ws_tiles / c.tiles) smax = ws_tiles / c.tiles;
+    for (int s = 2; s <= smax; ++s) {
+      const int items = c.tiles * s, rounds = (items + grid - 1) / grid;
+      const float eff = (float)items / (float)(rounds * grid);
+      if (eff > best + 0.08f) {
+        best = eff;
+        c.S = s;
+      }
+    }
+  }
+  c.kb_per = (num_kb + c.S - 1) / c.S;
+  c.S = (num_kb + c.kb_per - 1) / c.kb_per;
+  c.total = c.tiles * c.S;
+  return c;
+}
+
+template <int EPI, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
-               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2, void* __restrict__ Cv,
-               const int32_t* __restrict__ n_active, int n_out, int K, int32_t* status, const QkvArgs qkv) {
+               const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+               const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+               const __grid_constant__ CUtensorMap tmW2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
+               int n_out, int K, int32_t* status, const QkvArgs qkv, float* __restrict__ ws, int* __restrict__ counters,
+               int ws_tiles, int wide_boxes) {
+  // tmB*: weight maps with 64-row boxes (any tile width); tmW*: the same matrices with 128-row boxes, used for
+  // 256-wide tiles so a stage is filled by fewer, larger TMA copies
+  constexpr int BN_MAX = 256;
   constexpr int A_BYTES = TC_BM * TC_BK * 2;              // 16 KB
-  constexpr int B_BYTES = BN * TC_BK * 2;                 // 32 KB (two 128-row halves)
+  constexpr int B_BYTES = BN_MAX * TC_BK * 2;             // up to 32 KB: 64-row boxes of the weight matrix
+  constexpr int BOX_BYTES = 64 * TC_BK * 2;               // 8 KB
   constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr int OUT_BN = EPI == EPI_SWIGLU ? BN / 2 : BN; // output columns per tile
-  constexpr uint32_t TMEM_COLS = 2 * BN;                  // two accumulators
-  static_assert(TMEM_COLS == 512 || TMEM_COLS == 256, "tensor memory allocation must be a power of two");
+  constexpr uint32_t TMEM_COLS = 2 * BN_MAX;              // two accumulators
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -51,6 +247,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // bars: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  volatile int* s_last = reinterpret_cast<volatile int*>(s_tmem + 2);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -78,36 +275,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const uint32_t tmem_base = *s_tmem;
 
   const int M = *n_active;
-  const int m_tiles = (M + TC_BM - 1) / TC_BM;
-  const int n_tiles = (n_out + OUT_BN - 1) / OUT_BN;
-  const int total = m_tiles * n_tiles;
   const int num_kb = (K + TC_BK - 1) / TC_BK;
+  const int min_bn = EPI == EPI_QKV ? (qkv.dh > 64 ? 128 : 64) : (EPI == EPI_SWIGLU ? 128 : 64);
+  const TileCfg tc = choose_tiles<EPI>(M, n_out, num_kb, (int)gridDim.x, ws != nullptr, ws_tiles, min_bn);
+  const int bn = tc.bn, S = tc.S, kb_per = tc.kb_per, m_tiles = tc.m_tiles, total = tc.total;
+  const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
+  const uint32_t stage_tx = (uint32_t)(A_BYTES + bn * TC_BK * 2);
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int t = blockIdx.x; t < total && ok; t += gridDim.x) {
-        const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * OUT_BN;
-        for (int kb = 0; kb < num_kb; ++kb) {
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+        const int t = w / S, sp = w - t * S;
+        const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
+        const int kb0 = sp * kb_per, kb1 = kb0 + kb_per < num_kb ? kb0 + kb_per : num_kb;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(stage), STAGE_BYTES);
+          mbar_expect_tx(full_bar(stage), stage_tx);
           tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(stage));
+          const bool wide = bn == 256 && wide_boxes;
           if (EPI == EPI_SWIGLU) {
-            tma_load_2d(sb, &tmB0, kb * TC_BK, n0, full_bar(stage));
-            tma_load_2d(sb + B_BYTES / 2, &tmB1, kb * TC_BK, n0, full_bar(stage));
-          } else if (EPI == EPI_QKV) {
-            const int src = n0 / qkv.hd, ln0 = n0 - src * qkv.hd;      // a tile never straddles two matrices
-            const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
-#pragma unroll
-            for (int hb = 0; hb < BN / 128; ++hb)
-              tma_load_2d(sb + hb * (B_BYTES / (BN / 128)), mp, kb * TC_BK, ln0 + hb * 128, full_bar(stage));
+            if (wide) {
+              tma_load_2d(sb, &tmW0, kb * TC_BK, n0, full_bar(stage));
+              tma_load_2d(sb + 2 * BOX_BYTES, &tmW1, kb * TC_BK, n0, full_bar(stage));
+            } else {
+              const int hb = bn >> 7;                                  // 64-row boxes per half
+              for (int i = 0; i < hb; ++i) {
+                tma_load_2d(sb + i * BOX_BYTES, &tmB0, kb * TC_BK, n0 + 64 * i, full_bar(stage));
+                tma_load_2d(sb + (hb + i) * BOX_BYTES, &tmB1, kb * TC_BK, n0 + 64 * i, full_bar(stage));
+              }
+            }
           } else {
-#pragma unroll
-            for (int hb = 0; hb < BN / 128; ++hb)
-              tma_load_2d(sb + hb * (B_BYTES / (BN / 128)), &tmB0, kb * TC_BK, n0 + hb * 128, full_bar(stage));
+            int src = 0, ln0 = n0;
+            if (EPI == EPI_QKV) {                                      // a tile never straddles two matrices
+              src = n0 / qkv.hd;
+              ln0 = n0 - src * qkv.hd;
+            }
+            if (wide) {
+              const CUtensorMap* mp = src == 0 ? &tmW0 : (src == 1 ? &tmW1 : &tmW2);
+              tma_load_2d(sb, mp, kb * TC_BK, ln0, full_bar(stage));
+              if (wide_boxes == 1) tma_load_2d(sb + 2 * BOX_BYTES, mp, kb * TC_BK, ln0 + 128, full_bar(stage));
+            } else {
+              const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
+              for (int i = 0; i < (bn >> 6); ++i)
+                tma_load_2d(sb + i * BOX_BYTES, mp, kb * TC_BK, ln0 + 64 * i, full_bar(stage));
+            }
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -115,25 +330,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_bf16_m128(BN);
+      const uint32_t idesc = idesc_bf16_m128(bn);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       int it = 0;
-      for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+        const int sp = w % S;
+        const int kb0 = sp * kb_per, kb1 = kb0 + kb_per < num_kb ? kb0 + kb_per : num_kb;
         const int acc = it & 1;
         const uint32_t use = (uint32_t)(it >> 1);
         if (!(ok = mbar_wait(acce_bar(acc), (use & 1) ^ 1, s_abort))) break;
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < num_kb; ++kb) {
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN_MAX);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(full_bar(stage), phase, s_abort))) break;
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
           const uint64_t adesc = smem_desc_k_sw128(sa), bdesc = smem_desc_k_sw128(sb);
 #pragma unroll
           for (int k = 0; k < TC_BK / 16; ++k)   // 16 bf16 = 32 bytes along K inside the 128-byte swizzle row
-            tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb | k) != 0);
+            tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb > kb0) | (k != 0));
           tc_commit(empty_bar(stage));
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -144,128 +361,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int quarter = warp & 3;             // tensor-memory lanes 32*quarter .. 32*quarter+31
     bool ok = true;
     int it = 0;
-    for (int t = blockIdx.x; t < total && ok; t += gridDim.x, ++it) {
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+      const int t = w / S, sp = w - t * S;
       const int acc = it & 1;
       const uint32_t use = (uint32_t)(it >> 1);
-      const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * OUT_BN;
+      const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int row = m0 + quarter * 32 + lane;
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
-      if (EPI == EPI_QKV) {
-        const int src = n0 / qkv.hd, ln0 = n0 - src * qkv.hd;
-        const bool live = row < M;
-        const int pos = live ? qkv.idx[row] : 0;
-        bf16* drow = src == 0 ? qkv.q + (long long)row * qkv.hd
-                              : (src == 1 ? qkv.kc : qkv.vc) + (long long)pos * qkv.hd;
-        if (src == 2) {
+      const int trow = quarter * 32 + lane;
+      const int row = m0 + trow;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
+      if (S == 1) {
+        epilogue_row<EPI>(TmemSrc{taddr}, bn, row, M, n0, n_out, Cv, qkv);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(acc));
+      } else {
+        // partial tile of this K-split -> workspace, then free the accumulator
+        float* prow = ws + ((size_t)(t * S + sp) * TC_BM + trow) * bn;
 #pragma unroll 1
-          for (int c0 = 0; c0 < BN; c0 += 32) {
-            uint32_t v[32];
-            tc_ld32(taddr + c0, v);
-            tc_wait_ld();
-            if (live) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8)
-                *reinterpret_cast<uint4*>(drow + ln0 + c0 + j) =
-                    make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
-                               pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
-                               pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
-                               pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
-            }
-          }
-        } else {
-          const int half = qkv.dh >> 1;
-          const float2* tr = qkv.rope + (long long)(pos % qkv.n_seq) * half;
-#pragma unroll 1
-          for (int hh = 0; hh < BN; hh += qkv.dh) {            // heads inside this tile
-#pragma unroll 1
-            for (int cc = 0; cc < half; cc += 32) {              // pair (j, j + dh/2), 32 pairs at a time
-              uint32_t lo[32], hi[32];
-              tc_ld32(taddr + hh + cc, lo);
-              tc_ld32(taddr + hh + half + cc, hi);
-              tc_wait_ld();
-              if (live) {
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                  const float2 cs = __ldg(tr + cc + j);
-                  const float a = __uint_as_float(lo[j]), b = __uint_as_float(hi[j]);
-                  lo[j] = __float_as_uint(a * cs.x - b * cs.y);
-                  hi[j] = __float_as_uint(b * cs.x + a * cs.y);
-                }
-                bf16* d0 = drow + ln0 + hh + cc;
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  *reinterpret_cast<uint4*>(d0 + j) =
-                      make_uint4(pack_bf16(__uint_as_float(lo[j]), __uint_as_float(lo[j + 1])),
-                                 pack_bf16(__uint_as_float(lo[j + 2]), __uint_as_float(lo[j + 3])),
-                                 pack_bf16(__uint_as_float(lo[j + 4]), __uint_as_float(lo[j + 5])),
-                                 pack_bf16(__uint_as_float(lo[j + 6]), __uint_as_float(lo[j + 7])));
-                  *reinterpret_cast<uint4*>(d0 + half + j) =
-                      make_uint4(pack_bf16(__uint_as_float(hi[j]), __uint_as_float(hi[j + 1])),
-                                 pack_bf16(__uint_as_float(hi[j + 2]), __uint_as_float(hi[j + 3])),
-                                 pack_bf16(__uint_as_float(hi[j + 4]), __uint_as_float(hi[j + 5])),
-                                 pack_bf16(__uint_as_float(hi[j + 6]), __uint_as_float(hi[j + 7])));
-                }
-              }
-            }
-          }
-        }
-      } else
-#pragma unroll 1
-      for (int c0 = 0; c0 < OUT_BN; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(taddr + c0, v);
-        if (EPI == EPI_SWIGLU) {
-          uint32_t u[32];
-          tc_ld32(taddr + OUT_BN + c0, u);
+        for (int c0 = 0; c0 < bn; c0 += 32) {
+          uint32_t v[32];
+          tc_ld32(taddr + c0, v);
           tc_wait_ld();
+          if (row < M) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float g = __uint_as_float(v[j]);
-            v[j] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
-          }
-        } else {
-          tc_wait_ld();
-        }
-        const int col = n0 + c0;
-        if (row < M && col < n_out) {
-          if (EPI == EPI_RESIDUAL) {
-            float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
-            if (col + 32 <= n_out) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                float4 o = *reinterpret_cast<float4*>(dst + j);
-                o.x += __uint_as_float(v[j]); o.y += __uint_as_float(v[j + 1]);
-                o.z += __uint_as_float(v[j + 2]); o.w += __uint_as_float(v[j + 3]);
-                *reinterpret_cast<float4*>(dst + j) = o;
-              }
-            } else {
-              for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] += __uint_as_float(v[j]);
-            }
-          } else {
-            bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
-            if (col + 32 <= n_out) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                uint4 o;
-                o.x = pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1]));
-                o.y = pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-                o.z = pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5]));
-                o.w = pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7]));
-                *reinterpret_cast<uint4*>(dst + j) = o;
-              }
-            } else {
-              for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-            }
+            for (int j = 0; j < 32; j += 4)
+              __stcg(reinterpret_cast<float4*>(prow + c0 + j),
+                     make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                                 __uint_as_float(v[j + 3])));
           }
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(acce_bar(acc));
+        __threadfence();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (warp == 2 && lane == 0) {
+          const int old = atomicAdd(&counters[t], 1);
+          const int last = old == S - 1;
+          if (last) counters[t] = 0;             // every split has arrived: leave the counter clean for the next launch
+          *s_last = last;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*s_last) {
+          __threadfence();
+          WsSrc src{ws + ((size_t)(t * S) * TC_BM + trow) * bn, (size_t)TC_BM * bn, S, row < M};
+          epilogue_row<EPI>(src, bn, row, M, n0, n_out, Cv, qkv);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // s_last is rewritten by the next item
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acce_bar(acc));
     }
   }
 
@@ -338,50 +485,62 @@ int get_tensor_map_2d(const void* ptr, long long rows, long long cols, int box_r
   return SL_OK;
 }
 
-template <int EPI, int BN, int STAGES>
-static int launch_cfg(const CUtensorMap& a, const CUtensorMap& b0, const CUtensorMap& b1, const CUtensorMap& b2, void* C,
+static int wide_boxes() {
+  static int v = -1;
+  if (v < 0) {
+    // tuning aid: SURELOCK_GEMM_BOX = 64 | 128 | 256 rows per weight copy of a 256-wide tile (default 256)
+    const char* e = getenv("SURELOCK_GEMM_BOX");
+    v = 2;
+    if (e && !strcmp(e, "64")) v = 0;
+    if (e && !strcmp(e, "128")) v = 1;
+  }
+  return v;
+}
+
+template <int EPI, int STAGES>
+static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensorMap* wb, void* C,
                       const int32_t* n_active, int max_rows, int n_out, int K, int32_t* status, const QkvArgs& qkv,
-                      cudaStream_t st) {
-  constexpr int SMEM = STAGES * (TC_BM * TC_BK * 2 + BN * TC_BK * 2) + 1024 + 256;
+                      const SplitWs& sw, cudaStream_t st) {
+  constexpr int SMEM = STAGES * (TC_BM * TC_BK * 2 + 256 * TC_BK * 2) + 1024 + 256;
   static bool attr_set = false;
   if (!attr_set) {
-    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI, BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
+    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
     attr_set = true;
   }
-  constexpr int OUT_BN = EPI == EPI_SWIGLU ? BN / 2 : BN;
-  const long long tiles = (long long)((max_rows + TC_BM - 1) / TC_BM) * ((n_out + OUT_BN - 1) / OUT_BN);
-  int grid = sm_count();
-  if (tiles < grid) grid = (int)tiles;
-  if (grid < 1) grid = 1;
-  gemm_tc_kernel<EPI, BN, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b0, b1, b2, C, n_active, n_out, K, status, qkv);
+  (void)max_rows;
+  const int grid = sm_count();   // persistent: one CTA per SM; the tile shape is chosen on the device from M
+  gemm_tc_kernel<EPI, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b[0], b[1], b[2], wb[0], wb[1], wb[2], C, n_active,
+                                                              n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles,
+                                                              wide_boxes());
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }
 
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
-                   int n_out, int K, int epilogue, int32_t* status, cudaStream_t st) {
+                   int n_out, int K, int epilogue, int32_t* status, const SplitWs& sw, cudaStream_t st) {
   // TMA needs 16-byte aligned bases and row strides; the epilogue's 128-bit stores need n_out % 8 == 0
   if (K % 8 || n_out % 8 || max_rows < 1) return SL_EUNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(W2) |
        reinterpret_cast<uintptr_t>(C)) & 15)
     return SL_EUNSUPPORTED;
   if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
-  CUtensorMap a, b0, b1;
-  {
-    int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
+  CUtensorMap a, b[3], wb[3];
+  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
+  if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, 64, &b[0]);
+  const int wrows = (wide_boxes() == 2 && epilogue != EPI_SWIGLU) ? 256 : 128;
+  if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, wrows, &wb[0]);
+  if (rc != SL_OK) return rc;
+  b[1] = b[2] = b[0];
+  wb[1] = wb[2] = wb[0];
+  if (W2) {
+    rc = get_tensor_map_2d(W2, n_out, K, 64, &b[1]);
+    if (rc == SL_OK) rc = get_tensor_map_2d(W2, n_out, K, 128, &wb[1]);
     if (rc != SL_OK) return rc;
-    rc = get_tensor_map_2d(W, n_out, K, 128, &b0);
-    if (rc != SL_OK) return rc;
-    b1 = b0;
-    if (W2) {
-      rc = get_tensor_map_2d(W2, n_out, K, 128, &b1);
-      if (rc != SL_OK) return rc;
-    }
   }
   switch (epilogue) {
-    case EPI_STORE: return launch_cfg<EPI_STORE, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
-    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
-    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 256, 4>(a, b0, b1, b1, C, n_active, max_rows, n_out, K, status, QkvArgs{}, st);
+    case EPI_STORE: return launch_cfg<EPI_STORE, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
     default: return SL_EINVAL;
   }
 }
@@ -389,20 +548,22 @@ int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const 
 // Q/K/V projections in one launch with RoPE and the cache scatter in the epilogue (Algorithm 1 lines 10-11).
 int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
                        void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
-                       int n_seq, int hd, int dh, int K, int32_t* status, cudaStream_t st) {
+                       int n_seq, int hd, int dh, int K, int32_t* status, const SplitWs& sw, cudaStream_t st) {
   if (K % 8 || hd % 256 || (dh != 64 && dh != 128) || max_rows < 1) return SL_EUNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(A) | reinterpret_cast<uintptr_t>(Wq) | reinterpret_cast<uintptr_t>(Wk) |
        reinterpret_cast<uintptr_t>(Wv) | reinterpret_cast<uintptr_t>(q_out) | reinterpret_cast<uintptr_t>(k_cache) |
        reinterpret_cast<uintptr_t>(v_cache)) & 15)
     return SL_EUNSUPPORTED;
-  CUtensorMap a, b0, b1, b2;
+  CUtensorMap a, b[3], wb[3];
+  const void* W[3] = {Wq, Wk, Wv};
   int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
-  if (rc == SL_OK) rc = get_tensor_map_2d(Wq, hd, K, 128, &b0);
-  if (rc == SL_OK) rc = get_tensor_map_2d(Wk, hd, K, 128, &b1);
-  if (rc == SL_OK) rc = get_tensor_map_2d(Wv, hd, K, 128, &b2);
+  for (int i = 0; i < 3 && rc == SL_OK; ++i) {
+    rc = get_tensor_map_2d(W[i], hd, K, 64, &b[i]);
+    if (rc == SL_OK) rc = get_tensor_map_2d(W[i], hd, K, wide_boxes() == 2 ? 256 : 128, &wb[i]);
+  }
   if (rc != SL_OK) return rc;
   QkvArgs qa{(bf16*)q_out, (bf16*)k_cache, (bf16*)v_cache, idx, rope, n_seq, hd, dh};
-  return launch_cfg<EPI_QKV, 256, 4>(a, b0, b1, b2, nullptr, n_active, max_rows, 3 * hd, K, status, qa, st);
+  return launch_cfg<EPI_QKV, 4>(a, b, wb, nullptr, n_active, max_rows, 3 * hd, K, status, qa, sw, st);
 }
 
 }  // namespace sl

@@ -130,6 +130,15 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// Split-K workspace of the GEMM: room for `tiles` fp32 partial tiles of 128 x 256 and one arrival counter per output
+// tile (zero-initialised once; the kernel leaves them zero).  ws == nullptr disables split-K.
+struct SplitWs {
+  float* ws = nullptr;
+  int* counters = nullptr;
+  int tiles = 0;
+};
+constexpr size_t SPLIT_TILE_BYTES = 128 * 256 * sizeof(float);
+
 // 2-D bf16 row-major [rows][cols] tensor map, box = box_rows x 64 elements, 128-byte swizzle, zero fill out of
 // bounds.  Maps are cached per (pointer, shape).  Returns SL_OK / SL_ECUDA.
 int get_tensor_map_2d(const void* ptr, long long rows, long long cols, int box_rows, CUtensorMap* out);
