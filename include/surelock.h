@@ -225,12 +225,19 @@ int surelock_softmax_kl_sure(const void *logits, const void *prev_logits, const 
                              int vocab, int dtype, const uint8_t *mask_state, uint8_t *lock_mask, float kl_eps,
                              float *kl, float *conf, int32_t *argmax, float *lse_out, void *stream);
 
+/* Bytes of workspace that lets surelock_gemm split K when M is small (see below). */
+size_t surelock_gemm_workspace_bytes(void);
+
 /* Dense contraction on packed rows, C[r][n] = sum_k A[r][k] * W[n][k] for r < *n_active (the projections of
  * Algorithm 1 lines 10, 12, 15; FLOP terms of Sec. 2.3).  A: dev [M][K]; W: dev [n_out][K]; C: dev [M][n_out];
  * A, W, C of `dtype`; fp32 accumulation.  impl: 0 = best available (tcgen05 tensor cores for SL_BF16 when the
- * shape allows), 1 = force the CUDA-core kernel.  dev_status as for surelock_compact. */
+ * shape allows), 1 = force the CUDA-core kernel.
+ * workspace: dev, surelock_gemm_workspace_bytes() bytes, ZERO-FILLED by the caller before its first use (the kernel
+ * leaves it reusable), or NULL.  With a workspace and few output tiles (small M) the tensor-core kernel splits K
+ * across SMs and sums the partial tiles in a fixed order (deterministic); without one it never splits.
+ * dev_status as for surelock_compact. */
 int surelock_gemm(const void *A, const void *W, void *C, const int32_t *n_active, int max_rows, int n_out, int K,
-                  int dtype, int impl, int32_t *dev_status, void *stream);
+                  int dtype, int impl, void *workspace, int32_t *dev_status, void *stream);
 
 /* M x N bidirectional attention of the packed queries against the whole cache (Algorithm 1 line 12; Sec. 2.1:
  * "variable-length attention against the full key/value tables"): for packed row r at flat position

@@ -71,7 +71,8 @@ def lib() -> C.CDLL:
         "surelock_compact_noalloc_max_flags": (C.c_int64, []),
         "surelock_kv_scatter": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]),
         "surelock_softmax_kl_sure": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, f32, vp, vp, vp, vp, vp]),
-        "surelock_gemm": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp]),
+        "surelock_gemm": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]),
+        "surelock_gemm_workspace_bytes": (sz, []),
         "surelock_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -282,9 +283,14 @@ def surelock_softmax_kl_sure(logits, prev_logits, row_of_pos_prev, prev_lse, act
                                           _p(lse_out), _stream()), "surelock_softmax_kl_sure")
 
 
-def surelock_gemm(A, W, Cout, n_active, impl: int = 0, dev_status=None):
+def surelock_gemm_workspace_bytes() -> int:
+    return lib().surelock_gemm_workspace_bytes()
+
+
+def surelock_gemm(A, W, Cout, n_active, impl: int = 0, dev_status=None, workspace=None):
+    """workspace: zero-filled uint8 CUDA tensor of surelock_gemm_workspace_bytes() bytes (enables split-K), or None."""
     _check(lib().surelock_gemm(_p(A), _p(W), _p(Cout), _p(n_active), A.shape[0], W.shape[0], A.shape[1], _dt(A), impl,
-                               _p(dev_status), _stream()), "surelock_gemm")
+                               _p(workspace), _p(dev_status), _stream()), "surelock_gemm")
 
 
 def surelock_attention(q, k_cache, v_cache, active_idx, row_offsets, n_active, B: int, N: int, o, impl: int = 0,

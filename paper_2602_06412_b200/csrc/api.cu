@@ -473,12 +473,21 @@ int surelock_softmax_kl_sure(const void* logits, const void* prev_logits, const 
                                 dtype, mask_state, lock_mask, kl_eps, kl, conf, argmax, lse_out, (cudaStream_t)stream);
 }
 
+static size_t gemm_ws_tiles() { return 2 * (size_t)sm_count(); }
+size_t surelock_gemm_workspace_bytes(void) { return gemm_ws_tiles() * (SPLIT_TILE_BYTES + sizeof(int)); }
+
 int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active, int max_rows, int n_out, int K,
-                  int dtype, int impl, int32_t* dev_status, void* stream) {
+                  int dtype, int impl, void* workspace, int32_t* dev_status, void* stream) {
   if (!A || !W || !C || !n_active || max_rows < 0 || n_out <= 0 || K <= 0) return SL_EINVAL;
   if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
   if (dtype == SL_BF16 && impl == 0) {
-    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, SplitWs{}, (cudaStream_t)stream);
+    SplitWs sw;
+    if (workspace) {
+      sw.tiles = (int)gemm_ws_tiles();
+      sw.ws = reinterpret_cast<float*>(workspace);
+      sw.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(workspace) + gemm_ws_tiles() * SPLIT_TILE_BYTES);
+    }
+    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, sw, (cudaStream_t)stream);
     if (rc != SL_EUNSUPPORTED) return rc;
   }
   return launch_gemm_simt(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, (cudaStream_t)stream);

@@ -15,6 +15,7 @@
 // The number of rows M is read from device memory: tiles whose first row is >= M are never scheduled, TMA zero-fills
 // rows beyond the allocation, and the epilogue stores only rows < M.  Every mbarrier wait is bounded: when it runs out
 // the CTA records SL_DEV_GEMM_TIMEOUT, all roles leave their loops, tensor memory is freed and the kernel returns.
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -51,34 +52,31 @@ struct TmemSrc {
   }
 };
 struct WsSrc {
-  const float* row;       // this thread's row in the partial tile of split 0
+  const float* row;       // one row of the partial tile of split 0
   size_t split_stride;    // floats between consecutive splits of the same tile
   int S;
-  bool live;
+  // sum over the splits in split order (deterministic), four splits' loads in flight at a time
   __device__ __forceinline__ void load(int col, uint32_t* v) const {
     float acc[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-    if (live) {
-      int s = 0;
-      for (; s + 2 <= S; s += 2) {                     // two splits in flight; the sum order stays s = 0, 1, 2, ...
-        const float4* p0 = reinterpret_cast<const float4*>(row + (size_t)s * split_stride + col);
-        const float4* p1 = reinterpret_cast<const float4*>(row + (size_t)(s + 1) * split_stride + col);
-        float4 t0[8], t1[8];
+    for (int s0 = 0; s0 < S; s0 += 4) {
+      float4 t[4][8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { t0[j] = __ldcg(p0 + j); t1[j] = __ldcg(p1 + j); }
+      for (int q = 0; q < 4; ++q) {
+        if (s0 + q < S) {
+          const float4* p = reinterpret_cast<const float4*>(row + (size_t)(s0 + q) * split_stride + col);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          acc[4 * j] += t0[j].x; acc[4 * j + 1] += t0[j].y; acc[4 * j + 2] += t0[j].z; acc[4 * j + 3] += t0[j].w;
-          acc[4 * j] += t1[j].x; acc[4 * j + 1] += t1[j].y; acc[4 * j + 2] += t1[j].z; acc[4 * j + 3] += t1[j].w;
+          for (int j = 0; j < 8; ++j) t[q][j] = __ldcg(p + j);
         }
       }
-      for (; s < S; ++s) {
-        const float4* p = reinterpret_cast<const float4*>(row + (size_t)s * split_stride + col);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float4 t = __ldcg(p + j);
-          acc[4 * j] += t.x; acc[4 * j + 1] += t.y; acc[4 * j + 2] += t.z; acc[4 * j + 3] += t.w;
+      for (int q = 0; q < 4; ++q) {
+        if (s0 + q < S) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            acc[4 * j] += t[q][j].x; acc[4 * j + 1] += t[q][j].y; acc[4 * j + 2] += t[q][j].z; acc[4 * j + 3] += t[q][j].w;
+          }
         }
       }
     }
@@ -100,92 +98,94 @@ __device__ __forceinline__ void store_bf16x32(bf16* dst, const uint32_t* v) {
                                                     pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
 }
 
-// Fused epilogue of one 128 x BN tile for the row this thread owns.
+// The epilogue works in UNITS of one row: 32 output columns (64 for a rotated q/k pair block).  A 128 x bn tile has
+// units_per_row() units per row; unit u of row `row` is finished by epilogue_unit().  Reading the accumulator from
+// tensor memory ties a thread to its row (lane); reading summed partial tiles from the workspace does not, so the
+// split-K finisher spreads (row, unit) pairs over all epilogue threads.
+template <int EPI>
+__device__ __forceinline__ int units_per_row(int bn, int n0, const QkvArgs& qkv) {
+  if (EPI == EPI_SWIGLU) return bn >> 6;
+  if (EPI == EPI_QKV && n0 / qkv.hd != 2) return bn >> 6;   // (head, 32-pair block): bn/dh * (dh/2)/32
+  return bn >> 5;
+}
+
 template <int EPI, typename Src>
-__device__ __forceinline__ void epilogue_row(const Src& src, int bn, int row, int M, int n0, int n_out,
-                                             void* __restrict__ Cv, const QkvArgs& qkv) {
-  const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
-  const bool live = row < M;
+__device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, bool live, int u, int n0, int n_out,
+                                              void* __restrict__ Cv, const QkvArgs& qkv) {
   if (EPI == EPI_QKV) {
     const int srcm = n0 / qkv.hd, ln0 = n0 - srcm * qkv.hd;
     const int pos = live ? qkv.idx[row] : 0;
     bf16* drow = srcm == 0 ? qkv.q + (long long)row * qkv.hd : (srcm == 1 ? qkv.kc : qkv.vc) + (long long)pos * qkv.hd;
     if (srcm == 2) {
-#pragma unroll 1
-      for (int c0 = 0; c0 < bn; c0 += 32) {
-        uint32_t v[32];
-        src.load(c0, v);
-        if (live) store_bf16x32(drow + ln0 + c0, v);
-      }
+      uint32_t v[32];
+      src.load(u * 32, v);
+      if (live) store_bf16x32(drow + ln0 + u * 32, v);
     } else {
-      const int half = qkv.dh >> 1;
+      const int half = qkv.dh >> 1, per_head = half >> 5;
+      const int hh = (u / per_head) * qkv.dh, cc = (u % per_head) * 32;     // head offset, pair block
       const float2* tr = qkv.rope + (long long)(pos % qkv.n_seq) * half;
-#pragma unroll 1
-      for (int hh = 0; hh < bn; hh += qkv.dh) {              // heads inside this tile
-#pragma unroll 1
-        for (int cc = 0; cc < half; cc += 32) {                // pairs (j, j + dh/2), 32 at a time
-          uint32_t lo[32], hi[32];
-          src.load2(hh + cc, lo, hh + half + cc, hi);
-          if (live) {
+      uint32_t lo[32], hi[32];
+      src.load2(hh + cc, lo, hh + half + cc, hi);
+      if (live) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const float2 cs = __ldg(tr + cc + j);
-              const float a = __uint_as_float(lo[j]), b = __uint_as_float(hi[j]);
-              lo[j] = __float_as_uint(a * cs.x - b * cs.y);
-              hi[j] = __float_as_uint(b * cs.x + a * cs.y);
-            }
-            store_bf16x32(drow + ln0 + hh + cc, lo);
-            store_bf16x32(drow + ln0 + hh + half + cc, hi);
-          }
+        for (int j = 0; j < 32; ++j) {
+          const float2 cs = __ldg(tr + cc + j);
+          const float a = __uint_as_float(lo[j]), b = __uint_as_float(hi[j]);
+          lo[j] = __float_as_uint(a * cs.x - b * cs.y);
+          hi[j] = __float_as_uint(b * cs.x + a * cs.y);
         }
+        store_bf16x32(drow + ln0 + hh + cc, lo);
+        store_bf16x32(drow + ln0 + hh + half + cc, hi);
       }
     }
     return;
   }
-#pragma unroll 1
-  for (int c0 = 0; c0 < out_bn; c0 += 32) {
-    uint32_t v[32];
-    if (EPI == EPI_SWIGLU) {
-      uint32_t u[32];
-      src.load2(c0, v, out_bn + c0, u);
+  const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
+  const int c0 = u * 32;
+  uint32_t v[32];
+  if (EPI == EPI_SWIGLU) {
+    uint32_t g2[32];
+    src.load2(c0, v, out_bn + c0, g2);
 #pragma unroll
-      for (int j = 0; j < 32; ++j) {
-        const float g = __uint_as_float(v[j]);
-        v[j] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(u[j]));
-      }
-    } else {
-      src.load(c0, v);
+    for (int j = 0; j < 32; ++j) {
+      const float g = __uint_as_float(v[j]);
+      v[j] = __float_as_uint(g / (1.f + __expf(-g)) * __uint_as_float(g2[j]));
     }
-    const int col = n0 + c0;
-    if (live && col < n_out) {
-      if (EPI == EPI_RESIDUAL) {
-        float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
-        if (col + 32 <= n_out) {
+  } else {
+    src.load(c0, v);
+  }
+  const int col = n0 + c0;
+  if (live && col < n_out) {
+    if (EPI == EPI_RESIDUAL) {
+      float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
+      if (col + 32 <= n_out) {
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float4 o = *reinterpret_cast<float4*>(dst + j);
-            o.x += __uint_as_float(v[j]); o.y += __uint_as_float(v[j + 1]);
-            o.z += __uint_as_float(v[j + 2]); o.w += __uint_as_float(v[j + 3]);
-            *reinterpret_cast<float4*>(dst + j) = o;
-          }
-        } else {
-          for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] += __uint_as_float(v[j]);
+        for (int j = 0; j < 32; j += 4) {
+          float4 o = *reinterpret_cast<float4*>(dst + j);
+          o.x += __uint_as_float(v[j]); o.y += __uint_as_float(v[j + 1]);
+          o.z += __uint_as_float(v[j + 2]); o.w += __uint_as_float(v[j + 3]);
+          *reinterpret_cast<float4*>(dst + j) = o;
         }
       } else {
-        bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
-        if (col + 32 <= n_out) {
-          store_bf16x32(dst, v);
-        } else {
-          for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
-        }
+        for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] += __uint_as_float(v[j]);
+      }
+    } else {
+      bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
+      if (col + 32 <= n_out) {
+        store_bf16x32(dst, v);
+      } else {
+        for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
       }
     }
   }
 }
 
 // Tile width and K-split for this launch, derived on the device from M so that every role of every CTA agrees.
-// Wide tiles (256 weight rows) when there are enough of them to fill the GPU; narrower tiles when M is small; and
-// when even 64-wide tiles are too few (weight-streaming regime, M <= 128 rows and a narrow output), K is split.
+// Enough 256-wide tiles to fill the grid (large M): 256-wide, no split, the tensor-pipe-bound configuration.
+// A single row tile (M <= 128, the weight-streaming regime): 128-wide tiles and K split up to four ways.  In between:
+// the width that needs the fewest rounds of the grid.  (Measured on B200: wider splits, or splitting at M > 128,
+// cost more in partial-tile traffic than they gain in balance.)  Splits meet in the workspace; the last arriver of
+// a tile sums them in split order and runs the fused epilogue.
 struct TileCfg {
   int bn, S, kb_per, m_tiles, n_tiles, tiles, total;
 };
@@ -194,30 +194,39 @@ __device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, in
                                                 int min_bn) {
   TileCfg c;
   c.m_tiles = (M + TC_BM - 1) / TC_BM;
-  c.bn = 256;
   auto ntiles = [&](int bn) {
     const int ob = EPI == EPI_SWIGLU ? bn >> 1 : bn;
     return (n_out + ob - 1) / ob;
   };
-  while (c.bn > min_bn && c.m_tiles * ntiles(c.bn) < grid) c.bn >>= 1;
-  c.n_tiles = ntiles(c.bn);
-  c.tiles = c.m_tiles * c.n_tiles;
+  c.bn = 256;
   c.S = 1;
-  if (can_split && c.tiles > 0 && c.tiles < grid) {
-    // pick the split whose items fill whole rounds of the grid best; prefer fewer splits on near ties
-    float best = (float)c.tiles / (float)grid;
-    int smax = num_kb / 4;
-    if (smax > 8) smax = 8;
-    if (smax > ws_tiles / c.tiles) smax = ws_tiles / c.tiles;
-    for (int s = 2; s <= smax; ++s) {
-      const int items = c.tiles * s, rounds = (items + grid - 1) / grid;
-      const float eff = (float)items / (float)(rounds * grid);
-      if (eff > best + 0.08f) {
-        best = eff;
-        c.S = s;
+  if (c.m_tiles == 1) {
+    // weight-streaming regime: 128-wide tiles, K split so that about one item per SM exists
+    c.bn = min_bn > 128 ? min_bn : 128;
+    const int tiles = ntiles(c.bn);
+    if (can_split && tiles < grid) {
+      int sp = (grid + tiles / 2) / tiles;
+      if (sp > 4) sp = 4;
+      if (sp > num_kb / 4) sp = num_kb / 4;
+      if (sp > ws_tiles / tiles) sp = ws_tiles / tiles;
+      if (sp >= 2) c.S = sp;
+    }
+  } else if (c.m_tiles > 1 && c.m_tiles * ntiles(256) < grid) {
+    // a few row tiles: no split; the width with the fewest (rounds of the grid x relative time of one tile), where a
+    // narrower tile re-reads the activation tile and uses the tensor pipe less well
+    float best = 3.0e38f;
+    for (int bn = 256; bn >= min_bn; bn >>= 1) {
+      const float cbn = bn == 256 ? 1.0f : (bn == 128 ? 0.6f : 0.42f);
+      const int rounds = (c.m_tiles * ntiles(bn) + grid - 1) / grid;
+      const float cost = (float)rounds * cbn;
+      if (cost < best - 1e-6f) {
+        best = cost;
+        c.bn = bn;
       }
     }
   }
+  c.n_tiles = ntiles(c.bn);
+  c.tiles = c.m_tiles * c.n_tiles;
   c.kb_per = (num_kb + c.S - 1) / c.S;
   c.S = (num_kb + c.kb_per - 1) / c.kb_per;
   c.total = c.tiles * c.S;
@@ -231,7 +240,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
                int n_out, int K, int32_t* status, const QkvArgs qkv, float* __restrict__ ws, int* __restrict__ counters,
-               int ws_tiles, int wide_boxes) {
+               int ws_tiles, int wide_boxes, int force_bn, int force_s) {
   // tmB*: weight maps with 64-row boxes (any tile width); tmW*: the same matrices with 128-row boxes, used for
   // 256-wide tiles so a stage is filled by fewer, larger TMA copies
   constexpr int BN_MAX = 256;
@@ -277,7 +286,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int M = *n_active;
   const int num_kb = (K + TC_BK - 1) / TC_BK;
   const int min_bn = EPI == EPI_QKV ? (qkv.dh > 64 ? 128 : 64) : (EPI == EPI_SWIGLU ? 128 : 64);
-  const TileCfg tc = choose_tiles<EPI>(M, n_out, num_kb, (int)gridDim.x, ws != nullptr, ws_tiles, min_bn);
+  TileCfg tc = choose_tiles<EPI>(M, n_out, num_kb, (int)gridDim.x, ws != nullptr, ws_tiles, min_bn);
+  if (force_bn > 0) {   // tuning aid (host environment variable): fixed tile width and split
+    tc.bn = force_bn < min_bn ? min_bn : force_bn;
+    const int ob = EPI == EPI_SWIGLU ? tc.bn >> 1 : tc.bn;
+    tc.n_tiles = (n_out + ob - 1) / ob;
+    tc.tiles = tc.m_tiles * tc.n_tiles;
+    tc.S = ws != nullptr && force_s > 0 && tc.tiles * force_s <= ws_tiles ? force_s : 1;
+    tc.kb_per = (num_kb + tc.S - 1) / tc.S;
+    tc.S = (num_kb + tc.kb_per - 1) / tc.kb_per;
+    tc.total = tc.tiles * tc.S;
+  }
   const int bn = tc.bn, S = tc.S, kb_per = tc.kb_per, m_tiles = tc.m_tiles, total = tc.total;
   const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
   const uint32_t stage_tx = (uint32_t)(A_BYTES + bn * TC_BK * 2);
@@ -373,8 +392,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int trow = quarter * 32 + lane;
       const int row = m0 + trow;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
+      const int upr = units_per_row<EPI>(bn, n0, qkv);
       if (S == 1) {
-        epilogue_row<EPI>(TmemSrc{taddr}, bn, row, M, n0, n_out, Cv, qkv);
+#pragma unroll 1
+        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, bn, row, row < M, u, n0, n_out, Cv, qkv);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(acc));
@@ -408,8 +429,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (*s_last) {
           __threadfence();
-          WsSrc src{ws + ((size_t)(t * S) * TC_BM + trow) * bn, (size_t)TC_BM * bn, S, row < M};
-          epilogue_row<EPI>(src, bn, row, M, n0, n_out, Cv, qkv);
+          // all 128 epilogue threads share the live rows of the tile: (row, unit) pairs, units of a row adjacent
+          const int live_rows = M - m0 < TC_BM ? M - m0 : TC_BM;
+          const int e_tid = (warp - 2) * 32 + lane;
+#pragma unroll 1
+          for (int i = e_tid; i < live_rows * upr; i += 128) {
+            const int r = i / upr, u = i - r * upr;
+            WsSrc src{ws + ((size_t)(t * S) * TC_BM + r) * bn, (size_t)TC_BM * bn, S};
+            epilogue_unit<EPI>(src, bn, m0 + r, true, u, n0, n_out, Cv, qkv);
+          }
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");   // s_last is rewritten by the next item
       }
@@ -497,6 +525,16 @@ static int wide_boxes() {
   return v;
 }
 
+static int force_cfg(int which) {
+  static int v[2] = {-1, -1};
+  if (v[0] < 0) {
+    v[0] = v[1] = 0;
+    const char* e = getenv("SURELOCK_GEMM_FORCE");   // tuning aid: "bn,S", e.g. "128,3"
+    if (e) sscanf(e, "%d,%d", &v[0], &v[1]);
+  }
+  return v[which];
+}
+
 template <int EPI, int STAGES>
 static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensorMap* wb, void* C,
                       const int32_t* n_active, int max_rows, int n_out, int K, int32_t* status, const QkvArgs& qkv,
@@ -511,7 +549,7 @@ static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensor
   const int grid = sm_count();   // persistent: one CTA per SM; the tile shape is chosen on the device from M
   gemm_tc_kernel<EPI, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b[0], b[1], b[2], wb[0], wb[1], wb[2], C, n_active,
                                                               n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles,
-                                                              wide_boxes());
+                                                              wide_boxes(), force_cfg(0), force_cfg(1));
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

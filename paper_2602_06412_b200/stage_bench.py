@@ -86,7 +86,8 @@ def main(argv=None):
         W = (rnd(a.n_out, a.K) * 0.02).to(torch.bfloat16)
         Cout = torch.empty((a.M, a.n_out), dtype=torch.bfloat16, device=dev)
         n = torch.tensor([a.M], dtype=torch.int32, device=dev)
-        fn = lambda: SL.surelock_gemm(A, W, Cout, n, impl=a.impl, dev_status=status)
+        wsp = torch.zeros(SL.surelock_gemm_workspace_bytes(), dtype=torch.uint8, device=dev)
+        fn = lambda: SL.surelock_gemm(A, W, Cout, n, impl=a.impl, dev_status=status, workspace=wsp)
         flops = 2.0 * a.M * a.n_out * a.K
         byts = 2.0 * (a.M * a.K + a.n_out * a.K + a.M * a.n_out)
         res.update(shape=[a.M, a.n_out, a.K], flops=flops, bytes=byts)

@@ -206,22 +206,30 @@ def test_gemm_cuda_cores(dtype, tol, M, n_out, K):
     assert (out[M:] == 3.0).all()                                    # rows beyond M untouched
 
 
+@pytest.mark.parametrize("split", [False, True])
 @pytest.mark.parametrize("M,n_out,K", [(1, 256, 64), (100, 256, 256), (128, 512, 4096), (129, 136, 200), (300, 4096, 512),
-                                       (1000, 1024, 1024), (0, 256, 256)])
-def test_gemm_tensor_cores(M, n_out, K):
+                                       (1000, 1024, 1024), (0, 256, 256), (32, 4096, 12288), (130, 1024, 8192)])
+def test_gemm_tensor_cores(M, n_out, K, split):
     g = torch.Generator().manual_seed(M * 7 + K)
     cap = M + 37
     A = torch.randn((cap, K), generator=g).to(torch.bfloat16)
     W = (torch.randn((n_out, K), generator=g) * 0.05).to(torch.bfloat16)
     out = torch.full((cap, n_out), 3.0, dtype=torch.bfloat16, device=DEV)
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    SL.surelock_gemm(A.to(DEV), W.to(DEV), out, torch.tensor([M], dtype=torch.int32, device=DEV), impl=0, dev_status=status)
+    wsp = torch.zeros(SL.surelock_gemm_workspace_bytes(), dtype=torch.uint8, device=DEV) if split else None
+    Ad, Wd, n = A.to(DEV), W.to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV)
+    SL.surelock_gemm(Ad, Wd, out, n, impl=0, dev_status=status, workspace=wsp)
     torch.cuda.synchronize()
     assert status.item() == 0
     if M:
         ref = f64(A[:M]) @ f64(W).T
         assert rel_err_rows(f64(out[:M]), ref) < 2e-2
     assert (out[M:] == 3.0).all()                                    # rows beyond M untouched
+    if split:                                                        # the workspace is left reusable, the result is deterministic
+        out2 = torch.full_like(out, 3.0)
+        SL.surelock_gemm(Ad, Wd, out2, n, impl=0, dev_status=status, workspace=wsp)
+        torch.cuda.synchronize()
+        assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
 
 
 @pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
