@@ -25,8 +25,8 @@ struct MaxSum {
 __device__ __forceinline__ MaxSum combine(const MaxSum& a, const MaxSum& b) {
   MaxSum o;
   o.m = fmaxf(a.m, b.m);
-  const float ea = a.m == -INFINITY ? 0.f : exp2f((a.m - o.m) * LOG2E);
-  const float eb = b.m == -INFINITY ? 0.f : exp2f((b.m - o.m) * LOG2E);
+  const float ea = a.m == -INFINITY ? 0.f : fast_exp2((a.m - o.m) * LOG2E);
+  const float eb = b.m == -INFINITY ? 0.f : fast_exp2((b.m - o.m) * LOG2E);
   o.s = a.s * ea + b.s * eb;
   o.am = a.m > b.m ? a.am : (b.m > a.m ? b.am : (a.am < b.am ? a.am : b.am));
   return o;
@@ -71,7 +71,7 @@ __device__ __forceinline__ void accum_maxsum(const float (&f)[VEC], int c, MaxSu
 #pragma unroll
   for (int k = 1; k < VEC; ++k) vmax = fmaxf(vmax, f[k]);
   if (vmax > st.m) {
-    st.s *= exp2f((st.m - vmax) * LOG2E);   // st.m = -inf gives 0 * 0
+    st.s *= fast_exp2((st.m - vmax) * LOG2E);   // st.m = -inf gives 0 * 0
     st.m = vmax;
     if (track_arg) {
       int a = VEC - 1;
@@ -83,18 +83,19 @@ __device__ __forceinline__ void accum_maxsum(const float (&f)[VEC], int c, MaxSu
   }
   const float mb = st.m * LOG2E;
 #pragma unroll
-  for (int k = 0; k < VEC; ++k) st.s += exp2f(fmaf(f[k], LOG2E, -mb));
+  for (int k = 0; k < VEC; ++k) st.s += fast_exp2(fmaf(f[k], LOG2E, -mb));
 }
 
-__device__ __forceinline__ float kl_g(float r) {
-  // g(r) = r - 1 + exp(-r)
-  if (fabsf(r) < 0.125f) {
-    const float r2 = r * r;
-    // r^2/2 - r^3/6 + r^4/24 - r^5/120 + r^6/720
-    return r2 * (0.5f + r * (-1.f / 6.f + r * (1.f / 24.f + r * (-1.f / 120.f + r * (1.f / 720.f)))));
-  }
-  return r + (exp2f(-r * LOG2E) - 1.f);
+// g(r) = r - 1 + exp(-r) >= 0.  Series below 1/8 (relative error < 3e-7), exp beyond.
+__device__ __forceinline__ float kl_g_series(float r) {
+  const float r2 = r * r;   // r^2/2 - r^3/6 + r^4/24 - r^5/120 + r^6/720
+  return r2 * (0.5f + r * (-1.f / 6.f + r * (1.f / 24.f + r * (-1.f / 120.f + r * (1.f / 720.f)))));
 }
+__device__ __forceinline__ float kl_g(float r) {
+  return fabsf(r) < 0.125f ? kl_g_series(r) : r + (fast_exp2(-r * LOG2E) - 1.f);
+}
+
+constexpr int KL_UNROLL = 4;   // 128-bit loads in flight per thread and row: hides HBM latency at 1024 threads per SM
 
 template <typename T>
 __global__ void __launch_bounds__(KL_THREADS)
@@ -108,21 +109,38 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
   __shared__ double s_sum[KL_THREADS / 32];
   const int M = *n_active;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = V / VEC;
   for (int r = blockIdx.x; r < M; r += gridDim.x) {
     const int pos = idx ? idx[r] : r;
     const int prow = row_of_pos_prev ? row_of_pos_prev[pos] : r;
-    const T* z = logits + (long long)r * V;
-    const T* y = (prev && prow >= 0) ? prev + (long long)prow * V : nullptr;
+    const uint4* z = reinterpret_cast<const uint4*>(logits + (long long)r * V);
+    const uint4* y = (prev && prow >= 0) ? reinterpret_cast<const uint4*>(prev + (long long)prow * V) : nullptr;
     const bool need_q = y && !prev_lse;
 
+    // sweep 1: max, sum of exponentials and argmax of the current row (and of the previous row if its lse is unknown)
     MaxSum a{-INFINITY, 0.f, 0x7fffffff}, b{-INFINITY, 0.f, 0};
-    for (int c = tid * VEC; c < V; c += KL_THREADS * VEC) {
-      float f[VEC];
-      unpack<T, VEC>(__ldg(reinterpret_cast<const uint4*>(z + c)), f);
-      accum_maxsum<VEC>(f, c, a, true);
-      if (need_q) {
-        unpack<T, VEC>(__ldg(reinterpret_cast<const uint4*>(y + c)), f);
-        accum_maxsum<VEC>(f, c, b, false);
+    for (int v0 = tid; v0 < nvec; v0 += KL_THREADS * KL_UNROLL) {
+      uint4 zz[KL_UNROLL], yy[KL_UNROLL];
+#pragma unroll
+      for (int k = 0; k < KL_UNROLL; ++k) {
+        const int vi = v0 + k * KL_THREADS;
+        if (vi < nvec) {
+          zz[k] = __ldg(z + vi);
+          if (need_q) yy[k] = __ldg(y + vi);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < KL_UNROLL; ++k) {
+        const int vi = v0 + k * KL_THREADS;
+        if (vi < nvec) {
+          float f[VEC];
+          unpack<T, VEC>(zz[k], f);
+          accum_maxsum<VEC>(f, vi * VEC, a, true);
+          if (need_q) {
+            unpack<T, VEC>(yy[k], f);
+            accum_maxsum<VEC>(f, vi * VEC, b, false);
+          }
+        }
       }
     }
     a = block_combine(a, s_ms);
@@ -135,20 +153,43 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
       lse_q = prev_lse[prow];
     }
 
+    // sweep 2: KL as a sum of non-negative terms (the current row comes from L2)
     float kl = INFINITY;
     if (y) {
       const float dl = lse_p - lse_q;
       const float lp2 = lse_p * LOG2E;
       float acc = 0.f;
-      for (int c = tid * VEC; c < V; c += KL_THREADS * VEC) {
-        float fz[VEC], fy[VEC];
-        unpack<T, VEC>(__ldg(reinterpret_cast<const uint4*>(z + c)), fz);
-        unpack<T, VEC>(__ldg(reinterpret_cast<const uint4*>(y + c)), fy);
+      for (int v0 = tid; v0 < nvec; v0 += KL_THREADS * KL_UNROLL) {
+        uint4 zz[KL_UNROLL], yy[KL_UNROLL];
 #pragma unroll
-        for (int k = 0; k < VEC; ++k) {
-          const float rr = (fz[k] - fy[k]) - dl;
-          const float p = exp2f(fmaf(fz[k], LOG2E, -lp2));
-          acc = fmaf(p, kl_g(rr), acc);
+        for (int k = 0; k < KL_UNROLL; ++k) {
+          const int vi = v0 + k * KL_THREADS;
+          if (vi < nvec) {
+            zz[k] = __ldg(z + vi);
+            yy[k] = __ldg(y + vi);
+          }
+        }
+#pragma unroll
+        for (int k = 0; k < KL_UNROLL; ++k) {
+          const int vi = v0 + k * KL_THREADS;
+          if (vi < nvec) {
+            float fz[VEC], fy[VEC], rr[VEC];
+            unpack<T, VEC>(zz[k], fz);
+            unpack<T, VEC>(yy[k], fy);
+            float rmax = 0.f;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) {
+              rr[e] = (fz[e] - fy[e]) - dl;
+              rmax = fmaxf(rmax, fabsf(rr[e]));
+            }
+            if (rmax < 0.125f) {          // whole vector in the series range: no per-element branch
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) acc = fmaf(fast_exp2(fmaf(fz[e], LOG2E, -lp2)), kl_g_series(rr[e]), acc);
+            } else {
+#pragma unroll
+              for (int e = 0; e < VEC; ++e) acc = fmaf(fast_exp2(fmaf(fz[e], LOG2E, -lp2)), kl_g(rr[e]), acc);
+            }
+          }
         }
       }
       double d = (double)acc;
@@ -171,6 +212,220 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
   }
 }
 
+// ---- bf16 rows at full HBM rate -------------------------------------------------------------------------------
+// Same computation as the generic kernel above, arranged for the instruction budget of a B200 SM: at the HBM rate a
+// row pair (2 x V bf16) leaves ~20 issue slots per vocabulary entry, so the arithmetic runs on packed fp32x2
+// instructions (two entries per FFMA2/FADD2/FMUL2), the row maximum is taken on packed bf16 pairs, the series/exp
+// choice of g is made per 8-entry vector from sum(r^2), and the next vectors are loaded while the current ones are
+// processed.
+constexpr int KLF_THREADS = 256;
+
+__device__ __forceinline__ float2 unpack_pair(unsigned w) {   // (low bf16, high bf16) -> two floats
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+__device__ __forceinline__ float vec_max_bf16(const uint4& v) {
+  const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.x), *reinterpret_cast<const __nv_bfloat162*>(&v.y));
+  const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.z), *reinterpret_cast<const __nv_bfloat162*>(&v.w));
+  const __nv_bfloat162 m = __hmax2(a, b);
+  const unsigned w = *reinterpret_cast<const unsigned*>(&m);
+  return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+
+struct MaxSum2 {
+  float m;
+  float2 s;   // two partial sums (even / odd entries), added at the end
+  int am;
+};
+
+__device__ __forceinline__ void accum_maxsum_bf16(const uint4& v, int c, MaxSum2& st, bool track_arg) {
+  const float vmax = vec_max_bf16(v);
+  if (vmax > st.m) {
+    const float sc = fast_exp2((st.m - vmax) * LOG2E);   // st.m = -inf: 0
+    st.s.x *= sc;
+    st.s.y *= sc;
+    st.m = vmax;
+    if (track_arg) {
+      const unsigned w[4] = {v.x, v.y, v.z, v.w};
+      int a = 7;
+#pragma unroll
+      for (int k = 3; k >= 0; --k) {
+        if (__uint_as_float(w[k] & 0xffff0000u) == vmax) a = 2 * k + 1;
+        if (__uint_as_float(w[k] << 16) == vmax) a = 2 * k;
+      }
+      st.am = c + a;
+    }
+  }
+  const float mb = -st.m * LOG2E;
+  const float2 l2 = make_float2(LOG2E, LOG2E), mb2 = make_float2(mb, mb);
+  const unsigned w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const float2 t = __ffma2_rn(unpack_pair(w[k]), l2, mb2);
+    st.s = __fadd2_rn(st.s, make_float2(fast_exp2(t.x), fast_exp2(t.y)));
+  }
+}
+
+// sum_v p_v g(r_v) over the 8 entries of one vector pair
+__device__ __forceinline__ float2 kl_vec_bf16(const uint4& zv, const uint4& yv, float dl, float lp2, float2 acc) {
+  const unsigned zw[4] = {zv.x, zv.y, zv.z, zv.w}, yw[4] = {yv.x, yv.y, yv.z, yv.w};
+  const float2 ndl = make_float2(-dl, -dl), l2 = make_float2(LOG2E, LOG2E), nlp = make_float2(-lp2, -lp2);
+  const float2 neg1 = make_float2(-1.f, -1.f);
+  float2 z[4], r[4], r2[4];
+  float2 ss = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    z[k] = unpack_pair(zw[k]);
+    const float2 y = unpack_pair(yw[k]);
+    r[k] = __fadd2_rn(__ffma2_rn(y, neg1, z[k]), ndl);     // (z - y) - dl
+    r2[k] = __fmul2_rn(r[k], r[k]);
+    ss = __fadd2_rn(ss, r2[k]);
+  }
+  if (ss.x + ss.y < 0.015625f) {                             // every |r| < 1/8: series, two entries per instruction
+    const float2 c2 = make_float2(0.5f, 0.5f), c3 = make_float2(-1.f / 6.f, -1.f / 6.f);
+    const float2 c4 = make_float2(1.f / 24.f, 1.f / 24.f), c5 = make_float2(-1.f / 120.f, -1.f / 120.f);
+    const float2 c6 = make_float2(1.f / 720.f, 1.f / 720.f);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float2 h = __ffma2_rn(r[k], c6, c5);
+      h = __ffma2_rn(r[k], h, c4);
+      h = __ffma2_rn(r[k], h, c3);
+      h = __ffma2_rn(r[k], h, c2);
+      const float2 t = __ffma2_rn(z[k], l2, nlp);
+      const float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+      acc = __ffma2_rn(p, __fmul2_rn(r2[k], h), acc);
+    }
+  } else if (ss.x + ss.y < 0.25f) {                          // every |r| < 1/2: series up to r^9 (relative error < 3e-9)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      float2 h = __ffma2_rn(r[k], make_float2(-1.f / 362880.f, -1.f / 362880.f), make_float2(1.f / 40320.f, 1.f / 40320.f));
+      h = __ffma2_rn(r[k], h, make_float2(-1.f / 5040.f, -1.f / 5040.f));
+      h = __ffma2_rn(r[k], h, make_float2(1.f / 720.f, 1.f / 720.f));
+      h = __ffma2_rn(r[k], h, make_float2(-1.f / 120.f, -1.f / 120.f));
+      h = __ffma2_rn(r[k], h, make_float2(1.f / 24.f, 1.f / 24.f));
+      h = __ffma2_rn(r[k], h, make_float2(-1.f / 6.f, -1.f / 6.f));
+      h = __ffma2_rn(r[k], h, make_float2(0.5f, 0.5f));
+      const float2 t = __ffma2_rn(z[k], l2, nlp);
+      const float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+      acc = __ffma2_rn(p, __fmul2_rn(r2[k], h), acc);
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const float2 t = __ffma2_rn(z[k], l2, nlp);
+      acc.x = fmaf(fast_exp2(t.x), kl_g(r[k].x), acc.x);
+      acc.y = fmaf(fast_exp2(t.y), kl_g(r[k].y), acc.y);
+    }
+  }
+  return acc;
+}
+
+__global__ void __launch_bounds__(KLF_THREADS, 3)
+softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restrict__ prev,
+                            const int32_t* __restrict__ row_of_pos_prev, const float* __restrict__ prev_lse,
+                            const int32_t* __restrict__ idx, const int32_t* __restrict__ n_active, int V,
+                            const uint8_t* __restrict__ mask_state, uint8_t* __restrict__ lock_mask, float kl_eps,
+                            float* __restrict__ kl_out, float* __restrict__ conf_out, int32_t* __restrict__ argmax_out,
+                            float* __restrict__ lse_out) {
+  __shared__ float s_m[KLF_THREADS / 32], s_s[KLF_THREADS / 32];
+  __shared__ int s_a[KLF_THREADS / 32];
+  __shared__ double s_sum[KLF_THREADS / 32];
+  const int M = *n_active;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int nvec = V >> 3;
+  constexpr int STEP = 2 * KLF_THREADS;   // two vectors per thread and iteration
+
+  auto block_maxsum = [&](MaxSum2 st) -> MaxSum {
+    MaxSum v{st.m, st.s.x + st.s.y, st.am};
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      MaxSum t;
+      t.m = __shfl_xor_sync(0xffffffffu, v.m, o);
+      t.s = __shfl_xor_sync(0xffffffffu, v.s, o);
+      t.am = __shfl_xor_sync(0xffffffffu, v.am, o);
+      v = combine(v, t);
+    }
+    __syncthreads();
+    if (lane == 0) { s_m[warp] = v.m; s_s[warp] = v.s; s_a[warp] = v.am; }
+    __syncthreads();
+    MaxSum r{s_m[0], s_s[0], s_a[0]};
+    for (int w = 1; w < KLF_THREADS / 32; ++w) r = combine(r, MaxSum{s_m[w], s_s[w], s_a[w]});
+    return r;
+  };
+
+  for (int r = blockIdx.x; r < M; r += gridDim.x) {
+    const int pos = idx ? idx[r] : r;
+    const int prow = row_of_pos_prev ? row_of_pos_prev[pos] : r;
+    const uint4* z = reinterpret_cast<const uint4*>(logits + (long long)r * V);
+    const uint4* y = (prev && prow >= 0) ? reinterpret_cast<const uint4*>(prev + (long long)prow * V) : nullptr;
+    const bool need_q = y && !prev_lse;
+
+    // sweep 1 (current row; the previous row only if its log-sum-exp was not kept), next vectors prefetched
+    MaxSum2 a{-INFINITY, make_float2(0.f, 0.f), 0x7fffffff}, b{-INFINITY, make_float2(0.f, 0.f), 0};
+    {
+      const uint4 zero = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // eight times -inf
+      uint4 c0 = tid < nvec ? __ldg(z + tid) : zero;
+      uint4 c1 = tid + KLF_THREADS < nvec ? __ldg(z + tid + KLF_THREADS) : zero;
+      for (int v0 = tid; v0 < nvec; v0 += STEP) {
+        const int n0 = v0 + STEP, n1 = n0 + KLF_THREADS;
+        const uint4 p0 = n0 < nvec ? __ldg(z + n0) : zero;
+        const uint4 p1 = n1 < nvec ? __ldg(z + n1) : zero;
+        accum_maxsum_bf16(c0, v0 * 8, a, true);
+        if (v0 + KLF_THREADS < nvec) accum_maxsum_bf16(c1, (v0 + KLF_THREADS) * 8, a, true);
+        c0 = p0;
+        c1 = p1;
+      }
+      if (need_q) {
+        for (int v0 = tid; v0 < nvec; v0 += KLF_THREADS) accum_maxsum_bf16(__ldg(y + v0), v0 * 8, b, false);
+      }
+    }
+    const MaxSum ra = block_maxsum(a);
+    const float lse_p = ra.m + log2f(ra.s) * LN2;
+    float lse_q = 0.f;
+    if (need_q) {
+      const MaxSum rb = block_maxsum(b);
+      lse_q = rb.m + log2f(rb.s) * LN2;
+    } else if (y) {
+      lse_q = prev_lse[prow];
+    }
+
+    // sweep 2: KL as a sum of non-negative terms (the current row comes back from L2)
+    float kl = INFINITY;
+    if (y) {
+      const float dl = lse_p - lse_q, lp2 = lse_p * LOG2E;
+      float2 acc = make_float2(0.f, 0.f);
+      const uint4 zero = make_uint4(0, 0, 0, 0);
+      uint4 cz0 = tid < nvec ? __ldg(z + tid) : zero, cy0 = tid < nvec ? __ldg(y + tid) : zero;
+      uint4 cz1 = zero, cy1 = zero;
+      if (tid + KLF_THREADS < nvec) { cz1 = __ldg(z + tid + KLF_THREADS); cy1 = __ldg(y + tid + KLF_THREADS); }
+      for (int v0 = tid; v0 < nvec; v0 += STEP) {
+        const int n0 = v0 + STEP, n1 = n0 + KLF_THREADS;
+        uint4 pz0 = zero, py0 = zero, pz1 = zero, py1 = zero;
+        if (n0 < nvec) { pz0 = __ldg(z + n0); py0 = __ldg(y + n0); }
+        if (n1 < nvec) { pz1 = __ldg(z + n1); py1 = __ldg(y + n1); }
+        acc = kl_vec_bf16(cz0, cy0, dl, lp2, acc);
+        if (v0 + KLF_THREADS < nvec) acc = kl_vec_bf16(cz1, cy1, dl, lp2, acc);
+        cz0 = pz0; cy0 = py0; cz1 = pz1; cy1 = py1;
+      }
+      double d = (double)acc.x + (double)acc.y;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+      __syncthreads();
+      if (lane == 0) s_sum[warp] = d;
+      __syncthreads();
+      d = 0.0;
+      for (int w = 0; w < KLF_THREADS / 32; ++w) d += s_sum[w];
+      kl = (float)d;
+    }
+    if (tid == 0) {
+      kl_out[r] = kl;
+      conf_out[r] = 1.f / ra.s;          // exp(max - lse)
+      argmax_out[r] = ra.am;
+      if (lse_out) lse_out[r] = lse_p;
+      if (mask_state[pos] == 0 && kl <= kl_eps) lock_mask[pos] = 1;
+    }
+  }
+}
+
 int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
                            const float* prev_lse, const int32_t* idx, const int32_t* n_active, int max_rows, int vocab,
                            int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
@@ -180,11 +435,14 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
   int g = sm_count() * 2;
   if (g > max_rows) g = max_rows;
   if (g < 1) g = 1;
-  if (dtype == SL_BF16)
-    softmax_kl_sure_kernel<bf16><<<g, KL_THREADS, 0, st>>>((const bf16*)logits, (const bf16*)prev_logits, row_of_pos_prev,
-                                                          prev_lse, idx, n_active, vocab, mask_state, lock_mask, kl_eps,
-                                                          kl, conf, argmax, lse_out);
-  else
+  if (dtype == SL_BF16) {
+    int gb = sm_count() * 3;
+    if (gb > max_rows) gb = max_rows;
+    if (gb < 1) gb = 1;
+    softmax_kl_sure_bf16_kernel<<<gb, KLF_THREADS, 0, st>>>((const bf16*)logits, (const bf16*)prev_logits, row_of_pos_prev,
+                                                             prev_lse, idx, n_active, vocab, mask_state, lock_mask, kl_eps,
+                                                             kl, conf, argmax, lse_out);
+  } else
     softmax_kl_sure_kernel<float><<<g, KL_THREADS, 0, st>>>((const float*)logits, (const float*)prev_logits,
                                                            row_of_pos_prev, prev_lse, idx, n_active, vocab, mask_state,
                                                            lock_mask, kl_eps, kl, conf, argmax, lse_out);

@@ -124,11 +124,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ float fast_exp2(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
 
 // Split-K workspace of the GEMM: room for `tiles` fp32 partial tiles of 128 x 256 and one arrival counter per output
 // tile (zero-initialised once; the kernel leaves them zero).  ws == nullptr disables split-K.
