@@ -7,8 +7,10 @@
 //   warp 0    TMA producer: Q tile once, then K and V blocks (two stages each), token-major cache rows, 128-byte swizzle;
 //   warp 1    one thread issues S = Q K^T (tcgen05.mma, 128x128xd_h, accumulator in tensor memory, two S buffers so
 //             S of block j+1 is computed while block j is in the softmax) and O += P V (V is the MN-major operand);
-//   warps 2-5 softmax: each thread owns one query row: tcgen05.ld its 128 scores, online max / sum in fp32 with the
-//             1/sqrt(d_h) scale folded into an exp2, P written as bf16 into swizzled shared memory for the second MMA.
+//   warps 2-9 softmax: two threads share one query row, 64 of the block's 128 scores each (the exponentials of a block
+//             are bound by the SM's 16 special-function results per clock, so all four schedulers carry two softmax
+//             warps): tcgen05.ld the scores, online max / sum in fp32 with the 1/sqrt(d_h) scale folded into an exp2
+//             (row maximum exchanged through shared memory), P written as bf16 into swizzled shared memory.
 //             O stays in tensor memory; it is rescaled (tcgen05.ld / st) only when a row's running maximum grows by
 //             more than 2^8, so after the first blocks the correction is almost never taken.  The final O / l is
 //             stored as bf16.
@@ -17,7 +19,7 @@
 
 namespace sl {
 
-constexpr int AT_THREADS = 192;
+constexpr int AT_THREADS = 320;   // TMA warp, MMA warp, 8 softmax warps (two per tensor-memory lane quarter)
 constexpr int AT_BQ = 128, AT_BKV = 128;
 constexpr int AT_MAX_B = 1024;
 
@@ -41,12 +43,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint8_t* sV = sK + 2 * KV_BYTES;                     // 2 stages
   uint8_t* sP = sV + 2 * KV_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
-  // q_full, q_free, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], s_free[2], p_full, p_free, o_free
+  // q_full, q_free, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], s_free[2], p_full, p_free, o_free,
+  // x_max[2], x_sum (the two threads of a row meet here; mbarriers, so that these waits are bounded too)
   enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
-         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, NUM_BARS };
+         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, X_MAX, X_SUM = X_MAX + 2, NUM_BARS };
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  int* s_prefix = reinterpret_cast<int*>(s_tmem + 2);   // [B+1] work-item prefix per sequence
+  float* s_xmax = reinterpret_cast<float*>(s_tmem + 2);    // [2 parities][2 halves][128 rows] partial row maxima
+  float* s_xsum = s_xmax + 512;                          // [2 halves][128 rows] partial row sums at the end of an item
+  int* s_prefix = reinterpret_cast<int*>(s_xsum + 256);  // [B+1] work-item prefix per sequence
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -55,8 +60,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   if (threadIdx.x == 0) {
     for (int i = 0; i < NUM_BARS; ++i) {
       uint32_t cnt = 1;
-      if (i == S_FREE || i == S_FREE + 1 || i == O_FREE) cnt = 4;
-      if (i == P_FULL) cnt = 128;
+      if (i == S_FREE || i == S_FREE + 1 || i == O_FREE) cnt = 8;
+      if (i == P_FULL || i == X_MAX || i == X_MAX + 1 || i == X_SUM) cnt = 256;
       mbar_init(bar(i), cnt);
     }
     *s_abort = 0;
@@ -176,11 +181,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
   } else {
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;                    // which 64 of the block's 128 keys (and which half of O)
     const int trow = quarter * 32 + lane;                // query row of this thread inside the tile
     const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
-    uint32_t g = 0;
+    constexpr int OH = DH / 2;                           // O columns per thread
+    uint32_t g = 0, it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
       int b, h, row0, nrows;
       decode(w, b, h, row0, nrows);
       float m_used = 0.f, l = 0.f;
@@ -191,22 +198,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), ph, s_abort));
         if (!ok) break;
         tc_fence_after();
-        uint32_t s[128];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tc_ld32(tmem_base + tlane + sb * 128 + c * 32, s + 32 * c);
+        uint32_t s[64];
+        tc_ld32(tmem_base + tlane + sb * 128 + half * 64, s);
+        tc_ld32(tmem_base + tlane + sb * 128 + half * 64 + 32, s + 32);
         tc_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(S_FREE + sb));
-        const int nvalid = N - j * AT_BKV;               // keys of this block that exist
+        const int nvalid = N - j * AT_BKV - half * 64;   // keys of this thread's 64 that exist
         float mx = -INFINITY;
+        if (nvalid >= 64) {
 #pragma unroll
-        for (int c = 0; c < 128; ++c) {
-          float v = __uint_as_float(s[c]) * scale_log2;
-          if (c >= nvalid) v = -INFINITY;
-          s[c] = __float_as_uint(v);
-          mx = fmaxf(mx, v);
+          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 64; ++c) {
+            if (c >= nvalid) s[c] = 0xff800000u;         // -inf
+            mx = fmaxf(mx, __uint_as_float(s[c]));
+          }
         }
+        // the two threads of a row exchange their partial maxima (buffer alternates with the block parity)
+        float* xm = s_xmax + (gj & 1) * 256;
+        xm[half * 128 + trow] = mx;
+        mbar_arrive(bar(X_MAX + sb));
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(X_MAX + sb), ph, s_abort));
+        if (!ok) break;
+        mx = fmaxf(mx, xm[(half ^ 1) * 128 + trow]) * scale_log2;
         bool need = false;
         float corr = 1.f;
         if (j == 0) {
@@ -217,42 +234,42 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           m_used = mx;
           l *= corr;
         }
-        float sum = 0.f;
-        uint32_t pk[64];
+        float2 sum2 = make_float2(0.f, 0.f);
+        uint32_t pk[32];
+        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
 #pragma unroll
-        for (int c = 0; c < 128; c += 2) {
-          const float p0 = fast_exp2(__uint_as_float(s[c]) - m_used);
-          const float p1 = fast_exp2(__uint_as_float(s[c + 1]) - m_used);
-          sum += p0 + p1;
-          pk[c >> 1] = pack_bf16(p0, p1);
+        for (int c = 0; c < 64; c += 2) {
+          const float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+          const float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
+          sum2 = __fadd2_rn(sum2, p);
+          pk[c >> 1] = pack_bf16(p.x, p.y);
         }
-        l += sum;
+        l += sum2.x + sum2.y;
         if (gj > 0) {
           ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (gj - 1) & 1, s_abort));   // P V of the previous block done
           if (!ok) break;
         }
-        if (j > 0 && __any_sync(0xffffffffu, need)) {
+        if (j > 0 && __any_sync(0xffffffffu, need)) {      // both threads of a row take the same decision
           tc_fence_after();
 #pragma unroll 1
-          for (int c = 0; c < DH; c += 32) {
+          for (int c = 0; c < OH; c += 32) {
             uint32_t ov[32];
-            tc_ld32(tmem_base + tlane + O_COL + c, ov);
+            tc_ld32(tmem_base + tlane + O_COL + half * OH + c, ov);
             tc_wait_ld();
 #pragma unroll
             for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * corr);
-            tc_st32(tmem_base + tlane + O_COL + c, ov);
+            tc_st32(tmem_base + tlane + O_COL + half * OH + c, ov);
           }
           tc_wait_st();
         }
-        // P row -> shared memory, 128-byte swizzle: 16-byte chunk c of row r sits at chunk position c ^ (r & 7)
+        // P row -> shared memory, 128-byte swizzle: 16-byte chunk c of row r sits at chunk position c ^ (r & 7);
+        // this thread's 64 keys are exactly one 128-byte row of slab `half`
         {
-          uint8_t* prow = sP + (trow >> 3) * 1024 + (trow & 7) * 128;
+          uint8_t* prow = sP + half * SLAB_BYTES + (trow >> 3) * 1024 + (trow & 7) * 128;
 #pragma unroll
-          for (int ch = 0; ch < 16; ++ch) {
-            const int slab = ch >> 3, c = ch & 7;
-            *reinterpret_cast<uint4*>(prow + slab * SLAB_BYTES + ((c ^ (trow & 7)) << 4)) =
-                make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
-          }
+          for (int c = 0; c < 8; ++c)
+            *reinterpret_cast<uint4*>(prow + ((c ^ (trow & 7)) << 4)) =
+                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         }
         fence_async_smem();
         tc_fence_before();
@@ -260,15 +277,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       if (!ok) break;
       g += nblk;
+      // row sum: add the partner's half
+      s_xsum[half * 128 + trow] = l;
+      mbar_arrive(bar(X_SUM));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(X_SUM), it & 1, s_abort));
+      if (!ok) break;
+      l += s_xsum[(half ^ 1) * 128 + trow];
       ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (g - 1) & 1, s_abort));       // last P V of the item done
       if (!ok) break;
       tc_fence_after();
       const float inv = 1.f / l;
-      bf16* orow = o + ((long long)(row0 + trow) * H + h) * DH;
+      bf16* orow = o + ((long long)(row0 + trow) * H + h) * DH + half * OH;
 #pragma unroll 1
-      for (int c = 0; c < DH; c += 32) {
+      for (int c = 0; c < OH; c += 32) {
         uint32_t ov[32];
-        tc_ld32(tmem_base + tlane + O_COL + c, ov);
+        tc_ld32(tmem_base + tlane + O_COL + half * OH + c, ov);
         tc_wait_ld();
         if (trow < nrows) {
 #pragma unroll
@@ -301,7 +324,7 @@ template <int DH>
 static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
                      int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
   constexpr int SLABS = DH / 64;
-  const int smem = 5 * SLABS * 128 * 128 + 2 * 128 * 128 + 1024 + 512 + 4 * (B + 2);
+  const int smem = 5 * SLABS * 128 * 128 + 2 * 128 * 128 + 1024 + 512 + 3072 + 4 * (B + 2);
   static int attr_smem = 0;
   if (smem > attr_smem) {
     SL_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
