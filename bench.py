@@ -30,7 +30,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2602_06412_b200 import inputs  # noqa: E402
+from paper_2602_06412_b200 import dist_util, inputs  # noqa: E402
 
 WORKLOADS = {
     # name: (model shape, batch, N, prompt length, lock pattern)
@@ -117,7 +117,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_sample(cfg, B, N, rows=128, head_rows=32):
+def oracle_sample(cfg, B, N, rows=512, head_rows=128, repeat=3):
     """Times the CPU oracle, as it stands, on a bounded sample of the workload: ONE of the L blocks on `rows`
     active rows of one sequence against an N-row cache, plus final norm + LM head + softmax/KL/lock test on
     `head_rows` rows; the block time is scaled by L.  Returns (tokens_per_s, seconds, threads, description)."""
@@ -131,12 +131,14 @@ def oracle_sample(cfg, B, N, rows=128, head_rows=32):
     lw = {k: v.float().numpy() for k, v in inputs.make_layer_weights(cfg, 0, 1).items()}
     g = np.random.default_rng(0)
     d, H, dh, V = cfg["d_model"], cfg["n_heads"], cfg["head_dim"], cfg["vocab"]
+    rows = min(rows, N)
     x = g.standard_normal((rows, d))
     pos = np.sort(g.choice(N, size=rows, replace=False))
     Kc, Vc = g.standard_normal((N, H, dh)), g.standard_normal((N, H, dh))
     t0 = time.perf_counter()
-    O.layer_rows(oc, lw, x, pos, Kc, Vc)
-    t_layer = time.perf_counter() - t0
+    for _ in range(repeat):
+        O.layer_rows(oc, lw, x, pos, Kc, Vc)
+    t_layer = (time.perf_counter() - t0) / repeat
     head = inputs._normal((V, d), 0.02, 3, torch.bfloat16, "cpu").float().numpy()
     xh = g.standard_normal((head_rows, d))
     zprev = g.standard_normal((head_rows, V)) * 3
@@ -148,20 +150,29 @@ def oracle_sample(cfg, B, N, rows=128, head_rows=32):
     per_row = cfg["n_layers"] * t_layer / rows + t_head / head_rows
     desc = (f"1 of {cfg['n_layers']} blocks on {rows} active rows of one N={N} sequence (x{cfg['n_layers']}) + LM head/"
             f"softmax-KL on {head_rows} rows; extrapolated per row")
-    return 1.0 / per_row, t_layer + t_head, threads, desc
+    return 1.0 / per_row, repeat * t_layer + t_head, threads, desc
 
 
-def run_reference(args, cfgname, B, N):
+def workload_config(args, cfgname, cfg, B, N, pattern, M=None):
+    """The `config` object, shared by both arms so that they describe the same workload."""
+    return {"workload": f"{args.workload}: full {cfgname} stack ({cfg['n_layers']} layers, d={cfg['d_model']}, "
+                        f"vocab={cfg['vocab']}), batch {B}, N={N}, M/N={args.ratio} ragged per sequence, "
+                        f"{pattern} lock pattern", "batch": B, "seq_len": N, "active_rows": M,
+            "l2": "inputs larger than L2 (every step streams all weights, %.1f GB)" % (weight_bytes(cfg) / 1e9),
+            "multi_gpu": "replicas only (one independent batch per rank, no collective)"}
+
+
+def run_reference(args, cfgname, B, N, pattern):
     cfg = inputs.model_shape(cfgname)
     vals, secs = [], 0.0
     for _ in range(max(1, min(args.steps, 3))):
-        v, s, threads, desc = oracle_sample(cfg, B, N, rows=64, head_rows=16)
+        v, s, threads, desc = oracle_sample(cfg, B, N, rows=128, head_rows=32, repeat=1)
         vals.append(v); secs += s
     v = float(np.median(vals))
     return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": len(vals), "warmup": 0, "ms_per_step": 1e3 * secs / len(vals), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": args.workload, "batch": B, "seq_len": N, "note": "CPU oracle, bounded sample per step"},
+            "config": dict(workload_config(args, cfgname, cfg, B, N, pattern), note="CPU oracle, bounded sample per step"),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
@@ -178,14 +189,12 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    rank = int(os.environ.get("RANK", 0))
-    world = int(os.environ.get("WORLD_SIZE", 1))
-    local = int(os.environ.get("LOCAL_RANK", 0))
+    rank, world, local = dist_util.env_rank_world()
     cfgname, B, N, n_prompt, pattern = WORKLOADS[args.workload]
 
     if args.impl == "reference":
         if rank == 0:
-            print(json.dumps(run_reference(args, cfgname, B, N)), flush=True)
+            print(json.dumps(run_reference(args, cfgname, B, N, pattern)), flush=True)
         return 0
 
     from paper_2602_06412_b200 import binding as SL
@@ -200,7 +209,7 @@ def main():
     args.warmup = max(args.warmup, 3)
     cfg = inputs.model_shape(cfgname)
     dtype = torch.bfloat16 if cfgname != "tiny" else torch.float32
-    seed = 1234 + rank
+    seed = dist_util.replica_seed(1234, rank)
     w = inputs.make_weights(cfg, seed, dtype=dtype, device=dev)
     ctx = SL.surelock_init(cfg, w, N, B)
     tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], seed)
@@ -244,18 +253,14 @@ def main():
         barrier()
         if sampler:
             sampler.__exit__()
-        ms = e0.elapsed_time(e1) / steps
-        if world > 1:
-            t = torch.tensor([ms], device=dev)
-            torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = dist_util.max_over_ranks(e0.elapsed_time(e1) / steps, dev)
         return M, ms, launches, lock0
 
     pk, pk_kind = peaks()
     sampler = ClockSampler(local)
     M, ms, launches, lock0 = timed(args.ratio, args.steps, args.warmup, sampler)
     clocks = sampler.summary()
-    value = world * M / (ms * 1e-3)
+    value = dist_util.sum_over_ranks(M, dev) / (ms * 1e-3)    # all replicas' rows / slowest replica's time
 
     # per-kernel-class breakdown of the same step (separate pass: events around every launch)
     SL.surelock_set_option(ctx, "time_kernels", 1)
@@ -303,12 +308,8 @@ def main():
         lk.copy_(lk0)
         SL.surelock_step_host(ctx, tk, mk, lk, 1e-3, n_h, ai, klh, cfh, amh)
     torch.cuda.synchronize()
-    e2e_ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e = dict(value=world * int(n_h.item()) / (e2e_ms * 1e-3), unit="tokens/s", ms_per_step=e2e_ms,
+    e2e_ms = dist_util.max_over_ranks((time.perf_counter() - t0) * 1e3 / args.steps, dev)
+    e2e = dict(value=dist_util.sum_over_ranks(int(n_h.item()), dev) / (e2e_ms * 1e-3), unit="tokens/s", ms_per_step=e2e_ms,
                h2d_bytes_per_step=R * 4 + R + R, d2h_bytes_per_step=R + 4 + 4 * R * 4)
 
     sweep = []
@@ -317,7 +318,8 @@ def main():
             Ms, mss, _, _ = timed(r, max(2, args.steps // 2), 3)
             ideal_ms = max(Ms * gemm_flops_per_row(cfg) / (pk["bf16_tflops_sustained"] * 1e12),
                            wbytes / (pk["hbm_gbs"] * 1e9)) * 1e3
-            sweep.append(dict(ratio=r, M=Ms, ms_per_step=round(mss, 4), tokens_per_s=round(world * Ms / (mss * 1e-3), 1),
+            sweep.append(dict(ratio=r, M=Ms, ms_per_step=round(mss, 4),
+                              tokens_per_s=round(dist_util.sum_over_ranks(Ms, dev) / (mss * 1e-3), 1),
                               gemm_ideal_ms=round(ideal_ms, 4), frac_of_gemm_ideal=round(ideal_ms / mss, 4)))
 
     status = SL.surelock_status_poll(ctx)
@@ -325,11 +327,7 @@ def main():
         "metric": "active_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if dtype == torch.bfloat16 else "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: full {cfgname} stack ({cfg['n_layers']} layers, d={cfg['d_model']}, "
-                               f"vocab={cfg['vocab']}), batch {B}, N={N}, M/N={args.ratio} ragged per sequence (M={M}), "
-                               f"{pattern} lock pattern", "batch": B, "seq_len": N, "active_rows": M,
-                   "l2": "inputs larger than L2 (every step streams all weights, %.1f GB)" % (wbytes / 1e9),
-                   "multi_gpu": "replicas only (one independent batch per rank, no collective)"},
+        "config": workload_config(args, cfgname, cfg, B, N, pattern, M),
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "roofline": roof, "kernels": kernels, "sweep": sweep,
         "device_status": status,
     }
