@@ -10,11 +10,14 @@
 //   warps 2-9 softmax: two threads share one query row, 64 of the block's 128 scores each (the exponentials of a block
 //             are bound by the SM's 16 special-function results per clock, so all four schedulers carry two softmax
 //             warps): tcgen05.ld the scores, online max / sum in fp32 with the 1/sqrt(d_h) scale folded into an exp2
-//             (row maximum exchanged through shared memory), P written as bf16 into swizzled shared memory.
+//             (each thread also reads its partner's 64 scores for the row maximum: cheaper than an exchange),
+//             P written as bf16 into swizzled shared memory.
 //             O stays in tensor memory; it is rescaled (tcgen05.ld / st) only when a row's running maximum grows by
 //             more than 2^8, so after the first blocks the correction is almost never taken.  The final O / l is
 //             stored as bf16.
 // Keys beyond N in the last block are masked to -inf.  All waits are bounded (SL_DEV_ATTN_TIMEOUT).
+#include <stdio.h>
+
 #include "tc_common.cuh"
 
 namespace sl {
@@ -27,7 +30,7 @@ template <int DH>
 __global__ void __launch_bounds__(AT_THREADS, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
-                    bf16* __restrict__ o, float scale_log2, int32_t* status) {
+                    bf16* __restrict__ o, float scale_log2, int32_t* status, unsigned long long* prof) {
   constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
   constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
   constexpr int Q_BYTES = SLABS * SLAB_BYTES;
@@ -44,13 +47,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint8_t* sP = sV + 2 * KV_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
   // q_full, q_free, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], s_free[2], p_full, p_free, o_free,
-  // x_max[2], x_sum (the two threads of a row meet here; mbarriers, so that these waits are bounded too)
+  // x_sum (the two threads of a row add their partial sums here; an mbarrier, so that this wait is bounded too)
   enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
-         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, X_MAX, X_SUM = X_MAX + 2, NUM_BARS };
+         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, X_SUM, NUM_BARS };
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  float* s_xmax = reinterpret_cast<float*>(s_tmem + 2);    // [2 parities][2 halves][128 rows] partial row maxima
-  float* s_xsum = s_xmax + 512;                          // [2 halves][128 rows] partial row sums at the end of an item
+  float* s_xsum = reinterpret_cast<float*>(s_tmem + 2);    // [2 halves][128 rows] partial row sums at the end of an item
   int* s_prefix = reinterpret_cast<int*>(s_xsum + 256);  // [B+1] work-item prefix per sequence
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -61,7 +63,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     for (int i = 0; i < NUM_BARS; ++i) {
       uint32_t cnt = 1;
       if (i == S_FREE || i == S_FREE + 1 || i == O_FREE) cnt = 8;
-      if (i == P_FULL || i == X_MAX || i == X_MAX + 1 || i == X_SUM) cnt = 256;
+      if (i == P_FULL || i == X_SUM) cnt = 8;   // one elected arrival per softmax warp
       mbar_init(bar(i), cnt);
     }
     *s_abort = 0;
@@ -187,6 +189,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     constexpr int OH = DH / 2;                           // O columns per thread
     uint32_t g = 0, it = 0;
     bool ok = true;
+#ifdef ATT_PROFILE
+    unsigned long long tp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t0 = clock64(), t1;
+#define ATT_T(i) { t1 = clock64(); tp[i] += t1 - t0; t0 = t1; }
+#else
+#define ATT_T(i)
+#endif
     for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
       int b, h, row0, nrows;
       decode(w, b, h, row0, nrows);
@@ -195,35 +203,55 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t gj = g + j;
         const int sb = gj & 1;
         const uint32_t ph = (gj >> 1) & 1;
+        ATT_T(0)
         ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), ph, s_abort));
         if (!ok) break;
+        ATT_T(1)
         tc_fence_after();
-        uint32_t s[64];
+        // this thread's 64 scores, and the partner's 64 as well: the row maximum needs all 128, and reading them from
+        // tensor memory in the same batch is cheaper than an exchange through shared memory
+        uint32_t s[64], t[64];
         tc_ld32(tmem_base + tlane + sb * 128 + half * 64, s);
         tc_ld32(tmem_base + tlane + sb * 128 + half * 64 + 32, s + 32);
+        tc_ld32(tmem_base + tlane + sb * 128 + (half ^ 1) * 64, t);
+        tc_ld32(tmem_base + tlane + sb * 128 + (half ^ 1) * 64 + 32, t + 32);
         tc_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(S_FREE + sb));
+        ATT_T(2)
         const int nvalid = N - j * AT_BKV - half * 64;   // keys of this thread's 64 that exist
-        float mx = -INFINITY;
-        if (nvalid >= 64) {
+        if (nvalid < 64) {
 #pragma unroll
-          for (int c = 0; c < 64; ++c) mx = fmaxf(mx, __uint_as_float(s[c]));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 64; ++c) {
+          for (int c = 0; c < 64; ++c)
             if (c >= nvalid) s[c] = 0xff800000u;         // -inf
-            mx = fmaxf(mx, __uint_as_float(s[c]));
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+#pragma unroll
+        for (int c = 0; c < 64; c += 4) {
+          mx4[0] = fmaxf(mx4[0], __uint_as_float(s[c]));
+          mx4[1] = fmaxf(mx4[1], __uint_as_float(s[c + 1]));
+          mx4[2] = fmaxf(mx4[2], __uint_as_float(s[c + 2]));
+          mx4[3] = fmaxf(mx4[3], __uint_as_float(s[c + 3]));
+        }
+        {
+          const int ovalid = N - j * AT_BKV - (half ^ 1) * 64;
+          if (ovalid >= 64) {
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+              mx4[0] = fmaxf(mx4[0], __uint_as_float(t[c]));
+              mx4[1] = fmaxf(mx4[1], __uint_as_float(t[c + 1]));
+              mx4[2] = fmaxf(mx4[2], __uint_as_float(t[c + 2]));
+              mx4[3] = fmaxf(mx4[3], __uint_as_float(t[c + 3]));
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 64; ++c)
+              if (c < ovalid) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(t[c]));
           }
         }
-        // the two threads of a row exchange their partial maxima (buffer alternates with the block parity)
-        float* xm = s_xmax + (gj & 1) * 256;
-        xm[half * 128 + trow] = mx;
-        mbar_arrive(bar(X_MAX + sb));
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(X_MAX + sb), ph, s_abort));
-        if (!ok) break;
-        mx = fmaxf(mx, xm[(half ^ 1) * 128 + trow]) * scale_log2;
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+        ATT_T(3)
         bool need = false;
         float corr = 1.f;
         if (j == 0) {
@@ -234,21 +262,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           m_used = mx;
           l *= corr;
         }
-        float2 sum2 = make_float2(0.f, 0.f);
+        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
         uint32_t pk[32];
         const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
 #pragma unroll
         for (int c = 0; c < 64; c += 2) {
           const float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
           const float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
-          sum2 = __fadd2_rn(sum2, p);
+          sum2[(c >> 1) & 1] = __fadd2_rn(sum2[(c >> 1) & 1], p);
           pk[c >> 1] = pack_bf16(p.x, p.y);
         }
-        l += sum2.x + sum2.y;
+        l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+        ATT_T(4)
         if (gj > 0) {
           ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (gj - 1) & 1, s_abort));   // P V of the previous block done
           if (!ok) break;
         }
+        ATT_T(5)
         if (j > 0 && __any_sync(0xffffffffu, need)) {      // both threads of a row take the same decision
           tc_fence_after();
 #pragma unroll 1
@@ -273,13 +303,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         fence_async_smem();
         tc_fence_before();
-        mbar_arrive(bar(P_FULL));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(P_FULL));
+        ATT_T(6)
       }
       if (!ok) break;
       g += nblk;
       // row sum: add the partner's half
       s_xsum[half * 128 + trow] = l;
-      mbar_arrive(bar(X_SUM));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(X_SUM));
       ok = __all_sync(0xffffffffu, mbar_wait(bar(X_SUM), it & 1, s_abort));
       if (!ok) break;
       l += s_xsum[(half ^ 1) * 128 + trow];
@@ -308,7 +341,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(O_FREE));
+      ATT_T(7)
     }
+#ifdef ATT_PROFILE
+    if (prof && blockIdx.x == 0 && warp == 2 && lane == 0)
+      for (int i = 0; i < 8; ++i) prof[i] = tp[i];
+#endif
   }
 
   tc_fence_before();
@@ -335,7 +373,21 @@ static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorM
   if (items < grid) grid = (int)items;
   if (grid < 1) grid = 1;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  attention_tc_kernel<DH><<<grid, AT_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status);
+  unsigned long long* prof = nullptr;
+#ifdef ATT_PROFILE
+  static unsigned long long* d_prof = nullptr;
+  if (!d_prof) cudaMalloc(&d_prof, 64);
+  prof = d_prof;
+#endif
+  attention_tc_kernel<DH><<<grid, AT_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status, prof);
+#ifdef ATT_PROFILE
+  {
+    unsigned long long h[8];
+    cudaMemcpy(h, d_prof, 64, cudaMemcpyDeviceToHost);
+    fprintf(stderr, "ATT_PROFILE cycles: loop %llu waitS %llu ldS %llu max+xchg %llu exp %llu waitPV %llu writeP %llu epi %llu\n",
+            h[0], h[1], h[2], h[3], h[4], h[5], h[6], h[7]);
+  }
+#endif
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

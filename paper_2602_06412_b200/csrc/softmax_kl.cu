@@ -9,6 +9,8 @@
 // KL is ~1e-7 (terms of size |r| summing to r^2/2); this one does not, is exactly 0 for identical rows, and is
 // insensitive to first order to the rounding of the two log-sum-exps (d KL / d(lse_p - lse_q) = 1 - sum q = 0).
 // g uses its Taylor series for |r| < 1/8 and r + (exp(-r) - 1) beyond.
+#include <stdlib.h>
+
 #include "common.cuh"
 
 namespace sl {
@@ -436,7 +438,13 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
   if (g > max_rows) g = max_rows;
   if (g < 1) g = 1;
   if (dtype == SL_BF16) {
-    int gb = sm_count() * 3;
+    static int per_sm = 0;
+    if (!per_sm) {
+      const char* e = getenv("SURELOCK_KL_CTAS_PER_SM");   // tuning aid
+      per_sm = e ? atoi(e) : 3;
+      if (per_sm < 1 || per_sm > 3) per_sm = 3;
+    }
+    int gb = sm_count() * per_sm;
     if (gb > max_rows) gb = max_rows;
     if (gb < 1) gb = 1;
     softmax_kl_sure_bf16_kernel<<<gb, KLF_THREADS, 0, st>>>((const bf16*)logits, (const bf16*)prev_logits, row_of_pos_prev,
