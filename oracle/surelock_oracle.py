@@ -25,7 +25,10 @@ design notes of the repository):
     without a previous posterior has D = +inf (Algorithm 1, line 19);
   * the lock test reads the mask state the forward pass saw (the state passed
     to this step), so a row can lock only after a step that was fed its token;
-  * the optional confidence-percentile gate (Algorithm 1, line 21) is off.
+  * the optional confidence-percentile gate (Algorithm 1, line 21) is off unless asked for; when on, the
+    percentile is taken per sequence over the locking candidates Z_t (Algorithm 1) rather than over all active
+    rows (Sec. 2.2 prose), with linear interpolation between order statistics, and a row passes when
+    u <= theta_m.
 
 Parity pins (tests that run without a GPU) tie this file to closed forms, printed
 values of the paper's Table 2, library routines of a different library (torch
@@ -166,6 +169,39 @@ def sure_test(D: np.ndarray, masked: np.ndarray, kl_eps: float) -> np.ndarray:
     return (np.asarray(masked) == 0) & (D <= kl_eps)
 
 
+def percentile_linear(values: Sequence[float], m: float) -> float:
+    """Empirical m-th percentile (0 <= m <= 100) with linear interpolation between order statistics:
+    x sorted ascending, h = (n-1) m / 100, result x[floor h] + (h - floor h)(x[ceil h] - x[floor h]).
+    An empty set has no percentile: returns -inf (so that nothing passes a "<= theta" test)."""
+    x = sorted(float(v) for v in values)
+    n = len(x)
+    if n == 0:
+        return -np.inf
+    h = (n - 1) * (float(m) / 100.0)
+    lo = int(np.floor(h))
+    hi = min(lo + 1, n - 1)
+    return x[lo] + (h - lo) * (x[hi] - x[lo])
+
+
+def confidence_gate(conf: np.ndarray, candidate: np.ndarray, seq_of_row: np.ndarray, n_seq: int, m: float):
+    """Optional confidence gate (Algorithm 1 lines 18, 21 and 23; Sec. 2.2 "Optional: Confidence gate").
+
+    u_i = 1 - max_v p_i(v) = 1 - conf_i.  Per sequence, theta_m is the m-th percentile of u over the locking
+    candidates Z_t (active and unmasked rows of that sequence); a candidate passes when u_i <= theta_m, i.e. it is
+    among the top-m % most confident candidates.  Returns (passes [rows] bool, theta [n_seq]).
+    """
+    u = 1.0 - np.asarray(conf, F64)
+    candidate = np.asarray(candidate, bool)
+    seq_of_row = np.asarray(seq_of_row)
+    theta = np.full(n_seq, -np.inf, F64)
+    passes = np.zeros(len(u), bool)
+    for b in range(n_seq):
+        rows = np.flatnonzero((seq_of_row == b) & candidate)
+        theta[b] = percentile_linear(u[rows], m)
+        passes[rows] = u[rows] <= theta[b]
+    return passes, theta
+
+
 # --------------------------------------------------------------------------
 # Algorithmic FLOPs (Sec. 2.3)
 # --------------------------------------------------------------------------
@@ -256,7 +292,7 @@ class OracleState:
 
 
 def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.ndarray,
-         lock: np.ndarray, kl_eps: float, logits_round=None):
+         lock: np.ndarray, kl_eps: float, logits_round=None, conf_gate_m: Optional[float] = None):
     """One SureLock step (Algorithm 1, lines 6-15 and 18-24; line 16 belongs to the caller).
 
     weights: {"tok_emb": [V][d], "lm_head": [V][d], "final_norm_g": [d],
@@ -299,10 +335,14 @@ def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.n
     if has_prev.any():
         D[has_prev] = kl_rows(logp[has_prev], state.prev_logp[bb[has_prev], ii[has_prev]])
     lockable = sure_test(D, np.asarray(mask_state)[bb, ii], kl_eps)  # lines 20, 23
+    theta = None
+    if conf_gate_m is not None:                                   # line 21: u <= theta_m over the candidates Z_t
+        gate, theta = confidence_gate(conf, np.asarray(mask_state)[bb, ii] == 0, bb, B, conf_gate_m)
+        lockable = lockable & gate
     new_lock = np.array(lock, dtype=np.uint8, copy=True)
     new_lock[bb[lockable], ii[lockable]] = 1                      # line 24
     state.prev_logp[bb, ii] = logp                                # locked rows keep p_{t*}
     state.prev_valid[bb, ii] = True
     state.flops += flops
     return dict(active_idx=idx, row_offsets=offs, hidden=hidden, logits=logits, kl=D,
-                conf=conf, argmax=am, new_lock=new_lock, flops=flops)
+                conf=conf, argmax=am, new_lock=new_lock, flops=flops, theta=theta)

@@ -375,3 +375,49 @@ def test_brute_force_tiny():
         assert abs(r2["kl"][r] - kl) < 1e-13
         assert bool(r2["new_lock"][0, i]) == (mask[0, i] == 0 and kl <= 1e-3)
     assert r2["new_lock"][0, 0] == 1
+
+
+# ------------------------------------------------------------------ optional confidence gate (Algorithm 1 line 21)
+def test_percentile_and_confidence_gate():
+    rng = np.random.default_rng(11)
+    for n in (1, 2, 5, 40, 101):
+        x = rng.random(n)
+        for m in (0, 10, 20, 40, 50, 99.5, 100):
+            assert abs(O.percentile_linear(x, m) - np.percentile(x, m)) < 1e-15     # numpy's default (linear) rule
+    assert O.percentile_linear([], 20) == -np.inf
+    assert O.percentile_linear([3.0, 1.0, 2.0], 0) == 1.0 and O.percentile_linear([3.0, 1.0, 2.0], 100) == 3.0
+    assert O.percentile_linear([0.0, 10.0], 25) == 2.5                              # interpolation by hand
+    # gate: per sequence, over candidates only
+    conf = np.array([0.9, 0.5, 0.99, 0.2, 0.7, 0.6, 0.95])
+    cand = np.array([1, 1, 1, 0, 1, 1, 1], bool)
+    seq = np.array([0, 0, 0, 0, 1, 1, 1])
+    passes, theta = O.confidence_gate(conf, cand, seq, 3, 50)
+    # sequence 0: u = .1, .5, .01 -> median .1 -> rows with u <= .1; the non-candidate (u = .8) never passes
+    assert abs(theta[0] - 0.1) < 1e-15 and list(passes[:4]) == [True, False, True, False]
+    # sequence 1: u = .3, .4, .05 -> median .3
+    assert abs(theta[1] - 0.3) < 1e-15 and list(passes[4:]) == [True, False, True]
+    assert theta[2] == -np.inf                                                      # no candidates: nothing passes
+    p100, _ = O.confidence_gate(conf, cand, seq, 3, 100)
+    assert list(p100) == list(cand)                                                 # m = 100 passes every candidate
+    p0, _ = O.confidence_gate(conf, cand, seq, 3, 0)
+    assert list(p0) == [False, False, True, False, False, False, True]              # m = 0: only the most confident
+
+
+def test_step_with_confidence_gate_locks_a_subset():
+    c, oc, w, wn = _small(seed=13)
+    B, N = 2, 16
+    tokens, mask = inputs.make_tokens(B, N, 10, c["vocab"], 6)
+    lock0 = np.zeros((B, N), np.uint8)
+    a, b = O.OracleState(oc, B, N), O.OracleState(oc, B, N)
+    for st in (a, b):
+        O.step(st, wn, tokens.numpy(), mask.numpy(), lock0, 1e-3)
+    plain = O.step(a, wn, tokens.numpy(), mask.numpy(), lock0, 1e-3)                # stationary: every unmasked row locks
+    gated = O.step(b, wn, tokens.numpy(), mask.numpy(), lock0, 1e-3, conf_gate_m=20)
+    assert plain["new_lock"].sum() == 20
+    assert np.all(gated["new_lock"] <= plain["new_lock"])                          # the gate only removes locks
+    # 10 candidates per sequence, 20th percentile: h = 1.8 -> the two most confident rows pass
+    assert list(gated["new_lock"].sum(1)) == [2, 2]
+    for bb in range(B):
+        u = 1 - gated["conf"][bb * N: bb * N + 10]
+        assert set(np.flatnonzero(gated["new_lock"][bb])) == set(np.argsort(u)[:2])
+    np.testing.assert_array_equal(gated["logits"], plain["logits"])                 # the gate changes decisions only
