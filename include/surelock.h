@@ -135,6 +135,14 @@ int surelock_kv_cache(surelock_ctx *ctx, int layer, void **k, void **v, size_t *
  * or -1 when the position has no previous posterior.  Writing both lets a caller seed p_{t-1}. */
 int surelock_prev_logits(surelock_ctx *ctx, void **buf, int32_t **row_of_pos);
 
+/* Optional confidence gate (Algorithm 1 lines 18, 21, 23; Sec. 2.2): with 0 <= m_percent <= 100 every later
+ * surelock_step locks a candidate (active, unmasked row) only if, besides D <= kl_eps, its uncertainty
+ * u = 1 - max_v p(v) is <= theta_m, the m-th percentile (linear interpolation between order statistics) of u over
+ * the candidates of ITS sequence; a sequence without candidates locks nothing.  The paper's runs use m = 20.
+ * A negative m_percent (or NaN) switches the gate off (the default: the KL criterion alone).  N must be <= 8192
+ * while the gate is on.  *theta (may be NULL) receives a dev pointer to the B thresholds of the last step. */
+int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float **theta);
+
 /* Tuning / test switches.  "gemm_impl": 0 = tensor-core GEMM and attention when the shape allows (default),
  * 1 = force the CUDA-core kernels.  "time_kernels": 1 creates an event pool (once) and brackets every launch of
  * later steps with CUDA events for surelock_kernel_times().  "trace_layers": 1 allocates (once, here, not in the
@@ -154,8 +162,8 @@ int surelock_last_launch_count(surelock_ctx *ctx);
  * surelock_set_option(ctx, "time_kernels", 1) before that step (events add a few microseconds per launch, so time
  * whole steps with the option off).  Synchronises the stream.  ms[i], launches[i] (may be NULL) for class i:
  * 0 compaction, 1 embedding/row gather, 2 RMSNorm, 3 QKV GEMM, 4 RoPE, 5 K/V scatter, 6 attention, 7 O-proj GEMM,
- * 8 gate/up GEMM + SwiGLU, 9 down GEMM, 10 LM-head GEMM, 11 softmax-KL-lock.  n_classes >= 12. */
-#define SURELOCK_KERNEL_CLASSES 12
+ * 8 gate/up GEMM + SwiGLU, 9 down GEMM, 10 LM-head GEMM, 11 softmax-KL-lock, 12 confidence gate.  n_classes >= 13. */
+#define SURELOCK_KERNEL_CLASSES 13
 int surelock_kernel_times(surelock_ctx *ctx, float *ms, int32_t *launches, int n_classes);
 
 void surelock_destroy(surelock_ctx *ctx);
@@ -224,6 +232,14 @@ int surelock_softmax_kl_sure(const void *logits, const void *prev_logits, const 
                              const float *prev_lse, const int32_t *active_idx, const int32_t *n_active, int max_rows,
                              int vocab, int dtype, const uint8_t *mask_state, uint8_t *lock_mask, float kl_eps,
                              float *kl, float *conf, int32_t *argmax, float *lse_out, void *stream);
+
+/* The confidence gate alone (the kernel surelock_step runs when the gate is on): for each of the B sequences,
+ * theta = m-th percentile of u = 1 - conf over rows r in [row_offsets[b], row_offsets[b+1]) with
+ * mask_state[active_idx[r]] == 0; then lock_mask[active_idx[r]] = 1 for those rows with u <= theta and
+ * kl[r] <= kl_eps.  conf, kl: dev fp32 [M]; theta_out: dev fp32 [B] or NULL.  N <= 8192. */
+int surelock_conf_gate_lock(const float *conf, const float *kl, const int32_t *active_idx, const int32_t *row_offsets,
+                            int B, int N, const uint8_t *mask_state, uint8_t *lock_mask, float kl_eps, float m_percent,
+                            float *theta_out, void *stream);
 
 /* Bytes of workspace that lets surelock_gemm split K when M is small (see below). */
 size_t surelock_gemm_workspace_bytes(void);

@@ -61,6 +61,8 @@ def lib() -> C.CDLL:
         "surelock_prev_logits": (i32, [vp, C.POINTER(vp), C.POINTER(vp)]),
         "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
         "surelock_last_launch_count": (i32, [vp]),
+        "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
+        "surelock_conf_gate_lock": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, f32, f32, vp, vp]),
         "surelock_layer_trace": (i32, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "surelock_kernel_times": (i32, [vp, vp, vp, i32]),
         "surelock_destroy": (None, [vp]),
@@ -230,12 +232,27 @@ def surelock_layer_trace(ctx: Ctx) -> torch.Tensor:
     return device_view(buf.value, (ctx.cfg["n_layers"] + 1, ctx.B * ctx.N, ctx.cfg["d_model"]), torch.float32)
 
 
+def surelock_set_confidence_gate(ctx: Ctx, m_percent: float) -> torch.Tensor:
+    """Switch the optional confidence gate on (0 <= m_percent <= 100) or off (negative).  Returns a view of the B
+    per-sequence thresholds theta_m that later steps fill."""
+    th = C.c_void_p()
+    _check(lib().surelock_set_confidence_gate(ctx.handle, m_percent, C.byref(th)), "surelock_set_confidence_gate")
+    return device_view(th.value, (ctx.B,), torch.float32)
+
+
+def surelock_conf_gate_lock(conf, kl, active_idx, row_offsets, B: int, N: int, mask_state, lock_mask, kl_eps: float,
+                            m_percent: float, theta_out=None):
+    _check(lib().surelock_conf_gate_lock(_p(conf), _p(kl), _p(active_idx), _p(row_offsets), B, N, _p(mask_state),
+                                         _p(lock_mask), kl_eps, m_percent, _p(theta_out), _stream()),
+           "surelock_conf_gate_lock")
+
+
 def surelock_last_launch_count(ctx: Ctx) -> int:
     return lib().surelock_last_launch_count(ctx.handle)
 
 
 KERNEL_CLASSES = ("compact", "gather", "rmsnorm", "gemm_qkv", "rope", "kv_scatter", "attention", "gemm_o",
-                  "gemm_gateup", "gemm_down", "gemm_head", "softmax_kl")
+                  "gemm_gateup", "gemm_down", "gemm_head", "softmax_kl", "conf_gate")
 
 
 def surelock_kernel_times(ctx: Ctx):

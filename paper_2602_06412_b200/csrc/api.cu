@@ -39,6 +39,8 @@ struct surelock_ctx {
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
   std::vector<int> ev_cls;            // class of the launch bracketed by events 2i, 2i+1
   int n_ev = 0;
+  float gate_m = -1.f;                // confidence-gate percentile (Algorithm 1 line 21); < 0 = gate off
+  float* theta = nullptr;             // [B] gate thresholds of the last step
   SplitWs split;                      // split-K workspace of the tensor-core GEMM (bf16 only)
   float* trace = nullptr;             // [L+1][R][d] block inputs/outputs of the last step (only when switched on)
 
@@ -68,7 +70,7 @@ static int dev_alloc(surelock_ctx* c, P** p, size_t bytes) {
 
 // Kernel classes for the timing breakdown (order is part of the C ABI: surelock_kernel_times)
 enum { K_COMPACT = 0, K_GATHER, K_RMSNORM, K_GEMM_QKV, K_ROPE, K_SCATTER, K_ATTN, K_GEMM_O, K_GEMM_GATEUP, K_GEMM_DOWN,
-       K_GEMM_HEAD, K_SOFTMAX_KL, K_NUM };
+       K_GEMM_HEAD, K_SOFTMAX_KL, K_CONF_GATE, K_NUM };
 
 static inline void tick(surelock_ctx* c, int cls) {
   if (c->timing && c->n_ev + 2 <= (int)c->ev.size()) {
@@ -229,6 +231,7 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * sizeof(int), c->st) != cudaSuccess)
       rc = SL_ECUDA;
   }
+  A_(c->theta, ((size_t)batch + 1) * 4);
   A_(c->st_tokens, R * 4);
   A_(c->st_mask, R);
   A_(c->st_lock, R);
@@ -280,7 +283,11 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   SL_K(K_GEMM_HEAD, gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
   SL_K(K_SOFTMAX_KL, launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
                                             c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state,
-                                            lock_mask, kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st));
+                                            lock_mask, kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st,
+                                            c->gate_m < 0.f));
+  if (c->gate_m >= 0.f)
+    SL_K(K_CONF_GATE, launch_conf_gate_lock(c->conf, c->kl, c->idx, c->row_offsets, c->B, c->N, mask_state, lock_mask,
+                                            kl_eps, c->gate_m, c->theta, c->st));
   if (out) {
     out->active_idx = c->idx;
     out->row_offsets = c->row_offsets;
@@ -397,6 +404,14 @@ int surelock_layer_trace(surelock_ctx* c, float** buf, size_t* layer_stride_elem
   return c->trace ? SL_OK : SL_EINVAL;
 }
 
+int surelock_set_confidence_gate(surelock_ctx* c, float m_percent, const float** theta) {
+  if (!c) return SL_EINVAL;
+  if (m_percent > 100.f) return SL_EINVAL;
+  c->gate_m = (m_percent >= 0.f) ? m_percent : -1.f;     // negative or NaN: gate off
+  if (theta) *theta = c->theta;
+  return SL_OK;
+}
+
 int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
 
 int surelock_kernel_times(surelock_ctx* c, float* ms, int32_t* launches, int n_classes) {
@@ -475,6 +490,15 @@ int surelock_softmax_kl_sure(const void* logits, const void* prev_logits, const 
 
 static size_t gemm_ws_tiles() { return 2 * (size_t)sm_count(); }
 size_t surelock_gemm_workspace_bytes(void) { return gemm_ws_tiles() * (SPLIT_TILE_BYTES + sizeof(int)); }
+
+int surelock_conf_gate_lock(const float* conf, const float* kl, const int32_t* active_idx, const int32_t* row_offsets,
+                            int B, int N, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent,
+                            float* theta_out, void* stream) {
+  if (!conf || !kl || !active_idx || !row_offsets || !mask_state || !lock_mask || B <= 0 || N <= 0) return SL_EINVAL;
+  if (!(kl_eps >= 0.f) || !(m_percent >= 0.f) || m_percent > 100.f) return SL_EINVAL;
+  return launch_conf_gate_lock(conf, kl, active_idx, row_offsets, B, N, mask_state, lock_mask, kl_eps, m_percent,
+                               theta_out, (cudaStream_t)stream);
+}
 
 int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active, int max_rows, int n_out, int K,
                   int dtype, int impl, void* workspace, int32_t* dev_status, void* stream) {

@@ -105,7 +105,8 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
                        const float* __restrict__ prev_lse, const int32_t* __restrict__ idx,
                        const int32_t* __restrict__ n_active, int V, const uint8_t* __restrict__ mask_state,
                        uint8_t* __restrict__ lock_mask, float kl_eps, float* __restrict__ kl_out,
-                       float* __restrict__ conf_out, int32_t* __restrict__ argmax_out, float* __restrict__ lse_out) {
+                       float* __restrict__ conf_out, int32_t* __restrict__ argmax_out, float* __restrict__ lse_out,
+                       int apply_lock) {
   constexpr int VEC = 16 / sizeof(T);
   __shared__ MaxSum s_ms[KL_THREADS / 32];
   __shared__ double s_sum[KL_THREADS / 32];
@@ -209,7 +210,7 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
       conf_out[r] = 1.f / a.s;          // exp(max - lse)
       argmax_out[r] = a.am;
       if (lse_out) lse_out[r] = lse_p;
-      if (mask_state[pos] == 0 && kl <= kl_eps) lock_mask[pos] = 1;
+      if (apply_lock && mask_state[pos] == 0 && kl <= kl_eps) lock_mask[pos] = 1;
     }
   }
 }
@@ -327,7 +328,7 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
                             const int32_t* __restrict__ idx, const int32_t* __restrict__ n_active, int V,
                             const uint8_t* __restrict__ mask_state, uint8_t* __restrict__ lock_mask, float kl_eps,
                             float* __restrict__ kl_out, float* __restrict__ conf_out, int32_t* __restrict__ argmax_out,
-                            float* __restrict__ lse_out) {
+                            float* __restrict__ lse_out, int apply_lock) {
   __shared__ float s_m[KLF_THREADS / 32], s_s[KLF_THREADS / 32];
   __shared__ int s_a[KLF_THREADS / 32];
   __shared__ double s_sum[KLF_THREADS / 32];
@@ -423,7 +424,7 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
       conf_out[r] = 1.f / ra.s;          // exp(max - lse)
       argmax_out[r] = ra.am;
       if (lse_out) lse_out[r] = lse_p;
-      if (mask_state[pos] == 0 && kl <= kl_eps) lock_mask[pos] = 1;
+      if (apply_lock && mask_state[pos] == 0 && kl <= kl_eps) lock_mask[pos] = 1;
     }
   }
 }
@@ -431,7 +432,7 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
 int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
                            const float* prev_lse, const int32_t* idx, const int32_t* n_active, int max_rows, int vocab,
                            int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
-                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st) {
+                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st, bool apply_lock) {
   const int vec = dtype == SL_BF16 ? 8 : 4;
   if (vocab <= 0 || vocab % vec) return SL_EUNSUPPORTED;
   int g = sm_count() * 2;
@@ -449,11 +450,11 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
     if (gb < 1) gb = 1;
     softmax_kl_sure_bf16_kernel<<<gb, KLF_THREADS, 0, st>>>((const bf16*)logits, (const bf16*)prev_logits, row_of_pos_prev,
                                                              prev_lse, idx, n_active, vocab, mask_state, lock_mask, kl_eps,
-                                                             kl, conf, argmax, lse_out);
+                                                             kl, conf, argmax, lse_out, apply_lock ? 1 : 0);
   } else
     softmax_kl_sure_kernel<float><<<g, KL_THREADS, 0, st>>>((const float*)logits, (const float*)prev_logits,
                                                            row_of_pos_prev, prev_lse, idx, n_active, vocab, mask_state,
-                                                           lock_mask, kl_eps, kl, conf, argmax, lse_out);
+                                                           lock_mask, kl_eps, kl, conf, argmax, lse_out, apply_lock ? 1 : 0);
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

@@ -16,7 +16,7 @@ from tests.parity_util import f64, rel_err_rows, to_dev
 
 
 def run_side_by_side(cfg, dtype, B, N, n_prompt, steps, kl_eps, seed, tol_logits, tol_hidden=None, std=0.02,
-                     forced_p=0.0, kl_tol=1e-3, kl_floor=1e-9, check_kl_free_running=False, log=None):
+                     forced_p=0.0, kl_tol=1e-3, kl_floor=1e-9, check_kl_free_running=False, log=None, conf_gate_m=None):
     """Returns the per-step trace of M.  Raises AssertionError on the first parity violation."""
     tol_hidden = tol_hidden or tol_logits
     w = inputs.make_weights(cfg, seed, dtype=dtype, std=std)
@@ -24,6 +24,7 @@ def run_side_by_side(cfg, dtype, B, N, n_prompt, steps, kl_eps, seed, tol_logits
     wd = to_dev(w)
     oc = O.ModelCfg(**cfg)
     ctx = SL.surelock_init(cfg, wd, N, B)
+    theta_view = SL.surelock_set_confidence_gate(ctx, conf_gate_m) if conf_gate_m is not None else None
     st = O.OracleState(oc, B, N)
     tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], seed)
     lock = torch.zeros((B, N), dtype=torch.uint8)
@@ -77,6 +78,15 @@ def run_side_by_side(cfg, dtype, B, N, n_prompt, steps, kl_eps, seed, tol_logits
         bb, ii = idx // N, idx % N
         want = O.sure_test(kl_ref, mask.numpy()[bb, ii], kl_eps)
         near = np.isfinite(kl_ref) & (np.abs(kl_ref - kl_eps) <= kl_tol * kl_eps)
+        if conf_gate_m is not None:          # the gate, evaluated by the oracle on the confidences the GPU produced
+            conf_gpu = out.conf[:M].cpu().numpy().astype(np.float64)
+            gate, theta = O.confidence_gate(conf_gpu, mask.numpy()[bb, ii] == 0, bb, B, conf_gate_m)
+            want = want & gate
+            th_gpu = theta_view.cpu().numpy().astype(np.float64)
+            fin_t = np.isfinite(theta)
+            assert np.array_equal(np.isfinite(th_gpu), fin_t)
+            np.testing.assert_allclose(th_gpu[fin_t], theta[fin_t], rtol=1e-5, atol=1e-7)
+            near = near | (np.abs((1.0 - conf_gpu) - theta[bb]) <= 1e-6)
         new_lock = lock_d.cpu()
         got = new_lock.numpy()[bb, ii].astype(bool)
         assert np.array_equal(got[~near], want[~near]), (t, "lock decisions")

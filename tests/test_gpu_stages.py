@@ -282,3 +282,41 @@ def test_attention_tensor_cores(B, N, H, dh, n_act, qscale):
         ref = O.attention_rows(f64(q[r0:r1]), f64(Kc[b * N:(b + 1) * N]), f64(Vc[b * N:(b + 1) * N]))
         assert rel_err_rows(f64(o[r0:r1]).reshape(r1 - r0, -1), ref) < 2e-2, (b,)
     assert (o[M:] == 5.0).all()                                      # rows beyond M untouched
+
+
+@pytest.mark.parametrize("B,N,m", [(1, 128, 20.0), (3, 200, 50.0), (4, 4096, 20.0), (2, 33, 0.0), (2, 33, 100.0), (5, 8, 37.5)])
+def test_conf_gate_lock(B, N, m):
+    """Confidence gate alone: per-sequence percentile threshold and gated lock decisions against the oracle."""
+    g = torch.Generator().manual_seed(B * 100 + N)
+    n_act = [int(x) for x in torch.randint(0, N + 1, (B,), generator=g)]
+    n_act[0] = N
+    if B > 1:
+        n_act[1] = 0                                                 # a sequence without active rows
+    lock = inputs.random_lock(B, N, n_act, 21)
+    idx, offs = O.active_set(lock.numpy())
+    M = len(idx)
+    conf = torch.rand(max(M, 1), generator=g)
+    conf[:: 7] = conf[0]                                             # ties
+    kl = torch.rand(max(M, 1), generator=g) * 2e-3
+    mask = (torch.rand((B, N), generator=g) < 0.4).to(torch.uint8)
+    if B > 2:
+        mask[2] = 1                                                  # a sequence without candidates
+    lock_d = lock.to(DEV)
+    theta = torch.full((B,), 7.0, device=DEV)
+    SL.surelock_conf_gate_lock(conf.to(DEV), kl.to(DEV), torch.from_numpy(idx).to(DEV) if M else torch.zeros(1, dtype=torch.int32, device=DEV),
+                               torch.from_numpy(offs).to(DEV), B, N, mask.to(DEV), lock_d, 1e-3, m, theta)
+    torch.cuda.synchronize()
+    bb, ii = idx // N, idx % N
+    cand = mask.numpy()[bb, ii] == 0
+    gate, th = O.confidence_gate(f64(conf[:M]), cand, bb, B, m)
+    want = gate & O.sure_test(f64(kl[:M]), mask.numpy()[bb, ii], 1e-3)
+    thg = theta.cpu().numpy().astype(np.float64)
+    fin = np.isfinite(th)
+    assert np.array_equal(np.isfinite(thg), fin) and np.all(thg[~fin] < 0)
+    np.testing.assert_allclose(thg[fin], th[fin], rtol=1e-6, atol=1e-7)
+    near = np.abs((1.0 - f64(conf[:M])) - th[bb]) <= 1e-6
+    new = lock_d.cpu().numpy()
+    got = new[bb, ii].astype(bool)
+    assert np.array_equal(got[~near], want[~near])
+    assert np.array_equal(new[lock.numpy() == 1], lock.numpy()[lock.numpy() == 1])   # locked rows stay locked
+    assert not got[~cand].any()

@@ -46,6 +46,19 @@ def test_bf16_head_dim_128_ragged_batch():
                      std=0.04, forced_p=0.3)
 
 
+def test_confidence_gate_in_the_step():
+    """Algorithm 1 line 21 with the paper's default m = 20 %: fewer rows lock than with the KL criterion alone."""
+    cfg = inputs.model_shape("tiny")
+    plain, _, _ = run_side_by_side(cfg, torch.float32, B=2, N=96, n_prompt=40, steps=12, kl_eps=1e-3, seed=5,
+                                   tol_logits=1e-4)
+    gated, _, _ = run_side_by_side(cfg, torch.float32, B=2, N=96, n_prompt=40, steps=12, kl_eps=1e-3, seed=5,
+                                   tol_logits=1e-4, conf_gate_m=20.0)
+    assert gated[2] > plain[2]                       # at the third step the gate has held most candidates back
+    assert all(a >= b for a, b in zip(gated, gated[1:]))
+    run_side_by_side(cfg, torch.bfloat16, B=3, N=128, n_prompt=64, steps=6, kl_eps=1e-3, seed=6, tol_logits=5e-2,
+                     std=0.05, conf_gate_m=40.0)
+
+
 def test_locked_rows_cache_bytes_never_change_and_active_rows_are_rewritten():
     cfg = inputs.model_shape("tiny")
     w = inputs.make_weights(cfg, 5, dtype=torch.bfloat16, std=0.05)
