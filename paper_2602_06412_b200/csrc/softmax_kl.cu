@@ -223,6 +223,25 @@ softmax_kl_sure_kernel(const T* __restrict__ logits, const T* __restrict__ prev,
 // processed.
 constexpr int KLF_THREADS = 256;
 
+// The current row is read twice (sweep 1 from HBM, sweep 2 from L2): ask L2 to keep it; the previous row is read
+// once: mark it evict-first so that it does not push current rows out.
+__device__ __forceinline__ uint64_t l2_policy_keep() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_stream() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ uint4 ld_hint(const uint4* p, uint64_t pol) {
+  uint4 v;
+  asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0, %1, %2, %3}, [%4], %5;"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p), "l"(pol));
+  return v;
+}
+
 __device__ __forceinline__ float2 unpack_pair(unsigned w) {   // (low bf16, high bf16) -> two floats
   return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
@@ -336,6 +355,7 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = V >> 3;
   constexpr int STEP = 2 * KLF_THREADS;   // two vectors per thread and iteration
+  const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
 
   auto block_maxsum = [&](MaxSum2 st) -> MaxSum {
     MaxSum v{st.m, st.s.x + st.s.y, st.am};
@@ -366,19 +386,19 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
     MaxSum2 a{-INFINITY, make_float2(0.f, 0.f), 0x7fffffff}, b{-INFINITY, make_float2(0.f, 0.f), 0};
     {
       const uint4 zero = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // eight times -inf
-      uint4 c0 = tid < nvec ? __ldg(z + tid) : zero;
-      uint4 c1 = tid + KLF_THREADS < nvec ? __ldg(z + tid + KLF_THREADS) : zero;
+      uint4 c0 = tid < nvec ? ld_hint(z + tid, pol_keep) : zero;
+      uint4 c1 = tid + KLF_THREADS < nvec ? ld_hint(z + tid + KLF_THREADS, pol_keep) : zero;
       for (int v0 = tid; v0 < nvec; v0 += STEP) {
         const int n0 = v0 + STEP, n1 = n0 + KLF_THREADS;
-        const uint4 p0 = n0 < nvec ? __ldg(z + n0) : zero;
-        const uint4 p1 = n1 < nvec ? __ldg(z + n1) : zero;
+        const uint4 p0 = n0 < nvec ? ld_hint(z + n0, pol_keep) : zero;
+        const uint4 p1 = n1 < nvec ? ld_hint(z + n1, pol_keep) : zero;
         accum_maxsum_bf16(c0, v0 * 8, a, true);
         if (v0 + KLF_THREADS < nvec) accum_maxsum_bf16(c1, (v0 + KLF_THREADS) * 8, a, true);
         c0 = p0;
         c1 = p1;
       }
       if (need_q) {
-        for (int v0 = tid; v0 < nvec; v0 += KLF_THREADS) accum_maxsum_bf16(__ldg(y + v0), v0 * 8, b, false);
+        for (int v0 = tid; v0 < nvec; v0 += KLF_THREADS) accum_maxsum_bf16(ld_hint(y + v0, pol_stream), v0 * 8, b, false);
       }
     }
     const MaxSum ra = block_maxsum(a);
@@ -397,14 +417,14 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
       const float dl = lse_p - lse_q, lp2 = lse_p * LOG2E;
       float2 acc = make_float2(0.f, 0.f);
       const uint4 zero = make_uint4(0, 0, 0, 0);
-      uint4 cz0 = tid < nvec ? __ldg(z + tid) : zero, cy0 = tid < nvec ? __ldg(y + tid) : zero;
+      uint4 cz0 = tid < nvec ? ld_hint(z + tid, pol_keep) : zero, cy0 = tid < nvec ? ld_hint(y + tid, pol_stream) : zero;
       uint4 cz1 = zero, cy1 = zero;
-      if (tid + KLF_THREADS < nvec) { cz1 = __ldg(z + tid + KLF_THREADS); cy1 = __ldg(y + tid + KLF_THREADS); }
+      if (tid + KLF_THREADS < nvec) { cz1 = ld_hint(z + tid + KLF_THREADS, pol_keep); cy1 = ld_hint(y + tid + KLF_THREADS, pol_stream); }
       for (int v0 = tid; v0 < nvec; v0 += STEP) {
         const int n0 = v0 + STEP, n1 = n0 + KLF_THREADS;
         uint4 pz0 = zero, py0 = zero, pz1 = zero, py1 = zero;
-        if (n0 < nvec) { pz0 = __ldg(z + n0); py0 = __ldg(y + n0); }
-        if (n1 < nvec) { pz1 = __ldg(z + n1); py1 = __ldg(y + n1); }
+        if (n0 < nvec) { pz0 = ld_hint(z + n0, pol_keep); py0 = ld_hint(y + n0, pol_stream); }
+        if (n1 < nvec) { pz1 = ld_hint(z + n1, pol_keep); py1 = ld_hint(y + n1, pol_stream); }
         acc = kl_vec_bf16(cz0, cy0, dl, lp2, acc);
         if (v0 + KLF_THREADS < nvec) acc = kl_vec_bf16(cz1, cy1, dl, lp2, acc);
         cz0 = pz0; cy0 = py0; cz1 = pz1; cy1 = py1;
