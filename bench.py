@@ -188,6 +188,8 @@ def main():
     ap.add_argument("--ratios", default="1,0.5,0.25,0.125,0.05", help="M/N sweep ('' = none)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sampler-steps", type=int, default=32,
+                    help="diffusion steps of the decoding run (SureLock vs the no-locking baseline sampler); 0 = skip")
     args = ap.parse_args()
     rank, world, local = dist_util.env_rank_world()
     cfgname, B, N, n_prompt, pattern = WORKLOADS[args.workload]
@@ -328,6 +330,30 @@ def main():
                               tokens_per_s=round(dist_util.sum_over_ranks(Ms, dev) / (mss * 1e-3), 1),
                               gemm_ideal_ms=round(ideal_ms, 4), frac_of_gemm_ideal=round(ideal_ms / mss, 4)))
 
+    # the paper's own run metrics on a short decoding run: the sampler loop with and without SureLock
+    sampler_run = None
+    if args.sampler_steps > 0 and rank == 0:
+        from paper_2602_06412_b200 import sampler
+        block_len = {"c3": 32, "c4": 64, "c5": 64, "tiny": 64}[args.workload]
+        runs = {}
+        for mode in ("surelock", "baseline"):
+            tk, mk = tokens.to(dev), mask.to(dev)
+            r = sampler.run(ctx, tk, mk, n_prompt, block_len, args.sampler_steps, 1e-3, surelock=(mode == "surelock"))
+            runs[mode] = r
+        sampler_run = dict(
+            steps=args.sampler_steps, block_len=block_len, kl_eps=1e-3, confidence_gate="off",
+            r_bar=round(runs["surelock"]["r_bar"], 4), flops_ratio=round(runs["surelock"]["flops_ratio"], 4),
+            f_base_per_position=runs["baseline"]["f_base_per_position"],
+            f_prop_per_position=runs["surelock"]["f_prop_per_position"],
+            e2e_tps_surelock=round(runs["surelock"]["e2e_tps"], 2), e2e_tps_baseline=round(runs["baseline"]["e2e_tps"], 2),
+            tps_ratio=round(runs["surelock"]["e2e_tps"] / max(runs["baseline"]["e2e_tps"], 1e-9), 3),
+            M_trace=runs["surelock"]["M_trace"],
+            ms_per_step_surelock=[round(x, 3) for x in runs["surelock"]["ms_per_step"]],
+            ms_per_step_baseline_median=round(float(np.median(runs["baseline"]["ms_per_step"])), 3),
+            note="random-init weights: the lock trajectory is synthetic (posteriors barely move, so unmasked rows lock "
+                 "at their second step); the paper reports 0.54x FLOPs and 1.30x TPS for LLaDA-8B-Instruct on its GPU")
+        SL.surelock_reset(ctx)
+
     status = SL.surelock_status_poll(ctx)
     line = {
         "metric": "active_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
@@ -335,6 +361,7 @@ def main():
         "dtype": "bf16" if dtype == torch.bfloat16 else "f32", "data": "synthetic",
         "config": workload_config(args, cfgname, cfg, B, N, pattern, M),
         "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "roofline": roof, "kernels": kernels, "sweep": sweep,
+        "sampler_run": sampler_run,
         "device_status": status,
     }
     if rank == 0 and not args.no_cpu_baseline:
