@@ -146,12 +146,13 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
 /* Tuning / test switches.  "gemm_impl": 0 = tensor-core GEMM and attention when the shape allows (default),
  * 1 = force the CUDA-core kernels.  "time_kernels": 1 creates an event pool (once) and brackets every launch of
  * later steps with CUDA events for surelock_kernel_times().  "trace_layers": 1 allocates (once, here, not in the
- * step) a buffer [L+1][B*N][d] fp32 and makes every later surelock_step copy the packed residual stream into it:
- * slot 0 = block input of layer 0 (the embeddings), slot l+1 = output of layer l; for stage-wise parity checks.  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
+ * step) a buffer [2L+1][B*N][d] fp32 and makes every later surelock_step copy the packed residual stream into it:
+ * slot 2l = input of block l (slot 0 = the embeddings), slot 2l+1 = after the attention sub-block of block l,
+ * slot 2L = output of the last block; for stage-wise parity checks.  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
  * (after a caller seeded them), 0 forgets them.  Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
-/* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [L+1][B*N][d] (rows packed as in
+/* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [2L+1][B*N][d] (rows packed as in
  * that step), *layer_stride_elems = B*N*d.  SL_EINVAL if tracing was never switched on. */
 int surelock_layer_trace(surelock_ctx *ctx, float **buf, size_t *layer_stride_elems);
 

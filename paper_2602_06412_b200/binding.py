@@ -226,10 +226,11 @@ def surelock_set_option(ctx: Ctx, name: str, value: int):
 
 
 def surelock_layer_trace(ctx: Ctx) -> torch.Tensor:
-    """View [L+1][B*N][d] fp32 of the per-layer residual stream of the last step ("trace_layers" must be on)."""
+    """View [2L+1][B*N][d] fp32 of the residual stream of the last step: slot 2l = input of block l, 2l+1 = after
+    its attention sub-block, 2L = output of the last block ("trace_layers" must be on)."""
     buf, stride = C.c_void_p(), C.c_size_t()
     _check(lib().surelock_layer_trace(ctx.handle, C.byref(buf), C.byref(stride)), "surelock_layer_trace")
-    return device_view(buf.value, (ctx.cfg["n_layers"] + 1, ctx.B * ctx.N, ctx.cfg["d_model"]), torch.float32)
+    return device_view(buf.value, (2 * ctx.cfg["n_layers"] + 1, ctx.B * ctx.N, ctx.cfg["d_model"]), torch.float32)
 
 
 def surelock_set_confidence_gate(ctx: Ctx, m_percent: float) -> torch.Tensor:

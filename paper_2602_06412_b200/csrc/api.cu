@@ -42,7 +42,7 @@ struct surelock_ctx {
   float gate_m = -1.f;                // confidence-gate percentile (Algorithm 1 line 21); < 0 = gate off
   float* theta = nullptr;             // [B] gate thresholds of the last step
   SplitWs split;                      // split-K workspace of the tensor-core GEMM (bf16 only)
-  float* trace = nullptr;             // [L+1][R][d] block inputs/outputs of the last step (only when switched on)
+  float* trace = nullptr;             // [2L+1][R][d]: slot 2l = input of block l, 2l+1 = after its attention sub-block, 2L = output
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
   void* kcache(int l) const { return kv + (size_t)(2 * l) * kv_layer_bytes(); }
@@ -148,6 +148,9 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   }
   SL_K(K_ATTN, attention(c, l));
   SL_K(K_GEMM_O, gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
+  if (c->trace && x == c->x)
+    SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(2 * l + 1) * c->R * d, x, (size_t)c->R * d * sizeof(float),
+                                cudaMemcpyDeviceToDevice, c->st));
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->ffn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
   SL_K(K_GEMM_GATEUP, gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
   SL_K(K_GEMM_DOWN, gemm(c, c->act, c->w_down[l], nullptr, x, d, g.d_ff, EPI_RESIDUAL));
@@ -276,7 +279,7 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   for (int l = 0; l < g.n_layers; ++l) {
     SL_TRY(run_layer(c, l, c->x));
     if (c->trace)
-      SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(l + 1) * c->R * g.d_model, c->x, xbytes, cudaMemcpyDeviceToDevice,
+      SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(2 * l + 2) * c->R * g.d_model, c->x, xbytes, cudaMemcpyDeviceToDevice,
                                   c->st));
   }
   SL_K(K_RMSNORM, launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
@@ -375,7 +378,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
   if (!strcmp(name, "trace_layers")) {
     if (value && !c->trace) {
-      const size_t bytes = (size_t)(c->cfg.n_layers + 1) * c->R * c->cfg.d_model * sizeof(float);
+      const size_t bytes = (size_t)(2 * c->cfg.n_layers + 1) * c->R * c->cfg.d_model * sizeof(float);
       const int rc = dev_alloc(c, &c->trace, bytes);
       if (rc != SL_OK) return rc;
     }
