@@ -3,6 +3,8 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdio.h>
+#include <stdlib.h>
 
 #include "surelock.h"
 
@@ -15,10 +17,16 @@ enum {
   SL_DEV_BAD_INDEX = 4          // an index read from device memory was out of range and was skipped
 };
 
-#define SL_CUDA_TRY(expr)                       \
-  do {                                          \
-    cudaError_t e__ = (expr);                   \
-    if (e__ != cudaSuccess) return SL_ECUDA;    \
+// A failing CUDA runtime call makes the entry point return SL_ECUDA; with SURELOCK_DEBUG set in the environment the
+// call site and the runtime's message are also written to stderr.
+#define SL_CUDA_TRY(expr)                                                                              \
+  do {                                                                                                 \
+    cudaError_t e__ = (expr);                                                                          \
+    if (e__ != cudaSuccess) {                                                                          \
+      if (getenv("SURELOCK_DEBUG"))                                                                    \
+        fprintf(stderr, "surelock: %s:%d: %s: %s\n", __FILE__, __LINE__, #expr, cudaGetErrorString(e__)); \
+      return SL_ECUDA;                                                                                 \
+    }                                                                                                  \
   } while (0)
 
 namespace sl {

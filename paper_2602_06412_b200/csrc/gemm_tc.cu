@@ -233,6 +233,153 @@ __device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, in
   return c;
 }
 
+// ---- CTA-pair path (cta_group::2) for the tensor-pipe-bound regime ---------------------------------------------------
+// A cluster of two CTAs owns a 256 x 256 output tile: each CTA loads its own 128 rows of A and HALF of the weight tile
+// (128 of its 256 rows), the leader CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both CTAs' shared memory,
+// and each CTA's tensor memory receives the accumulator of its own 128 rows.  Per K block a CTA moves 32 KB instead of
+// 48 KB from L2 (the weight half is shared by the pair), which leaves room for six stages.  Barriers: "full" lives in
+// the leader (both CTAs' TMA loads count their bytes there), "empty" and "accumulator full" are reached in both CTAs by
+// a multicast tcgen05.commit, "accumulator empty" lives in the leader and is reached by the peer's epilogue with a
+// remote arrive.  All waits are bounded like in the single-CTA path.
+constexpr int TC2_STAGES = 6;
+
+template <int EPI>
+__device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorMap* tmW0, const CUtensorMap* tmW1,
+                                         const CUtensorMap* tmW2, void* __restrict__ Cv, int M, int n_out, int K,
+                                         int32_t* status, const QkvArgs& qkv, uint8_t* smem) {
+  constexpr int BN = 256;
+  constexpr int A_BYTES = TC_BM * TC_BK * 2;              // 16 KB: this CTA's 128 rows of A
+  constexpr int B_BYTES = 128 * TC_BK * 2;                // 16 KB: this CTA's half of the weight tile
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int STAGES = TC2_STAGES;
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr int OUT_BN = EPI == EPI_SWIGLU ? 128 : 256;
+
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const uint32_t bar0 = smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
+  auto accf_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + a); };
+  auto acce_bar = [&](int a) { return bar0 + 8u * (2 * STAGES + 2 + a); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(full_bar(s), 1);      // the leader's arrive.expect_tx; transaction bytes of both CTAs
+      mbar_init(empty_bar(s), 1);     // one multicast commit
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(accf_bar(a), 1);      // one multicast commit
+      mbar_init(acce_bar(a), 8);      // four epilogue warps of each CTA
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  if (warp == 1) tc_alloc_pair(smem_u32(s_tmem), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                 // the peer's barriers are initialised before anything arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  const int m_pairs = (M + 2 * TC_BM - 1) / (2 * TC_BM);
+  const int n_tiles = (n_out + OUT_BN - 1) / OUT_BN;
+  const int total = m_pairs * n_tiles;
+  const int num_kb = (K + TC_BK - 1) / TC_BK;
+  const int cid = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int w = cid; w < total && ok; w += n_clusters) {
+        const int m0 = (w % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (w / m_pairs) * OUT_BN;
+        // this CTA's half of the weight tile
+        const CUtensorMap* mp = tmW0;
+        int brow = n0 + (int)rank * 128;
+        if (EPI == EPI_SWIGLU) {                           // leader: gate rows, peer: up rows of the same features
+          mp = rank == 0 ? tmW0 : tmW1;
+          brow = n0;
+        } else if (EPI == EPI_QKV) {
+          const int src = n0 / qkv.hd;
+          mp = src == 0 ? tmW0 : (src == 1 ? tmW1 : tmW2);
+          brow = n0 - src * qkv.hd + (int)rank * 128;
+        }
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
+          const uint32_t fb = mapa_u32(full_bar(stage), 0);
+          if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
+          tma_load_2d_pair(sa, tmA, kb * TC_BK, m0, fb);
+          tma_load_2d_pair(sb, mp, kb * TC_BK, brow, fb);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = idesc_bf16_m128(BN, false, 256);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      int it = 0;
+      for (int w = cid; w < total && ok; w += n_clusters, ++it) {
+        const int acc = it & 1;
+        const uint32_t use = (uint32_t)(it >> 1);
+        if (!(ok = mbar_wait(acce_bar(acc), (use & 1) ^ 1, s_abort))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!(ok = mbar_wait(full_bar(stage), phase, s_abort))) break;
+          tc_fence_after();
+          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
+          const uint64_t adesc = smem_desc_k_sw128(sa), bdesc = smem_desc_k_sw128(sb);
+#pragma unroll
+          for (int k = 0; k < TC_BK / 16; ++k)
+            tc_mma_bf16_pair(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb > 0) | (k != 0));
+          tc_commit_pair_mcast(empty_bar(stage), 3);
+          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+        }
+        if (ok) tc_commit_pair_mcast(accf_bar(acc), 3);
+      }
+    }
+  } else {
+    const int quarter = warp & 3;
+    bool ok = true;
+    int it = 0;
+    for (int w = cid; w < total && ok; w += n_clusters, ++it) {
+      const int acc = it & 1;
+      const uint32_t use = (uint32_t)(it >> 1);
+      const int m0 = (w % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (w / m_pairs) * OUT_BN;
+      ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const int row = m0 + quarter * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
+      const int upr = units_per_row<EPI>(BN, n0, qkv);
+#pragma unroll 1
+      for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(acc), 0));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_GEMM_TIMEOUT);
+  cluster_sync_all();                 // neither CTA leaves (or frees tensor memory) while the pair may still use it
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc_pair(tmem_base, TMEM_COLS);
+  }
+}
+
 template <int EPI, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
@@ -240,7 +387,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
                const __grid_constant__ CUtensorMap tmW2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
                int n_out, int K, int32_t* status, const QkvArgs qkv, float* __restrict__ ws, int* __restrict__ counters,
-               int ws_tiles, int wide_boxes, int force_bn, int force_s) {
+               int ws_tiles, int wide_boxes, int force_bn, int force_s, int pair_mode) {
   // tmB*: weight maps with 64-row boxes (any tile width); tmW*: the same matrices with 128-row boxes, used for
   // 256-wide tiles so a stage is filled by fewer, larger TMA copies
   constexpr int BN_MAX = 256;
@@ -252,6 +399,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  if (pair_mode) {
+    // launched as clusters of two: when the grid can be filled with 256 x 256 pair tiles (large M) the CTA-pair path
+    // takes the whole launch; both CTAs of a pair read the same M and take the same branch
+    const int Mp = *n_active;
+    const int obn = EPI == EPI_SWIGLU ? 128 : 256;
+    if (((Mp + 255) / 256) * ((n_out + obn - 1) / obn) >= (int)(gridDim.x >> 1)) {
+      run_pair<EPI>(&tmA, &tmW0, &tmW1, &tmW2, Cv, Mp, n_out, K, status, qkv, smem);
+      return;
+    }
+  }
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
   // bars: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -513,6 +670,7 @@ int get_tensor_map_2d(const void* ptr, long long rows, long long cols, int box_r
   return SL_OK;
 }
 
+static int pair_mode();
 static int wide_boxes() {
   static int v = -1;
   if (v < 0) {
@@ -521,6 +679,16 @@ static int wide_boxes() {
     v = 2;
     if (e && !strcmp(e, "64")) v = 0;
     if (e && !strcmp(e, "128")) v = 1;
+    if (v == 2 && pair_mode()) v = 1;   // the CTA-pair path loads 128-row halves of a weight tile: share those maps
+  }
+  return v;
+}
+
+static int pair_mode() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SURELOCK_GEMM_PAIR");   // 0 disables the CTA-pair (cta_group::2) path
+    v = (e && e[0] == '0') ? 0 : 1;
   }
   return v;
 }
@@ -546,11 +714,25 @@ static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensor
     attr_set = true;
   }
   (void)max_rows;
-  const int grid = sm_count();   // persistent: one CTA per SM; the tile shape is chosen on the device from M
-  gemm_tc_kernel<EPI, STAGES><<<grid, TC_THREADS, SMEM, st>>>(a, b[0], b[1], b[2], wb[0], wb[1], wb[2], C, n_active,
-                                                              n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles,
-                                                              wide_boxes(), force_cfg(0), force_cfg(1));
-  SL_CUDA_TRY(cudaGetLastError());
+  // persistent: one CTA per SM; the tile shape is chosen on the device from M.  The kernel contains cta_group::2
+  // instructions, so it is always launched as clusters of two (an even grid) even when the pair path is switched off.
+  const int grid = sm_count() & ~1;
+  const int pair = pair_mode();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  SL_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, STAGES>, a, b[0], b[1], b[2], wb[0], wb[1], wb[2], C, n_active,
+                                 n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles, wide_boxes(), force_cfg(0),
+                                 force_cfg(1), pair));
   return SL_OK;
 }
 
