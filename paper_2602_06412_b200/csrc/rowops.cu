@@ -58,19 +58,32 @@ int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* 
 
 // ------------------------------------------------------------------------------------------------ RMSNorm
 // h = x * rsqrt(mean(x^2) + eps) * g; x fp32 residual stream, h in the storage type (the GEMM operand).
-template <typename T>
+// One CTA per row.  For d <= 8192 the row is read once and kept in registers (REGS float4 per thread) between the
+// sum of squares and the scaling; longer rows fall back to a second read.
+template <typename T, int REGS>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ h,
                const int32_t* __restrict__ n_active, int d, float eps) {
   __shared__ float s_part[8];
   const int M = *n_active;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nv = d >> 2;                                   // float4 per row
   for (int r = blockIdx.x; r < M; r += gridDim.x) {
-    const float* xr = x + (long long)r * d;
+    const float4* xr = reinterpret_cast<const float4*>(x + (long long)r * d);
+    float4 v[REGS > 0 ? REGS : 1];
     float ss = 0.f;
-    for (int c = threadIdx.x * 4; c < d; c += 1024) {
-      const float4 v = *reinterpret_cast<const float4*>(xr + c);
-      ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    if (REGS > 0) {
+#pragma unroll
+      for (int k = 0; k < REGS; ++k) {
+        const int c = threadIdx.x + k * 256;
+        v[k] = c < nv ? xr[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+      }
+    } else {
+      for (int c = threadIdx.x; c < nv; c += 256) {
+        const float4 t = xr[c];
+        ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+      }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
@@ -82,21 +95,40 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
     for (int w = 0; w < 8; ++w) tot += s_part[w];
     const float rstd = rsqrtf(tot / (float)d + eps);
     T* hr = h + (long long)r * d;
-    for (int c = threadIdx.x * 4; c < d; c += 1024) {
-      const float4 v = *reinterpret_cast<const float4*>(xr + c);   // second read hits L1/L2
-      const float o0 = v.x * rstd * to_f(gain[c]), o1 = v.y * rstd * to_f(gain[c + 1]);
-      const float o2 = v.z * rstd * to_f(gain[c + 2]), o3 = v.w * rstd * to_f(gain[c + 3]);
+    auto emit = [&](int c, const float4& t) {
+      const int e = c << 2;
+      const float o0 = t.x * rstd * to_f(gain[e]), o1 = t.y * rstd * to_f(gain[e + 1]);
+      const float o2 = t.z * rstd * to_f(gain[e + 2]), o3 = t.w * rstd * to_f(gain[e + 3]);
       if constexpr (sizeof(T) == 2) {
-        __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b = __floats2bfloat162_rn(o2, o3);
+        __nv_bfloat162 a = __floats2bfloat162_rn(o0, o1), b2 = __floats2bfloat162_rn(o2, o3);
         uint2 pk;
         pk.x = *reinterpret_cast<unsigned*>(&a);
-        pk.y = *reinterpret_cast<unsigned*>(&b);
-        *reinterpret_cast<uint2*>(hr + c) = pk;
+        pk.y = *reinterpret_cast<unsigned*>(&b2);
+        *reinterpret_cast<uint2*>(hr + e) = pk;
       } else {
-        *reinterpret_cast<float4*>(hr + c) = make_float4(o0, o1, o2, o3);
+        *reinterpret_cast<float4*>(hr + e) = make_float4(o0, o1, o2, o3);
       }
+    };
+    if (REGS > 0) {
+#pragma unroll
+      for (int k = 0; k < REGS; ++k) {
+        const int c = threadIdx.x + k * 256;
+        if (c < nv) emit(c, v[k]);
+      }
+    } else {
+      for (int c = threadIdx.x; c < nv; c += 256) emit(c, xr[c]);   // second read hits L1/L2
     }
   }
+}
+
+template <typename T>
+static void launch_rms_t(const float* x, const void* gain, void* h, const int32_t* n_active, int g, int d, float eps,
+                         cudaStream_t st) {
+  const int nv = d >> 2;
+  if (nv <= 256 * 2) rmsnorm_kernel<T, 2><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
+  else if (nv <= 256 * 4) rmsnorm_kernel<T, 4><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
+  else if (nv <= 256 * 8) rmsnorm_kernel<T, 8><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
+  else rmsnorm_kernel<T, 0><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
 }
 
 int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_active, int max_rows, int d, float eps,
@@ -104,9 +136,9 @@ int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_a
   if (d % 4) return SL_EUNSUPPORTED;
   const int g = row_grid(max_rows, 8);
   if (dtype == SL_BF16)
-    rmsnorm_kernel<bf16><<<g, 256, 0, st>>>(x, (const bf16*)gain, (bf16*)h, n_active, d, eps);
+    launch_rms_t<bf16>(x, gain, h, n_active, g, d, eps, st);
   else
-    rmsnorm_kernel<float><<<g, 256, 0, st>>>(x, (const float*)gain, (float*)h, n_active, d, eps);
+    launch_rms_t<float>(x, gain, h, n_active, g, d, eps, st);
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }
