@@ -392,7 +392,7 @@ static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorM
   return SL_OK;
 }
 
-int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+int launch_attention_tc1(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
   if ((head_dim != 64 && head_dim != 128) || B > AT_MAX_B || max_rows < 1 || !row_offsets) return SL_EUNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |

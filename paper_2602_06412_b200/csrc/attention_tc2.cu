@@ -1,0 +1,423 @@
+// Tensor-core M x N attention on sm_100a, two query tiles per CTA (Algorithm 1 line 12; Sec. 2.1: the packed queries of
+// the active rows attend to ALL N cached keys/values of their sequence, bidirectional, no mask).
+//
+// Work item = (sequence b, head h, up to 256 consecutive packed rows of that sequence = two tiles of 128); items never
+// straddle sequences.  Persistent CTAs take items round-robin, the row-tile index fastest, so CTAs working at the same
+// time read the same K/V head through L2.  Keys are streamed in blocks of 128.
+//   warp 0     TMA producer: both Q tiles once per item, then K and V blocks (two stages each), token-major cache rows,
+//              128-byte swizzle;
+//   warp 1     one thread issues, per key block and tile t: O_t += P_t V (previous block; P_t is read from TENSOR
+//              MEMORY as the A operand, V is the MN-major shared-memory operand) and then S_t = Q_t K^T;
+//   warps 2-5  softmax of tile 0, warps 6-9 softmax of tile 1: ONE thread per query row (no exchange between
+//              threads): tcgen05.ld the 128 scores, running max / sum in fp32 with 1/sqrt(d_h) folded into an exp2,
+//              P written back as packed bf16 over the first 64 columns of the S tile (tcgen05.st).
+// The two tiles alternate: while the softmax warps of one tile work, the tensor pipe runs the other tile's two
+// products, and each scheduler's special-function unit always has one of its two softmax warps to feed.
+// O stays in tensor memory and is rescaled only when a row's running maximum grows by more than 2^8; O / l is stored
+// as bf16 at the end of the item.  Keys beyond N in the last block are masked to -inf.  All waits are bounded
+// (SL_DEV_ATTN_TIMEOUT).
+//
+// Tensor memory (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+d_h)  O1 [256+d_h, 256+2 d_h).
+#include <stdio.h>
+#include <stdlib.h>
+
+#include "tc_common.cuh"
+
+namespace sl {
+
+namespace {
+
+constexpr int PP_THREADS = 320;   // TMA warp, MMA warp, 4 softmax warps per tile
+constexpr int PP_BQ = 128, PP_BKV = 128, PP_ITEM_ROWS = 256;
+constexpr int PP_MAX_B = 1024;
+
+// D[tmem] (+)= A[tmem] * B[smem]: A = 128 lanes x 8 columns, two bf16 per column (K = 16)
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+}  // namespace
+
+template <int DH>
+__global__ void __launch_bounds__(PP_THREADS, 1)
+attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
+                    bf16* __restrict__ o, float scale_log2, int32_t* status, unsigned long long* prof) {
+  constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
+  constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
+  constexpr int Q_BYTES = SLABS * SLAB_BYTES;          // one Q tile
+  constexpr int KV_BYTES = SLABS * SLAB_BYTES;         // one K or V block of 128 keys
+  constexpr uint32_t TMEM_COLS = 512;
+  constexpr uint32_t O_COL = 256;
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = smem;                                  // 2 tiles
+  uint8_t* sK = sQ + 2 * Q_BYTES;                      // 2 stages
+  uint8_t* sV = sK + 2 * KV_BYTES;                     // 2 stages
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * KV_BYTES);
+  enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
+         P_FULL = S_FULL + 2, O_FULL = P_FULL + 2, O_FREE = O_FULL + 2, NUM_BARS = O_FREE + 2 };
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  int* s_prefix = reinterpret_cast<int*>(s_tmem + 2);  // [B+1] work-item prefix per sequence
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto bar = [&](int i) { return bar0 + 8u * i; };
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < NUM_BARS; ++i) {
+      const bool per_warp = (i >= P_FULL && i < P_FULL + 2) || (i >= O_FREE && i < O_FREE + 2);
+      mbar_init(bar(i), per_warp ? 4 : 1);             // one elected arrival per softmax warp of the tile
+    }
+    *s_abort = 0;
+    fence_mbar_init();
+    int acc = 0;
+    s_prefix[0] = 0;
+    for (int b = 0; b < B; ++b) {
+      const int mb = row_offsets[b + 1] - row_offsets[b];
+      acc += ((mb + PP_ITEM_ROWS - 1) / PP_ITEM_ROWS) * H;
+      s_prefix[b + 1] = acc;
+    }
+  }
+  if (warp == 1) tc_alloc(smem_u32(s_tmem), TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+  const int total = s_prefix[B];
+  const int nblk = (N + PP_BKV - 1) / PP_BKV;
+
+  // item -> (b, h, first packed row, rows in the item (1..256))
+  auto decode = [&](int w, int& b, int& h, int& row0, int& nrows) {
+    int lo = 0, hi = B;                                 // largest b with prefix[b] <= w
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (s_prefix[mid] <= w) lo = mid; else hi = mid;
+    }
+    b = lo;
+    const int r0 = row_offsets[b], mb = row_offsets[b + 1] - r0;
+    const int parts = (mb + PP_ITEM_ROWS - 1) / PP_ITEM_ROWS;
+    const int local = w - s_prefix[b];
+    h = local / parts;
+    const int qt = local % parts;
+    row0 = r0 + qt * PP_ITEM_ROWS;
+    nrows = mb - qt * PP_ITEM_ROWS < PP_ITEM_ROWS ? mb - qt * PP_ITEM_ROWS : PP_ITEM_ROWS;
+  };
+
+  if (warp == 0) {
+    if (lane == 0) {
+      uint32_t kcnt = 0, qcnt = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++qcnt) {
+        int b, h, row0, nrows;
+        decode(w, b, h, row0, nrows);
+        const int ntile = nrows > PP_BQ ? 2 : 1;
+        if (!(ok = mbar_wait(bar(Q_FREE), (qcnt & 1) ^ 1, s_abort))) break;
+        mbar_expect_tx(bar(Q_FULL), ntile * Q_BYTES);
+        for (int t = 0; t < ntile; ++t)
+#pragma unroll
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sQ + t * Q_BYTES + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0 + t * PP_BQ, bar(Q_FULL));
+        for (int j = 0; j < nblk; ++j, ++kcnt) {
+          const int st = kcnt & 1;
+          const uint32_t ph = (kcnt >> 1) & 1;
+          const int key0 = b * N + j * PP_BKV;
+          if (!(ok = mbar_wait(bar(K_FREE + st), ph ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
+#pragma unroll
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sK + st * KV_BYTES + s * SLAB_BYTES), &tmK, h * DH + 64 * s, key0, bar(K_FULL + st));
+          if (!(ok = mbar_wait(bar(V_FREE + st), ph ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(V_FULL + st), KV_BYTES);
+#pragma unroll
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sV + st * KV_BYTES + s * SLAB_BYTES), &tmV, h * DH + 64 * s, key0, bar(V_FULL + st));
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = idesc_bf16_m128(PP_BKV, false);
+      constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
+      uint32_t kc = 0, it = 0;
+      uint32_t gt[2] = {0, 0}, itt[2] = {0, 0};          // per tile: key blocks and items so far
+      bool ok = true;
+      // S_t = Q_t K^T for the key block in stage kst
+      auto issue_s = [&](int t, int kst) {
+        const uint32_t qa = smem_u32(sQ + t * Q_BYTES), ka = smem_u32(sK + kst * KV_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < DH / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
+          tc_mma_bf16(tmem_base + t * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
+        }
+        tc_commit(bar(S_FULL + t));
+      };
+      // O_t (+)= P_t V for the key block in stage vst; jb = index of that block inside the item
+      auto issue_pv = [&](int t, int vst, int jb) -> bool {
+        if (!mbar_wait(bar(P_FULL + t), (gt[t] + jb) & 1, s_abort)) return false;
+        if (jb == 0 && !mbar_wait(bar(O_FREE + t), (itt[t] & 1) ^ 1, s_abort)) return false;
+        tc_fence_after();
+        const uint32_t va = smem_u32(sV + vst * KV_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < PP_BKV / 16; ++kk)
+          tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + kk * 8,
+                         smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, (jb | kk) != 0);
+        return true;
+      };
+      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+        int b, h, row0, nrows;
+        decode(w, b, h, row0, nrows);
+        const int ntile = nrows > PP_BQ ? 2 : 1;
+        if (!(ok = mbar_wait(bar(Q_FULL), it & 1, s_abort))) break;
+        for (int j = 0; j < nblk && ok; ++j) {
+          const int kst = (kc + j) & 1;
+          if (!(ok = mbar_wait(bar(K_FULL + kst), ((kc + j) >> 1) & 1, s_abort))) break;
+          const int vst = (kc + j - 1) & 1;
+          if (j > 0 && !(ok = mbar_wait(bar(V_FULL + vst), ((kc + j - 1) >> 1) & 1, s_abort))) break;
+          for (int t = 0; t < ntile && ok; ++t) {
+            if (j > 0) ok = issue_pv(t, vst, j - 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(t, kst);
+          }
+          if (!ok) break;
+          tc_commit(bar(K_FREE + kst));
+          if (j > 0) tc_commit(bar(V_FREE + vst));
+        }
+        if (!ok) break;
+        tc_commit(bar(Q_FREE));                          // every S product of this item has been issued
+        const int vst = (kc + nblk - 1) & 1;
+        if (!(ok = mbar_wait(bar(V_FULL + vst), ((kc + nblk - 1) >> 1) & 1, s_abort))) break;
+        for (int t = 0; t < ntile && ok; ++t) {
+          ok = issue_pv(t, vst, nblk - 1);
+          if (ok) tc_commit(bar(O_FULL + t));
+        }
+        if (!ok) break;
+        tc_commit(bar(V_FREE + vst));
+        kc += nblk;
+        for (int t = 0; t < ntile; ++t) {
+          gt[t] += nblk;
+          ++itt[t];
+        }
+      }
+    }
+  } else {
+    const int t = (warp - 2) >> 2;                       // tile of this warp
+    const int quarter = warp & 3;                        // tensor-memory lane quarter this warp may access
+    const int trow = quarter * 32 + lane;                // query row of this thread inside the tile
+    const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
+    const uint32_t s_addr = tmem_base + tlane + t * 128;
+    const uint32_t o_addr = tmem_base + tlane + O_COL + t * DH;
+    uint32_t g = 0, it = 0;
+    bool ok = true;
+#ifdef ATT_PROFILE
+    unsigned long long tp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t0 = clock64(), t1;
+#define ATT_T(i) { t1 = clock64(); tp[i] += t1 - t0; t0 = t1; }
+#else
+#define ATT_T(i)
+#endif
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+      int b, h, row0, nrows;
+      decode(w, b, h, row0, nrows);
+      const int rows_t = nrows - t * PP_BQ;              // rows of this tile (<= 0: the item has no second tile)
+      if (rows_t <= 0) continue;
+      float m_used = 0.f, l = 0.f;
+      for (int j = 0; j < nblk; ++j) {
+        ATT_T(0)
+        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + t), (g + j) & 1, s_abort));
+        if (!ok) break;
+        ATT_T(1)
+        tc_fence_after();
+        uint32_t s[128];
+        tc_ld32(s_addr, s);
+        tc_ld32(s_addr + 32, s + 32);
+        tc_ld32(s_addr + 64, s + 64);
+        tc_ld32(s_addr + 96, s + 96);
+        tc_wait_ld();
+        ATT_T(2)
+        const int nvalid = N - j * PP_BKV;               // keys of this block that exist
+        if (nvalid < PP_BKV) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c)
+            if (c >= nvalid) s[c] = 0xff800000u;         // -inf
+        }
+        float mx4[4] = {__uint_as_float(s[0]), __uint_as_float(s[1]), __uint_as_float(s[2]), __uint_as_float(s[3])};
+#pragma unroll
+        for (int c = 4; c < 124; c += 8) {
+          mx4[0] = max3(mx4[0], __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+          mx4[1] = max3(mx4[1], __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+          mx4[2] = max3(mx4[2], __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+          mx4[3] = max3(mx4[3], __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+        }
+        mx4[0] = max3(mx4[0], __uint_as_float(s[124]), __uint_as_float(s[125]));
+        mx4[1] = max3(mx4[1], __uint_as_float(s[126]), __uint_as_float(s[127]));
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+        ATT_T(3)
+        bool need = false;
+        float corr = 1.f;
+        if (j == 0) {
+          m_used = mx;
+        } else if (mx > m_used + 8.f) {
+          need = true;
+          corr = fast_exp2(m_used - mx);
+          m_used = mx;
+          l *= corr;
+        }
+        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
+#pragma unroll
+        for (int c = 0; c < 128; c += 2) {
+          const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
+          const float2 p = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+          sum2[(c >> 1) & 1] = __fadd2_rn(sum2[(c >> 1) & 1], p);
+          s[c >> 1] = pack_bf16(p.x, p.y);               // packed P over the registers whose scores are spent
+        }
+        l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+        ATT_T(4)
+        tc_st32(s_addr, s);                              // P: keys 2c, 2c+1 in column c of the S tile
+        tc_st32(s_addr + 32, s + 32);
+        if (j > 0 && __any_sync(0xffffffffu, need)) {    // S of this block is complete, so the previous P V is too
+#pragma unroll 1
+          for (int c = 0; c < DH; c += 32) {
+            uint32_t ov[32];
+            tc_ld32(o_addr + c, ov);
+            tc_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * corr);
+            tc_st32(o_addr + c, ov);
+          }
+        }
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(P_FULL + t));
+        ATT_T(5)
+      }
+      if (!ok) break;
+      g += nblk;
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(O_FULL + t), it & 1, s_abort));   // last P V of the item done
+      if (!ok) break;
+      ++it;
+      ATT_T(6)
+      tc_fence_after();
+      const float inv = 1.f / l;
+      bf16* orow = o + ((long long)(row0 + t * PP_BQ + trow) * H + h) * DH;
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 32) {
+        uint32_t ov[32];
+        tc_ld32(o_addr + c, ov);
+        tc_wait_ld();
+        if (trow < rows_t) {
+#pragma unroll
+          for (int k = 0; k < 32; k += 8) {
+            uint4 v;
+            v.x = pack_bf16(__uint_as_float(ov[k]) * inv, __uint_as_float(ov[k + 1]) * inv);
+            v.y = pack_bf16(__uint_as_float(ov[k + 2]) * inv, __uint_as_float(ov[k + 3]) * inv);
+            v.z = pack_bf16(__uint_as_float(ov[k + 4]) * inv, __uint_as_float(ov[k + 5]) * inv);
+            v.w = pack_bf16(__uint_as_float(ov[k + 6]) * inv, __uint_as_float(ov[k + 7]) * inv);
+            *reinterpret_cast<uint4*>(orow + c + k) = v;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(O_FREE + t));
+      ATT_T(7)
+    }
+#ifdef ATT_PROFILE
+    if (prof && blockIdx.x == 0 && (warp == 2 || warp == 6) && lane == 0)
+      for (int i = 0; i < 8; ++i) prof[(warp == 6 ? 8 : 0) + i] = tp[i];
+#endif
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_ATTN_TIMEOUT);
+  if (warp == 1) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+template <int DH>
+static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
+                        int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
+  constexpr int SLABS = DH / 64;
+  const int smem = 6 * SLABS * 128 * 128 + 1024 + 512 + 4 * (B + 2);
+  static int attr_smem = 0;
+  if (smem > attr_smem) {
+    SL_CUDA_TRY(cudaFuncSetAttribute(attention_pp_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_smem = smem;
+  }
+  long long items = (long long)H * ((max_rows + PP_ITEM_ROWS - 1) / PP_ITEM_ROWS + B);
+  int grid = sm_count();
+  if (items < grid) grid = (int)items;
+  if (grid < 1) grid = 1;
+  const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
+  unsigned long long* prof = nullptr;
+#ifdef ATT_PROFILE
+  static unsigned long long* d_prof = nullptr;
+  if (!d_prof) cudaMalloc(&d_prof, 128);
+  prof = d_prof;
+#endif
+  attention_pp_kernel<DH><<<grid, PP_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status, prof);
+#ifdef ATT_PROFILE
+  {
+    unsigned long long h[16];
+    cudaMemcpy(h, d_prof, 128, cudaMemcpyDeviceToHost);
+    for (int t = 0; t < 2; ++t)
+      fprintf(stderr, "ATT_PROFILE tile %d cycles: loop %llu waitS %llu ldS %llu max %llu exp %llu stP %llu waitO %llu epi %llu\n",
+              t, h[8 * t], h[8 * t + 1], h[8 * t + 2], h[8 * t + 3], h[8 * t + 4], h[8 * t + 5], h[8 * t + 6], h[8 * t + 7]);
+  }
+#endif
+  SL_CUDA_TRY(cudaGetLastError());
+  return SL_OK;
+}
+
+int launch_attention_tc2(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
+  if ((head_dim != 64 && head_dim != 128) || B > PP_MAX_B || max_rows < 1 || !row_offsets) return SL_EUNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |
+       reinterpret_cast<uintptr_t>(o)) & 15)
+    return SL_EUNSUPPORTED;
+  CUtensorMap tq, tk, tv;
+  const long long cols = (long long)H * head_dim;
+  int rc = get_tensor_map_2d(q, max_rows, cols, 128, &tq);
+  if (rc != SL_OK) return rc;
+  rc = get_tensor_map_2d(kc, (long long)B * N, cols, 128, &tk);
+  if (rc != SL_OK) return rc;
+  rc = get_tensor_map_2d(vc, (long long)B * N, cols, 128, &tv);
+  if (rc != SL_OK) return rc;
+  return head_dim == 128 ? launch_pp_dh<128>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st)
+                         : launch_pp_dh<64>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st);
+}
+
+int launch_attention_tc1(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
+
+// SURELOCK_ATT_IMPL=1 selects the single-tile kernel (for A/B measurements); default is the two-tile kernel.
+int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                        int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
+  static int impl = -1;
+  if (impl < 0) {
+    const char* e = getenv("SURELOCK_ATT_IMPL");
+    impl = e ? atoi(e) : 0;
+  }
+  return impl == 1 ? launch_attention_tc1(q, kc, vc, row_offsets, max_rows, B, N, H, head_dim, o, status, st)
+                   : launch_attention_tc2(q, kc, vc, row_offsets, max_rows, B, N, H, head_dim, o, status, st);
+}
+
+}  // namespace sl
