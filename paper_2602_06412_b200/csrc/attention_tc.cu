@@ -1,59 +1,81 @@
-// Tensor-core M x N attention on sm_100a (Algorithm 1 line 12; Sec. 2.1: the packed queries of the active rows
-// attend to ALL N cached keys/values of their sequence, bidirectional, no mask).
+// Tensor-core M x N attention on sm_100a, two query tiles per CTA (Algorithm 1 line 12; Sec. 2.1: the packed queries of
+// the active rows attend to ALL N cached keys/values of their sequence, bidirectional, no mask).
 //
-// Work item = (sequence b, head h, tile of up to 128 consecutive packed rows of that sequence); items never
-// straddle sequences.  Persistent CTAs take items round-robin; the q-tile index runs fastest so CTAs working at the
-// same time read the same K/V head through L2.  Per item the keys are streamed in blocks of 128:
-//   warp 0    TMA producer: Q tile once, then K and V blocks (two stages each), token-major cache rows, 128-byte swizzle;
-//   warp 1    one thread issues S = Q K^T (tcgen05.mma, 128x128xd_h, accumulator in tensor memory, two S buffers so
-//             S of block j+1 is computed while block j is in the softmax) and O += P V (V is the MN-major operand);
-//   warps 2-9 softmax: two threads share one query row, 64 of the block's 128 scores each (the exponentials of a block
-//             are bound by the SM's 16 special-function results per clock, so all four schedulers carry two softmax
-//             warps): tcgen05.ld the scores, online max / sum in fp32 with the 1/sqrt(d_h) scale folded into an exp2
-//             (each thread also reads its partner's 64 scores for the row maximum: cheaper than an exchange),
-//             P written as bf16 into swizzled shared memory.
-//             O stays in tensor memory; it is rescaled (tcgen05.ld / st) only when a row's running maximum grows by
-//             more than 2^8, so after the first blocks the correction is almost never taken.  The final O / l is
-//             stored as bf16.
-// Keys beyond N in the last block are masked to -inf.  All waits are bounded (SL_DEV_ATTN_TIMEOUT).
+// Work item = (sequence b, head h, up to 256 consecutive packed rows of that sequence = two tiles of 128; one tile
+// when that spreads a small problem over more SMs, decided on the device from the row counts); items never straddle
+// sequences.  Persistent CTAs take items round-robin, the row-tile index fastest, so CTAs working at the same
+// time read the same K/V head through L2.  Keys are streamed in blocks of 128.
+//   warp 0     TMA producer: both Q tiles once per item, then K and V blocks (two stages each), token-major cache rows,
+//              128-byte swizzle;
+//   warp 1     one thread issues, per key block and tile t: O_t += P_t V (previous block; P_t is read from TENSOR
+//              MEMORY as the A operand, V is the MN-major shared-memory operand) and then S_t = Q_t K^T;
+//   warps 2-5  softmax of tile 0, warps 6-9 softmax of tile 1: ONE thread per query row (no exchange between
+//              threads): tcgen05.ld the 128 scores, running max / sum in fp32 with 1/sqrt(d_h) folded into an exp2,
+//              P written back as packed bf16 over the last 64 columns of the S tile (tcgen05.st), in two halves so
+//              that the first half of P V runs under the second half of the exponentials.
+// The two tiles alternate: while the softmax warps of one tile work, the tensor pipe runs the other tile's two
+// products, and each scheduler's special-function unit always has one of its two softmax warps to feed.
+// O stays in tensor memory and is rescaled only when a row's running maximum grows by more than 2^8; O / l is stored
+// as bf16 at the end of the item.  Keys beyond N in the last block are masked to -inf.  All waits are bounded
+// (SL_DEV_ATTN_TIMEOUT).
+//
+// Tensor memory (512 columns): S0 [0,128)  S1 [128,256)  O0 [256,256+d_h)  O1 [256+d_h, 256+2 d_h).
 #include <stdio.h>
+#include <type_traits>
 
 #include "tc_common.cuh"
 
 namespace sl {
 
-constexpr int AT_THREADS = 320;   // TMA warp, MMA warp, 8 softmax warps (two per tensor-memory lane quarter)
-constexpr int AT_BQ = 128, AT_BKV = 128;
-constexpr int AT_MAX_B = 1024;
+namespace {
+
+constexpr int PP_THREADS = 320;   // TMA warp, MMA warp, 4 softmax warps per tile
+constexpr int PP_BQ = 128, PP_BKV = 128, PP_ITEM_ROWS = 256;
+constexpr int PP_MAX_B = 1024;
+
+// D[tmem] (+)= A[tmem] * B[smem]: A = 128 lanes x 8 columns, two bf16 per column (K = 16)
+__device__ __forceinline__ void tc_mma_bf16_ta(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accum) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accum)
+      : "memory");
+}
+
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+}  // namespace
 
 template <int DH>
-__global__ void __launch_bounds__(AT_THREADS, 1)
-attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+__global__ void __launch_bounds__(PP_THREADS, 1)
+attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
                     bf16* __restrict__ o, float scale_log2, int32_t* status, unsigned long long* prof) {
   constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
   constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
-  constexpr int Q_BYTES = SLABS * SLAB_BYTES;
+  constexpr int Q_BYTES = SLABS * SLAB_BYTES;          // one Q tile
   constexpr int KV_BYTES = SLABS * SLAB_BYTES;         // one K or V block of 128 keys
-  constexpr int P_BYTES = 2 * SLAB_BYTES;              // 128 queries x 128 keys, bf16
-  constexpr uint32_t TMEM_COLS = 512;                  // S0 [0,128) S1 [128,256) O [256,256+DH)
+  constexpr uint32_t TMEM_COLS = 512;
   constexpr uint32_t O_COL = 256;
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = smem;
-  uint8_t* sK = sQ + Q_BYTES;                          // 2 stages
+  uint8_t* sQ = smem;                                  // 2 tiles
+  uint8_t* sK = sQ + 2 * Q_BYTES;                      // 2 stages
   uint8_t* sV = sK + 2 * KV_BYTES;                     // 2 stages
-  uint8_t* sP = sV + 2 * KV_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sP + P_BYTES);
-  // q_full, q_free, k_full[2], k_free[2], v_full[2], v_free[2], s_full[2], s_free[2], p_full, p_free, o_free,
-  // x_sum (the two threads of a row add their partial sums here; an mbarrier, so that this wait is bounded too)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * KV_BYTES);
   enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
-         S_FREE = S_FULL + 2, P_FULL = S_FREE + 2, P_FREE, O_FREE, X_SUM, NUM_BARS };
+         P_HALF = S_FULL + 2, P_FULL = P_HALF + 2, O_FULL = P_FULL + 2, O_FREE = O_FULL + 2,
+         X_PROF = O_FREE + 2, NUM_BARS = X_PROF + 1 };
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  float* s_xsum = reinterpret_cast<float*>(s_tmem + 2);    // [2 halves][128 rows] partial row sums at the end of an item
-  int* s_prefix = reinterpret_cast<int*>(s_xsum + 256);  // [B+1] work-item prefix per sequence
+  int* s_item_rows = reinterpret_cast<int*>(s_tmem + 2);
+  int* s_prefix = reinterpret_cast<int*>(s_tmem + 3);  // [B+1] work-item prefix per sequence
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -61,20 +83,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < NUM_BARS; ++i) {
-      uint32_t cnt = 1;
-      if (i == S_FREE || i == S_FREE + 1 || i == O_FREE) cnt = 8;
-      if (i == P_FULL || i == X_SUM) cnt = 8;   // one elected arrival per softmax warp
-      mbar_init(bar(i), cnt);
+      const bool per_warp = (i >= P_HALF && i < P_FULL + 2) || (i >= O_FREE && i < O_FREE + 2);
+      mbar_init(bar(i), per_warp ? 4 : 1);             // one elected arrival per softmax warp of the tile
     }
     *s_abort = 0;
     fence_mbar_init();
-    int acc = 0;
-    s_prefix[0] = 0;
-    for (int b = 0; b < B; ++b) {
-      const int mb = row_offsets[b + 1] - row_offsets[b];
-      acc += ((mb + AT_BQ - 1) / AT_BQ) * H;
-      s_prefix[b + 1] = acc;
+    // items of two tiles, unless one-tile items finish sooner: a one-tile item takes about 0.8 of the time of a
+    // two-tile item (its softmax warps and the tensor pipe alternate instead of overlapping), so they win when they
+    // spread over idle SMs, i.e. when 4 * rounds(one-tile) < 5 * rounds(two-tile)
+    int rows = PP_ITEM_ROWS, rounds2 = 0;
+    for (int pass = 0; pass < 3; ++pass) {
+      int acc = 0;
+      s_prefix[0] = 0;
+      for (int b = 0; b < B; ++b) {
+        const int mb = row_offsets[b + 1] - row_offsets[b];
+        acc += ((mb + rows - 1) / rows) * H;
+        s_prefix[b + 1] = acc;
+      }
+      const int rounds = (acc + (int)gridDim.x - 1) / (int)gridDim.x;
+      if (pass == 0) {
+        rounds2 = rounds;
+        rows = PP_BQ;                                    // try one-tile items
+      } else if (pass == 1) {
+        if (4 * rounds < 5 * rounds2) break;             // keep one-tile items
+        rows = PP_ITEM_ROWS;                             // back to two-tile items
+      } else {
+        break;
+      }
     }
+    *s_item_rows = rows;
   }
   if (warp == 1) tc_alloc(smem_u32(s_tmem), TMEM_COLS);
   tc_fence_before();
@@ -82,9 +119,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
   const int total = s_prefix[B];
-  const int nblk = (N + AT_BKV - 1) / AT_BKV;
+  const int item_rows = *s_item_rows;
+  const int nblk = (N + PP_BKV - 1) / PP_BKV;
 
-  // item -> (b, h, first packed row, rows in tile)
+  // item -> (b, h, first packed row, rows in the item (1..256))
   auto decode = [&](int w, int& b, int& h, int& row0, int& nrows) {
     int lo = 0, hi = B;                                 // largest b with prefix[b] <= w
     while (hi - lo > 1) {
@@ -93,12 +131,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     b = lo;
     const int r0 = row_offsets[b], mb = row_offsets[b + 1] - r0;
-    const int tiles = (mb + AT_BQ - 1) / AT_BQ;
+    const int parts = (mb + item_rows - 1) / item_rows;
     const int local = w - s_prefix[b];
-    h = local / tiles;
-    const int qt = local % tiles;
-    row0 = r0 + qt * AT_BQ;
-    nrows = mb - qt * AT_BQ < AT_BQ ? mb - qt * AT_BQ : AT_BQ;
+    h = local / parts;
+    const int qt = local % parts;
+    row0 = r0 + qt * item_rows;
+    nrows = mb - qt * item_rows < item_rows ? mb - qt * item_rows : item_rows;
   };
 
   if (warp == 0) {
@@ -108,14 +146,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++qcnt) {
         int b, h, row0, nrows;
         decode(w, b, h, row0, nrows);
+        const int ntile = nrows > PP_BQ ? 2 : 1;
         if (!(ok = mbar_wait(bar(Q_FREE), (qcnt & 1) ^ 1, s_abort))) break;
-        mbar_expect_tx(bar(Q_FULL), Q_BYTES);
+        mbar_expect_tx(bar(Q_FULL), ntile * Q_BYTES);
+        for (int t = 0; t < ntile; ++t)
 #pragma unroll
-        for (int s = 0; s < SLABS; ++s) tma_load_2d(smem_u32(sQ + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0, bar(Q_FULL));
+          for (int s = 0; s < SLABS; ++s)
+            tma_load_2d(smem_u32(sQ + t * Q_BYTES + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0 + t * PP_BQ, bar(Q_FULL));
         for (int j = 0; j < nblk; ++j, ++kcnt) {
           const int st = kcnt & 1;
           const uint32_t ph = (kcnt >> 1) & 1;
-          const int key0 = b * N + j * AT_BKV;
+          const int key0 = b * N + j * PP_BKV;
           if (!(ok = mbar_wait(bar(K_FREE + st), ph ^ 1, s_abort))) break;
           mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
 #pragma unroll
@@ -131,127 +172,174 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16_m128(AT_BKV, false);
+      constexpr uint32_t idesc_s = idesc_bf16_m128(PP_BKV, false);
       constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
-      uint32_t g = 0, it = 0;
+      uint32_t kc = 0, it = 0;
+      uint32_t gt[2] = {0, 0}, itt[2] = {0, 0};          // per tile: key blocks and items so far
       bool ok = true;
-      // S(gi) = Q K^T for global block gi into S buffer gi & 1
-      auto issue_s = [&](uint32_t gi) -> bool {
-        const int st = gi & 1;
-        const uint32_t ph = (gi >> 1) & 1;
-        if (!mbar_wait(bar(K_FULL + st), ph, s_abort)) return false;
-        if (!mbar_wait(bar(S_FREE + st), ph ^ 1, s_abort)) return false;
-        tc_fence_after();
-        const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * KV_BYTES);
+#ifdef ATT_PROFILE
+      unsigned long long mp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, m0 = clock64(), m1;
+      uint32_t xp = 0;
+#define ATT_M(i) { m1 = clock64(); mp[i] += m1 - m0; m0 = m1; }
+#else
+#define ATT_M(i)
+#endif
+      // S_t = Q_t K^T for the key block in stage kst
+      auto issue_s = [&](int t, int kst) {
+#ifdef ATT_PROFILE2
+        ATT_M(0)
+#endif
+        const uint32_t qa = smem_u32(sQ + t * Q_BYTES), ka = smem_u32(sK + kst * KV_BYTES);
 #pragma unroll
         for (int kk = 0; kk < DH / 16; ++kk) {
           const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
-          tc_mma_bf16(tmem_base + st * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
+          tc_mma_bf16(tmem_base + t * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
         }
-        tc_commit(bar(K_FREE + st));
-        tc_commit(bar(S_FULL + st));
+        tc_commit(bar(S_FULL + t));
+#ifdef ATT_PROFILE2
+        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(6) }
+#endif
+      };
+      // O_t (+)= P_t V for the key block in stage vst; jb = index of that block inside the item
+      auto issue_pv = [&](int t, int vst, int jb) -> bool {
+        const uint32_t va = smem_u32(sV + vst * KV_BYTES);
+        ATT_M(0)
+        if (!mbar_wait(bar(P_HALF + t), (gt[t] + jb) & 1, s_abort)) return false;
+        ATT_M(1 + t)
+        if (jb == 0 && !mbar_wait(bar(O_FREE + t), (itt[t] & 1) ^ 1, s_abort)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < PP_BKV / 32; ++kk)
+          tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                         smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, (jb | kk) != 0);
+#ifdef ATT_PROFILE2
+        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(7) }
+#else
+        ATT_M(0)
+#endif
+        if (!mbar_wait(bar(P_FULL + t), (gt[t] + jb) & 1, s_abort)) return false;
+        ATT_M(3 + t)
+        tc_fence_after();
+#pragma unroll
+        for (int kk = PP_BKV / 32; kk < PP_BKV / 16; ++kk)
+          tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                         smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, 1);
+#ifdef ATT_PROFILE2
+        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(7) }
+#endif
         return true;
       };
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+        int b, h, row0, nrows;
+        decode(w, b, h, row0, nrows);
+        const int ntile = nrows > PP_BQ ? 2 : 1;
         if (!(ok = mbar_wait(bar(Q_FULL), it & 1, s_abort))) break;
-        if (!(ok = issue_s(g))) break;
         for (int j = 0; j < nblk && ok; ++j) {
-          const uint32_t gj = g + j;
-          if (j + 1 < nblk) {
-            if (!(ok = issue_s(gj + 1))) break;
-          } else {
-            tc_commit(bar(Q_FREE));                      // every S MMA of this item has been issued
+          const int kst = (kc + j) & 1;
+          ATT_M(0)
+          if (!(ok = mbar_wait(bar(K_FULL + kst), ((kc + j) >> 1) & 1, s_abort))) break;
+          const int vst = (kc + j - 1) & 1;
+          if (j > 0 && !(ok = mbar_wait(bar(V_FULL + vst), ((kc + j - 1) >> 1) & 1, s_abort))) break;
+          ATT_M(5)
+          for (int t = 0; t < ntile && ok; ++t) {
+            if (j > 0) ok = issue_pv(t, vst, j - 1);
+            if (!ok) break;
+            tc_fence_after();
+            issue_s(t, kst);
           }
-          const int st = gj & 1;
-          const uint32_t ph = (gj >> 1) & 1;
-          if (!(ok = mbar_wait(bar(P_FULL), gj & 1, s_abort))) break;
-          if (!(ok = mbar_wait(bar(V_FULL + st), ph, s_abort))) break;
-          if (j == 0 && !(ok = mbar_wait(bar(O_FREE), (it & 1) ^ 1, s_abort))) break;
-          tc_fence_after();
-          const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * KV_BYTES);
-#pragma unroll
-          for (int kk = 0; kk < AT_BKV / 16; ++kk) {
-            const uint64_t ad = smem_desc_k_sw128(pa + (kk >> 2) * SLAB_BYTES + (kk & 3) * 32);
-            const uint64_t bd = smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES);
-            tc_mma_bf16(tmem_base + O_COL, ad, bd, idesc_o, (j | kk) != 0);
-          }
-          tc_commit(bar(V_FREE + st));
-          tc_commit(bar(P_FREE));
+          if (!ok) break;
+          tc_commit(bar(K_FREE + kst));
+          if (j > 0) tc_commit(bar(V_FREE + vst));
         }
-        g += nblk;
+        if (!ok) break;
+        tc_commit(bar(Q_FREE));                          // every S product of this item has been issued
+        const int vst = (kc + nblk - 1) & 1;
+        if (!(ok = mbar_wait(bar(V_FULL + vst), ((kc + nblk - 1) >> 1) & 1, s_abort))) break;
+        for (int t = 0; t < ntile && ok; ++t) {
+          ok = issue_pv(t, vst, nblk - 1);
+          if (ok) tc_commit(bar(O_FULL + t));
+        }
+        if (!ok) break;
+        tc_commit(bar(V_FREE + vst));
+        kc += nblk;
+        for (int t = 0; t < ntile; ++t) {
+          gt[t] += nblk;
+          ++itt[t];
+        }
       }
+#ifdef ATT_PROFILE
+      ATT_M(0)
+      if (prof && blockIdx.x == 0)
+        for (int i = 0; i < 8; ++i) prof[16 + i] = mp[i];
+#endif
     }
   } else {
-    const int quarter = warp & 3;
-    const int half = (warp - 2) >> 2;                    // which 64 of the block's 128 keys (and which half of O)
+    const int t = (warp - 2) >> 2;                       // tile of this warp
+    const int quarter = warp & 3;                        // tensor-memory lane quarter this warp may access
     const int trow = quarter * 32 + lane;                // query row of this thread inside the tile
     const uint32_t tlane = (uint32_t)(quarter * 32) << 16;
-    constexpr int OH = DH / 2;                           // O columns per thread
+    const uint32_t s_addr = tmem_base + tlane + t * 128;
+    const uint32_t o_addr = tmem_base + tlane + O_COL + t * DH;
     uint32_t g = 0, it = 0;
     bool ok = true;
+    // O row *= corr (whole warp; rows whose maximum did not move pass 1)
+    auto rescale_o = [&](float corr) {
+#pragma unroll 1
+      for (int c = 0; c < DH; c += 32) {
+        uint32_t ov[32];
+        tc_ld32(o_addr + c, ov);
+        tc_wait_ld();
+#pragma unroll
+        for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * corr);
+        tc_st32(o_addr + c, ov);
+      }
+      tc_wait_st();
+    };
 #ifdef ATT_PROFILE
     unsigned long long tp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t0 = clock64(), t1;
 #define ATT_T(i) { t1 = clock64(); tp[i] += t1 - t0; t0 = t1; }
 #else
 #define ATT_T(i)
 #endif
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
       int b, h, row0, nrows;
       decode(w, b, h, row0, nrows);
+      const int rows_t = nrows - t * PP_BQ;              // rows of this tile (<= 0: the item has no second tile)
+      if (rows_t <= 0) continue;
       float m_used = 0.f, l = 0.f;
-      for (int j = 0; j < nblk; ++j) {
-        const uint32_t gj = g + j;
-        const int sb = gj & 1;
-        const uint32_t ph = (gj >> 1) & 1;
+      // one key block of this tile; MASKED only for a last block that reaches beyond key N (kept apart so that the
+      // common path is free of branches and the compiler can interleave loads, maxima and exponentials)
+      auto block = [&](int j, auto masked_tag) -> bool {
+        constexpr bool MASKED = decltype(masked_tag)::value;
         ATT_T(0)
-        ok = __all_sync(0xffffffffu, mbar_wait(bar(S_FULL + sb), ph, s_abort));
-        if (!ok) break;
+        if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + t), (g + j) & 1, s_abort))) return false;
         ATT_T(1)
         tc_fence_after();
-        // this thread's 64 scores, and the partner's 64 as well: the row maximum needs all 128, and reading them from
-        // tensor memory in the same batch is cheaper than an exchange through shared memory
-        uint32_t s[64], t[64];
-        tc_ld32(tmem_base + tlane + sb * 128 + half * 64, s);
-        tc_ld32(tmem_base + tlane + sb * 128 + half * 64 + 32, s + 32);
-        tc_ld32(tmem_base + tlane + sb * 128 + (half ^ 1) * 64, t);
-        tc_ld32(tmem_base + tlane + sb * 128 + (half ^ 1) * 64 + 32, t + 32);
+        uint32_t s[128];
+        tc_ld32(s_addr, s);
+        tc_ld32(s_addr + 32, s + 32);
+        tc_ld32(s_addr + 64, s + 64);
+        tc_ld32(s_addr + 96, s + 96);
         tc_wait_ld();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(S_FREE + sb));
         ATT_T(2)
-        const int nvalid = N - j * AT_BKV - half * 64;   // keys of this thread's 64 that exist
-        if (nvalid < 64) {
+        if (MASKED) {
+          const int nvalid = N - j * PP_BKV;             // keys of this block that exist
 #pragma unroll
-          for (int c = 0; c < 64; ++c)
+          for (int c = 0; c < 128; ++c)
             if (c >= nvalid) s[c] = 0xff800000u;         // -inf
         }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+        float mx8[8];
 #pragma unroll
-        for (int c = 0; c < 64; c += 4) {
-          mx4[0] = fmaxf(mx4[0], __uint_as_float(s[c]));
-          mx4[1] = fmaxf(mx4[1], __uint_as_float(s[c + 1]));
-          mx4[2] = fmaxf(mx4[2], __uint_as_float(s[c + 2]));
-          mx4[3] = fmaxf(mx4[3], __uint_as_float(s[c + 3]));
+        for (int c = 0; c < 8; ++c) mx8[c] = __uint_as_float(s[c]);
+#pragma unroll
+        for (int c = 8; c < 120; c += 16) {
+#pragma unroll
+          for (int k = 0; k < 8; ++k) mx8[k] = max3(mx8[k], __uint_as_float(s[c + 2 * k]), __uint_as_float(s[c + 2 * k + 1]));
         }
-        {
-          const int ovalid = N - j * AT_BKV - (half ^ 1) * 64;
-          if (ovalid >= 64) {
 #pragma unroll
-            for (int c = 0; c < 64; c += 4) {
-              mx4[0] = fmaxf(mx4[0], __uint_as_float(t[c]));
-              mx4[1] = fmaxf(mx4[1], __uint_as_float(t[c + 1]));
-              mx4[2] = fmaxf(mx4[2], __uint_as_float(t[c + 2]));
-              mx4[3] = fmaxf(mx4[3], __uint_as_float(t[c + 3]));
-            }
-          } else {
-#pragma unroll
-            for (int c = 0; c < 64; ++c)
-              if (c < ovalid) mx4[c & 3] = fmaxf(mx4[c & 3], __uint_as_float(t[c]));
-          }
-        }
-        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
-        ATT_T(3)
+        for (int k = 0; k < 4; ++k) mx8[k] = max3(mx8[k], __uint_as_float(s[120 + 2 * k]), __uint_as_float(s[121 + 2 * k]));
+        const float mx = max3(max3(mx8[0], mx8[1], mx8[2]), max3(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])) * scale_log2;
+        // the running maximum is replaced only when it grows by more than 2^8
         bool need = false;
         float corr = 1.f;
         if (j == 0) {
@@ -262,71 +350,57 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
           m_used = mx;
           l *= corr;
         }
-        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-        uint32_t pk[32];
-        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
-#pragma unroll
-        for (int c = 0; c < 64; c += 2) {
-          const float2 t = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);
-          const float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
-          sum2[(c >> 1) & 1] = __fadd2_rn(sum2[(c >> 1) & 1], p);
-          pk[c >> 1] = pack_bf16(p.x, p.y);
-        }
-        l += (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+        // S of this block is complete, so the previous block's P V is too, and this block's has not been issued
+        if (j > 0 && __any_sync(0xffffffffu, need)) rescale_o(corr);
+        ATT_T(3)
         ATT_T(4)
-        if (gj > 0) {
-          ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (gj - 1) & 1, s_abort));   // P V of the previous block done
-          if (!ok) break;
-        }
-        ATT_T(5)
-        if (j > 0 && __any_sync(0xffffffffu, need)) {      // both threads of a row take the same decision
-          tc_fence_after();
-#pragma unroll 1
-          for (int c = 0; c < OH; c += 32) {
-            uint32_t ov[32];
-            tc_ld32(tmem_base + tlane + O_COL + half * OH + c, ov);
-            tc_wait_ld();
-#pragma unroll
-            for (int k = 0; k < 32; ++k) ov[k] = __float_as_uint(__uint_as_float(ov[k]) * corr);
-            tc_st32(tmem_base + tlane + O_COL + half * OH + c, ov);
-          }
-          tc_wait_st();
-        }
-        // P row -> shared memory, 128-byte swizzle: 16-byte chunk c of row r sits at chunk position c ^ (r & 7);
-        // this thread's 64 keys are exactly one 128-byte row of slab `half`
-        {
-          uint8_t* prow = sP + half * SLAB_BYTES + (trow >> 3) * 1024 + (trow & 7) * 128;
-#pragma unroll
-          for (int c = 0; c < 8; ++c)
-            *reinterpret_cast<uint4*>(prow + ((c ^ (trow & 7)) << 4)) =
-                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-        }
-        fence_async_smem();
+        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
+        float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#define PP_EXP32(c0)                                                                                                   \
+  _Pragma("unroll") for (int c = (c0); c < (c0) + 32; c += 2) {                                                        \
+    const float2 x = __ffma2_rn(make_float2(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), sc2, nm2);              \
+    const float2 p = make_float2(fast_exp2(x.x), fast_exp2(x.y));                                                      \
+    sum2[(c >> 1) & 3] = __fadd2_rn(sum2[(c >> 1) & 3], p);                                                            \
+    s[c >> 1] = pack_bf16(p.x, p.y);                     /* packed P over the registers whose scores are spent */      \
+  }
+        PP_EXP32(0)
+        PP_EXP32(32)
+        // P: keys 2c, 2c+1 in column 64 + c of the S tile (whose scores are all in registers by now)
+        tc_st32(s_addr + 64, s);                         // keys 0..63
+        PP_EXP32(64)
+        tc_wait_st();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(bar(P_FULL));
+        if (lane == 0) mbar_arrive(bar(P_HALF + t));     // the first half of P V can start
+        ATT_T(5)
+        PP_EXP32(96)
+        tc_st32(s_addr + 96, s + 32);                    // keys 64..127
+        sum2[0] = __fadd2_rn(__fadd2_rn(sum2[0], sum2[1]), __fadd2_rn(sum2[2], sum2[3]));
+        l += sum2[0].x + sum2[0].y;
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(P_FULL + t));
         ATT_T(6)
-      }
+        return true;
+      };
+      const int nfast = (N % PP_BKV) ? nblk - 1 : nblk;
+      for (int j = 0; j < nfast && ok; ++j) ok = block(j, std::false_type{});
+      if (ok && nfast < nblk) ok = block(nblk - 1, std::true_type{});
       if (!ok) break;
       g += nblk;
-      // row sum: add the partner's half
-      s_xsum[half * 128 + trow] = l;
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(X_SUM));
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(X_SUM), it & 1, s_abort));
+      ok = __all_sync(0xffffffffu, mbar_wait(bar(O_FULL + t), it & 1, s_abort));   // last P V of the item done
       if (!ok) break;
-      l += s_xsum[(half ^ 1) * 128 + trow];
-      ok = __all_sync(0xffffffffu, mbar_wait(bar(P_FREE), (g - 1) & 1, s_abort));       // last P V of the item done
-      if (!ok) break;
+      ++it;
       tc_fence_after();
       const float inv = 1.f / l;
-      bf16* orow = o + ((long long)(row0 + trow) * H + h) * DH + half * OH;
+      bf16* orow = o + ((long long)(row0 + t * PP_BQ + trow) * H + h) * DH;
 #pragma unroll 1
-      for (int c = 0; c < OH; c += 32) {
+      for (int c = 0; c < DH; c += 32) {
         uint32_t ov[32];
-        tc_ld32(tmem_base + tlane + O_COL + half * OH + c, ov);
+        tc_ld32(o_addr + c, ov);
         tc_wait_ld();
-        if (trow < nrows) {
+        if (trow < rows_t) {
 #pragma unroll
           for (int k = 0; k < 32; k += 8) {
             uint4 v;
@@ -340,12 +414,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(O_FREE));
+      if (lane == 0) mbar_arrive(bar(O_FREE + t));
       ATT_T(7)
     }
 #ifdef ATT_PROFILE
-    if (prof && blockIdx.x == 0 && warp == 2 && lane == 0)
-      for (int i = 0; i < 8; ++i) prof[i] = tp[i];
+    if (prof && blockIdx.x == 0 && (warp == 2 || warp == 6) && lane == 0)
+      for (int i = 0; i < 8; ++i) prof[(warp == 6 ? 8 : 0) + i] = tp[i];
 #endif
   }
 
@@ -359,16 +433,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }
 
 template <int DH>
-static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
-                     int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
+static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
+                        int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
   constexpr int SLABS = DH / 64;
-  const int smem = 5 * SLABS * 128 * 128 + 2 * 128 * 128 + 1024 + 512 + 3072 + 4 * (B + 2);
+  const int smem = 6 * SLABS * 128 * 128 + 1024 + 512 + 4 * (B + 3);
   static int attr_smem = 0;
   if (smem > attr_smem) {
-    SL_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    SL_CUDA_TRY(cudaFuncSetAttribute(attention_pp_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
     attr_smem = smem;
   }
-  long long items = (long long)H * ((max_rows + AT_BQ - 1) / AT_BQ + B);
+  long long items = (long long)H * ((max_rows + PP_BQ - 1) / PP_BQ + B);
   int grid = sm_count();
   if (items < grid) grid = (int)items;
   if (grid < 1) grid = 1;
@@ -376,25 +450,28 @@ static int launch_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorM
   unsigned long long* prof = nullptr;
 #ifdef ATT_PROFILE
   static unsigned long long* d_prof = nullptr;
-  if (!d_prof) cudaMalloc(&d_prof, 64);
+  if (!d_prof) cudaMalloc(&d_prof, 192);
   prof = d_prof;
 #endif
-  attention_tc_kernel<DH><<<grid, AT_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status, prof);
+  attention_pp_kernel<DH><<<grid, PP_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status, prof);
 #ifdef ATT_PROFILE
   {
-    unsigned long long h[8];
-    cudaMemcpy(h, d_prof, 64, cudaMemcpyDeviceToHost);
-    fprintf(stderr, "ATT_PROFILE cycles: loop %llu waitS %llu ldS %llu max+xchg %llu exp %llu waitPV %llu writeP %llu epi %llu\n",
-            h[0], h[1], h[2], h[3], h[4], h[5], h[6], h[7]);
+    unsigned long long h[24];
+    cudaMemcpy(h, d_prof, 192, cudaMemcpyDeviceToHost);
+    fprintf(stderr, "ATT_PROFILE mma thread cycles: issue+other %llu waitPhalf0 %llu waitPhalf1 %llu waitPfull0 %llu waitPfull1 %llu waitKV %llu  S-product %llu  PV-product %llu\n",
+            h[16], h[17], h[18], h[19], h[20], h[21], h[22], h[23]);
+    for (int t = 0; t < 2; ++t)
+      fprintf(stderr, "ATT_PROFILE tile %d cycles: loop %llu waitS %llu ldS %llu max %llu turn %llu exp-to-half %llu rest %llu waitO+epi %llu\n",
+              t, h[8 * t], h[8 * t + 1], h[8 * t + 2], h[8 * t + 3], h[8 * t + 4], h[8 * t + 5], h[8 * t + 6], h[8 * t + 7]);
   }
 #endif
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }
 
-int launch_attention_tc1(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
-                        int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
-  if ((head_dim != 64 && head_dim != 128) || B > AT_MAX_B || max_rows < 1 || !row_offsets) return SL_EUNSUPPORTED;
+int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st) {
+  if ((head_dim != 64 && head_dim != 128) || B > PP_MAX_B || max_rows < 1 || !row_offsets) return SL_EUNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |
        reinterpret_cast<uintptr_t>(o)) & 15)
     return SL_EUNSUPPORTED;
@@ -406,8 +483,8 @@ int launch_attention_tc1(const void* q, const void* kc, const void* vc, const in
   if (rc != SL_OK) return rc;
   rc = get_tensor_map_2d(vc, (long long)B * N, cols, 128, &tv);
   if (rc != SL_OK) return rc;
-  return head_dim == 128 ? launch_dh<128>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st)
-                         : launch_dh<64>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st);
+  return head_dim == 128 ? launch_pp_dh<128>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st)
+                         : launch_pp_dh<64>(tq, tk, tv, row_offsets, max_rows, B, N, H, o, status, st);
 }
 
 }  // namespace sl
