@@ -228,10 +228,10 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
   A_(c->scratch, compact_scratch_bytes((int64_t)R));
   A_(c->rope, (size_t)N * (cfg->head_dim / 2) * sizeof(float2));
   if (cfg->dtype == SL_BF16) {
-    c->split.tiles = 2 * sm_count();
+    c->split.tiles = 4 * sm_count();
     A_(c->split.ws, (size_t)c->split.tiles * SPLIT_TILE_BYTES);
-    A_(c->split.counters, (size_t)c->split.tiles * sizeof(int));
-    if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * sizeof(int), c->st) != cudaSuccess)
+    A_(c->split.counters, (size_t)c->split.tiles * 3 * sizeof(int));
+    if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * 3 * sizeof(int), c->st) != cudaSuccess)
       rc = SL_ECUDA;
   }
   A_(c->theta, ((size_t)batch + 1) * 4);
@@ -491,8 +491,8 @@ int surelock_softmax_kl_sure(const void* logits, const void* prev_logits, const 
                                 dtype, mask_state, lock_mask, kl_eps, kl, conf, argmax, lse_out, (cudaStream_t)stream);
 }
 
-static size_t gemm_ws_tiles() { return 2 * (size_t)sm_count(); }
-size_t surelock_gemm_workspace_bytes(void) { return gemm_ws_tiles() * (SPLIT_TILE_BYTES + sizeof(int)); }
+static size_t gemm_ws_tiles() { return 4 * (size_t)sm_count(); }
+size_t surelock_gemm_workspace_bytes(void) { return gemm_ws_tiles() * (SPLIT_TILE_BYTES + 3 * sizeof(int)); }
 
 int surelock_conf_gate_lock(const float* conf, const float* kl, const int32_t* active_idx, const int32_t* row_offsets,
                             int B, int N, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent,

@@ -27,6 +27,22 @@
 namespace sl {
 
 constexpr int TC_BM = 128, TC_BK = 64, TC_THREADS = 192;
+constexpr int TC_MAX_STAGES = 16;
+constexpr unsigned long long SPLIT_HELP_CYCLES = 200000ull;   // how long a split waits for its siblings before leaving (~0.1 ms)
+constexpr int TC_DATA_BYTES = 216 * 1024;   // operand stages: 4 x 48 KB (128 rows of A + a 256-wide weight tile) ... 16 x 12 KB
+
+#ifdef GEMM_PROFILE
+// development aid: per-CTA time stamps (ns) of the first item of a launch
+__device__ unsigned long long g_gemm_prof[160 * 8];
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define GP(i) { g_gemm_prof[blockIdx.x * 8 + (i)] = gtime(); }
+#else
+#define GP(i) {}
+#endif
 constexpr int EPI_QKV = 3;   // three weight matrices side by side; epilogue = RoPE + packed q + K/V cache scatter
 
 struct QkvArgs {
@@ -51,8 +67,11 @@ struct TmemSrc {
     tc_wait_ld();
   }
 };
+// Partial tiles are stored column-group-major: element (r, c) of a tile at float ((c / 4) * 128 + r) * 4 + c % 4, so
+// that the 32 rows of a warp write (and the finisher's threads read) 512 contiguous bytes per float4.
 struct WsSrc {
-  const float* row;       // one row of the partial tile of split 0
+  const float* base;      // partial tile of split 0
+  int r;                  // row inside the tile
   size_t split_stride;    // floats between consecutive splits of the same tile
   int S;
   // sum over the splits in split order (deterministic), four splits' loads in flight at a time
@@ -60,14 +79,15 @@ struct WsSrc {
     float acc[32];
 #pragma unroll
     for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+    const float* p0 = base + ((size_t)(col >> 2) * TC_BM + r) * 4;
     for (int s0 = 0; s0 < S; s0 += 4) {
       float4 t[4][8];
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         if (s0 + q < S) {
-          const float4* p = reinterpret_cast<const float4*>(row + (size_t)(s0 + q) * split_stride + col);
+          const float* p = p0 + (size_t)(s0 + q) * split_stride;
 #pragma unroll
-          for (int j = 0; j < 8; ++j) t[q][j] = __ldcg(p + j);
+          for (int j = 0; j < 8; ++j) t[q][j] = __ldcg(reinterpret_cast<const float4*>(p + (size_t)j * TC_BM * 4));
         }
       }
 #pragma unroll
@@ -187,7 +207,7 @@ __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, b
 // cost more in partial-tile traffic than they gain in balance.)  Splits meet in the workspace; the last arriver of
 // a tile sums them in split order and runs the fused epilogue.
 struct TileCfg {
-  int bn, S, kb_per, m_tiles, n_tiles, tiles, total;
+  int bn, S, m_tiles, n_tiles, tiles, total;   // split sp of a tile covers K blocks [sp * num_kb / S, (sp + 1) * num_kb / S)
 };
 template <int EPI>
 __device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, int grid, bool can_split, int ws_tiles,
@@ -201,34 +221,45 @@ __device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, in
   c.bn = 256;
   c.S = 1;
   if (c.m_tiles == 1) {
-    // weight-streaming regime: 128-wide tiles, K split so that about one item per SM exists
-    c.bn = min_bn > 128 ? min_bn : 128;
-    const int tiles = ntiles(c.bn);
-    if (can_split && tiles < grid) {
-      int sp = (grid + tiles / 2) / tiles;
-      if (sp > 4) sp = 4;
-      if (sp > num_kb / 4) sp = num_kb / 4;
-      if (sp > ws_tiles / tiles) sp = ws_tiles / tiles;
-      if (sp >= 2) c.S = sp;
+    // Weight-streaming regime: the widest tiles (most bytes per copy) that, with K split at most four ways and all
+    // items in ONE round of the grid, keep at least 0.6 of the SMs streaming.  (Measured on B200: more than four splits
+    // or a second round cost more in the hand-over through the workspace than the idle SMs do; narrow tiles without a
+    // split are bounded by the ~280 ns one K block takes whatever its size.)
+    c.bn = 128 > min_bn ? 128 : min_bn;
+    for (int bn = 256; bn >= 128 && bn >= min_bn; bn >>= 1) {
+      const int tiles = ntiles(bn);
+      int sp = grid / tiles;
+      sp = sp < 1 ? 1 : (sp > 4 ? 4 : sp);
+      if (sp * 4 > num_kb) sp = num_kb / 4 > 0 ? num_kb / 4 : 1;
+      if (!can_split || sp * tiles > ws_tiles) sp = 1;
+      c.bn = bn;
+      c.S = sp;
+      if (5 * tiles * sp >= 3 * grid) break;
     }
   } else if (c.m_tiles > 1 && c.m_tiles * ntiles(256) < grid) {
-    // a few row tiles: no split; the width with the fewest (rounds of the grid x relative time of one tile), where a
-    // narrower tile re-reads the activation tile and uses the tensor pipe less well
+    // a few row tiles: tile width and K split with the least estimated time, in units of one 256-wide K block:
+    // rounds of the grid x (K blocks of an item x relative cost of a block at this width + the cost of meeting in the
+    // workspace when K is split).  A narrower tile re-reads the activation tile and uses the tensor pipe less well.
     float best = 3.0e38f;
-    for (int bn = 256; bn >= min_bn; bn >>= 1) {
-      const float cbn = bn == 256 ? 1.0f : (bn == 128 ? 0.6f : 0.42f);
-      const int rounds = (c.m_tiles * ntiles(bn) + grid - 1) / grid;
-      const float cost = (float)rounds * cbn;
-      if (cost < best - 1e-6f) {
-        best = cost;
-        c.bn = bn;
+    for (int bn = 256; bn >= min_bn && bn >= 128; bn >>= 1) {
+      const float cbn = bn == 256 ? 1.0f : 0.6f;
+      const int tiles = c.m_tiles * ntiles(bn);
+      for (int sp = 1; sp <= 8 && sp * 4 <= num_kb; ++sp) {
+        if (sp > 1 && (!can_split || sp * tiles > ws_tiles)) break;
+        const int rounds = (tiles * sp + grid - 1) / grid;
+        const float cost = (float)rounds * ((float)((num_kb + sp - 1) / sp) * cbn + (sp > 1 ? 6.f + 10.f * cbn : 0.f));
+        if (cost < best - 1e-6f) {
+          best = cost;
+          c.bn = bn;
+          c.S = sp;
+        }
       }
     }
   }
   c.n_tiles = ntiles(c.bn);
   c.tiles = c.m_tiles * c.n_tiles;
-  c.kb_per = (num_kb + c.S - 1) / c.S;
-  c.S = (num_kb + c.kb_per - 1) / c.kb_per;
+  if (c.S > num_kb) c.S = num_kb;
+  if (c.S < 1) c.S = 1;
   c.total = c.tiles * c.S;
   return c;
 }
@@ -382,38 +413,44 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
 
 template <int EPI, int STAGES>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA32,
+               const __grid_constant__ CUtensorMap tmA64, const __grid_constant__ CUtensorMap tmB0,
                const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
-               const __grid_constant__ CUtensorMap tmW2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
+               const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX0,
+               const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
                int n_out, int K, int32_t* status, const QkvArgs qkv, float* __restrict__ ws, int* __restrict__ counters,
-               int ws_tiles, int wide_boxes, int force_bn, int force_s, int pair_mode) {
-  // tmB*: weight maps with 64-row boxes (any tile width); tmW*: the same matrices with 128-row boxes, used for
-  // 256-wide tiles so a stage is filled by fewer, larger TMA copies
+               int ws_tiles, int force_bn, int force_s, int pair_mode) {
+  // tmA / tmA32 / tmA64: the activation matrix with 128-, 32- and 64-row boxes; tmB*: weight maps with 64-row boxes
+  // (any tile width); tmW* / tmX*: the same matrices with 128- and 256-row boxes: a 256-wide tile is one 256-row copy
+  // (gate/up: two 128-row copies), the CTA-pair path loads 128-row halves
   constexpr int BN_MAX = 256;
-  constexpr int A_BYTES = TC_BM * TC_BK * 2;              // 16 KB
-  constexpr int B_BYTES = BN_MAX * TC_BK * 2;             // up to 32 KB: 64-row boxes of the weight matrix
   constexpr int BOX_BYTES = 64 * TC_BK * 2;               // 8 KB
-  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
   constexpr uint32_t TMEM_COLS = 2 * BN_MAX;              // two accumulators
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   if (pair_mode) {
-    // launched as clusters of two: when the grid can be filled with 256 x 256 pair tiles (large M) the CTA-pair path
-    // takes the whole launch; both CTAs of a pair read the same M and take the same branch
+    // launched as clusters of two: the CTA-pair path takes the whole launch when 256 x 256 pair tiles fill the grid
+    // (large M) and need no more time than single tiles: rounds of pair tiles against rounds of 128 x 256 tiles, which
+    // cost about 1.15 x as much per round (more L2 -> SM traffic).  Both CTAs of a pair read the same M and take the
+    // same branch.
     const int Mp = *n_active;
     const int obn = EPI == EPI_SWIGLU ? 128 : 256;
-    if (((Mp + 255) / 256) * ((n_out + obn - 1) / obn) >= (int)(gridDim.x >> 1)) {
+    const int nt = (n_out + obn - 1) / obn, half = (int)(gridDim.x >> 1);
+    const int pairs = ((Mp + 255) / 256) * nt, singles = ((Mp + 127) / 128) * nt;
+    const int rounds_p = (pairs + half - 1) / half, rounds_s = (singles + (int)gridDim.x - 1) / (int)gridDim.x;
+    if (pairs >= half && 20 * rounds_p <= 23 * rounds_s) {
       run_pair<EPI>(&tmA, &tmW0, &tmW1, &tmW2, Cv, Mp, n_out, K, status, qkv, smem);
       return;
     }
   }
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * STAGE_BYTES);
+  if (threadIdx.x == 0) GP(0)
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TC_DATA_BYTES);
   // bars: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  volatile int* s_last = reinterpret_cast<volatile int*>(s_tmem + 2);
+  volatile int* s_fin = reinterpret_cast<volatile int*>(s_tmem + 2);   // [3] split finishing: role, ticket, claim result
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -439,6 +476,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  if (threadIdx.x == 0) GP(1)
 
   const int M = *n_active;
   const int num_kb = (K + TC_BK - 1) / TC_BK;
@@ -450,12 +488,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc.n_tiles = (n_out + ob - 1) / ob;
     tc.tiles = tc.m_tiles * tc.n_tiles;
     tc.S = ws != nullptr && force_s > 0 && tc.tiles * force_s <= ws_tiles ? force_s : 1;
-    tc.kb_per = (num_kb + tc.S - 1) / tc.S;
-    tc.S = (num_kb + tc.kb_per - 1) / tc.kb_per;
+    if (tc.S > num_kb) tc.S = num_kb;
     tc.total = tc.tiles * tc.S;
   }
-  const int bn = tc.bn, S = tc.S, kb_per = tc.kb_per, m_tiles = tc.m_tiles, total = tc.total;
+  const int bn = tc.bn, S = tc.S, m_tiles = tc.m_tiles, total = tc.total;
   const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
+  // Stage layout, chosen from M like the tiles: with a single row tile of few rows only 32 or 64 activation rows are
+  // copied per stage (the MMA still reads 128 rows of shared memory; rows >= M are never stored), which leaves room for
+  // more stages: what bounds the weight-streaming regime is the number of weight bytes one SM keeps in flight.
+  const int a_rows = m_tiles > 1 || M > 64 ? TC_BM : (M > 32 ? 64 : 32);
+  const CUtensorMap* mapA = a_rows == TC_BM ? &tmA : (a_rows == 64 ? &tmA64 : &tmA32);
+  const int A_BYTES = a_rows * TC_BK * 2;
+  const int STAGE_BYTES = A_BYTES + bn * TC_BK * 2;
+  const int nst = TC_DATA_BYTES / STAGE_BYTES < STAGES ? TC_DATA_BYTES / STAGE_BYTES : STAGES;   // 4 .. 16
   const uint32_t stage_tx = (uint32_t)(A_BYTES + bn * TC_BK * 2);
 
   if (warp == 0) {
@@ -466,13 +511,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
         const int t = w / S, sp = w - t * S;
         const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
-        const int kb0 = sp * kb_per, kb1 = kb0 + kb_per < num_kb ? kb0 + kb_per : num_kb;
+        const int kb0 = sp * num_kb / S, kb1 = (sp + 1) * num_kb / S;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
           mbar_expect_tx(full_bar(stage), stage_tx);
-          tma_load_2d(sa, &tmA, kb * TC_BK, m0, full_bar(stage));
-          const bool wide = bn == 256 && wide_boxes;
+          tma_load_2d(sa, mapA, kb * TC_BK, m0, full_bar(stage));
+          const bool wide = bn == 256;
           if (EPI == EPI_SWIGLU) {
             if (wide) {
               tma_load_2d(sb, &tmW0, kb * TC_BK, n0, full_bar(stage));
@@ -491,16 +536,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               ln0 = n0 - src * qkv.hd;
             }
             if (wide) {
-              const CUtensorMap* mp = src == 0 ? &tmW0 : (src == 1 ? &tmW1 : &tmW2);
+              const CUtensorMap* mp = src == 0 ? &tmX0 : (src == 1 ? &tmX1 : &tmX2);
               tma_load_2d(sb, mp, kb * TC_BK, ln0, full_bar(stage));
-              if (wide_boxes == 1) tma_load_2d(sb + 2 * BOX_BYTES, mp, kb * TC_BK, ln0 + 128, full_bar(stage));
             } else {
               const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
               for (int i = 0; i < (bn >> 6); ++i)
                 tma_load_2d(sb + i * BOX_BYTES, mp, kb * TC_BK, ln0 + 64 * i, full_bar(stage));
             }
           }
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == nst) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -513,7 +557,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int it = 0;
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
         const int sp = w % S;
-        const int kb0 = sp * kb_per, kb1 = kb0 + kb_per < num_kb ? kb0 + kb_per : num_kb;
+        const int kb0 = sp * num_kb / S, kb1 = (sp + 1) * num_kb / S;
         const int acc = it & 1;
         const uint32_t use = (uint32_t)(it >> 1);
         if (!(ok = mbar_wait(acce_bar(acc), (use & 1) ^ 1, s_abort))) break;
@@ -521,6 +565,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN_MAX);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(full_bar(stage), phase, s_abort))) break;
+          if (it == 0 && kb == kb0) GP(2)
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
           const uint64_t adesc = smem_desc_k_sw128(sa), bdesc = smem_desc_k_sw128(sb);
@@ -528,9 +573,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < TC_BK / 16; ++k)   // 16 bf16 = 32 bytes along K inside the 128-byte swizzle row
             tc_mma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc, (kb > kb0) | (k != 0));
           tc_commit(empty_bar(stage));
-          if (++stage == STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == nst) { stage = 0; phase ^= 1; }
         }
         if (ok) tc_commit(accf_bar(acc));
+        if (it == 0) GP(3)
       }
     }
   } else {
@@ -545,6 +591,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      if (it == 0 && warp == 2 && lane == 0) GP(4)
       tc_fence_after();
       const int trow = quarter * 32 + lane;
       const int row = m0 + trow;
@@ -558,7 +605,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) mbar_arrive(acce_bar(acc));
       } else {
         // partial tile of this K-split -> workspace, then free the accumulator
-        float* prow = ws + ((size_t)(t * S + sp) * TC_BM + trow) * bn;
+        float* ptile = ws + (size_t)(t * S + sp) * TC_BM * bn + (size_t)trow * 4;
 #pragma unroll 1
         for (int c0 = 0; c0 < bn; c0 += 32) {
           uint32_t v[32];
@@ -567,7 +614,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (row < M) {
 #pragma unroll
             for (int j = 0; j < 32; j += 4)
-              __stcg(reinterpret_cast<float4*>(prow + c0 + j),
+              __stcg(reinterpret_cast<float4*>(ptile + (size_t)((c0 + j) >> 2) * TC_BM * 4),
                      make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
                                  __uint_as_float(v[j + 3])));
           }
@@ -575,34 +622,89 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(acc));
+        // The splits of a tile meet here.  Each takes a ticket; the finishing work (sum of the partial tiles in split
+        // order + fused epilogue) is cut into S shares of the tile's (row, unit) list.  The last arriver always
+        // finishes: its own share, then every share nobody has claimed.  A split that arrives earlier and has no other
+        // item to compute waits (bounded) for the rest and finishes the share of its ticket, so that in the usual
+        // single-round launch the S CTAs of a tile finish it together.  Shares are claimed with an atomic OR, so each
+        // is done exactly once whoever gets there first; the last CTA to leave zeroes the tile's three counters.
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (warp == 2 && lane == 0) {
-          const int old = atomicAdd(&counters[t], 1);
-          const int last = old == S - 1;
-          if (last) counters[t] = 0;             // every split has arrived: leave the counter clean for the next launch
-          *s_last = last;
+        // With little finishing work per tile (few live rows) the hand-over costs more than it saves: then only
+        // the last arriver finishes, as one share, and no share is claimed.
+        const int live_rows = M - m0 < TC_BM ? M - m0 : TC_BM;
+        const int items = live_rows * upr;
+        const bool coop = items >= 384;
+        const int shares = coop ? S : 1;
+        int* arrived = counters + t;
+        unsigned* claimed = reinterpret_cast<unsigned*>(counters + ws_tiles + t);
+        int* left = counters + 2 * ws_tiles + t;
+        const int e_tid = (warp - 2) * 32 + lane;
+        if (e_tid == 0) {
+          const int ticket = atomicAdd(arrived, 1);
+          int role = 0;                                // 0: leave, 1: finish the share of my ticket, 2: last arriver
+          if (ticket == S - 1) {
+            role = 2;
+          } else if (coop && w + (int)gridDim.x >= total) {
+            const unsigned long long t0 = clock64();
+            while (clock64() - t0 < SPLIT_HELP_CYCLES) {
+              if (*reinterpret_cast<volatile int*>(arrived) >= S) {
+                role = 1;
+                break;
+              }
+            }
+          }
+          s_fin[0] = role;
+          s_fin[1] = ticket;
+          if (it == 0) GP(5)
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        if (*s_last) {
+        const int role = s_fin[0], ticket = s_fin[1];
+        if (role) {
           __threadfence();
-          // all 128 epilogue threads share the live rows of the tile: (row, unit) pairs, units of a row adjacent
-          const int live_rows = M - m0 < TC_BM ? M - m0 : TC_BM;
-          const int e_tid = (warp - 2) * 32 + lane;
+          auto finish_share = [&](int k) {
+            const int lo = (int)((long long)k * items / shares), hi = (int)((long long)(k + 1) * items / shares);
 #pragma unroll 1
-          for (int i = e_tid; i < live_rows * upr; i += 128) {
-            const int r = i / upr, u = i - r * upr;
-            WsSrc src{ws + ((size_t)(t * S) * TC_BM + r) * bn, (size_t)TC_BM * bn, S};
-            epilogue_unit<EPI>(src, bn, m0 + r, true, u, n0, n_out, Cv, qkv);
+            for (int i = lo + e_tid; i < hi; i += 128) {   // rows fastest: a warp reads contiguous partials
+              const int u = i / live_rows, r = i - u * live_rows;
+              WsSrc src{ws + (size_t)(t * S) * TC_BM * bn, r, (size_t)TC_BM * bn, S};
+              epilogue_unit<EPI>(src, bn, m0 + r, true, u, n0, n_out, Cv, qkv);
+            }
+          };
+          const int nk = role == 2 ? shares : 1;       // the last arriver tries its own share first, then all others
+#pragma unroll 1
+          for (int q = 0; q < nk; ++q) {
+            const int k = role == 2 ? (q == 0 ? shares - 1 : q - 1) : ticket;
+            if (coop) {
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+              if (e_tid == 0) s_fin[2] = (int)((atomicOr(claimed, 1u << k) >> k) & 1u);   // 1: somebody else has it
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+              if (s_fin[2]) continue;
+            }
+            finish_share(k);
           }
         }
-        asm volatile("bar.sync 1, 128;" ::: "memory");   // s_last is rewritten by the next item
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (e_tid == 0) {
+          if (coop) {
+            __threadfence();
+            if (atomicAdd(left, 1) == S - 1) {
+              *arrived = 0;
+              *claimed = 0u;
+              *left = 0;
+            }
+          } else if (role == 2) {
+            *arrived = 0;                              // every split has arrived and only this CTA is still here
+          }
+        }
+        if (it == 0 && warp == 2 && lane == 0) GP(6)
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) GP(7)
   if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_GEMM_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
@@ -670,20 +772,6 @@ int get_tensor_map_2d(const void* ptr, long long rows, long long cols, int box_r
   return SL_OK;
 }
 
-static int pair_mode();
-static int wide_boxes() {
-  static int v = -1;
-  if (v < 0) {
-    // tuning aid: SURELOCK_GEMM_BOX = 64 | 128 | 256 rows per weight copy of a 256-wide tile (default 256)
-    const char* e = getenv("SURELOCK_GEMM_BOX");
-    v = 2;
-    if (e && !strcmp(e, "64")) v = 0;
-    if (e && !strcmp(e, "128")) v = 1;
-    if (v == 2 && pair_mode()) v = 1;   // the CTA-pair path loads 128-row halves of a weight tile: share those maps
-  }
-  return v;
-}
-
 static int pair_mode() {
   static int v = -1;
   if (v < 0) {
@@ -694,20 +782,17 @@ static int pair_mode() {
 }
 
 static int force_cfg(int which) {
-  static int v[2] = {-1, -1};
-  if (v[0] < 0) {
-    v[0] = v[1] = 0;
-    const char* e = getenv("SURELOCK_GEMM_FORCE");   // tuning aid: "bn,S", e.g. "128,3"
-    if (e) sscanf(e, "%d,%d", &v[0], &v[1]);
-  }
+  int v[2] = {0, 0};
+  const char* e = getenv("SURELOCK_GEMM_FORCE");   // tuning aid, read at every launch: "bn,S", e.g. "128,3"
+  if (e) sscanf(e, "%d,%d", &v[0], &v[1]);
   return v[which];
 }
 
 template <int EPI, int STAGES>
-static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensorMap* wb, void* C,
+static int launch_cfg(const CUtensorMap* a, const CUtensorMap* b, const CUtensorMap* wb, const CUtensorMap* xb, void* C,
                       const int32_t* n_active, int max_rows, int n_out, int K, int32_t* status, const QkvArgs& qkv,
                       const SplitWs& sw, cudaStream_t st) {
-  constexpr int SMEM = STAGES * (TC_BM * TC_BK * 2 + 256 * TC_BK * 2) + 1024 + 256;
+  constexpr int SMEM = TC_DATA_BYTES + 1024 + 512;
   static bool attr_set = false;
   if (!attr_set) {
     SL_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<EPI, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
@@ -730,9 +815,32 @@ static int launch_cfg(const CUtensorMap& a, const CUtensorMap* b, const CUtensor
   at[0].val.clusterDim.z = 1;
   cfg.attrs = at;
   cfg.numAttrs = 1;
-  SL_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, STAGES>, a, b[0], b[1], b[2], wb[0], wb[1], wb[2], C, n_active,
-                                 n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles, wide_boxes(), force_cfg(0),
+  SL_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, STAGES>, a[0], a[1], a[2], b[0], b[1], b[2], wb[0], wb[1], wb[2], xb[0], xb[1], xb[2], C, n_active,
+                                 n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles, force_cfg(0),
                                  force_cfg(1), pair));
+#ifdef GEMM_PROFILE
+  {
+    static unsigned long long h[160 * 8];
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(h, g_gemm_prof, sizeof(h));
+    unsigned long long t0 = ~0ull;
+    for (int c = 0; c < grid; ++c) if (h[c * 8] && h[c * 8] < t0) t0 = h[c * 8];
+    const char* names[8] = {"entry", "prologue", "first-stage", "mma-issued", "acc-ready", "partial+count", "finisher", "exit"};
+    fprintf(stderr, "GEMM_PROFILE epi %d n_out %d K %d (us after the first CTA's entry; min / mean / max over CTAs that report)\n", EPI, n_out, K);
+    for (int i = 0; i < 8; ++i) {
+      double mn = 1e30, mx = 0, sum = 0; int n = 0;
+      for (int c = 0; c < grid; ++c) {
+        const unsigned long long v = h[c * 8 + i];
+        if (v < t0) continue;
+        const double d = (double)(v - t0) * 1e-3;
+        mn = d < mn ? d : mn; mx = d > mx ? d : mx; sum += d; ++n;
+      }
+      if (n) fprintf(stderr, "  %-14s n %3d  %7.2f %7.2f %7.2f\n", names[i], n, mn, sum / n, mx);
+    }
+    static unsigned long long z[160 * 8];
+    cudaMemcpyToSymbol(g_gemm_prof, z, sizeof(z));
+  }
+#endif
   return SL_OK;
 }
 
@@ -744,23 +852,26 @@ int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const 
        reinterpret_cast<uintptr_t>(C)) & 15)
     return SL_EUNSUPPORTED;
   if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
-  CUtensorMap a, b[3], wb[3];
-  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
+  CUtensorMap a[3], b[3], wb[3], xb[3];
+  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a[0]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(A, max_rows, K, 32, &a[1]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(A, max_rows, K, 64, &a[2]);
   if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, 64, &b[0]);
-  const int wrows = (wide_boxes() == 2 && epilogue != EPI_SWIGLU) ? 256 : 128;
-  if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, wrows, &wb[0]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, 128, &wb[0]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(W, n_out, K, 256, &xb[0]);
   if (rc != SL_OK) return rc;
   b[1] = b[2] = b[0];
   wb[1] = wb[2] = wb[0];
+  xb[1] = xb[2] = xb[0];
   if (W2) {
     rc = get_tensor_map_2d(W2, n_out, K, 64, &b[1]);
     if (rc == SL_OK) rc = get_tensor_map_2d(W2, n_out, K, 128, &wb[1]);
     if (rc != SL_OK) return rc;
   }
   switch (epilogue) {
-    case EPI_STORE: return launch_cfg<EPI_STORE, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
-    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
-    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, 4>(a, b, wb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_STORE: return launch_cfg<EPI_STORE, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
     default: return SL_EINVAL;
   }
 }
@@ -774,16 +885,19 @@ int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void
        reinterpret_cast<uintptr_t>(Wv) | reinterpret_cast<uintptr_t>(q_out) | reinterpret_cast<uintptr_t>(k_cache) |
        reinterpret_cast<uintptr_t>(v_cache)) & 15)
     return SL_EUNSUPPORTED;
-  CUtensorMap a, b[3], wb[3];
+  CUtensorMap a[3], b[3], wb[3], xb[3];
   const void* W[3] = {Wq, Wk, Wv};
-  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a);
+  int rc = get_tensor_map_2d(A, max_rows, K, TC_BM, &a[0]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(A, max_rows, K, 32, &a[1]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(A, max_rows, K, 64, &a[2]);
   for (int i = 0; i < 3 && rc == SL_OK; ++i) {
     rc = get_tensor_map_2d(W[i], hd, K, 64, &b[i]);
-    if (rc == SL_OK) rc = get_tensor_map_2d(W[i], hd, K, wide_boxes() == 2 ? 256 : 128, &wb[i]);
+    if (rc == SL_OK) rc = get_tensor_map_2d(W[i], hd, K, 128, &wb[i]);
+    if (rc == SL_OK) rc = get_tensor_map_2d(W[i], hd, K, 256, &xb[i]);
   }
   if (rc != SL_OK) return rc;
   QkvArgs qa{(bf16*)q_out, (bf16*)k_cache, (bf16*)v_cache, idx, rope, n_seq, hd, dh};
-  return launch_cfg<EPI_QKV, 4>(a, b, wb, nullptr, n_active, max_rows, 3 * hd, K, status, qa, sw, st);
+  return launch_cfg<EPI_QKV, TC_MAX_STAGES>(a, b, wb, xb, nullptr, n_active, max_rows, 3 * hd, K, status, qa, sw, st);
 }
 
 }  // namespace sl

@@ -173,8 +173,9 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Split-K workspace of the GEMM: room for `tiles` fp32 partial tiles of 128 x 256 and one arrival counter per output
-// tile (zero-initialised once; the kernel leaves them zero).  ws == nullptr disables split-K.
+// Split-K workspace of the GEMM: room for `tiles` fp32 partial tiles of 128 x 256 and three counters per output tile
+// ([3][tiles] ints: arrived, claimed shares, left; zero-initialised once; the kernel leaves them zero).
+// ws == nullptr disables split-K.
 struct SplitWs {
   float* ws = nullptr;
   int* counters = nullptr;
