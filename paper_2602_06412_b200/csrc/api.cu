@@ -229,6 +229,7 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
   A_(c->rope, (size_t)N * (cfg->head_dim / 2) * sizeof(float2));
   if (cfg->dtype == SL_BF16) {
     c->split.tiles = 4 * sm_count();
+    c->split.prefetch_w = true;   // inside a step a GEMM never directly follows the kernel that writes n_active
     A_(c->split.ws, (size_t)c->split.tiles * SPLIT_TILE_BYTES);
     A_(c->split.counters, (size_t)c->split.tiles * 3 * sizeof(int));
     if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * 3 * sizeof(int), c->st) != cudaSuccess)

@@ -88,6 +88,12 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     *s_abort = 0;
     fence_mbar_init();
+  }
+  if (warp == 1) tc_alloc(smem_u32(s_tmem), TMEM_COLS);
+  // everything above overlaps the tail of the previous kernel; nothing below may run before it has completed
+  griddep_wait();
+  griddep_launch();
+  if (threadIdx.x == 0) {
     // items of two tiles, unless one-tile items finish sooner: a one-tile item takes about 0.8 of the time of a
     // two-tile item (its softmax warps and the tensor pipe alternate instead of overlapping), so they win when they
     // spread over idle SMs, i.e. when 4 * rounds(one-tile) < 5 * rounds(two-tile)
@@ -113,7 +119,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
     *s_item_rows = rows;
   }
-  if (warp == 1) tc_alloc(smem_u32(s_tmem), TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -453,7 +458,8 @@ static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtens
   if (!d_prof) cudaMalloc(&d_prof, 192);
   prof = d_prof;
 #endif
-  attention_pp_kernel<DH><<<grid, PP_THREADS, smem, st>>>(q, k, v, row_offsets, B, N, H, (bf16*)o, scale_log2, status, prof);
+  SL_CUDA_TRY(launch_pdl(attention_pp_kernel<DH>, dim3(grid), dim3(PP_THREADS), (size_t)smem, st, q, k, v, row_offsets, B, N, H,
+                         (bf16*)o, scale_log2, status, prof));
 #ifdef ATT_PROFILE
   {
     unsigned long long h[24];

@@ -50,6 +50,43 @@ __device__ __forceinline__ void set_status(int32_t* status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// ---- programmatic dependent launch ------------------------------------------------------------------------------------
+// The kernels of a step run back to back on one stream.  Launched with the programmatic-serialization attribute, a
+// kernel may start while its predecessor is still draining: everything it does before griddep_wait() (barrier set-up,
+// tensor-memory allocation, in the GEMM the first weight copies, which depend on no earlier kernel) overlaps the
+// predecessor's tail and the launch latency.  griddep_wait() returns once the predecessor grid has completed and its
+// writes are visible; griddep_launch() (always after the wait, so at most two kernels are in flight) lets the successor
+// start.  Both are no-ops in a kernel launched without the attribute.  SURELOCK_PDL=0 in the environment switches the
+// attribute off.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+inline bool pdl_enabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SURELOCK_PDL");
+    v = (e && e[0] == '0') ? 0 : 1;
+  }
+  return v != 0;
+}
+
+// <<<grid, block, smem, st>>> with the programmatic-serialization attribute; only for kernels that call griddep_wait()
+// before they touch anything an earlier kernel wrote.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline int sm_count() {
   static int n = 0;
   if (!n) {

@@ -420,7 +420,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmX0,
                const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2, void* __restrict__ Cv, const int32_t* __restrict__ n_active,
                int n_out, int K, int32_t* status, const QkvArgs qkv, float* __restrict__ ws, int* __restrict__ counters,
-               int ws_tiles, int force_bn, int force_s, int pair_mode) {
+               int ws_tiles, int force_bn, int force_s, int pair_mode, int prefetch_w) {
   // tmA / tmA32 / tmA64: the activation matrix with 128-, 32- and 64-row boxes; tmB*: weight maps with 64-row boxes
   // (any tile width); tmW* / tmX*: the same matrices with 128- and 256-row boxes: a 256-wide tile is one 256-row copy
   // (gate/up: two 128-row copies), the CTA-pair path loads 128-row halves
@@ -430,6 +430,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // prefetch_w: the caller states that neither *n_active nor the weights were written by the kernel launched just
+  // before this one (true inside a step): M may then be read, and the first weight copies issued, while that kernel is
+  // still draining.  Otherwise nothing is read before it has completed.
+  if (!prefetch_w) {
+    griddep_wait();
+    griddep_launch();
+  }
   if (pair_mode) {
     // launched as clusters of two: the CTA-pair path takes the whole launch when 256 x 256 pair tiles fill the grid
     // (large M) and need no more time than single tiles: rounds of pair tiles against rounds of 128 x 256 tiles, which
@@ -441,6 +448,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int pairs = ((Mp + 255) / 256) * nt, singles = ((Mp + 127) / 128) * nt;
     const int rounds_p = (pairs + half - 1) / half, rounds_s = (singles + (int)gridDim.x - 1) / (int)gridDim.x;
     if (pairs >= half && 20 * rounds_p <= 23 * rounds_s) {
+      if (prefetch_w) {
+        griddep_wait();
+        griddep_launch();
+      }
       run_pair<EPI>(&tmA, &tmW0, &tmW1, &tmW2, Cv, Mp, n_out, K, status, qkv, smem);
       return;
     }
@@ -508,47 +519,81 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // the weight part of stage `st` for K block kb of the tile at column n0
+      auto load_w = [&](int st, int kb, int n0) {
+        const uint32_t sb = smem_u32(smem + st * STAGE_BYTES) + A_BYTES;
+        const bool wide = bn == 256;
+        if (EPI == EPI_SWIGLU) {
+          if (wide) {
+            tma_load_2d(sb, &tmW0, kb * TC_BK, n0, full_bar(st));
+            tma_load_2d(sb + 2 * BOX_BYTES, &tmW1, kb * TC_BK, n0, full_bar(st));
+          } else {
+            const int hb = bn >> 7;                                  // 64-row boxes per half
+            for (int i = 0; i < hb; ++i) {
+              tma_load_2d(sb + i * BOX_BYTES, &tmB0, kb * TC_BK, n0 + 64 * i, full_bar(st));
+              tma_load_2d(sb + (hb + i) * BOX_BYTES, &tmB1, kb * TC_BK, n0 + 64 * i, full_bar(st));
+            }
+          }
+        } else {
+          int src = 0, ln0 = n0;
+          if (EPI == EPI_QKV) {                                      // a tile never straddles two matrices
+            src = n0 / qkv.hd;
+            ln0 = n0 - src * qkv.hd;
+          }
+          if (wide) {
+            const CUtensorMap* mp = src == 0 ? &tmX0 : (src == 1 ? &tmX1 : &tmX2);
+            tma_load_2d(sb, mp, kb * TC_BK, ln0, full_bar(st));
+          } else {
+            const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
+            for (int i = 0; i < (bn >> 6); ++i)
+              tma_load_2d(sb + i * BOX_BYTES, mp, kb * TC_BK, ln0 + 64 * i, full_bar(st));
+          }
+        }
+      };
+      bool waited = !prefetch_w;
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
         const int t = w / S, sp = w - t * S;
         const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
         const int kb0 = sp * num_kb / S, kb1 = (sp + 1) * num_kb / S;
-        for (int kb = kb0; kb < kb1; ++kb) {
-          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
-          const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
-          mbar_expect_tx(full_bar(stage), stage_tx);
-          tma_load_2d(sa, mapA, kb * TC_BK, m0, full_bar(stage));
-          const bool wide = bn == 256;
-          if (EPI == EPI_SWIGLU) {
-            if (wide) {
-              tma_load_2d(sb, &tmW0, kb * TC_BK, n0, full_bar(stage));
-              tma_load_2d(sb + 2 * BOX_BYTES, &tmW1, kb * TC_BK, n0, full_bar(stage));
-            } else {
-              const int hb = bn >> 7;                                  // 64-row boxes per half
-              for (int i = 0; i < hb; ++i) {
-                tma_load_2d(sb + i * BOX_BYTES, &tmB0, kb * TC_BK, n0 + 64 * i, full_bar(stage));
-                tma_load_2d(sb + (hb + i) * BOX_BYTES, &tmB1, kb * TC_BK, n0 + 64 * i, full_bar(stage));
-              }
-            }
-          } else {
-            int src = 0, ln0 = n0;
-            if (EPI == EPI_QKV) {                                      // a tile never straddles two matrices
-              src = n0 / qkv.hd;
-              ln0 = n0 - src * qkv.hd;
-            }
-            if (wide) {
-              const CUtensorMap* mp = src == 0 ? &tmX0 : (src == 1 ? &tmX1 : &tmX2);
-              tma_load_2d(sb, mp, kb * TC_BK, ln0, full_bar(stage));
-            } else {
-              const CUtensorMap* mp = src == 0 ? &tmB0 : (src == 1 ? &tmB1 : &tmB2);
-              for (int i = 0; i < (bn >> 6); ++i)
-                tma_load_2d(sb + i * BOX_BYTES, mp, kb * TC_BK, ln0 + 64 * i, full_bar(stage));
-            }
+        int kb = kb0;
+        if (!waited) {
+          // first item: the weight halves of the first stages go out now, the activation halves once the previous
+          // kernel has completed (the stages are fresh, so there is no "empty" wait)
+          const int npre = kb1 - kb0 < nst ? kb1 - kb0 : nst;
+          for (int i = 0; i < npre; ++i) {
+            mbar_expect_tx(full_bar(i), stage_tx);
+            load_w(i, kb0 + i, n0);
           }
+          griddep_wait();
+          griddep_launch();
+          waited = true;
+          for (int i = 0; i < npre; ++i)
+            tma_load_2d(smem_u32(smem + i * STAGE_BYTES), mapA, (kb0 + i) * TC_BK, m0, full_bar(i));
+          stage = npre;
+          if (stage == nst) { stage = 0; phase ^= 1; }
+          kb = kb0 + npre;
+        }
+        for (; kb < kb1; ++kb) {
+          if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
+          mbar_expect_tx(full_bar(stage), stage_tx);
+          tma_load_2d(smem_u32(smem + stage * STAGE_BYTES), mapA, kb * TC_BK, m0, full_bar(stage));
+          load_w(stage, kb, n0);
           if (++stage == nst) { stage = 0; phase ^= 1; }
         }
       }
+      if (!waited) {
+        griddep_wait();
+        griddep_launch();
+      }
+    } else if (prefetch_w) {
+      griddep_wait();
+      griddep_launch();
     }
   } else if (warp == 1) {
+    if (prefetch_w) {
+      griddep_wait();
+      griddep_launch();
+    }
     if (lane == 0) {
       const uint32_t idesc = idesc_bf16_m128(bn);
       int stage = 0;
@@ -580,6 +625,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
     }
   } else {
+    if (prefetch_w) {
+      griddep_wait();
+      griddep_launch();
+    }
     const int quarter = warp & 3;             // tensor-memory lanes 32*quarter .. 32*quarter+31
     bool ok = true;
     int it = 0;
@@ -808,16 +857,18 @@ static int launch_cfg(const CUtensorMap* a, const CUtensorMap* b, const CUtensor
   cfg.blockDim = dim3(TC_THREADS);
   cfg.dynamicSmemBytes = SMEM;
   cfg.stream = st;
-  cudaLaunchAttribute at[1];
+  cudaLaunchAttribute at[2];
   at[0].id = cudaLaunchAttributeClusterDimension;
   at[0].val.clusterDim.x = 2;
   at[0].val.clusterDim.y = 1;
   at[0].val.clusterDim.z = 1;
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = at;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = pdl_enabled() ? 2 : 1;
   SL_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, STAGES>, a[0], a[1], a[2], b[0], b[1], b[2], wb[0], wb[1], wb[2], xb[0], xb[1], xb[2], C, n_active,
                                  n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles, force_cfg(0),
-                                 force_cfg(1), pair));
+                                 force_cfg(1), pair, sw.prefetch_w ? 1 : 0));
 #ifdef GEMM_PROFILE
   {
     static unsigned long long h[160 * 8];

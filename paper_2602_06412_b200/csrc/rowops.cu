@@ -18,6 +18,8 @@ __global__ void __launch_bounds__(256)
 gather_rows_kernel(const T* __restrict__ table, const int32_t* __restrict__ tokens, const int32_t* __restrict__ idx,
                    const int32_t* __restrict__ n_active, int d, int table_rows, float* __restrict__ x,
                    int32_t* status) {
+  griddep_wait();
+  griddep_launch();
   const int M = *n_active;
   constexpr int VEC = 16 / sizeof(T);
   for (int r = blockIdx.x; r < M; r += gridDim.x) {
@@ -47,10 +49,10 @@ int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* 
   const int g = row_grid(max_rows, 8);
   if (dtype == SL_BF16) {
     if (d % 8) return SL_EUNSUPPORTED;
-    gather_rows_kernel<bf16><<<g, 256, 0, st>>>((const bf16*)table, tokens, idx, n_active, d, table_rows, x, status);
+    SL_CUDA_TRY(launch_pdl(gather_rows_kernel<bf16>, dim3(g), dim3(256), 0, st, (const bf16*)table, tokens, idx, n_active, d, table_rows, x, status));
   } else {
     if (d % 4) return SL_EUNSUPPORTED;
-    gather_rows_kernel<float><<<g, 256, 0, st>>>((const float*)table, tokens, idx, n_active, d, table_rows, x, status);
+    SL_CUDA_TRY(launch_pdl(gather_rows_kernel<float>, dim3(g), dim3(256), 0, st, (const float*)table, tokens, idx, n_active, d, table_rows, x, status));
   }
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
@@ -65,6 +67,8 @@ __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ h,
                const int32_t* __restrict__ n_active, int d, float eps) {
   __shared__ float s_part[8];
+  griddep_wait();
+  griddep_launch();
   const int M = *n_active;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nv = d >> 2;                                   // float4 per row
@@ -122,23 +126,23 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
 }
 
 template <typename T>
-static void launch_rms_t(const float* x, const void* gain, void* h, const int32_t* n_active, int g, int d, float eps,
+static int launch_rms_t(const float* x, const void* gain, void* h, const int32_t* n_active, int g, int d, float eps,
                          cudaStream_t st) {
   const int nv = d >> 2;
-  if (nv <= 256 * 2) rmsnorm_kernel<T, 2><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
-  else if (nv <= 256 * 4) rmsnorm_kernel<T, 4><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
-  else if (nv <= 256 * 8) rmsnorm_kernel<T, 8><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
-  else rmsnorm_kernel<T, 0><<<g, 256, 0, st>>>(x, (const T*)gain, (T*)h, n_active, d, eps);
+  if (nv <= 256 * 2) SL_CUDA_TRY(launch_pdl(rmsnorm_kernel<T, 2>, dim3(g), dim3(256), 0, st, x, (const T*)gain, (T*)h, n_active, d, eps));
+  else if (nv <= 256 * 4) SL_CUDA_TRY(launch_pdl(rmsnorm_kernel<T, 4>, dim3(g), dim3(256), 0, st, x, (const T*)gain, (T*)h, n_active, d, eps));
+  else if (nv <= 256 * 8) SL_CUDA_TRY(launch_pdl(rmsnorm_kernel<T, 8>, dim3(g), dim3(256), 0, st, x, (const T*)gain, (T*)h, n_active, d, eps));
+  else SL_CUDA_TRY(launch_pdl(rmsnorm_kernel<T, 0>, dim3(g), dim3(256), 0, st, x, (const T*)gain, (T*)h, n_active, d, eps));
+  return SL_OK;
 }
 
 int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_active, int max_rows, int d, float eps,
                    int dtype, cudaStream_t st) {
   if (d % 4) return SL_EUNSUPPORTED;
   const int g = row_grid(max_rows, 8);
-  if (dtype == SL_BF16)
-    launch_rms_t<bf16>(x, gain, h, n_active, g, d, eps, st);
-  else
-    launch_rms_t<float>(x, gain, h, n_active, g, d, eps, st);
+  const int rc = dtype == SL_BF16 ? launch_rms_t<bf16>(x, gain, h, n_active, g, d, eps, st)
+                                  : launch_rms_t<float>(x, gain, h, n_active, g, d, eps, st);
+  if (rc != SL_OK) return rc;
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

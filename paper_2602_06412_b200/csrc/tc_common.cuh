@@ -180,6 +180,9 @@ struct SplitWs {
   float* ws = nullptr;
   int* counters = nullptr;
   int tiles = 0;
+  // the caller states that neither *n_active nor the weights were written by the kernel launched just before the
+  // GEMM: it may then read M and start its first weight copies before that kernel has completed
+  bool prefetch_w = false;
 };
 constexpr size_t SPLIT_TILE_BYTES = 128 * 256 * sizeof(float);
 
