@@ -282,7 +282,7 @@ def main():
     # operand bytes = 148.0 MB / 167.8 MB on M=2048 x 12288 x 4096) to this step's algorithmic operand bytes
     d_, F_, V_, L_ = cfg["d_model"], cfg["d_ff"], cfg["vocab"], cfg["n_layers"]
     act_bytes = M * (L_ * (2 * d_ + 2 * 3 * d_ + 2 * d_ + 8 * d_ + 2 * d_ + 2 * F_ + 2 * F_ + 8 * d_) + 2 * d_ + 2 * V_)
-    traffic = 0.895 * (wbytes + act_bytes) / max(gemm_launch, 1)
+    traffic = 0.89 * (wbytes + act_bytes) / max(gemm_launch, 1)
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     if M >= ridge:
         ach = flops / (gemm_ms * 1e-3) / 1e12

@@ -166,3 +166,14 @@ def test_long_context_contiguous_plus_random_locks():
     w0, w1 = _two_steps(cfg, B=B, N=N, n_prompt=3584, n_active=na, seed=41, layers=[0, 1], seqs=[0, 2, 3], n_rows=8,
                         w_device=DEV, lock_fn=inputs.contiguous_plus_random_lock)
     print("worst stage errors, long context:", w0, w1)
+
+
+@pytest.mark.parametrize("n_active", [[23], [103], [305]])
+def test_single_sequence_few_active_rows(n_active):
+    """Weight-streaming regime of the GEMMs (single sequence, N = 512, LLaDA-8B layer shape, 2 layers): M = 23 and 103
+    take one row tile (32 / 128 activation rows per stage, K split with the fused QKV, SwiGLU and residual epilogues
+    finishing in the workspace), M = 305 three row tiles."""
+    cfg = inputs.model_shape("llada8b", n_layers=2, vocab=8192)
+    w0, w1 = _two_steps(cfg, B=1, N=512, n_prompt=128, n_active=n_active, seed=50 + n_active[0], layers=[0, 1], seqs=[0],
+                        n_rows=12, w_device=DEV)
+    print("worst stage errors, single sequence:", n_active, w0, w1)
