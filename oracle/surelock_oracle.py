@@ -203,6 +203,47 @@ def confidence_gate(conf: np.ndarray, candidate: np.ndarray, seq_of_row: np.ndar
 
 
 # --------------------------------------------------------------------------
+# Unmasking policy (Algorithm 1 line 16)
+# --------------------------------------------------------------------------
+def update_mask(tokens: np.ndarray, mask_state: np.ndarray, conf: np.ndarray, argmax: np.ndarray,
+                active_idx: np.ndarray, lo: int, hi: int, k: int, mask_token: int):
+    """UpdateMASK (Algorithm 1 line 16), the confidence-ordered policy the paper describes for masked-diffusion
+    samplers (App. "semantically distant options": per step a fixed number of masked positions with the highest
+    posterior probability become concrete tokens) restricted to one semi-autoregressive block (Sec. 4 set-up).
+
+    Per sequence: among the positions lo <= n < hi that are still masked, the k with the largest conf = max_v p(v)
+    (ties: lowest position) take their argmax token and become unmasked; everything else is unchanged.  A position
+    whose argmax is the mask token itself takes token 0 (a sampler never emits the mask token).  The Algorithm leaves
+    the policy open; this reading is the harness's, not part of the method.
+
+    tokens int [B][N], mask_state uint8 [B][N] (1 = masked), conf / argmax per packed active row, active_idx the
+    flat position b * N + n of each packed row.  Returns (new tokens, new mask_state, revealed per sequence).
+    """
+    tokens = np.array(tokens, dtype=np.int64)
+    mask_state = np.array(mask_state, dtype=np.uint8)
+    B, N = tokens.shape
+    conf = np.asarray(conf, F64)
+    revealed = np.zeros(B, np.int64)
+    for b in range(B):
+        cand = []                                      # (position, row) of masked block positions that were computed
+        for r, flat in enumerate(np.asarray(active_idx)):
+            bb, n = divmod(int(flat), N)
+            if bb == b and lo <= n < hi and mask_state[b, n] == 1:
+                cand.append((n, r))
+        for _ in range(k):
+            if not cand:
+                break
+            best = max(cand, key=lambda nr: (conf[nr[1]], -nr[0]))      # highest conf, then lowest position
+            n, r = best
+            tok = int(argmax[r])
+            tokens[b, n] = 0 if tok == mask_token else tok
+            mask_state[b, n] = 0
+            revealed[b] += 1
+            cand.remove(best)
+    return tokens, mask_state, revealed
+
+
+# --------------------------------------------------------------------------
 # Algorithmic FLOPs (Sec. 2.3)
 # --------------------------------------------------------------------------
 def flops_base_step(cfg: ModelCfg, B: int, N: int, n_kv_heads: Optional[int] = None) -> int:

@@ -421,3 +421,53 @@ def test_step_with_confidence_gate_locks_a_subset():
         u = 1 - gated["conf"][bb * N: bb * N + 10]
         assert set(np.flatnonzero(gated["new_lock"][bb])) == set(np.argsort(u)[:2])
     np.testing.assert_array_equal(gated["logits"], plain["logits"])                 # the gate changes decisions only
+
+
+def test_update_mask_reveals_the_most_confident_masked_block_positions():
+    """UpdateMASK (Algorithm 1 line 16) against a different library's routine (torch.topk on a stable ordering) and
+    against the properties that define the policy: per sequence exactly min(k, masked-and-computed block positions)
+    reveals, every revealed confidence >= every confidence left masked in the block, ties to the lowest position,
+    nothing outside the block or already unmasked changes, the mask token is never written."""
+    rng = np.random.default_rng(5)
+    B, N, V = 3, 40, 11
+    mask_tok = V - 1
+    for trial in range(20):
+        lo, hi, k = int(rng.integers(0, 20)), int(rng.integers(20, 41)), int(rng.integers(1, 6))
+        tokens = rng.integers(0, V - 1, (B, N))
+        mask = (rng.random((B, N)) < 0.5).astype(np.uint8)
+        tokens[mask == 1] = mask_tok
+        lock = (rng.random((B, N)) < 0.3) & (mask == 0)               # masked positions are never locked
+        idx, _ = O.active_set(lock.astype(np.uint8))
+        conf = np.round(rng.random(len(idx)), 1)                      # coarse values: many ties
+        am = rng.integers(0, V, len(idx))                             # may propose the mask token
+        t2, m2, rev = O.update_mask(tokens, mask, conf, am, idx, lo, hi, k, mask_tok)
+        conf_pos = np.full(B * N, -1.0)
+        conf_pos[idx] = conf
+        am_pos = np.zeros(B * N, np.int64)
+        am_pos[idx] = am
+        for b in range(B):
+            blk = np.arange(lo, hi)
+            cand = blk[mask[b, blk] == 1]
+            n_rev = min(k, len(cand))
+            assert rev[b] == n_rev
+            # torch.topk on (conf, -position) via a stable sort key
+            key = torch.tensor(conf_pos[b * N + cand]) * 1000 - torch.tensor(cand, dtype=torch.float64) * 1e-3
+            chosen = set(cand[torch.topk(key, n_rev).indices.numpy()].tolist()) if n_rev else set()
+            changed = set(np.flatnonzero(m2[b] != mask[b]).tolist())
+            assert changed == chosen
+            for n in chosen:
+                want = am_pos[b * N + n]
+                assert t2[b, n] == (0 if want == mask_tok else want) and t2[b, n] != mask_tok and m2[b, n] == 0
+            untouched = np.setdiff1d(np.arange(N), list(chosen))
+            assert np.array_equal(t2[b, untouched], tokens[b, untouched])
+            left = [n for n in cand if n not in chosen]
+            if chosen and left:
+                assert min(conf_pos[b * N + n] for n in chosen) >= max(conf_pos[b * N + n] for n in left)
+    # worked example: block [2, 6), k = 2, confidences 0.9 (pos 2), 0.9 (pos 4), 0.95 (pos 5); position 3 is unmasked
+    tokens = np.array([[7, 7, 9, 1, 9, 9, 9]])
+    mask = np.array([[0, 0, 1, 0, 1, 1, 1]], np.uint8)
+    idx = np.arange(7)
+    conf = np.array([0.1, 0.1, 0.9, 0.99, 0.9, 0.95, 0.999])
+    am = np.array([0, 0, 3, 3, 4, 9, 6])
+    t2, m2, rev = O.update_mask(tokens, mask, conf, am, idx, 2, 6, 2, 9)
+    assert t2.tolist() == [[7, 7, 3, 1, 9, 0, 9]] and m2.tolist() == [[0, 0, 0, 0, 1, 0, 1]] and rev.tolist() == [2]
