@@ -242,6 +242,24 @@ int surelock_conf_gate_lock(const float *conf, const float *kl, const int32_t *a
                             int B, int N, const uint8_t *mask_state, uint8_t *lock_mask, float kl_eps, float m_percent,
                             float *theta_out, void *stream);
 
+/* UpdateMASK (Algorithm 1 line 16) on the device: the confidence-ordered unmasking policy the paper describes for
+ * masked-diffusion samplers (a fixed number of masked positions with the highest posterior probability become concrete
+ * tokens each step), restricted to the semi-autoregressive block [lo, hi) (Sec. 4 set-up).  The Algorithm leaves the
+ * policy to the sampler; this call is the one the decoding harness uses between two surelock_step calls, so that a
+ * decoding loop needs no host round-trip.
+ * For each of the B sequences: among the positions lo <= n < hi with mask_state == 1, the k with the largest conf
+ * (ties: lowest position) get tokens[b][n] = argmax of that row (0 when that is mask_token) and mask_state[b][n] = 0.
+ *   conf        dev fp32  [M]   max_v p(v) per packed row (surelock_step_out.conf)
+ *   argmax      dev int32 [M]   (surelock_step_out.argmax)
+ *   active_idx  dev int32 [M], row_offsets dev int32 [B+1]: the packing of the step that produced conf / argmax
+ *   tokens      dev int32 [B][N], mask_state dev uint8 [B][N]: updated in place
+ *   n_revealed  dev int32 [B] or NULL: how many positions of each sequence were revealed (< k when fewer were masked)
+ * Masked positions are never locked, so every masked position of the block has a row.  0 <= lo <= hi <= N, k >= 0.
+ * Returns SL_EINVAL on bad arguments, SL_ECUDA on a launch failure.  Asynchronous on `stream`. */
+int surelock_update_mask(const float *conf, const int32_t *argmax, const int32_t *active_idx, const int32_t *row_offsets,
+                         int B, int N, int lo, int hi, int k, int32_t mask_token, int32_t *tokens, uint8_t *mask_state,
+                         int32_t *n_revealed, void *stream);
+
 /* Bytes of workspace that lets surelock_gemm split K when M is small (see below). */
 size_t surelock_gemm_workspace_bytes(void);
 

@@ -63,6 +63,7 @@ def lib() -> C.CDLL:
         "surelock_last_launch_count": (i32, [vp]),
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
         "surelock_conf_gate_lock": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, f32, f32, vp, vp]),
+        "surelock_update_mask": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
         "surelock_layer_trace": (i32, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "surelock_kernel_times": (i32, [vp, vp, vp, i32]),
         "surelock_destroy": (None, [vp]),
@@ -246,6 +247,13 @@ def surelock_conf_gate_lock(conf, kl, active_idx, row_offsets, B: int, N: int, m
     _check(lib().surelock_conf_gate_lock(_p(conf), _p(kl), _p(active_idx), _p(row_offsets), B, N, _p(mask_state),
                                          _p(lock_mask), kl_eps, m_percent, _p(theta_out), _stream()),
            "surelock_conf_gate_lock")
+
+
+def surelock_update_mask(conf, argmax, active_idx, row_offsets, B: int, N: int, lo: int, hi: int, k: int,
+                         mask_token: int, tokens, mask_state, n_revealed=None):
+    """UpdateMASK (Algorithm 1 line 16) on the device; tokens int32 [B][N] and mask_state uint8 [B][N] in place."""
+    _check(lib().surelock_update_mask(_p(conf), _p(argmax), _p(active_idx), _p(row_offsets), B, N, lo, hi, k, mask_token,
+                                      _p(tokens), _p(mask_state), _p(n_revealed), _stream()), "surelock_update_mask")
 
 
 def surelock_last_launch_count(ctx: Ctx) -> int:

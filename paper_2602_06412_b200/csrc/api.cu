@@ -521,6 +521,16 @@ int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active
   return launch_gemm_simt(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, (cudaStream_t)stream);
 }
 
+int surelock_update_mask(const float* conf, const int32_t* argmax, const int32_t* active_idx, const int32_t* row_offsets,
+                         int B, int N, int lo, int hi, int k, int32_t mask_token, int32_t* tokens, uint8_t* mask_state,
+                         int32_t* n_revealed, void* stream) {
+  if (!conf || !argmax || !active_idx || !row_offsets || !tokens || !mask_state || B <= 0 || N <= 0 || lo < 0 ||
+      hi < lo || hi > N || k < 0)
+    return SL_EINVAL;
+  return launch_update_mask(conf, argmax, active_idx, row_offsets, B, N, lo, hi, k, mask_token, tokens, mask_state,
+                            n_revealed, (cudaStream_t)stream);
+}
+
 int surelock_attention(const void* q, const void* k_cache, const void* v_cache, const int32_t* active_idx,
                        const int32_t* row_offsets, const int32_t* n_active, int max_rows, int B, int N, int H,
                        int head_dim, void* o, int dtype, int impl, int32_t* dev_status, void* stream) {

@@ -140,4 +140,8 @@ int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
                           cudaStream_t st);
 
+int launch_update_mask(const float* conf, const int32_t* argmax, const int32_t* idx, const int32_t* row_offsets, int B,
+                       int N, int lo, int hi, int k, int32_t mask_token, int32_t* tokens, uint8_t* mask_state,
+                       int32_t* n_revealed, cudaStream_t st);
+
 }  // namespace sl

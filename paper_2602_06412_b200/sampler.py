@@ -1,10 +1,10 @@
 """Decoding harness around the SureLock step: the sampler loop of Algorithm 1 with the unmasking policy on the device.
 
-The library call (`surelock_step`) is Algorithm 1 lines 6-15 and 18-24; this module plays line 5 (the loop over
-diffusion steps) and line 16 (`UpdateMASK`): semi-autoregressive blocks, and in every step each sequence reveals the
-`k` masked positions of its current block whose posterior is most confident, with their argmax tokens (temperature 0,
-"low-confidence remasking": the rest stay masked).  Everything here is torch device arithmetic on the step's packed
-outputs, so the loop never waits for the GPU; per-step times are CUDA events read at the end.
+The library call `surelock_step` is Algorithm 1 lines 6-15 and 18-24, `surelock_update_mask` is line 16
+(`UpdateMASK`); this module plays line 5 (the loop over diffusion steps): semi-autoregressive blocks, and in every step
+each sequence reveals the `k` masked positions of its current block whose posterior is most confident, with their
+argmax tokens (temperature 0, "low-confidence remasking": the rest stay masked).  Both calls are kernels of the
+library working on device buffers, so the loop never waits for the GPU; per-step times are CUDA events read at the end.
 
 It also computes what the paper reports from such a run: the per-step active-row trace M_t, the micro-averaged active
 ratio r_bar, the algorithmic-FLOP ratio F_prop / F_base (Sec. 2.3), E2E-TPS and StepTPS (unmasked tokens per
@@ -26,22 +26,6 @@ def algorithmic_flops_per_step(cfg: Dict, B: int, N: int) -> int:
     return L * (4 * B * H * N * N * dh + 2 * B * N * d * d + 2 * B * N * d * d + 4 * B * N * d * H * dh + 6 * B * N * d * F)
 
 
-def update_mask(tokens, mask_state, conf_pos, argmax_pos, lo: int, hi: int, k: int, mask_token: int):
-    """UpdateMASK: in block [lo, hi) of every sequence reveal the k masked positions with the highest confidence
-    (lowest index on ties) with their argmax token.  All arguments are device tensors [B][N]; in place; no sync."""
-    for _ in range(k):
-        blk_mask = mask_state[:, lo:hi] == 1
-        score = torch.where(blk_mask, conf_pos[:, lo:hi], torch.full_like(conf_pos[:, lo:hi], -1.0))
-        j = torch.argmax(score, dim=1, keepdim=True)                         # first maximum = lowest index
-        has = blk_mask.any(dim=1, keepdim=True)
-        tok = torch.gather(argmax_pos[:, lo:hi], 1, j)
-        tok = torch.where(tok == mask_token, torch.zeros_like(tok), tok)     # never "reveal" the mask token itself
-        cur_t = torch.gather(tokens[:, lo:hi], 1, j)
-        cur_m = torch.gather(mask_state[:, lo:hi], 1, j)
-        tokens[:, lo:hi].scatter_(1, j, torch.where(has, tok, cur_t))
-        mask_state[:, lo:hi].scatter_(1, j, torch.where(has, torch.zeros_like(cur_m), cur_m))
-
-
 def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: int, block_len: int, steps: int,
         kl_eps: float, surelock: bool = True, unmask_per_step: int = 1) -> Dict:
     """Run `steps` diffusion steps on device tensors tokens int32 [B][N], mask_state uint8 [B][N] (both updated in
@@ -55,9 +39,7 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
     lock = torch.zeros((B, N), dtype=torch.uint8, device=dev)
     m_trace = torch.zeros(steps, dtype=torch.int32, device=dev)
     unmasked_trace = torch.zeros(steps, dtype=torch.int32, device=dev)
-    conf_pos = torch.empty(R + 1, dtype=torch.float32, device=dev)
-    argmax_pos = torch.empty(R + 1, dtype=torch.int32, device=dev)
-    rows = torch.arange(R, device=dev, dtype=torch.int32)
+    n_rev = torch.zeros(B, dtype=torch.int32, device=dev)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
     SL.surelock_reset(ctx)
     ev[0].record()
@@ -66,19 +48,12 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
         if not surelock:
             lock.zero_()                                                     # baseline sampler: nothing stays locked
         m_trace[t:t + 1] = out.n_active
-        # packed (row) -> position; rows >= M are routed to the dummy slot R
-        valid = rows < out.n_active
-        dst = torch.where(valid, out.active_idx, torch.full_like(out.active_idx, R)).long()
-        conf_pos.fill_(-1.0)
-        conf_pos.scatter_(0, dst, out.conf)
-        argmax_pos.scatter_(0, dst, out.argmax)
         blk = min(t // steps_per_block, max((N - n_prompt + block_len - 1) // block_len - 1, 0))
         lo = n_prompt + blk * block_len
         hi = min(lo + block_len, N)
-        before = mask_state.sum(dtype=torch.int32)
-        update_mask(tokens, mask_state, conf_pos[:R].view(B, N), argmax_pos[:R].view(B, N), lo, hi, unmask_per_step,
-                    mask_token)
-        unmasked_trace[t:t + 1] = before - mask_state.sum(dtype=torch.int32)
+        SL.surelock_update_mask(out.conf, out.argmax, out.active_idx, out.row_offsets, B, N, lo, hi, unmask_per_step,
+                                mask_token, tokens, mask_state, n_rev)
+        unmasked_trace[t:t + 1] = n_rev.sum(dtype=torch.int32)
         ev[t + 1].record()
     torch.cuda.synchronize()
     ms = [ev[t].elapsed_time(ev[t + 1]) for t in range(steps)]

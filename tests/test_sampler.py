@@ -1,5 +1,5 @@
-"""The decoding harness: the unmasking policy (pure torch, checked on CPU against a loop) and, on the GPU, the
-sampler loop with and without SureLock (trace invariants and the paper's run metrics)."""
+"""The decoding harness: the on-device unmasking policy against the oracle and, on the GPU, the sampler loop with and
+without SureLock (trace invariants and the paper's run metrics)."""
 import numpy as np
 import pytest
 import torch
@@ -7,29 +7,38 @@ import torch
 from paper_2602_06412_b200 import inputs, sampler
 
 
-def test_update_mask_policy_matches_a_plain_loop():
-    g = torch.Generator().manual_seed(3)
-    B, N, lo, hi, mask_tok = 4, 40, 16, 32, 99
-    for k in (1, 3):
-        tokens = torch.randint(0, 50, (B, N), generator=g, dtype=torch.int32)
-        mask = (torch.rand((B, N), generator=g) < 0.5).to(torch.uint8)
-        mask[1, lo:hi] = 0                                  # a sequence whose block is already fully revealed
-        mask[2, lo:hi] = 1
-        conf = torch.rand((B, N), generator=g)
-        conf[2, lo + 3] = conf[2, lo + 7] = 2.0             # a tie: the lower index wins
-        am = torch.randint(0, 100, (B, N), generator=g, dtype=torch.int32)
-        am[2, lo + 3] = mask_tok                            # the argmax happens to be the mask token: reveal token 0
-        t_ref, m_ref = tokens.clone(), mask.clone()
-        for b in range(B):
-            for _ in range(k):
-                cand = [i for i in range(lo, hi) if m_ref[b, i] == 1]
-                if not cand:
-                    break
-                best = max(cand, key=lambda i: (float(conf[b, i]), -i))
-                t_ref[b, best] = 0 if int(am[b, best]) == mask_tok else int(am[b, best])
-                m_ref[b, best] = 0
-        sampler.update_mask(tokens, mask, conf, am, lo, hi, k, mask_tok)
-        assert torch.equal(tokens, t_ref) and torch.equal(mask, m_ref)
+@pytest.mark.gpu
+@pytest.mark.parametrize("B,N,lo,hi,k", [(4, 40, 16, 32, 1), (4, 40, 16, 32, 3), (3, 700, 0, 700, 5), (2, 1536, 512, 576, 64),
+                                         (1, 64, 10, 10, 2), (5, 33, 0, 33, 0)])
+def test_update_mask_kernel_matches_the_oracle(B, N, lo, hi, k):
+    """surelock_update_mask (Algorithm 1 line 16) against the oracle, bit-exact: ragged active sets, ties in the
+    confidence (coarse values), a sequence whose block is already revealed, a fully masked block, argmax equal to the
+    mask token, an empty block, k = 0, more reveals asked for than masked positions."""
+    from oracle import surelock_oracle as O
+    from paper_2602_06412_b200 import binding as SL
+    rng = np.random.default_rng(B * 1000 + N + k)
+    V = 50
+    mask_tok = V - 1
+    tokens = rng.integers(0, V - 1, (B, N)).astype(np.int32)
+    mask = (rng.random((B, N)) < 0.5).astype(np.uint8)
+    if hi > lo:
+        mask[min(1, B - 1), lo:hi] = 0
+        mask[B - 1, lo:hi] = 1
+    tokens[mask == 1] = mask_tok
+    lock = ((rng.random((B, N)) < 0.4) & (mask == 0)).astype(np.uint8)
+    idx, offs = O.active_set(lock)
+    conf = np.round(rng.random(len(idx)), 1).astype(np.float32)
+    am = rng.integers(0, V, len(idx)).astype(np.int32)
+    t_ref, m_ref, rev_ref = O.update_mask(tokens, mask, conf, am, idx, lo, hi, k, mask_tok)
+    dev = "cuda"
+    t_d, m_d = torch.from_numpy(tokens).to(dev), torch.from_numpy(mask).to(dev)
+    rev = torch.full((B,), -1, dtype=torch.int32, device=dev)
+    SL.surelock_update_mask(torch.from_numpy(conf).to(dev), torch.from_numpy(am).to(dev),
+                            torch.from_numpy(idx.astype(np.int32)).to(dev), torch.from_numpy(offs.astype(np.int32)).to(dev),
+                            B, N, lo, hi, k, mask_tok, t_d, m_d, rev)
+    torch.cuda.synchronize()
+    assert np.array_equal(t_d.cpu().numpy(), t_ref) and np.array_equal(m_d.cpu().numpy(), m_ref)
+    assert np.array_equal(rev.cpu().numpy(), rev_ref)
 
 
 def test_flop_accounting_matches_section_2_3_formula():
