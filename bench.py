@@ -338,22 +338,31 @@ def main():
         runs = {}
         tk, mk = tokens.to(dev), mask.to(dev)
         sampler.run(ctx, tk, mk, n_prompt, block_len, 2, 1e-3)               # untimed: first-use costs of the loop's torch ops
-        for mode in ("surelock", "baseline"):
+        for mode in ("surelock", "baseline", "selection", "hybrid"):
             tk, mk = tokens.to(dev), mask.to(dev)
-            r = sampler.run(ctx, tk, mk, n_prompt, block_len, args.sampler_steps, 1e-3, surelock=(mode == "surelock"))
+            r = sampler.run(ctx, tk, mk, n_prompt, block_len, args.sampler_steps, 1e-3,
+                            surelock=mode in ("surelock", "hybrid"),
+                            select_fraction=0.8 if mode in ("selection", "hybrid") else None)
             runs[mode] = r
+        base_tps = max(runs["baseline"]["e2e_tps"], 1e-9)
         sampler_run = dict(
             steps=args.sampler_steps, block_len=block_len, kl_eps=1e-3, confidence_gate="off",
             r_bar=round(runs["surelock"]["r_bar"], 4), flops_ratio=round(runs["surelock"]["flops_ratio"], 4),
             f_base_per_position=runs["baseline"]["f_base_per_position"],
             f_prop_per_position=runs["surelock"]["f_prop_per_position"],
             e2e_tps_surelock=round(runs["surelock"]["e2e_tps"], 2), e2e_tps_baseline=round(runs["baseline"]["e2e_tps"], 2),
-            tps_ratio=round(runs["surelock"]["e2e_tps"] / max(runs["baseline"]["e2e_tps"], 1e-9), 3),
+            tps_ratio=round(runs["surelock"]["e2e_tps"] / base_tps, 3),
+            # Experiment 5: selection surrogate (0.8 of the positions) alone and combined with SureLock
+            selection=dict(fraction=0.8, tps_ratio=round(runs["selection"]["e2e_tps"] / base_tps, 3),
+                           flops_ratio=round(runs["selection"]["r_bar"], 4)),
+            hybrid=dict(fraction=0.8, tps_ratio=round(runs["hybrid"]["e2e_tps"] / base_tps, 3),
+                        flops_ratio=round(runs["hybrid"]["r_bar"], 4)),
             M_trace=runs["surelock"]["M_trace"],
             ms_per_step_surelock=[round(x, 3) for x in runs["surelock"]["ms_per_step"]],
             ms_per_step_baseline_median=round(float(np.median(runs["baseline"]["ms_per_step"])), 3),
             note="random-init weights: the lock trajectory is synthetic (posteriors barely move, so unmasked rows lock "
-                 "at their second step); the paper reports 0.54x FLOPs and 1.30x TPS for LLaDA-8B-Instruct on its GPU")
+                 "at their second step); the paper reports 0.54x FLOPs and 1.30x TPS for SureLock, 0.64x / 1.18x for "
+                 "selection at 0.8 and 0.28x / 1.73x for the combination (LLaDA-8B-Instruct on its GPU)")
         SL.surelock_reset(ctx)
 
     status = SL.surelock_status_poll(ctx)

@@ -26,11 +26,32 @@ def algorithmic_flops_per_step(cfg: Dict, B: int, N: int) -> int:
     return L * (4 * B * H * N * N * dh + 2 * B * N * d * d + 2 * B * N * d * d + 4 * B * N * d * H * dh + 6 * B * N * d * F)
 
 
+def selection_skip_mask(lock: torch.Tensor, mask_state: torch.Tensor, fraction: float, step: int, seed: int):
+    """Surrogate of a selection-based method (Experiment 5): compute only a fixed `fraction` of the positions that are
+    not locked.  Which ones is the selection method's business; this surrogate draws them with a seeded generator,
+    per sequence, and never skips a masked position (the sampler needs its posterior).  Returns uint8 [B][N], 1 = skip
+    this step.  Device arithmetic on the lock mask only; the step itself is unchanged."""
+    B, N = lock.shape
+    g = torch.Generator(device=lock.device).manual_seed(seed * 1000003 + step)
+    score = torch.rand((B, N), generator=g, device=lock.device)
+    eligible = (lock == 0) & (mask_state == 0)                       # may be skipped
+    n_unlocked = (lock == 0).sum(dim=1, keepdim=True)
+    n_skip = torch.minimum(torch.floor(n_unlocked * (1.0 - fraction)).long(), eligible.sum(dim=1, keepdim=True))
+    score = torch.where(eligible, score, torch.full_like(score, 2.0))
+    rank = score.argsort(dim=1).argsort(dim=1)                       # 0 = first to be skipped
+    return ((rank < n_skip) & eligible).to(torch.uint8)
+
+
 def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: int, block_len: int, steps: int,
-        kl_eps: float, surelock: bool = True, unmask_per_step: int = 1) -> Dict:
+        kl_eps: float, surelock: bool = True, unmask_per_step: int = 1, select_fraction: float = None,
+        select_seed: int = 0) -> Dict:
     """Run `steps` diffusion steps on device tensors tokens int32 [B][N], mask_state uint8 [B][N] (both updated in
     place).  Generation positions n_prompt.. are decoded block by block (`block_len` positions, `steps_per_block` =
-    ceil(block_len / unmask_per_step) steps each).  Returns the trace and the paper's metrics."""
+    ceil(block_len / unmask_per_step) steps each).  `select_fraction` (Experiment 5, e.g. 0.8) adds the selection
+    surrogate: every step only that fraction of the not-yet-locked positions is computed; with `surelock` this is the
+    paper's combination, without it the selection baseline.  A skipped row keeps its cached K/V; it has no posterior in
+    that step, so it cannot lock in the step in which it returns (D needs the previous step's posterior).
+    Returns the trace and the paper's metrics."""
     B, N = tokens.shape
     dev = tokens.device
     R = B * N
@@ -44,7 +65,13 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
     SL.surelock_reset(ctx)
     ev[0].record()
     for t in range(steps):
-        out = SL.surelock_step(ctx, tokens, mask_state, lock, kl_eps)
+        if select_fraction is None:
+            out = SL.surelock_step(ctx, tokens, mask_state, lock, kl_eps)
+        else:
+            skip = selection_skip_mask(lock, mask_state, select_fraction, t, select_seed)
+            step_lock = lock | skip                                          # skipped rows are simply not active
+            out = SL.surelock_step(ctx, tokens, mask_state, step_lock, kl_eps)
+            lock |= step_lock & (skip ^ 1)                                   # new locks come from computed rows only
         if not surelock:
             lock.zero_()                                                     # baseline sampler: nothing stays locked
         m_trace[t:t + 1] = out.n_active

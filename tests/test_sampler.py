@@ -72,3 +72,50 @@ def test_sampler_run_with_and_without_surelock():
     assert abs(sure["r_bar"] - sum(M) / (64 * B * N)) < 1e-12 and sure["flops_ratio"] == sure["r_bar"] < 1.0
     assert abs(sure["f_prop_per_position"] / sure["f_base_per_position"] - sure["r_bar"]) < 1e-12
     assert sure["e2e_tps"] > 0 and len(sure["step_tps"]) == 64
+
+
+@pytest.mark.gpu
+def test_selection_hybrid_run():
+    """Experiment 5's three settings on a tiny model: selection alone computes a fixed fraction of all positions,
+    SureLock alone the unlocked ones, the combination that fraction of the unlocked ones (never skipping a masked
+    position), so it computes no more than selection alone; decoding still completes."""
+    from paper_2602_06412_b200 import binding as SL
+    from tests.parity_util import to_dev
+    cfg = inputs.model_shape("tiny")
+    w = to_dev(inputs.make_weights(cfg, 9, dtype=torch.float32))
+    B, N, n_prompt, blk, steps, k = 2, 128, 64, 32, 64, 0.8
+    res = {}
+    for name, sure, frac in (("sure", True, None), ("select", False, k), ("hybrid", True, k)):
+        ctx = SL.surelock_init(cfg, w, N, B)
+        tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], 9)
+        tokens, mask = tokens.cuda(), mask.cuda()
+        res[name] = sampler.run(ctx, tokens, mask, n_prompt, blk, steps=steps, kl_eps=1e-3, surelock=sure,
+                                select_fraction=frac, select_seed=4)
+        assert SL.surelock_status_poll(ctx) == 0
+        assert res[name]["masked_at_end"] == 0 and res[name]["unmasked_per_step"] == [B] * steps
+    sel, hyb, sure = res["select"], res["hybrid"], res["sure"]
+    # selection alone: floor(0.2 * N) positions per sequence skipped whenever enough unmasked ones exist
+    for t, M in enumerate(sel["M_trace"]):
+        masked = B * max(N - n_prompt - t, 0)                           # one reveal per sequence and step
+        assert B * N - B * int(N * (1 - k)) <= M <= B * N and M >= masked
+    assert sel["locked_at_end"] == 0
+    # (a skipped row cannot lock in the step in which it returns, so the combination locks later than SureLock alone;
+    # with these synthetic posteriors, where rows lock right after being revealed, it need not beat SureLock alone)
+    assert hyb["r_bar"] < sel["r_bar"] < 1.0 and sure["r_bar"] < 1.0 and hyb["locked_at_end"] > 0
+    assert all(m <= s for m, s in zip(hyb["M_trace"][2:], sel["M_trace"][2:]))
+
+
+def test_selection_skip_mask_properties():
+    g = torch.Generator().manual_seed(1)
+    B, N = 3, 50
+    lock = (torch.rand((B, N), generator=g) < 0.3).to(torch.uint8)
+    mask = ((torch.rand((B, N), generator=g) < 0.3) & (lock == 0)).to(torch.uint8)
+    mask[2] = (lock[2] == 0).to(torch.uint8)                             # every unlocked position still masked
+    skip = sampler.selection_skip_mask(lock, mask, 0.8, 5, 7)
+    assert not (skip & lock).any() and not (skip & mask).any()          # only computed, unmasked positions are skipped
+    for b in range(B):
+        unlocked = int((lock[b] == 0).sum())
+        eligible = int(((lock[b] == 0) & (mask[b] == 0)).sum())
+        assert int(skip[b].sum()) == min(int(unlocked * 0.2), eligible)
+    assert torch.equal(skip, sampler.selection_skip_mask(lock, mask, 0.8, 5, 7))   # seeded
+    assert not torch.equal(skip, sampler.selection_skip_mask(lock, mask, 0.8, 6, 7))
