@@ -165,12 +165,14 @@ def workload_config(args, cfgname, cfg, B, N, pattern, M=None):
 def run_reference(args, cfgname, B, N, pattern):
     cfg = inputs.model_shape(cfgname)
     vals, secs = [], 0.0
-    for _ in range(max(1, min(args.steps, 3))):
+    for _ in range(max(0, args.warmup)):                              # untimed, like the GPU arm's warm-up steps
+        oracle_sample(cfg, B, N, rows=32, head_rows=8, repeat=1)
+    for _ in range(max(1, args.steps)):                               # each step: a bounded sample of the workload
         v, s, threads, desc = oracle_sample(cfg, B, N, rows=128, head_rows=32, repeat=1)
         vals.append(v); secs += s
     v = float(np.median(vals))
     return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
-            "steps": len(vals), "warmup": 0, "ms_per_step": 1e3 * secs / len(vals), "higher_is_better": True,
+            "steps": len(vals), "warmup": max(0, args.warmup), "ms_per_step": 1e3 * secs / len(vals), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": dict(workload_config(args, cfgname, cfg, B, N, pattern), note="CPU oracle, bounded sample per step"),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
