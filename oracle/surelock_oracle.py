@@ -371,7 +371,10 @@ def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.n
     logp = log_softmax(logits)
     conf, am = posterior_stats(logits)                            # line 18
     bb, ii = idx // N, idx % N
-    D = np.full(M, np.inf, F64)                                   # line 19
+    D = np.full(M, np.inf, F64)                                   # line 19: KL(p_t || p_{t-1}) if t > 1 else inf
+    # p_{t-1} is the posterior computed at step t-1.  Under Algorithm 1 the active set only shrinks, so every active row
+    # has one from the second step on; a row that an extension (un-locking, a selection method) returns to the active
+    # set after steps in which it was not computed has none, and gets inf like a first step.
     has_prev = state.prev_valid[bb, ii]
     if has_prev.any():
         D[has_prev] = kl_rows(logp[has_prev], state.prev_logp[bb[has_prev], ii[has_prev]])
@@ -383,6 +386,7 @@ def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.n
     new_lock = np.array(lock, dtype=np.uint8, copy=True)
     new_lock[bb[lockable], ii[lockable]] = 1                      # line 24
     state.prev_logp[bb, ii] = logp                                # locked rows keep p_{t*}
+    state.prev_valid[:] = False                                   # "previous" means computed in the step just taken
     state.prev_valid[bb, ii] = True
     state.flops += flops
     return dict(active_idx=idx, row_offsets=offs, hidden=hidden, logits=logits, kl=D,

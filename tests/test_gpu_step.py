@@ -183,3 +183,57 @@ def test_single_layer_llada_shape(M_list):
         assert ek < 2e-2 and ev < 2e-2, (M, ek, ev)
         Kc[:] = f64(kg)
         Vc[:] = f64(vg)
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 2e-4), (torch.bfloat16, 5e-2)])
+def test_degenerate_active_sets(dtype, tol):
+    """The degenerate cases of the active set: every position locked (M = 0: nothing is computed or written, the call
+    still succeeds), one sequence of the batch fully locked next to a sequence with a single active row, and a row that
+    returns to the active set after a step in which it was not computed (D = inf in its first step back)."""
+    cfg = inputs.model_shape("tiny")
+    B, N, eps = 3, 96, 1e-3
+    w = inputs.make_weights(cfg, 11, dtype=dtype, std=0.05)
+    wn, wd = inputs.weights_to_numpy(w), to_dev(w)
+    ctx = SL.surelock_init(cfg, wd, N, B)
+    st = O.OracleState(O.ModelCfg(**cfg), B, N)
+    tokens, mask = inputs.make_tokens(B, N, 40, cfg["vocab"], 11)
+    rnd = (lambda a: torch.from_numpy(a).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()) \
+        if dtype == torch.bfloat16 else None
+
+    def both(lock):
+        ld = lock.to(DEV)
+        out = SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), ld, eps)
+        assert SL.surelock_status_poll(ctx) == 0
+        ref = O.step(st, wn, tokens.numpy(), mask.numpy(), lock.numpy(), eps, logits_round=rnd)
+        M = out.M()
+        assert M == len(ref["active_idx"])
+        assert np.array_equal(out.active_idx[:M].cpu().numpy(), ref["active_idx"])
+        assert np.array_equal(out.row_offsets.cpu().numpy(), ref["row_offsets"])
+        if M:
+            assert rel_err_rows(f64(out.logits[:M]), ref["logits"]) < tol
+        return out, ref, ld.cpu()
+
+    lock = torch.zeros((B, N), dtype=torch.uint8)
+    both(lock)                                                           # step 1: everything active
+    kv_before = [t.clone() for t in SL.surelock_kv_cache(ctx, 0)]
+    # every position locked
+    full = torch.ones((B, N), dtype=torch.uint8)
+    out, ref, after = both(full)
+    assert out.M() == 0 and torch.equal(after, full)
+    for a, b in zip(kv_before, SL.surelock_kv_cache(ctx, 0)):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    # sequence 0 fully locked, sequence 1 with one active row, sequence 2 ragged
+    lock = torch.ones((B, N), dtype=torch.uint8)
+    lock[1, 57] = 0
+    lock[2, 5:70:3] = 0
+    out, ref, after = both(lock)
+    M = out.M()
+    assert M == 1 + len(range(5, 70, 3)) and out.row_offsets.cpu().tolist() == [0, 0, 1, M]
+    assert torch.isinf(out.kl[:M]).all()                                 # none of them was computed in the previous step
+    assert torch.equal(after, lock)                                      # so none of them can lock
+    # the same rows once more: now they have a previous posterior
+    out, ref, after = both(lock)
+    kl = out.kl[:M].cpu().numpy().astype(np.float64)
+    assert np.isfinite(kl).all()
+    fin = np.isfinite(ref["kl"])
+    assert fin.all() and np.all(np.abs(kl - ref["kl"]) <= (2e-2 if dtype == torch.bfloat16 else 1e-3) * ref["kl"] + 1e-6)

@@ -471,3 +471,32 @@ def test_update_mask_reveals_the_most_confident_masked_block_positions():
     am = np.array([0, 0, 3, 3, 4, 9, 6])
     t2, m2, rev = O.update_mask(tokens, mask, conf, am, idx, 2, 6, 2, 9)
     assert t2.tolist() == [[7, 7, 3, 1, 9, 0, 9]] and m2.tolist() == [[0, 0, 0, 0, 1, 0, 1]] and rev.tolist() == [2]
+
+
+def test_kl_is_stepwise_a_returning_row_starts_over():
+    """Algorithm 1 line 19: D_t = KL(p_t || p_{t-1}) if t > 1 else inf.  Pinned by hand on a tiny model: the rows of a
+    second step have D equal to the KL between the two steps' softmaxes (scipy), and a row that sat out one step has
+    D = inf in the step in which it returns, whatever posterior it had before."""
+    c, oc, w, wn = _small(seed=8)
+    B, N = 1, 10
+    tokens, mask = inputs.make_tokens(B, N, 4, c["vocab"], 8)
+    st = O.OracleState(oc, B, N)
+    lock = np.zeros((B, N), np.uint8)
+    r1 = O.step(st, wn, tokens.numpy(), mask.numpy(), lock, 1e-3)
+    assert np.isinf(r1["kl"]).all()
+    tok2 = tokens.numpy().copy()
+    tok2[0, 5] = 3
+    m2 = mask.numpy().copy()
+    m2[0, 5] = 0
+    lock2 = lock.copy()
+    lock2[0, 2] = 1                                                   # position 2 sits this step out
+    r2 = O.step(st, wn, tok2, m2, lock2, 0.0)
+    p1 = scipy.special.softmax(r1["logits"], axis=1)
+    p2 = scipy.special.softmax(r2["logits"], axis=1)
+    rows1 = r2["active_idx"]                                          # step-1 rows were all positions in order
+    want = np.array([scipy.special.rel_entr(p2[i], p1[pos]).sum() for i, pos in enumerate(rows1)])
+    np.testing.assert_allclose(r2["kl"], want, rtol=1e-9, atol=1e-15)
+    r3 = O.step(st, wn, tok2, m2, lock, 1e-3)                         # position 2 is back
+    back = int(np.flatnonzero(r3["active_idx"] == 2)[0])
+    assert np.isinf(r3["kl"][back]) and np.isfinite(np.delete(r3["kl"], back)).all()
+    assert r3["new_lock"][0, 2] == 0
