@@ -210,7 +210,7 @@ def test_gemm_cuda_cores(dtype, tol, M, n_out, K):
 @pytest.mark.parametrize("M,n_out,K", [(1, 256, 64), (100, 256, 256), (128, 512, 4096), (129, 136, 200), (300, 4096, 512),
                                        (1000, 1024, 1024), (0, 256, 256), (32, 4096, 12288), (130, 1024, 8192),
                                        (20, 4096, 4096), (60, 12288, 4096), (128, 4096, 12288), (305, 4096, 12288),
-                                       (305, 12288, 4096), (700, 12288, 1024)])
+                                       (305, 12288, 4096), (700, 12288, 1024), (638, 4096, 12288), (1534, 4096, 4096)])
 def test_gemm_tensor_cores(M, n_out, K, split):
     """Covers every tiling regime: one row tile with 32 / 64 / 128 activation rows per stage and K split (the last
     arriver finishes alone, or the splits of a tile finish it together), a few row tiles with K split, single-CTA tiles
