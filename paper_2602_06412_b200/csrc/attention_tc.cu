@@ -2,11 +2,17 @@
 // the active rows attend to ALL N cached keys/values of their sequence, bidirectional, no mask).
 //
 // Work item = (sequence b, head h, up to 256 consecutive packed rows of that sequence = two tiles of 128; one tile
-// when that spreads a small problem over more SMs, decided on the device from the row counts); items never straddle
-// sequences.  Persistent CTAs take items round-robin, the row-tile index fastest, so CTAs working at the same
-// time read the same K/V head through L2.  Keys are streamed in blocks of 128.
-//   warp 0     TMA producer: both Q tiles once per item, then K and V blocks (two stages each), token-major cache rows,
-//              128-byte swizzle;
+// when that spreads a small problem over more SMs); items never straddle sequences.  Persistent CTAs take items
+// round-robin, the row-tile index fastest, so CTAs working at the same time read the same K/V head through L2.  Keys
+// are streamed in blocks of 128.  Two modes, chosen on the device from the row counts of the sequences:
+//  * PAIRS (dense active sets): the two tiles of an item share every K/V block (two stages each);
+//  * STREAMS (at least as many lone tiles as pairs, e.g. every sequence has <= 128 active rows): a CTA runs two
+//    independent streams of one-tile items (stream CTA + t * grid), each with its own Q tile, ONE K and ONE V buffer and
+//    its own producer warp, so that any two tiles share an SM; every tile of a launch takes the same number of key
+//    blocks, so the streams advance in step.  (K/V blocks are then copied once per tile, which costs 3-9 % when the
+//    tiles could have shared them: hence the two modes.)
+//   warp 0     TMA producer (of stream 0; warp 10 of stream 1): Q once per item, then K and V blocks, token-major
+//              cache rows, 128-byte swizzle;
 //   warp 1     one thread issues, per key block and tile t: O_t += P_t V (previous block; P_t is read from TENSOR
 //              MEMORY as the A operand, V is the MN-major shared-memory operand) and then S_t = Q_t K^T;
 //   warps 2-5  softmax of tile 0, warps 6-9 softmax of tile 1: ONE thread per query row (no exchange between
@@ -29,7 +35,7 @@ namespace sl {
 
 namespace {
 
-constexpr int PP_THREADS = 320;   // TMA warp, MMA warp, 4 softmax warps per tile
+constexpr int PP_THREADS = 352;   // TMA warp, MMA warp, 4 softmax warps per tile, second TMA warp (STREAMS mode)
 constexpr int PP_BQ = 128, PP_BKV = 128, PP_ITEM_ROWS = 256;
 constexpr int PP_MAX_B = 1024;
 
@@ -69,13 +75,14 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   uint8_t* sK = sQ + 2 * Q_BYTES;                      // 2 stages
   uint8_t* sV = sK + 2 * KV_BYTES;                     // 2 stages
   uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * KV_BYTES);
-  enum { Q_FULL = 0, Q_FREE, K_FULL, K_FREE = K_FULL + 2, V_FULL = K_FREE + 2, V_FREE = V_FULL + 2, S_FULL = V_FREE + 2,
-         P_HALF = S_FULL + 2, P_FULL = P_HALF + 2, O_FULL = P_FULL + 2, O_FREE = O_FULL + 2,
-         X_PROF = O_FREE + 2, NUM_BARS = X_PROF + 1 };
+  // every barrier name has two slots: per K/V stage or per tile in PAIRS mode (Q: slot 0), per stream in STREAMS mode
+  enum { Q_FULL = 0, Q_FREE = 2, K_FULL = 4, K_FREE = 6, V_FULL = 8, V_FREE = 10, S_FULL = 12, P_HALF = 14, P_FULL = 16,
+         O_FULL = 18, O_FREE = 20, NUM_BARS = 22 };
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   int* s_item_rows = reinterpret_cast<int*>(s_tmem + 2);
-  int* s_prefix = reinterpret_cast<int*>(s_tmem + 3);  // [B+1] work-item prefix per sequence
+  int* s_streams = reinterpret_cast<int*>(s_tmem + 3);
+  int* s_prefix = reinterpret_cast<int*>(s_tmem + 4);  // [B+1] work-item prefix per sequence
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -94,11 +101,20 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   griddep_wait();
   griddep_launch();
   if (threadIdx.x == 0) {
-    // items of two tiles, unless one-tile items finish sooner: a one-tile item takes about 0.8 of the time of a
+    // STREAMS when lone tiles (a sequence's odd tile) are at least as many as tile pairs
+    int lone = 0, pairs = 0;
+    for (int b = 0; b < B; ++b) {
+      const int tb = (row_offsets[b + 1] - row_offsets[b] + PP_BQ - 1) / PP_BQ;
+      lone += tb & 1;
+      pairs += tb >> 1;
+    }
+    const int streams = lone >= pairs;
+    *s_streams = streams;
+    // PAIRS: items of two tiles, unless one-tile items finish sooner: a one-tile item takes about 0.8 of the time of a
     // two-tile item (its softmax warps and the tensor pipe alternate instead of overlapping), so they win when they
-    // spread over idle SMs, i.e. when 4 * rounds(one-tile) < 5 * rounds(two-tile)
-    int rows = PP_ITEM_ROWS, rounds2 = 0;
-    for (int pass = 0; pass < 3; ++pass) {
+    // spread over idle SMs, i.e. when 4 * rounds(one-tile) < 5 * rounds(two-tile).  STREAMS: one-tile items.
+    int rows = streams ? PP_BQ : PP_ITEM_ROWS, rounds2 = 0;
+    for (int pass = streams ? 2 : 0; pass < 3; ++pass) {
       int acc = 0;
       s_prefix[0] = 0;
       for (int b = 0; b < B; ++b) {
@@ -125,6 +141,8 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
   const uint32_t tmem_base = *s_tmem;
   const int total = s_prefix[B];
   const int item_rows = *s_item_rows;
+  const bool streams = *s_streams != 0;
+  const int nstream = 2 * (int)gridDim.x;
   const int nblk = (N + PP_BKV - 1) / PP_BKV;
 
   // item -> (b, h, first packed row, rows in the item (1..256))
@@ -144,141 +162,204 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     nrows = mb - qt * item_rows < item_rows ? mb - qt * item_rows : item_rows;
   };
 
-  if (warp == 0) {
-    if (lane == 0) {
-      uint32_t kcnt = 0, qcnt = 0;
-      bool ok = true;
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++qcnt) {
-        int b, h, row0, nrows;
-        decode(w, b, h, row0, nrows);
-        const int ntile = nrows > PP_BQ ? 2 : 1;
-        if (!(ok = mbar_wait(bar(Q_FREE), (qcnt & 1) ^ 1, s_abort))) break;
-        mbar_expect_tx(bar(Q_FULL), ntile * Q_BYTES);
-        for (int t = 0; t < ntile; ++t)
-#pragma unroll
+  if (streams) {
+    if (warp == 0 || warp == 10) {
+      if (lane == 0) {
+        const int t = warp == 0 ? 0 : 1;                   // stream of this producer
+        uint32_t kcnt = 0, qcnt = 0;
+        bool ok = true;
+        for (int w = (int)blockIdx.x + t * (int)gridDim.x; w < total && ok; w += nstream, ++qcnt) {
+          int b, h, row0, nrows;
+          decode(w, b, h, row0, nrows);
+          if (!(ok = mbar_wait(bar(Q_FREE + t), (qcnt & 1) ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(Q_FULL + t), Q_BYTES);
+  #pragma unroll
           for (int s = 0; s < SLABS; ++s)
-            tma_load_2d(smem_u32(sQ + t * Q_BYTES + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0 + t * PP_BQ, bar(Q_FULL));
-        for (int j = 0; j < nblk; ++j, ++kcnt) {
-          const int st = kcnt & 1;
-          const uint32_t ph = (kcnt >> 1) & 1;
-          const int key0 = b * N + j * PP_BKV;
-          if (!(ok = mbar_wait(bar(K_FREE + st), ph ^ 1, s_abort))) break;
-          mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
-#pragma unroll
-          for (int s = 0; s < SLABS; ++s)
-            tma_load_2d(smem_u32(sK + st * KV_BYTES + s * SLAB_BYTES), &tmK, h * DH + 64 * s, key0, bar(K_FULL + st));
-          if (!(ok = mbar_wait(bar(V_FREE + st), ph ^ 1, s_abort))) break;
-          mbar_expect_tx(bar(V_FULL + st), KV_BYTES);
-#pragma unroll
-          for (int s = 0; s < SLABS; ++s)
-            tma_load_2d(smem_u32(sV + st * KV_BYTES + s * SLAB_BYTES), &tmV, h * DH + 64 * s, key0, bar(V_FULL + st));
+            tma_load_2d(smem_u32(sQ + t * Q_BYTES + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0, bar(Q_FULL + t));
+          for (int j = 0; j < nblk; ++j, ++kcnt) {
+            const uint32_t ph = kcnt & 1;
+            const int key0 = b * N + j * PP_BKV;
+            if (!(ok = mbar_wait(bar(K_FREE + t), ph ^ 1, s_abort))) break;
+            mbar_expect_tx(bar(K_FULL + t), KV_BYTES);
+  #pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+              tma_load_2d(smem_u32(sK + t * KV_BYTES + s * SLAB_BYTES), &tmK, h * DH + 64 * s, key0, bar(K_FULL + t));
+            if (!(ok = mbar_wait(bar(V_FREE + t), ph ^ 1, s_abort))) break;
+            mbar_expect_tx(bar(V_FULL + t), KV_BYTES);
+  #pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+              tma_load_2d(smem_u32(sV + t * KV_BYTES + s * SLAB_BYTES), &tmV, h * DH + 64 * s, key0, bar(V_FULL + t));
+          }
         }
       }
-    }
-  } else if (warp == 1) {
-    if (lane == 0) {
-      constexpr uint32_t idesc_s = idesc_bf16_m128(PP_BKV, false);
-      constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
-      uint32_t kc = 0, it = 0;
-      uint32_t gt[2] = {0, 0}, itt[2] = {0, 0};          // per tile: key blocks and items so far
-      bool ok = true;
-#ifdef ATT_PROFILE
-      unsigned long long mp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, m0 = clock64(), m1;
-      uint32_t xp = 0;
-#define ATT_M(i) { m1 = clock64(); mp[i] += m1 - m0; m0 = m1; }
-#else
-#define ATT_M(i)
-#endif
-      // S_t = Q_t K^T for the key block in stage kst
-      auto issue_s = [&](int t, int kst) {
-#ifdef ATT_PROFILE2
-        ATT_M(0)
-#endif
-        const uint32_t qa = smem_u32(sQ + t * Q_BYTES), ka = smem_u32(sK + kst * KV_BYTES);
-#pragma unroll
-        for (int kk = 0; kk < DH / 16; ++kk) {
-          const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
-          tc_mma_bf16(tmem_base + t * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
-        }
-        tc_commit(bar(S_FULL + t));
-#ifdef ATT_PROFILE2
-        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(6) }
-#endif
-      };
-      // O_t (+)= P_t V for the key block in stage vst; jb = index of that block inside the item
-      auto issue_pv = [&](int t, int vst, int jb) -> bool {
-        const uint32_t va = smem_u32(sV + vst * KV_BYTES);
-        ATT_M(0)
-        if (!mbar_wait(bar(P_HALF + t), (gt[t] + jb) & 1, s_abort)) return false;
-        ATT_M(1 + t)
-        if (jb == 0 && !mbar_wait(bar(O_FREE + t), (itt[t] & 1) ^ 1, s_abort)) return false;
-        tc_fence_after();
-#pragma unroll
-        for (int kk = 0; kk < PP_BKV / 32; ++kk)
-          tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
-                         smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, (jb | kk) != 0);
-#ifdef ATT_PROFILE2
-        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(7) }
-#else
-        ATT_M(0)
-#endif
-        if (!mbar_wait(bar(P_FULL + t), (gt[t] + jb) & 1, s_abort)) return false;
-        ATT_M(3 + t)
-        tc_fence_after();
-#pragma unroll
-        for (int kk = PP_BKV / 32; kk < PP_BKV / 16; ++kk)
-          tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
-                         smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, 1);
-#ifdef ATT_PROFILE2
-        { tc_commit(bar(X_PROF)); mbar_wait(bar(X_PROF), xp & 1, s_abort); ++xp; ATT_M(7) }
-#endif
-        return true;
-      };
-      for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
-        int b, h, row0, nrows;
-        decode(w, b, h, row0, nrows);
-        const int ntile = nrows > PP_BQ ? 2 : 1;
-        if (!(ok = mbar_wait(bar(Q_FULL), it & 1, s_abort))) break;
-        for (int j = 0; j < nblk && ok; ++j) {
-          const int kst = (kc + j) & 1;
-          ATT_M(0)
-          if (!(ok = mbar_wait(bar(K_FULL + kst), ((kc + j) >> 1) & 1, s_abort))) break;
-          const int vst = (kc + j - 1) & 1;
-          if (j > 0 && !(ok = mbar_wait(bar(V_FULL + vst), ((kc + j - 1) >> 1) & 1, s_abort))) break;
-          ATT_M(5)
-          for (int t = 0; t < ntile && ok; ++t) {
-            if (j > 0) ok = issue_pv(t, vst, j - 1);
-            if (!ok) break;
-            tc_fence_after();
-            issue_s(t, kst);
+    } else if (warp == 1) {
+      if (lane == 0) {
+        constexpr uint32_t idesc_s = idesc_bf16_m128(PP_BKV, false);
+        constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
+        uint32_t g = 0, it = 0;                            // key blocks and tiles so far (the same for both streams)
+        bool ok = true;
+        // S_t = Q_t K^T for the key block in the stream's K buffer
+        auto issue_s = [&](int t) {
+          const uint32_t qa = smem_u32(sQ + t * Q_BYTES), ka = smem_u32(sK + t * KV_BYTES);
+  #pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
+            tc_mma_bf16(tmem_base + t * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
+          }
+          tc_commit(bar(S_FULL + t));
+          tc_commit(bar(K_FREE + t));
+        };
+        // O_t (+)= P_t V for key block jb of the tile (global block number g + jb), V in the stream's V buffer
+        auto issue_pv = [&](int t, int jb) -> bool {
+          const uint32_t va = smem_u32(sV + t * KV_BYTES);
+          const uint32_t par = (g + jb) & 1;
+          if (!mbar_wait(bar(V_FULL + t), par, s_abort)) return false;
+          if (!mbar_wait(bar(P_HALF + t), par, s_abort)) return false;
+          if (jb == 0 && !mbar_wait(bar(O_FREE + t), (it & 1) ^ 1, s_abort)) return false;
+          tc_fence_after();
+  #pragma unroll
+          for (int kk = 0; kk < PP_BKV / 32; ++kk)
+            tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                           smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, (jb | kk) != 0);
+          if (!mbar_wait(bar(P_FULL + t), par, s_abort)) return false;
+          tc_fence_after();
+  #pragma unroll
+          for (int kk = PP_BKV / 32; kk < PP_BKV / 16; ++kk)
+            tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                           smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, 1);
+          tc_commit(bar(V_FREE + t));
+          return true;
+        };
+        // the two streams take their tiles in step: round `it` is tile CTA + t * grid + it * nstream of stream t
+        for (int w0 = (int)blockIdx.x; w0 < total && ok; w0 += nstream, ++it) {
+          const int nt = w0 + (int)gridDim.x < total ? 2 : 1;   // streams that still have a tile
+          for (int t = 0; t < nt && ok; ++t) ok = mbar_wait(bar(Q_FULL + t), it & 1, s_abort);
+          for (int j = 0; j < nblk && ok; ++j) {
+            for (int t = 0; t < nt && ok; ++t) {
+              if (j > 0) ok = issue_pv(t, j - 1);
+              if (!ok) break;
+              if (!(ok = mbar_wait(bar(K_FULL + t), (g + j) & 1, s_abort))) break;
+              tc_fence_after();
+              issue_s(t);
+            }
           }
           if (!ok) break;
-          tc_commit(bar(K_FREE + kst));
-          if (j > 0) tc_commit(bar(V_FREE + vst));
-        }
-        if (!ok) break;
-        tc_commit(bar(Q_FREE));                          // every S product of this item has been issued
-        const int vst = (kc + nblk - 1) & 1;
-        if (!(ok = mbar_wait(bar(V_FULL + vst), ((kc + nblk - 1) >> 1) & 1, s_abort))) break;
-        for (int t = 0; t < ntile && ok; ++t) {
-          ok = issue_pv(t, vst, nblk - 1);
-          if (ok) tc_commit(bar(O_FULL + t));
-        }
-        if (!ok) break;
-        tc_commit(bar(V_FREE + vst));
-        kc += nblk;
-        for (int t = 0; t < ntile; ++t) {
-          gt[t] += nblk;
-          ++itt[t];
+          for (int t = 0; t < nt; ++t) tc_commit(bar(Q_FREE + t));   // every S product of these tiles has been issued
+          for (int t = 0; t < nt && ok; ++t) {
+            ok = issue_pv(t, nblk - 1);
+            if (ok) tc_commit(bar(O_FULL + t));
+          }
+          g += nblk;
         }
       }
-#ifdef ATT_PROFILE
-      ATT_M(0)
-      if (prof && blockIdx.x == 0)
-        for (int i = 0; i < 8; ++i) prof[16 + i] = mp[i];
-#endif
     }
   } else {
+    if (warp == 0) {
+      if (lane == 0) {
+        uint32_t kcnt = 0, qcnt = 0;
+        bool ok = true;
+        for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++qcnt) {
+          int b, h, row0, nrows;
+          decode(w, b, h, row0, nrows);
+          const int ntile = nrows > PP_BQ ? 2 : 1;
+          if (!(ok = mbar_wait(bar(Q_FREE), (qcnt & 1) ^ 1, s_abort))) break;
+          mbar_expect_tx(bar(Q_FULL), ntile * Q_BYTES);
+          for (int t = 0; t < ntile; ++t)
+  #pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+              tma_load_2d(smem_u32(sQ + t * Q_BYTES + s * SLAB_BYTES), &tmQ, h * DH + 64 * s, row0 + t * PP_BQ, bar(Q_FULL));
+          for (int j = 0; j < nblk; ++j, ++kcnt) {
+            const int st = kcnt & 1;
+            const uint32_t ph = (kcnt >> 1) & 1;
+            const int key0 = b * N + j * PP_BKV;
+            if (!(ok = mbar_wait(bar(K_FREE + st), ph ^ 1, s_abort))) break;
+            mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
+  #pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+              tma_load_2d(smem_u32(sK + st * KV_BYTES + s * SLAB_BYTES), &tmK, h * DH + 64 * s, key0, bar(K_FULL + st));
+            if (!(ok = mbar_wait(bar(V_FREE + st), ph ^ 1, s_abort))) break;
+            mbar_expect_tx(bar(V_FULL + st), KV_BYTES);
+  #pragma unroll
+            for (int s = 0; s < SLABS; ++s)
+              tma_load_2d(smem_u32(sV + st * KV_BYTES + s * SLAB_BYTES), &tmV, h * DH + 64 * s, key0, bar(V_FULL + st));
+          }
+        }
+      }
+    } else if (warp == 1) {
+      if (lane == 0) {
+        constexpr uint32_t idesc_s = idesc_bf16_m128(PP_BKV, false);
+        constexpr uint32_t idesc_o = idesc_bf16_m128(DH, true);
+        uint32_t kc = 0, it = 0;
+        uint32_t gt[2] = {0, 0}, itt[2] = {0, 0};          // per tile: key blocks and items so far
+        bool ok = true;
+        // S_t = Q_t K^T for the key block in stage kst
+        auto issue_s = [&](int t, int kst) {
+          const uint32_t qa = smem_u32(sQ + t * Q_BYTES), ka = smem_u32(sK + kst * KV_BYTES);
+  #pragma unroll
+          for (int kk = 0; kk < DH / 16; ++kk) {
+            const uint32_t off = (kk >> 2) * SLAB_BYTES + (kk & 3) * 32;
+            tc_mma_bf16(tmem_base + t * 128, smem_desc_k_sw128(qa + off), smem_desc_k_sw128(ka + off), idesc_s, kk != 0);
+          }
+          tc_commit(bar(S_FULL + t));
+        };
+        // O_t (+)= P_t V for the key block in stage vst; jb = index of that block inside the item
+        auto issue_pv = [&](int t, int vst, int jb) -> bool {
+          const uint32_t va = smem_u32(sV + vst * KV_BYTES);
+          if (!mbar_wait(bar(P_HALF + t), (gt[t] + jb) & 1, s_abort)) return false;
+          if (jb == 0 && !mbar_wait(bar(O_FREE + t), (itt[t] & 1) ^ 1, s_abort)) return false;
+          tc_fence_after();
+  #pragma unroll
+          for (int kk = 0; kk < PP_BKV / 32; ++kk)
+            tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                           smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, (jb | kk) != 0);
+          if (!mbar_wait(bar(P_FULL + t), (gt[t] + jb) & 1, s_abort)) return false;
+          tc_fence_after();
+  #pragma unroll
+          for (int kk = PP_BKV / 32; kk < PP_BKV / 16; ++kk)
+            tc_mma_bf16_ta(tmem_base + O_COL + t * DH, tmem_base + t * 128 + 64 + kk * 8,
+                           smem_desc_mn_sw128(va + kk * 16 * 128, SLAB_BYTES), idesc_o, 1);
+          return true;
+        };
+        for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
+          int b, h, row0, nrows;
+          decode(w, b, h, row0, nrows);
+          const int ntile = nrows > PP_BQ ? 2 : 1;
+          if (!(ok = mbar_wait(bar(Q_FULL), it & 1, s_abort))) break;
+          for (int j = 0; j < nblk && ok; ++j) {
+            const int kst = (kc + j) & 1;
+            if (!(ok = mbar_wait(bar(K_FULL + kst), ((kc + j) >> 1) & 1, s_abort))) break;
+            const int vst = (kc + j - 1) & 1;
+            if (j > 0 && !(ok = mbar_wait(bar(V_FULL + vst), ((kc + j - 1) >> 1) & 1, s_abort))) break;
+            for (int t = 0; t < ntile && ok; ++t) {
+              if (j > 0) ok = issue_pv(t, vst, j - 1);
+              if (!ok) break;
+              tc_fence_after();
+              issue_s(t, kst);
+            }
+            if (!ok) break;
+            tc_commit(bar(K_FREE + kst));
+            if (j > 0) tc_commit(bar(V_FREE + vst));
+          }
+          if (!ok) break;
+          tc_commit(bar(Q_FREE));                          // every S product of this item has been issued
+          const int vst = (kc + nblk - 1) & 1;
+          if (!(ok = mbar_wait(bar(V_FULL + vst), ((kc + nblk - 1) >> 1) & 1, s_abort))) break;
+          for (int t = 0; t < ntile && ok; ++t) {
+            ok = issue_pv(t, vst, nblk - 1);
+            if (ok) tc_commit(bar(O_FULL + t));
+          }
+          if (!ok) break;
+          tc_commit(bar(V_FREE + vst));
+          kc += nblk;
+          for (int t = 0; t < ntile; ++t) {
+            gt[t] += nblk;
+            ++itt[t];
+          }
+        }
+      }
+    }
+  }
+  if (warp >= 2 && warp < 10) {
     const int t = (warp - 2) >> 2;                       // tile of this warp
     const int quarter = warp & 3;                        // tensor-memory lane quarter this warp may access
     const int trow = quarter * 32 + lane;                // query row of this thread inside the tile
@@ -306,10 +387,13 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #else
 #define ATT_T(i)
 #endif
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
+    // PAIRS: tile t of every item of this CTA; STREAMS: every item of stream t
+    const int w_first = (int)blockIdx.x + (streams ? t * (int)gridDim.x : 0), w_step = streams ? nstream : (int)gridDim.x;
+    const int t_off = streams ? 0 : t * PP_BQ;
+    for (int w = w_first; w < total && ok; w += w_step) {
       int b, h, row0, nrows;
       decode(w, b, h, row0, nrows);
-      const int rows_t = nrows - t * PP_BQ;              // rows of this tile (<= 0: the item has no second tile)
+      const int rows_t = nrows - t_off;                  // rows of this tile (<= 0: the item has no second tile)
       if (rows_t <= 0) continue;
       float m_used = 0.f, l = 0.f;
       // one key block of this tile; MASKED only for a last block that reaches beyond key N (kept apart so that the
@@ -399,7 +483,7 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ++it;
       tc_fence_after();
       const float inv = 1.f / l;
-      bf16* orow = o + ((long long)(row0 + t * PP_BQ + trow) * H + h) * DH;
+      bf16* orow = o + ((long long)(row0 + t_off + trow) * H + h) * DH;
 #pragma unroll 1
       for (int c = 0; c < DH; c += 32) {
         uint32_t ov[32];
@@ -441,7 +525,7 @@ template <int DH>
 static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets,
                         int max_rows, int B, int N, int H, void* o, int32_t* status, cudaStream_t st) {
   constexpr int SLABS = DH / 64;
-  const int smem = 6 * SLABS * 128 * 128 + 1024 + 512 + 4 * (B + 3);
+  const int smem = 6 * SLABS * 128 * 128 + 1024 + 512 + 4 * (B + 4);
   static int attr_smem = 0;
   if (smem > attr_smem) {
     SL_CUDA_TRY(cudaFuncSetAttribute(attention_pp_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -464,8 +548,6 @@ static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtens
   {
     unsigned long long h[24];
     cudaMemcpy(h, d_prof, 192, cudaMemcpyDeviceToHost);
-    fprintf(stderr, "ATT_PROFILE mma thread cycles: issue+other %llu waitPhalf0 %llu waitPhalf1 %llu waitPfull0 %llu waitPfull1 %llu waitKV %llu  S-product %llu  PV-product %llu\n",
-            h[16], h[17], h[18], h[19], h[20], h[21], h[22], h[23]);
     for (int t = 0; t < 2; ++t)
       fprintf(stderr, "ATT_PROFILE tile %d cycles: loop %llu waitS %llu ldS %llu max %llu turn %llu exp-to-half %llu rest %llu waitO+epi %llu\n",
               t, h[8 * t], h[8 * t + 1], h[8 * t + 2], h[8 * t + 3], h[8 * t + 4], h[8 * t + 5], h[8 * t + 6], h[8 * t + 7]);
