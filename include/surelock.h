@@ -135,6 +135,20 @@ int surelock_kv_cache(surelock_ctx *ctx, int layer, void **k, void **v, size_t *
  * or -1 when the position has no previous posterior.  Writing both lets a caller seed p_{t-1}. */
 int surelock_prev_logits(surelock_ctx *ctx, void **buf, int32_t **row_of_pos);
 
+/* Checkpoint / resume of a decoding run (the paper has no counterpart; the sampler state it lists in Algorithm 1's
+ * "Require" and lines 1-3 is the lock mask, the cache C and p_{t-1}; the lock mask, tokens and mask state are the
+ * caller's).  surelock_state_export writes what the ctx holds between two steps into a HOST buffer: a header (model
+ * shape, N, batch, element type, rows of the last step), the K/V cache of every layer, and the previous step's logits,
+ * their log-sum-exps and position -> row table.  surelock_state_import loads such a buffer into a ctx created with the
+ * same model shape, N, batch and element type (weights are not part of the state); the next surelock_step then
+ * continues bit for bit as the exporting ctx would have.  Both calls synchronise the ctx stream.
+ *   surelock_state_bytes: capacity that always suffices for this ctx (the export usually writes less: only the rows
+ *   of the last step's logits are stored).
+ * Returns SL_EINVAL on NULL / too small a buffer / a buffer that is not a state of this shape, SL_ECUDA on a failed copy. */
+size_t surelock_state_bytes(const surelock_ctx *ctx);
+int surelock_state_export(surelock_ctx *ctx, void *host_dst, size_t capacity, size_t *written);
+int surelock_state_import(surelock_ctx *ctx, const void *host_src, size_t bytes);
+
 /* Optional confidence gate (Algorithm 1 lines 18, 21, 23; Sec. 2.2): with 0 <= m_percent <= 100 every later
  * surelock_step locks a candidate (active, unmasked row) only if, besides D <= kl_eps, its uncertainty
  * u = 1 - max_v p(v) is <= theta_m, the m-th percentile (linear interpolation between order statistics) of u over

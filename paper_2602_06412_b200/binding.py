@@ -64,6 +64,9 @@ def lib() -> C.CDLL:
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
         "surelock_conf_gate_lock": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, f32, f32, vp, vp]),
         "surelock_update_mask": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
+        "surelock_state_bytes": (sz, [vp]),
+        "surelock_state_export": (i32, [vp, vp, sz, C.POINTER(sz)]),
+        "surelock_state_import": (i32, [vp, vp, sz]),
         "surelock_layer_trace": (i32, [vp, C.POINTER(vp), C.POINTER(sz)]),
         "surelock_kernel_times": (i32, [vp, vp, vp, i32]),
         "surelock_destroy": (None, [vp]),
@@ -254,6 +257,20 @@ def surelock_update_mask(conf, argmax, active_idx, row_offsets, B: int, N: int, 
     """UpdateMASK (Algorithm 1 line 16) on the device; tokens int32 [B][N] and mask_state uint8 [B][N] in place."""
     _check(lib().surelock_update_mask(_p(conf), _p(argmax), _p(active_idx), _p(row_offsets), B, N, lo, hi, k, mask_token,
                                       _p(tokens), _p(mask_state), _p(n_revealed), _stream()), "surelock_update_mask")
+
+
+def surelock_state_export(ctx: Ctx) -> bytes:
+    """Checkpoint of what the ctx holds between two steps (K/V cache, previous posterior), as host bytes."""
+    cap = lib().surelock_state_bytes(ctx.handle)
+    buf = (C.c_char * cap)()
+    n = C.c_size_t(0)
+    _check(lib().surelock_state_export(ctx.handle, C.cast(buf, C.c_void_p), cap, C.byref(n)), "surelock_state_export")
+    return bytes(memoryview(buf)[: n.value])
+
+
+def surelock_state_import(ctx: Ctx, state: bytes):
+    buf = (C.c_char * len(state)).from_buffer_copy(state)
+    _check(lib().surelock_state_import(ctx.handle, C.cast(buf, C.c_void_p), len(state)), "surelock_state_import")
 
 
 def surelock_last_launch_count(ctx: Ctx) -> int:

@@ -373,6 +373,85 @@ int surelock_prev_logits(surelock_ctx* c, void** buf, int32_t** row_of_pos) {
   return SL_OK;
 }
 
+// ---- checkpoint / resume
+struct StateHeader {
+  uint64_t magic;                       // "SLKSTAT1"
+  int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab, dtype, N, B;
+  int32_t have_prev, rows_prev;         // rows of the previous step's logits that are stored
+  int32_t reserved[5];
+};
+static const uint64_t STATE_MAGIC = 0x31544154534b4c53ull;
+
+static void fill_header(const surelock_ctx* c, StateHeader* h) {
+  memset(h, 0, sizeof(*h));
+  h->magic = STATE_MAGIC;
+  h->n_layers = c->cfg.n_layers; h->d_model = c->cfg.d_model; h->n_heads = c->cfg.n_heads; h->head_dim = c->cfg.head_dim;
+  h->d_ff = c->cfg.d_ff; h->vocab = c->cfg.vocab; h->dtype = c->cfg.dtype; h->N = c->N; h->B = c->B;
+}
+
+size_t surelock_state_bytes(const surelock_ctx* c) {
+  if (!c) return 0;
+  const size_t R = c->R, V = c->cfg.vocab;
+  return sizeof(StateHeader) + 2 * (size_t)c->cfg.n_layers * c->kv_layer_bytes() + R * V * c->esz + R * 4 + R * 4;
+}
+
+int surelock_state_export(surelock_ctx* c, void* host_dst, size_t capacity, size_t* written) {
+  if (!c || !host_dst) return SL_EINVAL;
+  SL_CUDA_TRY(cudaStreamSynchronize(c->st));
+  const int prv = c->cur ^ 1;           // the slot the last step wrote
+  StateHeader h;
+  fill_header(c, &h);
+  h.have_prev = c->have_prev ? 1 : 0;
+  int32_t m_prev = 0;
+  if (c->have_prev) SL_CUDA_TRY(cudaMemcpy(&m_prev, c->n_active, 4, cudaMemcpyDeviceToHost));
+  if (m_prev < 0 || m_prev > c->R) return SL_EDEVICE;
+  h.rows_prev = m_prev;
+  const size_t kvb = 2 * (size_t)c->cfg.n_layers * c->kv_layer_bytes();
+  const size_t lgb = (size_t)m_prev * c->cfg.vocab * c->esz, lsb = (size_t)m_prev * 4, rpb = (size_t)c->R * 4;
+  const size_t need = sizeof(h) + kvb + lgb + lsb + rpb;
+  if (capacity < need) return SL_EINVAL;
+  char* p = static_cast<char*>(host_dst);
+  memcpy(p, &h, sizeof(h));
+  p += sizeof(h);
+  SL_CUDA_TRY(cudaMemcpy(p, c->kv, kvb, cudaMemcpyDeviceToHost));
+  p += kvb;
+  if (lgb) SL_CUDA_TRY(cudaMemcpy(p, c->logits[prv], lgb, cudaMemcpyDeviceToHost));
+  p += lgb;
+  if (lsb) SL_CUDA_TRY(cudaMemcpy(p, c->lse[prv], lsb, cudaMemcpyDeviceToHost));
+  p += lsb;
+  SL_CUDA_TRY(cudaMemcpy(p, c->row_of_pos[prv], rpb, cudaMemcpyDeviceToHost));
+  if (written) *written = need;
+  return SL_OK;
+}
+
+int surelock_state_import(surelock_ctx* c, const void* host_src, size_t bytes) {
+  if (!c || !host_src || bytes < sizeof(StateHeader)) return SL_EINVAL;
+  StateHeader h, want;
+  memcpy(&h, host_src, sizeof(h));
+  fill_header(c, &want);
+  if (h.magic != STATE_MAGIC || h.n_layers != want.n_layers || h.d_model != want.d_model || h.n_heads != want.n_heads ||
+      h.head_dim != want.head_dim || h.d_ff != want.d_ff || h.vocab != want.vocab || h.dtype != want.dtype ||
+      h.N != want.N || h.B != want.B || h.rows_prev < 0 || h.rows_prev > c->R)
+    return SL_EINVAL;
+  const size_t kvb = 2 * (size_t)c->cfg.n_layers * c->kv_layer_bytes();
+  const size_t lgb = (size_t)h.rows_prev * c->cfg.vocab * c->esz, lsb = (size_t)h.rows_prev * 4, rpb = (size_t)c->R * 4;
+  if (bytes < sizeof(h) + kvb + lgb + lsb + rpb) return SL_EINVAL;
+  SL_CUDA_TRY(cudaStreamSynchronize(c->st));
+  SL_TRY(surelock_reset(c));
+  const int prv = c->cur ^ 1;
+  const char* p = static_cast<const char*>(host_src) + sizeof(h);
+  SL_CUDA_TRY(cudaMemcpyAsync(c->kv, p, kvb, cudaMemcpyHostToDevice, c->st));
+  p += kvb;
+  if (lgb) SL_CUDA_TRY(cudaMemcpyAsync(c->logits[prv], p, lgb, cudaMemcpyHostToDevice, c->st));
+  p += lgb;
+  if (lsb) SL_CUDA_TRY(cudaMemcpyAsync(c->lse[prv], p, lsb, cudaMemcpyHostToDevice, c->st));
+  p += lsb;
+  SL_CUDA_TRY(cudaMemcpyAsync(c->row_of_pos[prv], p, rpb, cudaMemcpyHostToDevice, c->st));
+  c->have_prev = h.have_prev != 0;
+  SL_CUDA_TRY(cudaStreamSynchronize(c->st));
+  return SL_OK;
+}
+
 int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }

@@ -237,3 +237,40 @@ def test_degenerate_active_sets(dtype, tol):
     assert np.isfinite(kl).all()
     fin = np.isfinite(ref["kl"])
     assert fin.all() and np.all(np.abs(kl - ref["kl"]) <= (2e-2 if dtype == torch.bfloat16 else 1e-3) * ref["kl"] + 1e-6)
+
+
+def test_checkpoint_resume_continues_bit_for_bit():
+    """surelock_state_export / _import: a second ctx that imports the state taken after three steps takes the fourth
+    step exactly as the first one does (same packing, logits, KL, lock decisions, cache bytes); a state of another
+    shape is refused."""
+    cfg = inputs.model_shape("tiny", d_model=512, n_heads=4, head_dim=128, d_ff=1536, vocab=4096, n_layers=2)
+    B, N, eps = 2, 160, 1e-3
+    wd = to_dev(inputs.make_weights(cfg, 21, dtype=torch.bfloat16, std=0.04))
+    a = SL.surelock_init(cfg, wd, N, B)
+    tokens, mask = inputs.make_tokens(B, N, 60, cfg["vocab"], 21)
+    tok_d, mask_d = tokens.to(DEV), mask.to(DEV)
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    for t in range(3):
+        SL.surelock_step(a, tok_d, mask_d, lock, eps)
+        lock = inputs.bernoulli_lock_schedule(lock.cpu(), mask == 0, 0.3, 500 + t).to(DEV)
+    state = SL.surelock_state_export(a)
+    b = SL.surelock_init(cfg, wd, N, B)
+    SL.surelock_state_import(b, state)
+    la, lb = lock.clone(), lock.clone()
+    oa = SL.surelock_step(a, tok_d, mask_d, la, eps)
+    ob = SL.surelock_step(b, tok_d, mask_d, lb, eps)
+    assert SL.surelock_status_poll(a) == 0 and SL.surelock_status_poll(b) == 0
+    M = oa.M()
+    assert M == ob.M() and 0 < M < B * N
+    assert torch.equal(oa.active_idx[:M], ob.active_idx[:M])
+    assert torch.equal(oa.logits[:M].view(torch.int16), ob.logits[:M].view(torch.int16))
+    assert torch.equal(oa.kl[:M].view(torch.int32), ob.kl[:M].view(torch.int32)) and torch.isfinite(oa.kl[:M]).any()
+    assert torch.equal(la, lb)
+    for l in range(cfg["n_layers"]):
+        for x, y in zip(SL.surelock_kv_cache(a, l), SL.surelock_kv_cache(b, l)):
+            assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    other = SL.surelock_init(cfg, wd, N + 32, B)
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_state_import(other, state)
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_state_import(b, state[: len(state) // 2])
