@@ -2,8 +2,9 @@
 // (the Q/K/V, output, SwiGLU and LM-head contractions of Algorithm 1 lines 10, 12 and 15).
 //
 // Persistent, warp-specialised CTAs, one per SM:
-//   warp 0   TMA producer: cp.async.bulk.tensor loads of a 128x64 A tile and two 128x64 W tiles per stage into
-//            128-byte-swizzled shared memory, completion counted on an mbarrier (no multicast);
+//   warp 0   TMA producer: cp.async.bulk.tensor loads of an A tile (128, 64 or 32 rows x 64) and a W tile (BN rows x 64,
+//            as one 256-row box when BN = 256) per stage into 128-byte-swizzled shared memory, completion counted on
+//            an mbarrier (no multicast); 4 to 16 stages in 216 KB, the stage size follows the tile;
 //   warp 1   allocates tensor memory and issues tcgen05.mma (128 x BN x 16, cta_group::1) from one thread, operands
 //            described by shared-memory matrix descriptors; tcgen05.commit hands smem stages back to the producer
 //            and finished accumulators to the epilogue;
@@ -12,6 +13,10 @@
 //            the row's ORIGINAL position, q stored packed, k and v written straight into the cache row of that
 //            position, which is Algorithm 1 line 11 done in the epilogue) and write with 128-bit stores.
 // Two accumulators live in tensor memory so the epilogue of tile i overlaps the main loop of tile i+1.
+// At large M the whole launch takes the CTA-pair path (run_pair below: cluster of two, cta_group::2, 256 x 256 tiles).
+// At small M the K dimension is split over several CTAs; they meet in a workspace (see the epilogue).  The kernel is
+// launched with programmatic stream serialization: set-up, and inside a step the first weight copies, run while the
+// previous kernel drains.
 // The number of rows M is read from device memory: tiles whose first row is >= M are never scheduled, TMA zero-fills
 // rows beyond the allocation, and the epilogue stores only rows < M.  Every mbarrier wait is bounded: when it runs out
 // the CTA records SL_DEV_GEMM_TIMEOUT, all roles leave their loops, tensor memory is freed and the kernel returns.
@@ -202,10 +207,9 @@ __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, b
 
 // Tile width and K-split for this launch, derived on the device from M so that every role of every CTA agrees.
 // Enough 256-wide tiles to fill the grid (large M): 256-wide, no split, the tensor-pipe-bound configuration.
-// A single row tile (M <= 128, the weight-streaming regime): 128-wide tiles and K split up to four ways.  In between:
-// the width that needs the fewest rounds of the grid.  (Measured on B200: wider splits, or splitting at M > 128,
-// cost more in partial-tile traffic than they gain in balance.)  Splits meet in the workspace; the last arriver of
-// a tile sums them in split order and runs the fused epilogue.
+// A single row tile (M <= 128, the weight-streaming regime): the widest tiles that, split at most four ways, fill one
+// round of the grid.  A few row tiles: width and split with the least estimated time.  Splits meet in the workspace;
+// the partial tiles are summed in split order (deterministic) and the fused epilogue runs on the sum.
 struct TileCfg {
   int bn, S, m_tiles, n_tiles, tiles, total;   // split sp of a tile covers K blocks [sp * num_kb / S, (sp + 1) * num_kb / S)
 };
