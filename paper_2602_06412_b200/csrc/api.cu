@@ -35,6 +35,7 @@ struct surelock_ctx {
   bool have_prev = false;
   int launches = 0;
   int gemm_impl = 0;                  // 0 = tensor cores when possible, 1 = CUDA cores
+  bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
   bool timing = false;                // per-kernel-class CUDA-event timing (off by default)
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
   std::vector<int> ev_cls;            // class of the launch bracketed by events 2i, 2i+1
@@ -42,6 +43,8 @@ struct surelock_ctx {
   float gate_m = -1.f;                // confidence-gate percentile (Algorithm 1 line 21); < 0 = gate off
   float* theta = nullptr;             // [B] gate thresholds of the last step
   SplitWs split;                      // split-K workspace of the tensor-core GEMM (bf16 only)
+  float4* lse_part = nullptr;         // [ceil(V/256)][R]: softmax statistics of the current logits, left by the LM head
+  int* lse_valid = nullptr;           // set by the LM-head GEMM when it wrote them
   float* trace = nullptr;             // [2L+1][R][d]: slot 2l = input of block l, 2l+1 = after its attention sub-block, 2L = output
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
@@ -114,8 +117,10 @@ static int attention(surelock_ctx* c, int l) {
 }
 
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
+  c->last_gemm_tc = false;
   if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->split, c->st);
+    c->last_gemm_tc = rc == SL_OK;
     if (rc != SL_EUNSUPPORTED) return rc;
   }
   return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
@@ -235,6 +240,11 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * 3 * sizeof(int), c->st) != cudaSuccess)
       rc = SL_ECUDA;
   }
+  if (cfg->dtype == SL_BF16 && V > 0) {
+    A_(c->lse_part, ((V + 255) / 256) * R * sizeof(float4));
+    A_(c->lse_valid, 16);
+    if (rc == SL_OK && cudaMemsetAsync(c->lse_valid, 0, 16, c->st) != cudaSuccess) rc = SL_ECUDA;
+  }
   A_(c->theta, ((size_t)batch + 1) * 4);
   A_(c->st_tokens, R * 4);
   A_(c->st_mask, R);
@@ -284,11 +294,18 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
                                   c->st));
   }
   SL_K(K_RMSNORM, launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
+  c->split.lse_part = c->lse_part;                 // the LM head leaves the rows' softmax statistics for the next kernel
+  c->split.lse_rows = c->R;
+  c->split.lse_valid = c->lse_valid;
   SL_K(K_GEMM_HEAD, gemm(c, c->h, c->lm_head, nullptr, c->logits[cur], g.vocab, g.d_model, EPI_STORE));
+  c->split.lse_part = nullptr;
+  c->split.lse_valid = nullptr;
+  const bool head_tc = c->last_gemm_tc;            // only the tensor-core kernel writes the statistics (and their flag)
   SL_K(K_SOFTMAX_KL, launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
                                             c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state,
                                             lock_mask, kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st,
-                                            c->gate_m < 0.f));
+                                            c->gate_m < 0.f, head_tc ? c->lse_part : nullptr,
+                                            (g.vocab + 255) / 256, c->R, c->lse_valid));
   if (c->gate_m >= 0.f)
     SL_K(K_CONF_GATE, launch_conf_gate_lock(c->conf, c->kl, c->idx, c->row_offsets, c->B, c->N, mask_state, lock_mask,
                                             kl_eps, c->gate_m, c->theta, c->st));

@@ -135,7 +135,9 @@ int launch_attention_simt(const void* q, const void* kc, const void* vc, const i
 int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
                            const float* prev_lse, const int32_t* idx, const int32_t* n_active, int max_rows, int vocab,
                            int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
-                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st, bool apply_lock = true);
+                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st, bool apply_lock = true,
+                           const float4* lse_part = nullptr, int part_tiles = 0, int part_rows = 0,
+                           const int* lse_valid = nullptr);   // lse_part: per-tile softmax statistics left by the LM head
 int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx, const int32_t* row_offsets, int B, int N,
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
                           cudaStream_t st);

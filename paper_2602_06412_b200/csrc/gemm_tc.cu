@@ -55,6 +55,17 @@ struct QkvArgs {
   const int32_t* idx;         // [M] flat position of each packed row
   const float2* rope;         // [n_seq][dh/2] (cos, sin)
   int n_seq, hd, dh;
+  // EPI_STORE only (the LM head): per (256-column tile, row) the running maximum, sum of exp(x - max) and arg-max of the
+  // stored (bf16-rounded) values, [n_tiles][lse_rows] float4 (m, s, index as int bits, 0); *lse_valid = 1 when this
+  // launch wrote them (256-wide tiles without K split).  nullptr: not wanted.
+  float4* lse_part;
+  int lse_rows;
+  int* lse_valid;
+};
+
+struct RowStat {
+  float m, s;
+  int am;
 };
 
 // ----------------------------------------------------------------------------------------------- kernel
@@ -121,6 +132,49 @@ __device__ __forceinline__ void store_bf16x32(bf16* dst, const uint32_t* v) {
                                                     pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
                                                     pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
                                                     pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+}
+
+// One 32-column unit of the LM head: store as bf16 and fold the stored values into the row's running softmax statistics
+// (Algorithm 1 line 15: the posterior's normaliser, and the arg-max / confidence of line 18, taken where the logits are
+// still in registers so that the softmax-KL kernel need not read the current row twice).
+template <typename Src>
+__device__ __forceinline__ void store_unit_with_stats(const Src& src, int row, bool live, int u, int n0, int n_out,
+                                                      void* __restrict__ Cv, RowStat& rs) {
+  const int c0 = u * 32, col = n0 + c0;
+  uint32_t v[32];
+  src.load(c0, v);
+  if (!live || col >= n_out) return;
+  float f[32];
+  float lm = -INFINITY;
+  int li = 0;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    f[j] = col + j < n_out ? __bfloat162float(__float2bfloat16_rn(__uint_as_float(v[j]))) : -INFINITY;
+    if (f[j] > lm) {                                   // strict: the lowest index wins a tie
+      lm = f[j];
+      li = j;
+    }
+  }
+  if (lm > rs.m) {
+    rs.s *= fast_exp2((rs.m - lm) * 1.4426950408889634f);   // rs.m = -inf: 0
+    rs.m = lm;
+    rs.am = col + li;
+  }
+  const float nb = -rs.m * 1.4426950408889634f;
+  float2 acc = make_float2(0.f, 0.f);
+#pragma unroll
+  for (int j = 0; j < 32; j += 2) {
+    const float2 t = __ffma2_rn(make_float2(f[j], f[j + 1]), make_float2(1.4426950408889634f, 1.4426950408889634f),
+                                make_float2(nb, nb));
+    acc = __fadd2_rn(acc, make_float2(fast_exp2(t.x), fast_exp2(t.y)));
+  }
+  rs.s += acc.x + acc.y;
+  bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
+  if (col + 32 <= n_out) {
+    store_bf16x32(dst, v);
+  } else {
+    for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
+  }
 }
 
 // The epilogue works in UNITS of one row: 32 output columns (64 for a rotated q/k pair block).  A 128 x bn tile has
@@ -397,8 +451,16 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
       const int row = m0 + quarter * 32 + lane;
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN);
       const int upr = units_per_row<EPI>(BN, n0, qkv);
+      if (EPI == EPI_STORE && qkv.lse_part) {
+        RowStat rs{-INFINITY, 0.f, 0};
 #pragma unroll 1
-      for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv);
+        for (int u = 0; u < upr; ++u) store_unit_with_stats(TmemSrc{taddr}, row, row < M, u, n0, n_out, Cv, rs);
+        if (row < M)
+          qkv.lse_part[(size_t)(n0 / BN) * qkv.lse_rows + row] = make_float4(rs.m, rs.s, __int_as_float(rs.am), 0.f);
+      } else {
+#pragma unroll 1
+        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv);
+      }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(acc), 0));
@@ -456,6 +518,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         griddep_wait();
         griddep_launch();
       }
+      if (EPI == EPI_STORE && qkv.lse_valid && blockIdx.x == 0 && threadIdx.x == 0) *qkv.lse_valid = 1;
       run_pair<EPI>(&tmA, &tmW0, &tmW1, &tmW2, Cv, Mp, n_out, K, status, qkv, smem);
       return;
     }
@@ -507,6 +570,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc.total = tc.tiles * tc.S;
   }
   const int bn = tc.bn, S = tc.S, m_tiles = tc.m_tiles, total = tc.total;
+  if (EPI == EPI_STORE && qkv.lse_valid && blockIdx.x == 0 && threadIdx.x == 0) *qkv.lse_valid = (S == 1 && bn == 256) ? 1 : 0;
   const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
   // Stage layout, chosen from M like the tiles: with a single row tile of few rows only 32 or 64 activation rows are
   // copied per stage (the MMA still reads 128 rows of shared memory; rows >= M are never stored), which leaves room for
@@ -651,8 +715,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * BN_MAX);
       const int upr = units_per_row<EPI>(bn, n0, qkv);
       if (S == 1) {
+        if (EPI == EPI_STORE && qkv.lse_part && bn == 256) {
+          RowStat rs{-INFINITY, 0.f, 0};
 #pragma unroll 1
-        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, bn, row, row < M, u, n0, n_out, Cv, qkv);
+          for (int u = 0; u < upr; ++u) store_unit_with_stats(TmemSrc{taddr}, row, row < M, u, n0, n_out, Cv, rs);
+          if (row < M)
+            qkv.lse_part[(size_t)(n0 / 256) * qkv.lse_rows + row] = make_float4(rs.m, rs.s, __int_as_float(rs.am), 0.f);
+        } else {
+#pragma unroll 1
+          for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, bn, row, row < M, u, n0, n_out, Cv, qkv);
+        }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(acce_bar(acc));
@@ -924,7 +996,13 @@ int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const 
     if (rc != SL_OK) return rc;
   }
   switch (epilogue) {
-    case EPI_STORE: return launch_cfg<EPI_STORE, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
+    case EPI_STORE: {
+      QkvArgs qa{};
+      qa.lse_part = sw.lse_part;
+      qa.lse_rows = sw.lse_rows;
+      qa.lse_valid = sw.lse_valid;
+      return launch_cfg<EPI_STORE, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, qa, sw, st);
+    }
     case EPI_RESIDUAL: return launch_cfg<EPI_RESIDUAL, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
     case EPI_SWIGLU: return launch_cfg<EPI_SWIGLU, TC_MAX_STAGES>(a, b, wb, xb, C, n_active, max_rows, n_out, K, status, QkvArgs{}, sw, st);
     default: return SL_EINVAL;
@@ -951,7 +1029,7 @@ int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void
     if (rc == SL_OK) rc = get_tensor_map_2d(W[i], hd, K, 256, &xb[i]);
   }
   if (rc != SL_OK) return rc;
-  QkvArgs qa{(bf16*)q_out, (bf16*)k_cache, (bf16*)v_cache, idx, rope, n_seq, hd, dh};
+  QkvArgs qa{(bf16*)q_out, (bf16*)k_cache, (bf16*)v_cache, idx, rope, n_seq, hd, dh, nullptr, 0, nullptr};
   return launch_cfg<EPI_QKV, TC_MAX_STAGES>(a, b, wb, xb, nullptr, n_active, max_rows, 3 * hd, K, status, qa, sw, st);
 }
 

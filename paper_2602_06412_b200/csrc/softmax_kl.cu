@@ -347,7 +347,8 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
                             const int32_t* __restrict__ idx, const int32_t* __restrict__ n_active, int V,
                             const uint8_t* __restrict__ mask_state, uint8_t* __restrict__ lock_mask, float kl_eps,
                             float* __restrict__ kl_out, float* __restrict__ conf_out, int32_t* __restrict__ argmax_out,
-                            float* __restrict__ lse_out, int apply_lock) {
+                            float* __restrict__ lse_out, int apply_lock, const float4* __restrict__ lse_part,
+                            int part_tiles, int part_rows, const int* __restrict__ lse_valid) {
   __shared__ float s_m[KLF_THREADS / 32], s_s[KLF_THREADS / 32];
   __shared__ int s_a[KLF_THREADS / 32];
   __shared__ double s_sum[KLF_THREADS / 32];
@@ -355,6 +356,9 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int nvec = V >> 3;
   constexpr int STEP = 2 * KLF_THREADS;   // two vectors per thread and iteration
+  // the LM head may have left the current rows' softmax statistics per 256-column tile: then sweep 1 is a reduction
+  // of part_tiles small records instead of a pass over the row
+  const bool have_part = lse_part != nullptr && *lse_valid != 0;
   const uint64_t pol_keep = l2_policy_keep(), pol_stream = l2_policy_stream();
 
   auto block_maxsum = [&](MaxSum2 st) -> MaxSum {
@@ -384,7 +388,19 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
 
     // sweep 1 (current row; the previous row only if its log-sum-exp was not kept), next vectors prefetched
     MaxSum2 a{-INFINITY, make_float2(0.f, 0.f), 0x7fffffff}, b{-INFINITY, make_float2(0.f, 0.f), 0};
-    {
+    if (have_part) {
+      MaxSum acc{-INFINITY, 0.f, 0x7fffffff};
+      for (int t = tid; t < part_tiles; t += KLF_THREADS) {
+        const float4 p = __ldcs(lse_part + (size_t)t * part_rows + r);
+        acc = combine(acc, MaxSum{p.x, p.y, __float_as_int(p.z)});
+      }
+      a.m = acc.m;
+      a.s = make_float2(acc.s, 0.f);
+      a.am = acc.am;
+      if (need_q) {
+        for (int v0 = tid; v0 < nvec; v0 += KLF_THREADS) accum_maxsum_bf16(ld_hint(y + v0, pol_stream), v0 * 8, b, false);
+      }
+    } else {
       const uint4 zero = make_uint4(0xff80ff80u, 0xff80ff80u, 0xff80ff80u, 0xff80ff80u);   // eight times -inf
       uint4 c0 = tid < nvec ? ld_hint(z + tid, pol_keep) : zero;
       uint4 c1 = tid + KLF_THREADS < nvec ? ld_hint(z + tid + KLF_THREADS, pol_keep) : zero;
@@ -452,7 +468,8 @@ softmax_kl_sure_bf16_kernel(const bf16* __restrict__ logits, const bf16* __restr
 int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const int32_t* row_of_pos_prev,
                            const float* prev_lse, const int32_t* idx, const int32_t* n_active, int max_rows, int vocab,
                            int dtype, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float* kl,
-                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st, bool apply_lock) {
+                           float* conf, int32_t* argmax, float* lse_out, cudaStream_t st, bool apply_lock,
+                           const float4* lse_part, int part_tiles, int part_rows, const int* lse_valid) {
   const int vec = dtype == SL_BF16 ? 8 : 4;
   if (vocab <= 0 || vocab % vec) return SL_EUNSUPPORTED;
   int g = sm_count() * 2;
@@ -470,7 +487,8 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
     if (gb < 1) gb = 1;
     softmax_kl_sure_bf16_kernel<<<gb, KLF_THREADS, 0, st>>>((const bf16*)logits, (const bf16*)prev_logits, row_of_pos_prev,
                                                              prev_lse, idx, n_active, vocab, mask_state, lock_mask, kl_eps,
-                                                             kl, conf, argmax, lse_out, apply_lock ? 1 : 0);
+                                                             kl, conf, argmax, lse_out, apply_lock ? 1 : 0, lse_part,
+                                                             part_tiles, part_rows, lse_valid);
   } else
     softmax_kl_sure_kernel<float><<<g, KL_THREADS, 0, st>>>((const float*)logits, (const float*)prev_logits,
                                                            row_of_pos_prev, prev_lse, idx, n_active, vocab, mask_state,

@@ -183,6 +183,11 @@ struct SplitWs {
   // the caller states that neither *n_active nor the weights were written by the kernel launched just before the
   // GEMM: it may then read M and start its first weight copies before that kernel has completed
   bool prefetch_w = false;
+  // EPI_STORE (LM head) only: where the epilogue leaves per-(256-column tile, row) softmax statistics of the stored
+  // logits, [ceil(n_out / 256)][lse_rows] float4, and the flag it sets when it did (see gemm_tc.cu); nullptr = off
+  float4* lse_part = nullptr;
+  int lse_rows = 0;
+  int* lse_valid = nullptr;
 };
 constexpr size_t SPLIT_TILE_BYTES = 128 * 256 * sizeof(float);
 
