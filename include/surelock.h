@@ -121,8 +121,12 @@ int surelock_step_host(surelock_ctx *ctx, const int32_t *tokens, const uint8_t *
 int surelock_layer_step(surelock_ctx *ctx, int layer, const void *hidden_in, const uint8_t *lock_mask,
                         float *hidden_out, surelock_step_out *out);
 
-/* Synchronise the ctx stream and report: *device_status = 0, or the code a kernel stored (see SL_DEV_* in
- * the source) ; returns SL_EDEVICE if non-zero, SL_ECUDA if the stream reported a CUDA error. */
+/* Synchronise the ctx stream and report: *device_status = 0, or the first code a kernel stored since the last
+ * surelock_reset: 1 = the compaction's bounded look-back wait ran out, 2 = a bounded barrier wait of the tensor-core
+ * GEMM ran out, 3 = the same in the attention kernel (in all three the kernel gave up and returned: the step's
+ * results are invalid), 4 = a token id or row index read from device memory was out of range and was skipped,
+ * 5 = with "check_cache" on, a position entered a step locked although its K/V were never written.
+ * Returns SL_EDEVICE if non-zero, SL_ECUDA if the stream reported a CUDA error. */
 int surelock_status_poll(surelock_ctx *ctx, int *device_status);
 
 /* K/V cache of one layer (Algorithm 1 line 11: K^all / V^all): dev pointers to [B*N][H][d_h] arrays of
@@ -163,7 +167,14 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * step) a buffer [2L+1][B*N][d] fp32 and makes every later surelock_step copy the packed residual stream into it:
  * slot 2l = input of block l (slot 0 = the embeddings), slot 2l+1 = after the attention sub-block of block l,
  * slot 2L = output of the last block; for stage-wise parity checks.  "have_prev": 1 declares the buffers returned by surelock_prev_logits() valid
- * (after a caller seeded them), 0 forgets them.  Unknown names return SL_EINVAL. */
+ * (after a caller seeded them), 0 forgets them.  "check_cache": checks, at the start of every later surelock_step, the
+ * one precondition the host cannot see: a position that enters the step locked must have K/V in the caches (Algorithm 1
+ * line 12 attends to them), i.e. it was active in an earlier step since the last reset / this call, or the caller
+ * filled the caches.  1 = on, no position valid yet; 2 = on, every position declared valid (after a pre-fill through
+ * surelock_kv_cache()); 0 = off (default).  A violation stores device status 5 and the step goes on; one small kernel
+ * per step, one flag byte per position (allocated here).  surelock_reset() invalidates all positions,
+ * surelock_state_import() validates all.  surelock_layer_step() neither checks nor marks.
+ * Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
 /* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [2L+1][B*N][d] (rows packed as in

@@ -45,6 +45,8 @@ struct surelock_ctx {
   SplitWs split;                      // split-K workspace of the tensor-core GEMM (bf16 only)
   float4* lse_part = nullptr;         // [ceil(V/256)][R]: softmax statistics of the current logits, left by the LM head
   int* lse_valid = nullptr;           // set by the LM-head GEMM when it wrote them
+  uint8_t* kv_valid = nullptr;        // [R] "check_cache": 1 = every layer's K/V of the position was written since the last reset
+  bool check_cache = false;
   float* trace = nullptr;             // [2L+1][R][d]: slot 2l = input of block l, 2l+1 = after its attention sub-block, 2L = output
 
   size_t kv_layer_bytes() const { return (size_t)R * cfg.n_heads * cfg.head_dim * esz; }
@@ -73,7 +75,7 @@ static int dev_alloc(surelock_ctx* c, P** p, size_t bytes) {
 
 // Kernel classes for the timing breakdown (order is part of the C ABI: surelock_kernel_times)
 enum { K_COMPACT = 0, K_GATHER, K_RMSNORM, K_GEMM_QKV, K_ROPE, K_SCATTER, K_ATTN, K_GEMM_O, K_GEMM_GATEUP, K_GEMM_DOWN,
-       K_GEMM_HEAD, K_SOFTMAX_KL, K_CONF_GATE, K_NUM };
+       K_GEMM_HEAD, K_SOFTMAX_KL, K_CONF_GATE, K_NUM };   // the cache check counts as K_COMPACT
 
 static inline void tick(surelock_ctx* c, int cls) {
   if (c->timing && c->n_ev + 2 <= (int)c->ev.size()) {
@@ -269,6 +271,7 @@ int surelock_reset(surelock_ctx* c) {
   for (int i = 0; i < 2; ++i) SL_CUDA_TRY(cudaMemsetAsync(c->row_of_pos[i], 0xff, (size_t)c->R * 4, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->status, 0, 16, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->n_active, 0, 16, c->st));
+  if (c->kv_valid) SL_CUDA_TRY(cudaMemsetAsync(c->kv_valid, 0, (size_t)c->R, c->st));   // cache contents are undefined now
   return SL_OK;
 }
 
@@ -281,6 +284,7 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   c->launches = 0;
   const int cur = c->cur, prv = cur ^ 1;
   c->n_ev = 0;
+  if (c->check_cache) SL_K(K_COMPACT, launch_cache_check(lock_mask, c->kv_valid, c->R, c->status, c->st));
   SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur],
                                  c->scratch, c->status, c->st));
   SL_K(K_GATHER, launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype,
@@ -459,6 +463,7 @@ int surelock_state_import(surelock_ctx* c, const void* host_src, size_t bytes) {
   const char* p = static_cast<const char*>(host_src) + sizeof(h);
   SL_CUDA_TRY(cudaMemcpyAsync(c->kv, p, kvb, cudaMemcpyHostToDevice, c->st));
   p += kvb;
+  if (c->kv_valid) SL_CUDA_TRY(cudaMemsetAsync(c->kv_valid, 1, (size_t)c->R, c->st));   // an imported cache counts as filled
   if (lgb) SL_CUDA_TRY(cudaMemcpyAsync(c->logits[prv], p, lgb, cudaMemcpyHostToDevice, c->st));
   p += lgb;
   if (lsb) SL_CUDA_TRY(cudaMemcpyAsync(c->lse[prv], p, lsb, cudaMemcpyHostToDevice, c->st));
@@ -473,6 +478,15 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
+  if (!strcmp(name, "check_cache")) {
+    if (value && !c->kv_valid) {
+      const int rc = dev_alloc(c, &c->kv_valid, (size_t)c->R);
+      if (rc != SL_OK) return rc;
+    }
+    if (value) SL_CUDA_TRY(cudaMemsetAsync(c->kv_valid, value == 2 ? 1 : 0, (size_t)c->R, c->st));
+    c->check_cache = value != 0;
+    return SL_OK;
+  }
   if (!strcmp(name, "trace_layers")) {
     if (value && !c->trace) {
       const size_t bytes = (size_t)(2 * c->cfg.n_layers + 1) * c->R * c->cfg.d_model * sizeof(float);
@@ -545,7 +559,9 @@ const char* surelock_strerror(int s) {
     case SL_EINVAL: return "invalid argument";
     case SL_ENOMEM: return "device allocation failed";
     case SL_ECUDA: return "CUDA runtime error";
-    case SL_EDEVICE: return "a kernel reported an error through the status word";
+    case SL_EDEVICE:
+      return "a kernel reported an error through the status word (1 compaction wait, 2 GEMM wait, 3 attention wait ran "
+             "out; 4 index out of range; 5 locked position without valid K/V)";
     case SL_EUNSUPPORTED: return "shape or type not supported";
     case SL_ELIMIT: return "size exceeds the fixed capacity of the allocation-free entry point";
     default: return "unknown status";

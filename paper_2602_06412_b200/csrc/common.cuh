@@ -14,7 +14,8 @@ enum {
   SL_DEV_COMPACT_TIMEOUT = 1,   // decoupled look-back of the compaction gave up waiting for a predecessor chunk
   SL_DEV_GEMM_TIMEOUT = 2,      // an mbarrier wait in the tcgen05 GEMM ran out
   SL_DEV_ATTN_TIMEOUT = 3,      // an mbarrier wait in the tcgen05 attention ran out
-  SL_DEV_BAD_INDEX = 4          // an index read from device memory was out of range and was skipped
+  SL_DEV_BAD_INDEX = 4,         // an index read from device memory was out of range and was skipped
+  SL_DEV_STALE_CACHE = 5        // "check_cache" is on and a position entered a step locked without valid K/V
 };
 
 // A failing CUDA runtime call makes the entry point return SL_ECUDA; with SURELOCK_DEBUG set in the environment the
@@ -141,6 +142,9 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
 int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx, const int32_t* row_offsets, int B, int N,
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
                           cudaStream_t st);
+
+// step precondition check (cache_check.cu): locked positions need kv_valid, active ones become valid
+int launch_cache_check(const uint8_t* lock, uint8_t* kv_valid, int total, int32_t* status, cudaStream_t st);
 
 int launch_update_mask(const float* conf, const int32_t* argmax, const int32_t* idx, const int32_t* row_offsets, int B,
                        int N, int lo, int hi, int k, int32_t mask_token, int32_t* tokens, uint8_t* mask_state,

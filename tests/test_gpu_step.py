@@ -274,3 +274,48 @@ def test_checkpoint_resume_continues_bit_for_bit():
         SL.surelock_state_import(other, state)
     with pytest.raises(SL.SurelockError):
         SL.surelock_state_import(b, state[: len(state) // 2])
+
+
+def test_cache_check_flags_a_locked_position_without_keys_and_values():
+    """The "check_cache" switch: a position that enters a step locked although no step ever wrote its K/V (the one
+    precondition the host cannot see) is reported as device status 5; legal schedules, a declared pre-fill and an
+    imported state pass; surelock_reset invalidates the positions again."""
+    cfg = inputs.model_shape("tiny")
+    B, N, eps = 2, 96, 1e-3
+    wd = to_dev(inputs.make_weights(cfg, 31, dtype=torch.float32))
+    ctx = SL.surelock_init(cfg, wd, N, B)
+    tokens, mask = inputs.make_tokens(B, N, 40, cfg["vocab"], 31)
+    tok_d, mask_d = tokens.to(DEV), mask.to(DEV)
+    SL.surelock_set_option(ctx, "check_cache", 1)
+    n0 = None
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    for t in range(4):                                    # every position is active in the first step: all later locks are legal
+        SL.surelock_step(ctx, tok_d, mask_d, lock, eps)
+        n0 = SL.surelock_last_launch_count(ctx)
+        lock = inputs.bernoulli_lock_schedule(lock.cpu(), mask == 0, 0.3, 700 + t).to(DEV)
+    assert SL.surelock_status_poll(ctx) == 0
+    SL.surelock_set_option(ctx, "check_cache", 0)
+    SL.surelock_step(ctx, tok_d, mask_d, lock.clone(), eps)
+    assert SL.surelock_last_launch_count(ctx) == n0 - 1   # the check is one launch, and only when switched on
+
+    SL.surelock_reset(ctx)                                # cache contents are undefined again
+    SL.surelock_set_option(ctx, "check_cache", 1)
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    lock[1, 7] = 1                                        # locked before any step computed it
+    SL.surelock_step(ctx, tok_d, mask_d, lock, eps)
+    assert SL.surelock_status_poll(ctx) == 5
+    SL.surelock_reset(ctx)                                # clears the status word
+    assert SL.surelock_status_poll(ctx) == 0
+
+    SL.surelock_set_option(ctx, "check_cache", 2)         # the caller vouches for the caches (pre-fill)
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    lock[1, 7] = 1
+    SL.surelock_step(ctx, tok_d, mask_d, lock, eps)
+    assert SL.surelock_status_poll(ctx) == 0
+
+    state = SL.surelock_state_export(ctx)                 # an imported state counts as a filled cache
+    other = SL.surelock_init(cfg, wd, N, B)
+    SL.surelock_set_option(other, "check_cache", 1)
+    SL.surelock_state_import(other, state)
+    SL.surelock_step(other, tok_d, mask_d, lock, eps)
+    assert SL.surelock_status_poll(other) == 0
