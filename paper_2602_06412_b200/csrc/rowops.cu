@@ -61,7 +61,9 @@ int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* 
 // ------------------------------------------------------------------------------------------------ RMSNorm
 // h = x * rsqrt(mean(x^2) + eps) * g; x fp32 residual stream, h in the storage type (the GEMM operand).
 // One CTA per row.  For d <= 8192 the row is read once and kept in registers (REGS float4 per thread) between the
-// sum of squares and the scaling; longer rows fall back to a second read.
+// sum of squares and the scaling, and the CTA's NEXT row is already on its way while this one is reduced and
+// written (the loads of a persistent CTA otherwise stop during the two barriers and the stores: 0.66 -> 0.75 of
+// the copy rate at 6587 rows of 4096); longer rows fall back to a second read.
 template <typename T, int REGS>
 __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ h,
@@ -72,6 +74,16 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
   const int M = *n_active;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nv = d >> 2;                                   // float4 per row
+  float4 nxt[REGS > 0 ? REGS : 1];                        // the row after this one, in flight while this one is reduced
+  auto fetch = [&](int r) {
+    const float4* xr = reinterpret_cast<const float4*>(x + (long long)r * d);
+#pragma unroll
+    for (int k = 0; k < (REGS > 0 ? REGS : 1); ++k) {
+      const int c = threadIdx.x + k * 256;
+      nxt[k] = c < nv ? __ldcs(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+  if (REGS > 0 && (int)blockIdx.x < M) fetch(blockIdx.x);
   for (int r = blockIdx.x; r < M; r += gridDim.x) {
     const float4* xr = reinterpret_cast<const float4*>(x + (long long)r * d);
     float4 v[REGS > 0 ? REGS : 1];
@@ -79,10 +91,10 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
     if (REGS > 0) {
 #pragma unroll
       for (int k = 0; k < REGS; ++k) {
-        const int c = threadIdx.x + k * 256;
-        v[k] = c < nv ? xr[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        v[k] = nxt[k];
         ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
       }
+      if (r + (int)gridDim.x < M) fetch(r + gridDim.x);
     } else {
       for (int c = threadIdx.x; c < nv; c += 256) {
         const float4 t = xr[c];
@@ -139,7 +151,7 @@ static int launch_rms_t(const float* x, const void* gain, void* h, const int32_t
 int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_active, int max_rows, int d, float eps,
                    int dtype, cudaStream_t st) {
   if (d % 4) return SL_EUNSUPPORTED;
-  const int g = row_grid(max_rows, 8);
+  const int g = row_grid(max_rows, 4);   // 52 registers with the next row in flight: four CTAs per SM
   const int rc = dtype == SL_BF16 ? launch_rms_t<bf16>(x, gain, h, n_active, g, d, eps, st)
                                   : launch_rms_t<float>(x, gain, h, n_active, g, d, eps, st);
   if (rc != SL_OK) return rc;
