@@ -9,7 +9,9 @@
 //            described by shared-memory matrix descriptors; tcgen05.commit hands smem stages back to the producer
 //            and finished accumulators to the epilogue;
 //   warps 2-5 epilogue: tcgen05.ld the fp32 accumulator (one row per thread), apply the fused operation
-//            (store bf16 | add into the fp32 residual stream | silu(gate)*up | QKV: rotary embedding on q and k with
+//            (store bf16 | add into the fp32 residual stream, as 128-byte bulk reductions performed by the L2 from a
+//            per-thread staging slot wherever the stages leave 18 KB of shared memory, so that the epilogue never
+//            waits for a load of x | silu(gate)*up | QKV: rotary embedding on q and k with
 //            the row's ORIGINAL position, q stored packed, k and v written straight into the cache row of that
 //            position, which is Algorithm 1 line 11 done in the epilogue) and write with 128-bit stores.
 // Two accumulators live in tensor memory so the epilogue of tile i overlaps the main loop of tile i+1.
@@ -190,7 +192,7 @@ __device__ __forceinline__ int units_per_row(int bn, int n0, const QkvArgs& qkv)
 
 template <int EPI, typename Src>
 __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, bool live, int u, int n0, int n_out,
-                                              void* __restrict__ Cv, const QkvArgs& qkv) {
+                                              void* __restrict__ Cv, const QkvArgs& qkv, uint32_t red_slot = 0) {
   if (EPI == EPI_QKV) {
     const int srcm = n0 / qkv.hd, ln0 = n0 - srcm * qkv.hd;
     const int pos = live ? qkv.idx[row] : 0;
@@ -237,7 +239,16 @@ __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, b
   if (live && col < n_out) {
     if (EPI == EPI_RESIDUAL) {
       float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + col;
-      if (col + 32 <= n_out) {
+      if (col + 32 <= n_out && red_slot) {
+        // residual add done by the L2: the 128 bytes of this row go through the thread's staging slot into one bulk
+        // reduction, so the epilogue never waits for a load of x
+        bulk_wait_read0();                       // the previous unit's reduction has read the slot
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) st_shared_f4(red_slot + 4 * j, v[j], v[j + 1], v[j + 2], v[j + 3]);
+        fence_async_smem();
+        bulk_reduce_add_f32(dst, red_slot, 128);
+        bulk_commit();
+      } else if (col + 32 <= n_out) {
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
           float4 o = *reinterpret_cast<float4*>(dst + j);
@@ -440,6 +451,11 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
     const int quarter = warp & 3;
     bool ok = true;
     int it = 0;
+    // EPI_RESIDUAL: 144-byte staging slot of this thread above the stages and barriers (the odd stride keeps the eight
+    // 16-byte stores of a quarter warp on different banks)
+    const uint32_t red_slot = EPI == EPI_RESIDUAL
+        ? smem_u32(smem + STAGES * STAGE_BYTES + 1024) + (uint32_t)(quarter * 32 + lane) * 144u : 0u;
+    static_assert(STAGES * STAGE_BYTES + 1024 + 128 * 144 <= TC_DATA_BYTES, "staging slots must fit the allocation");
     for (int w = cid; w < total && ok; w += n_clusters, ++it) {
       const int acc = it & 1;
       const uint32_t use = (uint32_t)(it >> 1);
@@ -459,12 +475,13 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
           qkv.lse_part[(size_t)(n0 / BN) * qkv.lse_rows + row] = make_float4(rs.m, rs.s, __int_as_float(rs.am), 0.f);
       } else {
 #pragma unroll 1
-        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv);
+        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv, red_slot);
       }
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(mapa_u32(acce_bar(acc), 0));
     }
+    if (EPI == EPI_RESIDUAL) bulk_wait0();      // every reduction of this thread has been performed before the CTA leaves
   }
 
   tc_fence_before();
@@ -700,6 +717,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int quarter = warp & 3;             // tensor-memory lanes 32*quarter .. 32*quarter+31
     bool ok = true;
     int it = 0;
+    // EPI_RESIDUAL, when the stages leave room below the barriers: this thread's 144-byte staging slot for the
+    // residual add as an L2 bulk reduction (see epilogue_unit)
+    const uint32_t red_slot = EPI == EPI_RESIDUAL && nst * STAGE_BYTES + 128 * 144 <= TC_DATA_BYTES
+        ? smem_u32(smem + nst * STAGE_BYTES) + (uint32_t)((warp - 2) * 32 + lane) * 144u : 0u;
     for (int w = blockIdx.x; w < total && ok; w += gridDim.x, ++it) {
       const int t = w / S, sp = w - t * S;
       const int acc = it & 1;
@@ -723,7 +744,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             qkv.lse_part[(size_t)(n0 / 256) * qkv.lse_rows + row] = make_float4(rs.m, rs.s, __int_as_float(rs.am), 0.f);
         } else {
 #pragma unroll 1
-          for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, bn, row, row < M, u, n0, n_out, Cv, qkv);
+          for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, bn, row, row < M, u, n0, n_out, Cv, qkv, red_slot);
         }
         tc_fence_before();
         __syncwarp();
@@ -793,7 +814,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int i = lo + e_tid; i < hi; i += 128) {   // rows fastest: a warp reads contiguous partials
               const int u = i / live_rows, r = i - u * live_rows;
               WsSrc src{ws + (size_t)(t * S) * TC_BM * bn, r, (size_t)TC_BM * bn, S};
-              epilogue_unit<EPI>(src, bn, m0 + r, true, u, n0, n_out, Cv, qkv);
+              epilogue_unit<EPI>(src, bn, m0 + r, true, u, n0, n_out, Cv, qkv, red_slot);
             }
           };
           const int nk = role == 2 ? shares : 1;       // the last arriver tries its own share first, then all others
@@ -825,6 +846,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (it == 0 && warp == 2 && lane == 0) GP(6)
       }
     }
+    if (EPI == EPI_RESIDUAL) bulk_wait0();      // every reduction of this thread has been performed before the CTA leaves
   }
 
   tc_fence_before();
