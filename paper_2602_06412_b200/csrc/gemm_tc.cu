@@ -530,7 +530,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int nt = (n_out + obn - 1) / obn, half = (int)(gridDim.x >> 1);
     const int pairs = ((Mp + 255) / 256) * nt, singles = ((Mp + 127) / 128) * nt;
     const int rounds_p = (pairs + half - 1) / half, rounds_s = (singles + (int)gridDim.x - 1) / (int)gridDim.x;
-    if (pairs >= half && 20 * rounds_p <= 23 * rounds_s) {
+    // Also when the pair tiles only partly fill ONE round, if the single tiles are too many to split their K range two
+    // ways within a round (more than half the grid): a K block of a pair tile moves 32 instead of 48 KB per SM and takes
+    // ~0.8 of a single tile's (measured at 4096 x 4096, 4096 x 12288 and 12288 x 4096 for M = 160 ... 1024: 36-38 vs
+    // 42-43 us, 76-78 vs 82-94 us, 45 vs 51 us; with fewer single tiles the K split wins).
+    const bool take = (pairs >= half && 20 * rounds_p <= 23 * rounds_s) ||
+                      (Mp > TC_BM && pairs < half && 2 * singles > (int)gridDim.x && K >= 24 * TC_BK && force_bn <= 0);
+    if (take) {
       if (prefetch_w) {
         griddep_wait();
         griddep_launch();
