@@ -299,6 +299,17 @@ size_t surelock_gemm_workspace_bytes(void);
 int surelock_gemm(const void *A, const void *W, void *C, const int32_t *n_active, int max_rows, int n_out, int K,
                   int dtype, int impl, void *workspace, int32_t *dev_status, void *stream);
 
+/* The same contraction with the fused epilogues of the transformer block (Sec. 2.3: the output / down projections
+ * feed the residual stream, the gate and up projections feed SwiGLU), for stage-wise parity checks and timing:
+ *   epilogue 1: C is the fp32 residual stream, dev float [M][n_out]: C[r][n] += sum_k A[r][k] W[n][k]
+ *   epilogue 2: C[r][n] = silu(sum_k A[r][k] W[n][k]) * (sum_k A[r][k] W2[n][k]), C of `dtype`; W2: dev [n_out][K]
+ *   epilogue 0: surelock_gemm (W2 ignored)
+ * Other arguments as for surelock_gemm; rows >= *n_active of C are not touched.  SL_EINVAL for an unknown epilogue or a
+ * missing W2. */
+int surelock_gemm_fused(const void *A, const void *W, const void *W2, void *C, const int32_t *n_active, int max_rows,
+                        int n_out, int K, int dtype, int epilogue, int impl, void *workspace, int32_t *dev_status,
+                        void *stream);
+
 /* M x N bidirectional attention of the packed queries against the whole cache (Algorithm 1 line 12; Sec. 2.1:
  * "variable-length attention against the full key/value tables"): for packed row r at flat position
  * active_idx[r] = b*N+i and every head h, o[r][h] = softmax_j(q[r][h] . K[b*N+j][h] / sqrt(d_h)) V[b*N+j][h],

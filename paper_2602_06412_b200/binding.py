@@ -79,6 +79,7 @@ def lib() -> C.CDLL:
         "surelock_softmax_kl_sure": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, vp, vp, f32, vp, vp, vp, vp, vp]),
         "surelock_gemm": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]),
         "surelock_gemm_workspace_bytes": (sz, []),
+        "surelock_gemm_fused": (i32, [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp]),
         "surelock_attention": (i32, [vp, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, i32, i32, vp, vp]),
     }
     for name, (res, args) in sig.items():
@@ -334,6 +335,13 @@ def surelock_gemm(A, W, Cout, n_active, impl: int = 0, dev_status=None, workspac
     """workspace: zero-filled uint8 CUDA tensor of surelock_gemm_workspace_bytes() bytes (enables split-K), or None."""
     _check(lib().surelock_gemm(_p(A), _p(W), _p(Cout), _p(n_active), A.shape[0], W.shape[0], A.shape[1], _dt(A), impl,
                                _p(workspace), _p(dev_status), _stream()), "surelock_gemm")
+
+
+def surelock_gemm_fused(A, W, W2, Cout, n_active, epilogue: int, impl: int = 0, dev_status=None, workspace=None):
+    """epilogue 1: Cout (fp32) += A W^T; 2: Cout = silu(A W^T) * (A W2^T); 0: plain store."""
+    _check(lib().surelock_gemm_fused(_p(A), _p(W), _p(W2), _p(Cout), _p(n_active), A.shape[0], W.shape[0], A.shape[1],
+                                     _dt(A), epilogue, impl, _p(workspace), _p(dev_status), _stream()),
+           "surelock_gemm_fused")
 
 
 def surelock_attention(q, k_cache, v_cache, active_idx, row_offsets, n_active, B: int, N: int, o, impl: int = 0,

@@ -618,8 +618,18 @@ int surelock_conf_gate_lock(const float* conf, const float* kl, const int32_t* a
 
 int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active, int max_rows, int n_out, int K,
                   int dtype, int impl, void* workspace, int32_t* dev_status, void* stream) {
+  return surelock_gemm_fused(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, impl, workspace, dev_status,
+                             stream);
+}
+
+int surelock_gemm_fused(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
+                        int n_out, int K, int dtype, int epilogue, int impl, void* workspace, int32_t* dev_status,
+                        void* stream) {
   if (!A || !W || !C || !n_active || max_rows < 0 || n_out <= 0 || K <= 0) return SL_EINVAL;
   if (dtype != SL_BF16 && dtype != SL_FP32) return SL_EINVAL;
+  if (epilogue != EPI_STORE && epilogue != EPI_RESIDUAL && epilogue != EPI_SWIGLU) return SL_EINVAL;
+  if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
+  if (epilogue != EPI_SWIGLU) W2 = nullptr;
   if (dtype == SL_BF16 && impl == 0) {
     SplitWs sw;
     if (workspace) {
@@ -627,10 +637,10 @@ int surelock_gemm(const void* A, const void* W, void* C, const int32_t* n_active
       sw.ws = reinterpret_cast<float*>(workspace);
       sw.counters = reinterpret_cast<int*>(reinterpret_cast<char*>(workspace) + gemm_ws_tiles() * SPLIT_TILE_BYTES);
     }
-    const int rc = launch_gemm_tc(A, W, nullptr, C, n_active, max_rows, n_out, K, EPI_STORE, dev_status, sw, (cudaStream_t)stream);
+    const int rc = launch_gemm_tc(A, W, W2, C, n_active, max_rows, n_out, K, epilogue, dev_status, sw, (cudaStream_t)stream);
     if (rc != SL_EUNSUPPORTED) return rc;
   }
-  return launch_gemm_simt(A, W, nullptr, C, n_active, max_rows, n_out, K, dtype, EPI_STORE, (cudaStream_t)stream);
+  return launch_gemm_simt(A, W, W2, C, n_active, max_rows, n_out, K, dtype, epilogue, (cudaStream_t)stream);
 }
 
 int surelock_update_mask(const float* conf, const int32_t* argmax, const int32_t* active_idx, const int32_t* row_offsets,

@@ -237,6 +237,63 @@ def test_gemm_tensor_cores(M, n_out, K, split):
         assert torch.equal(out.view(torch.int16), out2.view(torch.int16))
 
 
+@pytest.mark.parametrize("impl", [0, 1])
+@pytest.mark.parametrize("M,n_out,K", [(20, 4096, 4096), (100, 4096, 12288), (128, 4096, 4096), (129, 136, 200), (305, 4096, 4096),
+                                       (638, 4096, 4096), (700, 1024, 12288), (1312, 4096, 4096), (0, 256, 256)])
+def test_gemm_residual_epilogue(M, n_out, K, impl):
+    """x += A W^T into the fp32 residual stream (the output and down projections): every path of the epilogue: plain
+    read-modify-write (few activation rows per stage, or a ragged last unit), bulk reductions by the L2 from the
+    single-CTA tiles, from the K-split finisher and from the CTA-pair path (one partly filled round, several rounds);
+    rows beyond M stay untouched and two runs give the same bits."""
+    if impl == 1 and M * n_out * K > 3e10:
+        pytest.skip("CUDA-core kernel: small shapes only")
+    g = torch.Generator().manual_seed(M * 11 + K)
+    cap = M + 37
+    A = torch.randn((cap, K), generator=g).to(torch.bfloat16)
+    W = (torch.randn((n_out, K), generator=g) * 0.05).to(torch.bfloat16)
+    x0 = torch.randn((cap, n_out), generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    wsp = torch.zeros(SL.surelock_gemm_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    Ad, Wd, n = A.to(DEV), W.to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV)
+    outs = []
+    for _ in range(2):
+        x = x0.to(DEV)
+        SL.surelock_gemm_fused(Ad, Wd, None, x, n, 1, impl=impl, dev_status=status, workspace=wsp)
+        torch.cuda.synchronize()
+        outs.append(x)
+    assert status.item() == 0
+    x = outs[0]
+    if M:
+        ref = f64(x0[:M]) + f64(A[:M]) @ f64(W).T
+        assert rel_err_rows(f64(x[:M]), ref) < (2e-2 if impl == 0 else 1e-4) and torch.isfinite(x[:M]).all()
+        # bf16 operands are exact and the sums are fp32: the stream must come out far inside the parity bar
+        assert np.abs(f64(x[:M]) - ref).max() < 1e-3 * (1 + np.abs(ref).max())
+    assert torch.equal(x[M:].cpu(), x0[M:])                          # rows beyond M untouched, bit for bit
+    assert torch.equal(outs[0].view(torch.int32), outs[1].view(torch.int32))
+
+
+@pytest.mark.parametrize("M,n_out,K", [(20, 1024, 4096), (129, 136, 200), (305, 12288, 1024), (1312, 2048, 4096)])
+def test_gemm_swiglu_epilogue(M, n_out, K):
+    """silu(A Wg^T) * (A Wu^T) in one launch (gate and up projections), against the oracle's silu."""
+    g = torch.Generator().manual_seed(M * 13 + K)
+    cap = M + 5
+    A = torch.randn((cap, K), generator=g).to(torch.bfloat16)
+    Wg = (torch.randn((n_out, K), generator=g) * 0.03).to(torch.bfloat16)
+    Wu = (torch.randn((n_out, K), generator=g) * 0.03).to(torch.bfloat16)
+    out = torch.full((cap, n_out), 3.0, dtype=torch.bfloat16, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    wsp = torch.zeros(SL.surelock_gemm_workspace_bytes(), dtype=torch.uint8, device=DEV)
+    SL.surelock_gemm_fused(A.to(DEV), Wg.to(DEV), Wu.to(DEV), out, torch.tensor([M], dtype=torch.int32, device=DEV), 2,
+                           dev_status=status, workspace=wsp)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    ref = O.silu(f64(A[:M]) @ f64(Wg).T) * (f64(A[:M]) @ f64(Wu).T)
+    assert rel_err_rows(f64(out[:M]), ref) < 2e-2
+    assert (out[M:] == 3.0).all()
+    with pytest.raises(SL.SurelockError):
+        SL.surelock_gemm_fused(A.to(DEV), Wg.to(DEV), None, out, torch.tensor([M], dtype=torch.int32, device=DEV), 2)
+
+
 @pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
 @pytest.mark.parametrize("B,N,H,dh,n_act", [(2, 77, 3, 64, [20, 77]), (1, 200, 2, 128, [9]), (3, 33, 1, 64, [0, 33, 1])])
 def test_attention_cuda_cores(dtype, tol, B, N, H, dh, n_act):
