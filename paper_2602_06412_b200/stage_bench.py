@@ -60,6 +60,7 @@ def main(argv=None):
     ap.add_argument("--n_out", type=int, default=12288)
     ap.add_argument("--K", type=int, default=4096)
     ap.add_argument("--impl", type=int, default=0)
+    ap.add_argument("--epilogue", type=int, default=0, help="gemm: 0 store, 1 += into the fp32 residual stream, 2 SwiGLU")
     ap.add_argument("--B", type=int, default=8)
     ap.add_argument("--N", type=int, default=1536)
     ap.add_argument("--H", type=int, default=32)
@@ -87,10 +88,19 @@ def main(argv=None):
         Cout = torch.empty((a.M, a.n_out), dtype=torch.bfloat16, device=dev)
         n = torch.tensor([a.M], dtype=torch.int32, device=dev)
         wsp = torch.zeros(SL.surelock_gemm_workspace_bytes(), dtype=torch.uint8, device=dev)
-        fn = lambda: SL.surelock_gemm(A, W, Cout, n, impl=a.impl, dev_status=status, workspace=wsp)
         flops = 2.0 * a.M * a.n_out * a.K
         byts = 2.0 * (a.M * a.K + a.n_out * a.K + a.M * a.n_out)
-        res.update(shape=[a.M, a.n_out, a.K], flops=flops, bytes=byts)
+        if a.epilogue == 1:                                   # fp32 stream read and written
+            Cout = torch.zeros((a.M, a.n_out), dtype=torch.float32, device=dev)
+            fn = lambda: SL.surelock_gemm_fused(A, W, None, Cout, n, 1, impl=a.impl, dev_status=status, workspace=wsp)
+            byts = 2.0 * (a.M * a.K + a.n_out * a.K) + 8.0 * a.M * a.n_out
+        elif a.epilogue == 2:                                 # gate and up matrices
+            W2 = (rnd(a.n_out, a.K) * 0.02).to(torch.bfloat16)
+            fn = lambda: SL.surelock_gemm_fused(A, W, W2, Cout, n, 2, impl=a.impl, dev_status=status, workspace=wsp)
+            flops, byts = 2 * flops, byts + 2.0 * a.n_out * a.K
+        else:
+            fn = lambda: SL.surelock_gemm(A, W, Cout, n, impl=a.impl, dev_status=status, workspace=wsp)
+        res.update(shape=[a.M, a.n_out, a.K], epilogue=a.epilogue, flops=flops, bytes=byts)
     elif a.stage == "attention":
         B, N, H, dh = a.B, a.N, a.H, a.dh
         na = [max(1, int(N * a.ratio))] * B
