@@ -34,6 +34,7 @@ from paper_2602_06412_b200 import dist_util, inputs  # noqa: E402
 
 WORKLOADS = {
     # name: (model shape, batch, N, prompt length, lock pattern)
+    "c2": ("llada8b-layer", 1, 1024, 0, "random"),      # single-layer microbench: see run_single_layer()
     "c3": ("llada8b", 1, 512, 256, "random"),
     "c4": ("llada8b", 8, 1536, 512, "random"),
     "c5": ("llada8b", 4, 4096, 3584, "contiguous_plus_random"),
@@ -163,6 +164,34 @@ def workload_config(args, cfgname, cfg, B, N, pattern, M=None):
 
 
 def run_reference(args, cfgname, B, N, pattern):
+    if args.workload == "c2":                                         # the single-layer microbench: the oracle's layer alone
+        from oracle import surelock_oracle as O
+        cfg = inputs.model_shape("llada8b", n_layers=1, vocab=0)
+        oc = O.ModelCfg(**cfg)
+        lw = {k: v.float().numpy() for k, v in inputs.make_layer_weights(cfg, 0, 1).items()}
+        g = np.random.default_rng(0)
+        rows, vals, secs = 128, [], 0.0
+        Kc, Vc = (g.standard_normal((N, cfg["n_heads"], cfg["head_dim"])) for _ in range(2))
+        for i in range(max(0, args.warmup) + max(1, args.steps)):
+            x, pos = g.standard_normal((rows, cfg["d_model"])), np.sort(g.choice(N, size=rows, replace=False))
+            t0 = time.perf_counter()
+            O.layer_rows(oc, lw, x, pos, Kc, Vc)
+            if i >= max(0, args.warmup):
+                vals.append(rows / (time.perf_counter() - t0)); secs += time.perf_counter() - t0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        v = float(np.median(vals))
+        desc = f"the layer on {rows} active rows against the N={N} cache per step"
+        return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
+                "steps": len(vals), "warmup": max(0, args.warmup), "ms_per_step": 1e3 * secs / len(vals),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "config": {"workload": "c2: ONE LLaDA-8B-shaped layer, batch 1, N=1024 (CPU oracle, bounded sample per step)",
+                           "batch": 1, "seq_len": N},
+                "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
+                "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     cfg = inputs.model_shape(cfgname)
     vals, secs = [], 0.0
     for _ in range(max(0, args.warmup)):                              # untimed, like the GPU arm's warm-up steps
@@ -177,6 +206,132 @@ def run_reference(args, cfgname, B, N, pattern):
             "config": dict(workload_config(args, cfgname, cfg, B, N, pattern), note="CPU oracle, bounded sample per step"),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+
+
+# ----------------------------------------------------------------------------------------------------- single layer
+def run_single_layer(args, rank, world, local):
+    """Single LLaDA-8B-shaped layer (RMSNorm, QKV + RoPE + cache scatter, M x N attention, O, SwiGLU FFN; no embedding,
+    LM head or KL), batch 1, N = 1024, cache pre-filled by one full pass, seeded random active subsets of
+    M in {1024, 512, 256, 128, 32} rows, through surelock_layer_step.  One "step" is one call."""
+    from paper_2602_06412_b200 import binding as SL
+    SL.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    args.warmup = max(args.warmup, 3)
+    cfg = inputs.model_shape("llada8b", n_layers=1, vocab=0)
+    N, d, F = 1024, cfg["d_model"], cfg["d_ff"]
+    seed = dist_util.replica_seed(1234, rank)
+    w = dict(layers=[{k: v.to(dev) for k, v in inputs.make_layer_weights(cfg, 0, seed, dtype=torch.bfloat16).items()}])
+    ctx = SL.surelock_init(cfg, w, N, 1)
+    H0, H1 = inputs.hidden_states(N, d, 1).to(dev), inputs.hidden_states(N, d, 2).to(dev)
+    out = torch.zeros((N, d), dtype=torch.float32, device=dev)
+    SL.surelock_layer_step(ctx, 0, H0, torch.zeros((1, N), dtype=torch.uint8, device=dev), out)   # pre-fill of the cache
+    torch.cuda.synchronize()
+    pk, pk_kind = peaks()
+    hd = cfg["n_heads"] * cfg["head_dim"]
+    wbytes = 2 * (4 * hd * d + 3 * d * F)
+    flops_row = 2 * d * 3 * hd + 2 * hd * d + 6 * d * F
+
+    def timed(M, steps, warmup):
+        lock = inputs.random_lock(1, N, [M], 100 + M).to(dev) if M < N else torch.zeros((1, N), dtype=torch.uint8, device=dev)
+        for _ in range(warmup):
+            SL.surelock_layer_step(ctx, 0, H1, lock, out)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            o = SL.surelock_layer_step(ctx, 0, H1, lock, out)
+        e1.record()
+        torch.cuda.synchronize()
+        assert o.M() == M
+        return dist_util.max_over_ranks(e0.elapsed_time(e1) / steps, dev), lock
+
+    steps = max(args.steps, 20)
+    M0 = 512
+    sampler = ClockSampler(local)
+    with sampler:
+        ms, lock0 = timed(M0, 50 * steps, args.warmup)
+    clocks = sampler.summary()
+    launches = 50 * steps * SL.surelock_last_launch_count(ctx)
+    SL.surelock_set_option(ctx, "time_kernels", 1)
+    SL.surelock_layer_step(ctx, 0, H1, lock0, out)
+    kt = SL.surelock_kernel_times(ctx)
+    SL.surelock_set_option(ctx, "time_kernels", 0)
+    total_k = sum(v[0] for v in kt.values())
+    kernels = {k: dict(ms=round(v[0], 4), launches=v[1], share=round(v[0] / total_k, 4)) for k, v in kt.items()}
+    gemm_ms = sum(v[0] for k, v in kt.items() if k.startswith("gemm"))
+    gemm_n = sum(v[1] for k, v in kt.items() if k.startswith("gemm"))
+    ach = M0 * flops_row / (gemm_ms * 1e-3) / 1e12
+    roof = dict(kernel="gemm_tc (the four GEMM launches of the layer)", bound="tensor", achieved=ach,
+                peak=pk["bf16_tflops"], unit="TFLOP/s", frac=ach / pk["bf16_tflops"],
+                traffic=0.89 * (wbytes + M0 * (2 * d + 6 * hd + 2 * hd + 8 * d + 2 * d + 4 * F + 8 * d)) / max(gemm_n, 1),
+                traffic_note="bytes per average launch, scaled from a small-case ncu capture",
+                peak_kind=f"{pk_kind}, burst (kernels timed one by one)", launches_per_step=gemm_n,
+                avg_launch_ms=gemm_ms / max(gemm_n, 1))
+    # end to end: the hidden states come from pinned host memory and the packed output rows go back, every call
+    hin = inputs.hidden_states(N, d, 2).pin_memory()
+    hout = torch.zeros((N, d), dtype=torch.float32).pin_memory()
+    hdev = torch.empty_like(H1)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        hdev.copy_(hin, non_blocking=True)
+        SL.surelock_layer_step(ctx, 0, hdev, lock0, out)
+        hout[:M0].copy_(out[:M0], non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = dist_util.max_over_ranks((time.perf_counter() - t0) * 1e3 / steps, dev)
+    sweep = []
+    for M in (1024, 512, 256, 128, 32):
+        t, _ = timed(M, 20 * steps, 3)
+        ideal = max(M * flops_row / (pk["bf16_tflops_sustained"] * 1e12) + 4.0 * M * N * hd / (pk["bf16_tflops_sustained"] * 1e12),
+                    wbytes / (pk["hbm_gbs"] * 1e9)) * 1e3
+        sweep.append(dict(M=M, ms_per_step=round(t, 5), tokens_per_s=round(dist_util.sum_over_ranks(M, dev) / (t * 1e-3), 1),
+                          ideal_ms=round(ideal, 5), frac_of_ideal=round(ideal / t, 4)))
+    line = {
+        "metric": "active_tokens_per_s", "value": dist_util.sum_over_ranks(M0, dev) / (ms * 1e-3), "unit": "tokens/s",
+        "n_gpus": world, "steps": 50 * steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "c2: ONE LLaDA-8B-shaped layer (d=4096, 32 heads x 128, FFN 12288), batch 1, N=1024, "
+                               f"M={M0} active rows (seeded random subset), through surelock_layer_step", "batch": 1,
+                   "seq_len": N, "active_rows": M0,
+                   "l2": "inputs larger than L2 (every call streams the layer's weights, %.0f MB)" % (wbytes / 1e6),
+                   "multi_gpu": "replicas only (one independent layer per rank, no collective)"},
+        "e2e": dict(value=dist_util.sum_over_ranks(M0, dev) / (e2e_ms * 1e-3), unit="tokens/s", ms_per_step=e2e_ms,
+                    h2d_bytes_per_step=N * d * 2, d2h_bytes_per_step=M0 * d * 4),
+        "gpu_launches": launches, "clocks": clocks, "roofline": roof, "kernels": kernels, "sweep": sweep,
+        "device_status": SL.surelock_status_poll(ctx),
+    }
+    if rank == 0 and not args.no_cpu_baseline:
+        from oracle import surelock_oracle as O
+        oc = O.ModelCfg(**cfg)
+        lw = {k: v.float().cpu().numpy() for k, v in w["layers"][0].items()}
+        g = np.random.default_rng(0)
+        rows = 256
+        pos = np.sort(g.choice(N, size=rows, replace=False))
+        Kc, Vc = g.standard_normal((N, cfg["n_heads"], cfg["head_dim"])), g.standard_normal((N, cfg["n_heads"], cfg["head_dim"]))
+        x = g.standard_normal((rows, d))
+        t0 = time.perf_counter()
+        for _ in range(3):
+            O.layer_rows(oc, lw, x, pos, Kc, Vc)
+        secs = time.perf_counter() - t0
+        try:
+            from threadpoolctl import threadpool_info
+            threads = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            threads = os.cpu_count() or 1
+        line["cpu_baseline"] = {"value": 3 * rows / secs, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                                "sample": f"the layer on {rows} active rows against the N={N} cache, 3 times",
+                                "seconds": round(secs, 2)}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+    return 0
 
 
 # ----------------------------------------------------------------------------------------------------- GPU leg
@@ -200,6 +355,9 @@ def main():
         if rank == 0:
             print(json.dumps(run_reference(args, cfgname, B, N, pattern)), flush=True)
         return 0
+
+    if args.workload == "c2":
+        return run_single_layer(args, rank, world, local)
 
     from paper_2602_06412_b200 import binding as SL
     SL.lib()                                       # fail loudly if the CUDA library is missing

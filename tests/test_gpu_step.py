@@ -147,7 +147,7 @@ def test_argument_errors_are_reported_not_fatal():
     assert SL.surelock_status_poll(ctx) == 0
 
 
-@pytest.mark.parametrize("M_list", [[1024, 256, 32]])
+@pytest.mark.parametrize("M_list", [[1024, 512, 256, 128, 32]])
 def test_single_layer_llada_shape(M_list):
     """Single LLaDA-8B-shaped layer, N=1024: cache pre-filled by one full pass, then seeded random active subsets."""
     cfg = inputs.model_shape("llada8b", n_layers=1, vocab=0)
