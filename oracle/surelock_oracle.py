@@ -25,6 +25,14 @@ design notes of the repository):
     without a previous posterior has D = +inf (Algorithm 1, line 19);
   * the lock test reads the mask state the forward pass saw (the state passed
     to this step), so a row can lock only after a step that was fed its token;
+    Algorithm 1 read literally updates the masked set (line 16) before the test
+    (line 20): step(..., unmask=...) plays that order;
+  * p_{t-1} of a row that was NOT computed in step t-1 (it cannot happen under
+    Algorithm 1's monotone locks; un-locking and selection methods make it
+    happen): OracleState(prev_policy="previous_step") gives such a row D = +inf
+    (Algorithm 1 line 19 compares with the posterior of step t-1, which the row
+    does not have); prev_policy="keep_last" compares with the last posterior the
+    row ever had (Sec. 2.1: a locked row keeps p_t <- p_{t*});
   * the optional confidence-percentile gate (Algorithm 1, line 21) is off unless asked for; when on, the
     percentile is taken per sequence over the locking candidates Z_t (Algorithm 1) rather than over all active
     rows (Sec. 2.2 prose), with linear interpolation between order statistics, and a row passes when
@@ -316,9 +324,16 @@ class OracleState:
 
     K, V: [L][B][N][H][d_h] float64.  prev_logp: [B][N][V] float64 with
     prev_valid [B][N]; an invalid row stands for "p_{t-1} = None".
+
+    prev_policy decides what p_{t-1} is for a row that was not computed in the step just before (see the module
+    header): "previous_step" -> it has none (D = +inf), "keep_last" -> the last posterior it ever had.  Under
+    Algorithm 1 itself (locks only grow, every unlocked row is computed every step) the two never differ.
     """
 
-    def __init__(self, cfg: ModelCfg, B: int, N: int):
+    def __init__(self, cfg: ModelCfg, B: int, N: int, prev_policy: str = "previous_step"):
+        if prev_policy not in ("previous_step", "keep_last"):
+            raise ValueError(prev_policy)
+        self.prev_policy = prev_policy
         self.cfg, self.B, self.N = cfg, B, N
         shp = (cfg.n_layers, B, N, cfg.n_heads, cfg.head_dim)
         self.K = np.zeros(shp, F64)
@@ -333,8 +348,25 @@ class OracleState:
 
 
 def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.ndarray,
-         lock: np.ndarray, kl_eps: float, logits_round=None, conf_gate_m: Optional[float] = None):
+         lock: np.ndarray, kl_eps: float, logits_round=None, conf_gate_m: Optional[float] = None,
+         unmask=None, skip: Optional[np.ndarray] = None, kl_eps_rows: Optional[np.ndarray] = None,
+         may_lock: Optional[np.ndarray] = None):
     """One SureLock step (Algorithm 1, lines 6-15 and 18-24; line 16 belongs to the caller).
+
+    unmask: None (default) = the lock test of lines 20-23 reads the mask state that was passed in, i.e. the state
+    the forward pass saw.  A callable plays Algorithm 1 in its LITERAL order: it is line 16, called after the
+    posteriors of line 15 as unmask(tokens, mask_state, conf, argmax, active_idx) -> (tokens', mask_state'), and
+    the candidates of line 20 are then taken from mask_state' (a position revealed in this step can lock in this
+    step, with K/V that were computed from the mask token).  The result carries tokens' / mask_state'.
+
+    skip: optional [B][N] of 0/1, the selection surrogate of Experiment 5: an unlocked position with skip = 1 is not
+    computed in this step (it is not in the active set; its cached K/V and its lock bit stay as they are, it gets no
+    posterior), so that only a fraction of the not-yet-locked positions is recomputed; new locks come from computed
+    rows only.
+
+    kl_eps_rows / may_lock: optional [B][N] arrays used by the un-locking extension (App. "Optional Unlocking"):
+    a per-position threshold that replaces kl_eps (the stricter rho * eps of a position that was un-locked before)
+    and a per-position permission (0 during the cool-down after an un-lock).
 
     weights: {"tok_emb": [V][d], "lm_head": [V][d], "final_norm_g": [d],
               "layers": [ {attn_norm_g, wq, wk, wv, wo, ffn_norm_g, w_gate, w_up, w_down} ]}.
@@ -349,7 +381,10 @@ def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.n
     """
     cfg, B, N = state.cfg, state.B, state.N
     tokens = np.asarray(tokens)
-    idx, offs = active_set(lock)
+    not_computed = np.asarray(lock) != 0
+    if skip is not None:
+        not_computed = not_computed | (np.asarray(skip) != 0)
+    idx, offs = active_set(not_computed.astype(np.uint8))
     M = len(idx)
     emb = np.asarray(weights["tok_emb"])
     hidden = np.zeros((M, cfg.d_model), F64)
@@ -378,16 +413,150 @@ def step(state: OracleState, weights: Dict, tokens: np.ndarray, mask_state: np.n
     has_prev = state.prev_valid[bb, ii]
     if has_prev.any():
         D[has_prev] = kl_rows(logp[has_prev], state.prev_logp[bb[has_prev], ii[has_prev]])
-    lockable = sure_test(D, np.asarray(mask_state)[bb, ii], kl_eps)  # lines 20, 23
+    new_tokens, new_mask = tokens, np.asarray(mask_state)
+    if unmask is not None:                                        # line 16 in its literal place, before line 20
+        new_tokens, new_mask = unmask(tokens, np.asarray(mask_state), conf, am, idx)
+        new_tokens, new_mask = np.asarray(new_tokens), np.asarray(new_mask)
+    eps_rows = kl_eps if kl_eps_rows is None else np.asarray(kl_eps_rows, F64)[bb, ii]
+    lockable = sure_test(D, new_mask[bb, ii], eps_rows)           # lines 20, 23
+    if may_lock is not None:
+        lockable = lockable & (np.asarray(may_lock)[bb, ii] != 0)
     theta = None
     if conf_gate_m is not None:                                   # line 21: u <= theta_m over the candidates Z_t
-        gate, theta = confidence_gate(conf, np.asarray(mask_state)[bb, ii] == 0, bb, B, conf_gate_m)
+        gate, theta = confidence_gate(conf, new_mask[bb, ii] == 0, bb, B, conf_gate_m)
         lockable = lockable & gate
     new_lock = np.array(lock, dtype=np.uint8, copy=True)
     new_lock[bb[lockable], ii[lockable]] = 1                      # line 24
-    state.prev_logp[bb, ii] = logp                                # locked rows keep p_{t*}
-    state.prev_valid[:] = False                                   # "previous" means computed in the step just taken
+    state.prev_logp[bb, ii] = logp                                # rows that were not computed keep their last posterior
+    if state.prev_policy == "previous_step":
+        state.prev_valid[:] = False                               # "previous" means computed in the step just taken
     state.prev_valid[bb, ii] = True
     state.flops += flops
     return dict(active_idx=idx, row_offsets=offs, hidden=hidden, logits=logits, kl=D,
-                conf=conf, argmax=am, new_lock=new_lock, flops=flops, theta=theta)
+                conf=conf, argmax=am, new_lock=new_lock, flops=flops, theta=theta, logp=logp,
+                tokens=new_tokens, mask_state=new_mask)
+
+
+# --------------------------------------------------------------------------
+# Optional un-locking (App. "Optional Unlocking")
+# --------------------------------------------------------------------------
+# The appendix leaves open what the "budgeted proxy" is, how theta_t treats a sequence without active rows, and says
+# "if any holds" above an equation whose three conditions are joined by AND.  Readings taken here:
+#   * the proxy recomputes the LOCKED rows as queries through the whole stack against the caches as they stand
+#     (variable-length attention over all N cached keys / values) WITHOUT writing their K/V back: probe_rows();
+#   * the rule is the printed equation: all three conditions must hold;
+#   * theta_t is, per sequence, the m-th percentile (linear interpolation, as for the confidence gate) of
+#     u = 1 - max_v p over the rows that were ACTIVE in step t; a sequence with no active row has no reference
+#     uncertainty and un-locks nothing (theta = +inf);
+#   * a position un-locked after step t is active from step t+1 on; "invalidate cached K/V" needs no action because
+#     every active row's K/V is rewritten in every step; it may lock again from step t + D_cool + 1 on, and from then
+#     on under the threshold rho * eps.
+@dataclasses.dataclass
+class UnlockParams:
+    period: int            # P: the probe runs after every P-th step
+    eps_unlock: float      # drift threshold on KL(p_hat_t || p_{t*})
+    d_interval: int        # a position stays locked for more than this many steps before it may be un-locked
+    d_cool: int            # steps after an un-lock during which the position cannot lock again
+    rho: float             # re-lock threshold factor, rho <= 1
+    m: float               # percentile (0..100) of the active rows' uncertainty that gives theta_t
+
+
+class UnlockState:
+    """What un-locking needs beyond Algorithm 1's state: per position the step t* at which it locked, the posterior
+    p_{t*} it had then (as log-probabilities), the last step of its cool-down, and whether it was ever un-locked."""
+
+    def __init__(self, B: int, N: int, V: int):
+        self.t_star = np.full((B, N), -1, np.int64)
+        self.frozen_logp = np.zeros((B, N, V), F64)
+        self.cool_until = np.full((B, N), -1, np.int64)
+        self.relock = np.zeros((B, N), bool)
+
+
+def record_locks(ustate: UnlockState, t: int, lock_before: np.ndarray, step_out: Dict, N: int) -> None:
+    """After step t: every position that this step locked gets t* = t and keeps its posterior of step t as p_{t*}."""
+    idx = np.asarray(step_out["active_idx"])
+    bb, ii = idx // N, idx % N
+    newly = (np.asarray(step_out["new_lock"])[bb, ii] != 0) & (np.asarray(lock_before)[bb, ii] == 0)
+    ustate.t_star[bb[newly], ii[newly]] = t
+    ustate.frozen_logp[bb[newly], ii[newly]] = np.asarray(step_out["logp"])[newly]
+
+
+def relock_thresholds(ustate: UnlockState, kl_eps: float, rho: float, t: int):
+    """Per-position lock threshold and permission for step t: rho * eps for a position that was un-locked before,
+    eps otherwise; no locking while t <= cool_until (the D_cool steps after the un-lock)."""
+    eps_rows = np.where(ustate.relock, rho * kl_eps, kl_eps).astype(F64)
+    may_lock = (t > ustate.cool_until).astype(np.uint8)
+    return eps_rows, may_lock
+
+
+def probe_rows(state: OracleState, weights: Dict, tokens: np.ndarray, lock: np.ndarray):
+    """The proxy: posteriors p_hat_t of the LOCKED rows, recomputed against the caches as they stand.
+
+    For every sequence the locked positions (ascending) go through every block like active rows do in step()
+    (lines 7, 10, 12, 15), except that line 11 is not executed: their fresh k, v are discarded and attention reads
+    all N cached rows, their own frozen entries included.  Nothing in `state` is modified.
+    Returns (locked_idx flat ascending, logits [n][V], logp [n][V], conf [n]).
+    """
+    cfg, B, N = state.cfg, state.B, state.N
+    tokens = np.asarray(tokens)
+    idx, offs = active_set(1 - (np.asarray(lock) != 0).astype(np.uint8))      # positions with lock = 1
+    n = len(idx)
+    hidden = np.zeros((n, cfg.d_model), F64)
+    emb = np.asarray(weights["tok_emb"])
+    for b in range(B):
+        r0, r1 = int(offs[b]), int(offs[b + 1])
+        if r1 == r0:
+            continue
+        pos = (idx[r0:r1] - b * N).astype(np.int64)
+        x = np.asarray(emb[tokens[b, pos]], F64)
+        for l, lw in enumerate(weights["layers"]):
+            q, _, _ = qkv_rows(cfg, lw, x, pos)
+            o = attention_rows(q, state.K[l, b], state.V[l, b])
+            x = ffn_rows(cfg, lw, x + o @ np.asarray(lw["wo"], F64).T)
+        hidden[r0:r1] = x
+    logits = rmsnorm(hidden, weights["final_norm_g"], cfg.rms_eps) @ np.asarray(weights["lm_head"], F64).T
+    logp = log_softmax(logits)
+    conf, _ = posterior_stats(logits)
+    return idx, logits, logp, conf
+
+
+def unlock_test(u_probe, D_probe, theta, t: int, t_star, p: UnlockParams) -> np.ndarray:
+    """The un-lock rule: u~ > theta_t  AND  D~ > eps_unlock  AND  t - t* > D_interval (element-wise)."""
+    return (np.asarray(u_probe, F64) > np.asarray(theta, F64)) & (np.asarray(D_probe, F64) > p.eps_unlock) & \
+           ((t - np.asarray(t_star)) > p.d_interval)
+
+
+def active_uncertainty_threshold(conf_active: np.ndarray, active_idx: np.ndarray, B: int, N: int, m: float):
+    """theta_t per sequence: the m-th percentile of u = 1 - conf over the rows that were active in step t;
+    +inf for a sequence without active rows."""
+    u = 1.0 - np.asarray(conf_active, F64)
+    seq = np.asarray(active_idx) // N
+    theta = np.full(B, np.inf, F64)
+    for b in range(B):
+        rows = np.flatnonzero(seq == b)
+        if len(rows):
+            theta[b] = percentile_linear(u[rows], m)
+    return theta
+
+
+def probe_unlock(state: OracleState, ustate: UnlockState, weights: Dict, tokens: np.ndarray, lock: np.ndarray, t: int,
+                 conf_active: np.ndarray, active_idx: np.ndarray, p: UnlockParams, logits_round=None):
+    """The probe after step t (called when t is a multiple of P): proxy posteriors of the locked rows, drift against
+    p_{t*}, the un-lock rule, and the state changes of an un-lock.  `lock` is the mask after step t's lock update;
+    conf_active / active_idx are step t's outputs.  Returns dict(new_lock, locked_idx, u, drift, theta, unlocked)."""
+    B, N = state.B, state.N
+    idx, logits, logp, conf = probe_rows(state, weights, tokens, lock)
+    if logits_round is not None:
+        logits = np.asarray(logits_round(logits), F64)
+        logp = log_softmax(logits)
+        conf, _ = posterior_stats(logits)
+    bb, ii = idx // N, idx % N
+    drift = kl_rows(logp, ustate.frozen_logp[bb, ii])
+    theta = active_uncertainty_threshold(conf_active, active_idx, B, N, p.m)
+    u = 1.0 - conf
+    fire = unlock_test(u, drift, theta[bb], t, ustate.t_star[bb, ii], p)
+    new_lock = np.array(lock, dtype=np.uint8, copy=True)
+    new_lock[bb[fire], ii[fire]] = 0
+    ustate.cool_until[bb[fire], ii[fire]] = t + p.d_cool
+    ustate.relock[bb[fire], ii[fire]] = True
+    return dict(new_lock=new_lock, locked_idx=idx, u=u, drift=drift, theta=theta, unlocked=fire, logits=logits)

@@ -17,6 +17,20 @@ def rel_err_rows(got, ref):
     return float(np.max(np.abs(got - ref) / den))
 
 
+def rel_err_stats(got, ref):
+    """The same per-entry relative error as rel_err_rows, summarised three ways: its maximum, its root mean square
+    and its 99.99th percentile over all entries."""
+    got = np.asarray(got, np.float64)
+    ref = np.asarray(ref, np.float64)
+    got = got.reshape(-1, got.shape[-1])
+    ref = ref.reshape(-1, ref.shape[-1])
+    if ref.size == 0:
+        return dict(max=0.0, rms=0.0, p9999=0.0)
+    rms = np.sqrt(np.mean(ref * ref, axis=-1, keepdims=True))
+    e = np.abs(got - ref) / np.maximum(np.abs(ref), np.maximum(rms, 1e-300))
+    return dict(max=float(e.max()), rms=float(np.sqrt(np.mean(e * e))), p9999=float(np.percentile(e, 99.99)))
+
+
 def f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to("cpu", torch.float64).numpy()
 

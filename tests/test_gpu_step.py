@@ -13,6 +13,12 @@ from tests.stepper import run_side_by_side
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
+# Whole-step bf16 runs against the ALL-fp64 oracle (free running: every bf16 rounding of an activation since the
+# embedding is in the difference).  The 2e-2 bar of the bf16 path is enforced stage by stage, from the GPU's own traced
+# inputs, in test_gpu_teacher_forced.py; here the per-entry relative error is rounding noise that has passed through
+# 2-3 layers, and what is bounded is its distribution: root mean square <= 1e-2 (measured 0.43-0.61 %), 99.99th
+# percentile <= 3e-2 (measured 2.0-2.5 %), maximum over 10^5..10^6 entries <= 5e-2 (measured 2.2-3.5 %).
+BF16_FREE_RUNNING = dict(tol_logits=5e-2, tol_rms=1e-2, tol_p9999=3e-2)
 
 
 def test_tiny_fp32_sampler_natural_locks():
@@ -36,14 +42,14 @@ def test_tiny_fp32_forced_lock_schedule_and_peaked_posteriors():
 
 def test_tiny_bf16_step():
     cfg = inputs.model_shape("tiny")
-    run_side_by_side(cfg, torch.bfloat16, B=2, N=128, n_prompt=64, steps=10, kl_eps=1e-3, seed=3, tol_logits=5e-2,
-                     std=0.05, forced_p=0.2)
+    run_side_by_side(cfg, torch.bfloat16, B=2, N=128, n_prompt=64, steps=10, kl_eps=1e-3, seed=3, std=0.05, forced_p=0.2,
+                     **BF16_FREE_RUNNING)
 
 
 def test_bf16_head_dim_128_ragged_batch():
     cfg = inputs.model_shape("tiny", d_model=512, n_heads=4, head_dim=128, d_ff=1536, vocab=4096, n_layers=3)
-    run_side_by_side(cfg, torch.bfloat16, B=3, N=200, n_prompt=90, steps=8, kl_eps=1e-3, seed=4, tol_logits=5e-2,
-                     std=0.04, forced_p=0.3)
+    run_side_by_side(cfg, torch.bfloat16, B=3, N=200, n_prompt=90, steps=8, kl_eps=1e-3, seed=4, std=0.04, forced_p=0.3,
+                     **BF16_FREE_RUNNING)
 
 
 def test_confidence_gate_in_the_step():
@@ -55,8 +61,8 @@ def test_confidence_gate_in_the_step():
                                    tol_logits=1e-4, conf_gate_m=20.0)
     assert gated[2] > plain[2]                       # at the third step the gate has held most candidates back
     assert all(a >= b for a, b in zip(gated, gated[1:]))
-    run_side_by_side(cfg, torch.bfloat16, B=3, N=128, n_prompt=64, steps=6, kl_eps=1e-3, seed=6, tol_logits=5e-2,
-                     std=0.05, conf_gate_m=40.0)
+    run_side_by_side(cfg, torch.bfloat16, B=3, N=128, n_prompt=64, steps=6, kl_eps=1e-3, seed=6, std=0.05, conf_gate_m=40.0,
+                     **BF16_FREE_RUNNING)
 
 
 def test_locked_rows_cache_bytes_never_change_and_active_rows_are_rewritten():
@@ -199,6 +205,7 @@ def test_degenerate_active_sets(dtype, tol):
     tokens, mask = inputs.make_tokens(B, N, 40, cfg["vocab"], 11)
     rnd = (lambda a: torch.from_numpy(a).to(torch.float32).to(torch.bfloat16).to(torch.float64).numpy()) \
         if dtype == torch.bfloat16 else None
+    gpu_logits = []                                      # the logits the GPU materialised, step by step
 
     def both(lock):
         ld = lock.to(DEV)
@@ -211,6 +218,7 @@ def test_degenerate_active_sets(dtype, tol):
         assert np.array_equal(out.row_offsets.cpu().numpy(), ref["row_offsets"])
         if M:
             assert rel_err_rows(f64(out.logits[:M]), ref["logits"]) < tol
+        gpu_logits.append(f64(out.logits[:M]))
         return out, ref, ld.cpu()
 
     lock = torch.zeros((B, N), dtype=torch.uint8)
@@ -235,8 +243,12 @@ def test_degenerate_active_sets(dtype, tol):
     out, ref, after = both(lock)
     kl = out.kl[:M].cpu().numpy().astype(np.float64)
     assert np.isfinite(kl).all()
-    fin = np.isfinite(ref["kl"])
-    assert fin.all() and np.all(np.abs(kl - ref["kl"]) <= (2e-2 if dtype == torch.bfloat16 else 1e-3) * ref["kl"] + 1e-6)
+    # the same packed rows in both steps: the oracle's KL on the logits the GPU stored in these two steps
+    kl_ref = O.kl_from_logits(gpu_logits[-1], gpu_logits[-2])
+    assert np.all(np.abs(kl - kl_ref) <= 1e-3 * kl_ref + 1e-9)
+    if dtype == torch.float32:                           # fp32 path: also against the all-fp64 run
+        fin = np.isfinite(ref["kl"])
+        assert fin.all() and np.all(np.abs(kl - ref["kl"]) <= 1e-3 * ref["kl"] + 1e-6)
 
 
 def test_checkpoint_resume_continues_bit_for_bit():

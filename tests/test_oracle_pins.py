@@ -500,3 +500,250 @@ def test_kl_is_stepwise_a_returning_row_starts_over():
     back = int(np.flatnonzero(r3["active_idx"] == 2)[0])
     assert np.isinf(r3["kl"][back]) and np.isfinite(np.delete(r3["kl"], back)).all()
     assert r3["new_lock"][0, 2] == 0
+
+
+def test_keep_last_policy_compares_a_returning_row_with_its_last_posterior():
+    """The other reading of p_{t-1} for a row that sat out a step (Sec. 2.1: a locked row keeps p_{t*}): with
+    prev_policy="keep_last" the returning row's D is the KL between its new posterior and the one it had two steps
+    ago, by hand with scipy; every row that never sat out gets the same D under both policies."""
+    c, oc, w, wn = _small(seed=8)
+    B, N = 1, 10
+    tokens, mask = inputs.make_tokens(B, N, 4, c["vocab"], 8)
+    tok2 = tokens.numpy().copy()
+    tok2[0, 5] = 3
+    m2 = mask.numpy().copy()
+    m2[0, 5] = 0
+    lock0 = np.zeros((B, N), np.uint8)
+    lock2 = lock0.copy()
+    lock2[0, 2] = 1
+    out = {}
+    for pol in ("previous_step", "keep_last"):
+        st = O.OracleState(oc, B, N, prev_policy=pol)
+        r1 = O.step(st, wn, tokens.numpy(), mask.numpy(), lock0, 1e-3)
+        O.step(st, wn, tok2, m2, lock2, 0.0)
+        out[pol] = (r1, O.step(st, wn, tok2, m2, lock0, 1e-3))
+    r1, r3 = out["keep_last"]
+    p1 = scipy.special.softmax(r1["logits"][2])
+    p3 = scipy.special.softmax(r3["logits"][2])
+    np.testing.assert_allclose(r3["kl"][2], scipy.special.rel_entr(p3, p1).sum(), rtol=1e-9)
+    assert np.isinf(out["previous_step"][1]["kl"][2])
+    others = np.arange(N) != 2
+    np.testing.assert_array_equal(r3["kl"][others], out["previous_step"][1]["kl"][others])
+    np.testing.assert_array_equal(r3["logits"], out["previous_step"][1]["logits"])   # the forward itself is the same
+    with pytest.raises(ValueError):
+        O.OracleState(oc, B, N, prev_policy="something else")
+
+
+def test_literal_algorithm_order_lets_a_position_lock_in_the_step_that_reveals_it():
+    """Algorithm 1 line 16 (UpdateMASK) stands before line 20 (candidates = active and unmasked).  Read literally, a
+    position revealed in step t is a candidate in step t.  On a stationary sequence (D = 0 for every row in step 2):
+    the default reading locks exactly the rows that were fed as tokens; the literal order also locks the position
+    that step 2 reveals, and its cached K/V are then those of the MASK token it was fed as."""
+    c, oc, w, wn = _small(seed=6)
+    B, N = 1, 12
+    tokens, mask = inputs.make_tokens(B, N, 8, c["vocab"], 4)
+    tk, mk = tokens.numpy(), mask.numpy()
+    mask_tok = c["vocab"] - 1
+    calls = []
+
+    def reveal_position_9(tok, msk, conf, am, idx):
+        calls.append((conf.copy(), am.copy(), idx.copy()))
+        tok, msk = tok.copy(), msk.copy()
+        tok[0, 9], msk[0, 9] = 5, 0
+        return tok, msk
+
+    res = {}
+    for name, fn in (("default", None), ("literal", reveal_position_9)):
+        st = O.OracleState(oc, B, N)
+        O.step(st, wn, tk, mk, np.zeros((B, N), np.uint8), 1e-3)
+        res[name] = (O.step(st, wn, tk, mk, np.zeros((B, N), np.uint8), 1e-3, unmask=fn), st)
+    rd, rl = res["default"][0], res["literal"][0]
+    assert np.all(rd["kl"] == 0.0) and np.all(rl["kl"] == 0.0)
+    assert rd["new_lock"].tolist() == [[1] * 8 + [0] * 4]
+    assert rl["new_lock"].tolist() == [[1] * 8 + [0, 1, 0, 0]]
+    assert rl["tokens"][0, 9] == 5 and rl["mask_state"][0, 9] == 0 and rd["mask_state"][0, 9] == 1
+    assert len(calls) == 1 and list(calls[0][2]) == list(range(N))
+    np.testing.assert_array_equal(calls[0][0], rl["conf"])                        # line 16 sees this step's posteriors
+    # the forward ran before the reveal: the K/V that position 9 is locked with are those of the mask token
+    st = res["literal"][1]
+    assert tk[0, 9] == mask_tok
+    x = np.asarray(wn["tok_emb"], np.float64)[[mask_tok]]
+    _, k, v = O.qkv_rows(oc, wn["layers"][0], x, np.array([9]))
+    np.testing.assert_allclose(st.K[0, 0, 9], k[0], rtol=1e-12, atol=1e-14)
+    np.testing.assert_allclose(st.V[0, 0, 9], v[0], rtol=1e-12, atol=1e-14)
+    np.testing.assert_array_equal(rd["logits"], rl["logits"])
+
+
+def test_selection_skip_rows_are_not_computed_and_cannot_lock():
+    """Experiment 5's selection surrogate as a skip mask: a skipped unlocked position is not in the active set, keeps
+    its K/V and its lock bit, gets no posterior; the step equals a step in which those positions are locked, and the
+    lock update touches computed rows only.  With the previous-step reading a skipped row has D = inf when it returns,
+    with keep-last it compares with its older posterior."""
+    c, oc, w, wn = _small(seed=9)
+    B, N = 2, 10
+    tokens, mask = inputs.make_tokens(B, N, 6, c["vocab"], 9)
+    tk, mk = tokens.numpy(), mask.numpy()
+    lock = np.zeros((B, N), np.uint8)
+    lock[0, 1] = 1
+    skip = np.zeros((B, N), np.uint8)
+    skip[0, 3] = skip[1, 0] = skip[1, 4] = 1
+    a = O.OracleState(oc, B, N)
+    b = O.OracleState(oc, B, N)
+    for st in (a, b):
+        O.step(st, wn, tk, mk, np.zeros((B, N), np.uint8), 1e-3)
+    K0 = a.K.copy()
+    ra = O.step(a, wn, tk, mk, lock, 1e-3, skip=skip)
+    rb = O.step(b, wn, tk, mk, lock | skip, 1e-3)
+    want_idx = [i for i in range(B * N) if i not in (1, 3, 10, 14)]
+    assert list(ra["active_idx"]) == want_idx and ra["row_offsets"].tolist() == [0, 8, 16]
+    np.testing.assert_array_equal(ra["logits"], rb["logits"])
+    np.testing.assert_array_equal(a.K[:, 0, 3], K0[:, 0, 3])                      # a skipped row's K/V stay
+    # stationary tokens: D = 0 for every computed row, so every computed unmasked row locks; skipped ones do not
+    want_lock = ((mk == 0) & (skip == 0)).astype(np.uint8) | lock
+    assert np.array_equal(ra["new_lock"], want_lock)
+    assert ra["new_lock"][0, 3] == 0 and ra["new_lock"][1, 0] == 0 and ra["new_lock"][1, 4] == 0
+    assert np.array_equal(rb["new_lock"], want_lock | skip)                       # the locked-instead run keeps skip bits
+    r3 = O.step(a, wn, tk, mk, ra["new_lock"], 1e-3)                              # the skipped rows return
+    back = [int(np.flatnonzero(r3["active_idx"] == p)[0]) for p in (3, 10, 14)]
+    assert np.isinf(r3["kl"][back]).all() and not r3["new_lock"][0, 3]
+    kl = O.OracleState(oc, B, N, prev_policy="keep_last")
+    O.step(kl, wn, tk, mk, np.zeros((B, N), np.uint8), 1e-3)
+    r2k = O.step(kl, wn, tk, mk, lock, 1e-3, skip=skip)
+    r3k = O.step(kl, wn, tk, mk, r2k["new_lock"], 1e-3)
+    assert np.all(np.abs(r3k["kl"][back]) < 1e-12) and r3k["new_lock"][0, 3] == 1
+
+
+# ------------------------------------------------------------------ optional un-locking (App. "Optional Unlocking")
+def test_unlock_rule_truth_table():
+    """The printed rule: u~ > theta AND D~ > eps_unlock AND t - t* > D_interval; strict inequalities."""
+    p = O.UnlockParams(period=4, eps_unlock=0.01, d_interval=3, d_cool=2, rho=0.5, m=20.0)
+    u = np.array([0.5, 0.5, 0.5, 0.5, 0.2, 0.5, 0.5, 0.3])
+    D = np.array([0.02, 0.02, 0.02, 0.01, 0.02, 0.005, 0.02, 0.02])
+    t_star = np.array([1, 5, 4, 1, 1, 1, 2, 1])
+    theta = np.full(8, 0.3)
+    fire = O.unlock_test(u, D, theta, 8, t_star, p)
+    #      all hold | 8-5=3 not >3 | 8-4=4 | D == eps | u < theta | D < eps | fine | u == theta
+    assert fire.tolist() == [True, False, True, False, False, False, True, False]
+    assert not O.unlock_test(u, D, np.full(8, np.inf), 8, t_star, p).any()        # no reference uncertainty: nothing
+
+
+def test_active_uncertainty_threshold_is_numpy_percentile_per_sequence():
+    rng = np.random.default_rng(3)
+    N, B = 9, 3
+    idx = np.array([0, 2, 3, 7, 8, 18, 19, 20, 21, 22, 23, 24])                   # sequence 1 has no active row
+    conf = rng.random(len(idx))
+    th = O.active_uncertainty_threshold(conf, idx, B, N, 20.0)
+    assert th[1] == np.inf
+    np.testing.assert_allclose(th[0], np.percentile(1 - conf[:5], 20.0), rtol=1e-12)
+    np.testing.assert_allclose(th[2], np.percentile(1 - conf[5:], 20.0), rtol=1e-12)
+
+
+def test_probe_is_a_dense_forward_over_the_cached_keys_and_changes_nothing():
+    """probe_rows: the locked rows as queries against the caches as they stand.  Pinned against the independent dense
+    torch forward in which the K/V of EVERY position are overridden by the cache contents (so each probed row's result
+    is what that forward gives at its position), and by stationarity: if nothing changed since the rows locked, the
+    probe reproduces their frozen posterior and the drift is 0."""
+    c, oc, w, wn = _small(seed=11)
+    B, N, V = 2, 12, c["vocab"]
+    tokens, mask = inputs.make_tokens(B, N, 7, V, 5)
+    tk, mk = tokens.numpy(), mask.numpy()
+    st = O.OracleState(oc, B, N)
+    us = O.UnlockState(B, N, V)
+    zero = np.zeros((B, N), np.uint8)
+    O.step(st, wn, tk, mk, zero, 1e-3)
+    r2 = O.step(st, wn, tk, mk, zero, 1e-3)                                       # stationary: unmasked rows lock
+    O.record_locks(us, 2, zero, r2, N)
+    lock = r2["new_lock"]
+    assert lock.sum() == 14 and np.all(us.t_star[lock == 1] == 2) and np.all(us.t_star[lock == 0] == -1)
+    K0, V0 = st.K.copy(), st.V.copy()
+    idx, logits, logp, conf = O.probe_rows(st, wn, tk, lock)
+    assert np.array_equal(st.K, K0) and np.array_equal(st.V, V0)                  # line 11 is not executed
+    assert list(idx) == [b * N + i for b in range(B) for i in range(7)]
+    bb, ii = idx // N, idx % N
+    np.testing.assert_allclose(logp, us.frozen_logp[bb, ii], rtol=0, atol=1e-11)
+    assert np.all(np.abs(O.kl_rows(logp, us.frozen_logp[bb, ii])) < 1e-12)
+    # a context shift: the sampler reveals tokens, one more step rewrites the active rows' K/V
+    tk2, mk2 = tk.copy(), mk.copy()
+    tk2[:, 7:10] = [[3, 4, 5], [9, 8, 7]]
+    mk2[:, 7:10] = 0
+    O.step(st, wn, tk2, mk2, lock, 1e-3)
+    idx, logits, logp, conf = O.probe_rows(st, wn, tk2, lock)
+    for b in range(B):
+        allpos = torch.arange(N)
+        ov = {l: (allpos, torch.from_numpy(st.K[l, b]), torch.from_numpy(st.V[l, b])) for l in range(c["n_layers"])}
+        ref = DR.dense_forward(c, _w64(w), torch.from_numpy(tk2[b]), kv_override=ov).numpy()
+        got = logits[idx // N == b]
+        assert np.max(np.abs(got - ref[:7])) <= 1e-11 * np.max(np.abs(ref))
+    drift = O.kl_rows(logp, us.frozen_logp[bb, ii])
+    want = DR.kl_torch(torch.from_numpy(logits), torch.from_numpy(us.frozen_logp[bb, ii])).numpy()
+    np.testing.assert_allclose(drift, want, rtol=1e-9, atol=1e-15)
+    assert np.all(drift > 1e-9)                                                   # the frozen posteriors are stale now
+
+
+def test_unlock_cycle_by_hand_cool_down_and_stricter_relock():
+    """One position through the whole cycle on a tiny model, every decision checked by hand: it locks, the context
+    shifts, the probe un-locks it only once all three conditions hold (the interval is the last to be met), it is
+    active again from the next step and its K/V are rewritten then, it cannot lock during the cool-down, and
+    afterwards only under rho * eps."""
+    c, oc, w, wn = _small(seed=11)
+    B, N, V = 1, 12, c["vocab"]
+    tokens, mask = inputs.make_tokens(B, N, 7, V, 5)
+    tk, mk = tokens.numpy(), mask.numpy()
+    st = O.OracleState(oc, B, N)
+    us = O.UnlockState(B, N, V)
+    eps = 1e-3
+    P = O.UnlockParams(period=1, eps_unlock=1e-9, d_interval=2, d_cool=2, rho=1e-30, m=0.0)
+    zero = np.zeros((B, N), np.uint8)
+    O.step(st, wn, tk, mk, zero, eps)                                             # t = 1
+    r = O.step(st, wn, tk, mk, zero, eps)                                         # t = 2: rows 0..6 lock (stationary)
+    O.record_locks(us, 2, zero, r, N)
+    lock = r["new_lock"]
+    pr = O.probe_unlock(st, us, wn, tk, lock, 2, r["conf"], r["active_idx"], P)
+    assert not pr["unlocked"].any() and np.array_equal(pr["new_lock"], lock)      # no drift, and t - t* = 0
+    tk2, mk2 = tk.copy(), mk.copy()
+    tk2[0, 7:10] = [3, 4, 5]
+    mk2[0, 7:10] = 0
+    for t in (3, 4):                                                              # drift is there, the interval is not met
+        before = lock.copy()
+        e_rows, may = O.relock_thresholds(us, eps, P.rho, t)
+        r = O.step(st, wn, tk2, mk2, lock, eps, kl_eps_rows=e_rows, may_lock=may)
+        O.record_locks(us, t, before, r, N)
+        lock = r["new_lock"]
+        pr = O.probe_unlock(st, us, wn, tk2, lock, t, r["conf"], r["active_idx"], P)
+        early = us.t_star[0, pr["locked_idx"]] == 2
+        assert np.all(pr["drift"][early] > P.eps_unlock)
+        assert not pr["unlocked"].any(), t                                         # 3 - 2 and 4 - 2 are not > 2
+        lock = pr["new_lock"]
+    # t = 5: theta = min uncertainty of the active rows (m = 0); un-lock exactly the early rows above it
+    before = lock.copy()
+    e_rows, may = O.relock_thresholds(us, eps, P.rho, 5)
+    r = O.step(st, wn, tk2, mk2, lock, eps, kl_eps_rows=e_rows, may_lock=may)
+    O.record_locks(us, 5, before, r, N)
+    lock = r["new_lock"]
+    pr = O.probe_unlock(st, us, wn, tk2, lock, 5, r["conf"], r["active_idx"], P)
+    li = pr["locked_idx"]
+    want = (pr["u"] > pr["theta"][0]) & (pr["drift"] > P.eps_unlock) & (5 - us.t_star[0, li] > 2)
+    assert np.array_equal(pr["unlocked"], want) and want.any()
+    assert np.all(us.t_star[0, li[want]] == 2)                                    # only rows locked long enough ago
+    freed = li[want]
+    assert np.all(pr["new_lock"][0, freed] == 0) and np.all(us.cool_until[0, freed] == 7) and us.relock[0, freed].all()
+    lock = pr["new_lock"]
+    K_before = st.K[1, 0, freed].copy()            # second block: its keys depend on the context (the first block's do not)
+    # t = 6, 7: active again (K/V rewritten with the current context), cannot lock (cool-down); D = inf at t = 6 anyway
+    for t in (6, 7):
+        e_rows, may = O.relock_thresholds(us, eps, P.rho, t)
+        assert not may[0, freed].any() and np.all(e_rows[0, freed] == eps * P.rho)
+        r = O.step(st, wn, tk2, mk2, lock, eps, kl_eps_rows=e_rows, may_lock=may)
+        assert set(freed) <= set(r["active_idx"])
+        assert not r["new_lock"][0, freed].any(), t
+        lock = r["new_lock"]
+    assert np.all(np.any(st.K[1, 0, freed] != K_before, axis=(1, 2)))
+    # t = 8: cool-down over, but the threshold is rho * eps: D = 0 (stationary again) passes, a tiny positive D would not
+    e_rows, may = O.relock_thresholds(us, eps, P.rho, 8)
+    assert may[0, freed].all()
+    r = O.step(st, wn, tk2, mk2, lock, eps, kl_eps_rows=e_rows, may_lock=may)
+    rows = [int(np.flatnonzero(r["active_idx"] == p)[0]) for p in freed]
+    assert np.all(r["kl"][rows] <= 1e-12)
+    exact0 = r["kl"][rows] <= e_rows[0, freed]
+    assert np.array_equal(r["new_lock"][0, freed].astype(bool), exact0)
+    assert np.array_equal(O.sure_test(np.array([1e-31, 1e-4]), np.zeros(2), np.array([1e-33, 1e-3])), [False, True])
