@@ -87,7 +87,9 @@ int surelock_init(surelock_ctx **out, const surelock_model_cfg *cfg, const surel
                   int N, int batch, void *cuda_stream);
 
 /* Forget the previous posteriors (p_{t-1} = None, so the next step's KL is +inf for every row: Algorithm 1
- * line 19) and clear the device status word.  Cache contents are kept (a caller may have pre-filled them). */
+ * line 19), clear the device status word and the hand-over counters of the split-K GEMM (a kernel that gave up on a
+ * bounded wait, device status 2, may have left them half-way), and zero the fallback count.  Cache contents are kept
+ * (a caller may have pre-filled them). */
 int surelock_reset(surelock_ctx *ctx);
 
 /* One SureLock step (Algorithm 1 lines 6-15 and 18-24; the unmasking policy of line 16 is the caller's).
@@ -162,7 +164,9 @@ int surelock_state_import(surelock_ctx *ctx, const void *host_src, size_t bytes)
 int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float **theta);
 
 /* Tuning / test switches.  "gemm_impl": 0 = tensor-core GEMM and attention when the shape allows (default),
- * 1 = force the CUDA-core kernels.  "time_kernels": 1 creates an event pool (once) and brackets every launch of
+ * 1 = force the CUDA-core kernels.  "strict_tc": 1 = a bf16 contraction or attention whose shape the tensor-core
+ * kernels do not take makes the step return SL_EUNSUPPORTED instead of running on the CUDA-core kernels (0, the
+ * default, falls back and counts it: surelock_last_fallback_count()).  "time_kernels": 1 creates an event pool (once) and brackets every launch of
  * later steps with CUDA events for surelock_kernel_times().  "trace_layers": 1 allocates (once, here, not in the
  * step) a buffer [2L+1][B*N][d] fp32 and makes every later surelock_step copy the packed residual stream into it:
  * slot 2l = input of block l (slot 0 = the embeddings), slot 2l+1 = after the attention sub-block of block l,
@@ -183,6 +187,10 @@ int surelock_layer_trace(surelock_ctx *ctx, float **buf, size_t *layer_stride_el
 
 /* Number of kernels the last surelock_step / surelock_layer_step call launched (host-side count). */
 int surelock_last_launch_count(surelock_ctx *ctx);
+
+/* Number of launches since the last surelock_reset in which a bf16 ctx with "gemm_impl" 0 ran a CUDA-core kernel
+ * because the tensor-core kernel does not take the shape (host-side count; 0 for every benchmark configuration). */
+int surelock_last_fallback_count(surelock_ctx *ctx);
 
 /* Per-kernel-class device time of the LAST step, measured with CUDA events on the ctx stream; needs
  * surelock_set_option(ctx, "time_kernels", 1) before that step (events add a few microseconds per launch, so time
@@ -227,7 +235,9 @@ int surelock_compact(const uint8_t *lock_mask, int B, int N, int32_t *active_idx
  * cudaFree or other allocating call; it enqueues one cudaMemsetAsync (the array keeps the previous call's
  * contents, so the words this call uses are cleared first) and one kernel on `stream`.
  * The FIRST call on each device also asks the CUDA runtime for the array's device address (with that device
- * current) and caches it; make that first call outside any stream capture.
+ * current) and caches it for the life of the process; make that first call outside any stream capture.  The cached
+ * address does not survive cudaDeviceReset() or the destruction of the device's primary context: a process that does
+ * either must not call this entry point on that device afterwards.
  * All calls on a device share the one array: two calls whose kernels may overlap on the GPU (different streams,
  * or different host threads) race on it and give wrong results -- serialise them. */
 int surelock_compact_noalloc(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
@@ -293,7 +303,7 @@ size_t surelock_gemm_workspace_bytes(void);
  * A, W, C of `dtype`; fp32 accumulation.  impl: 0 = best available (tcgen05 tensor cores for SL_BF16 when the
  * shape allows), 1 = force the CUDA-core kernel.
  * workspace: dev, surelock_gemm_workspace_bytes() bytes, ZERO-FILLED by the caller before its first use (the kernel
- * leaves it reusable), or NULL.  With a workspace and few output tiles (small M) the tensor-core kernel splits K
+ * leaves it reusable, unless it gave up on a bounded wait: after device status 2 zero-fill it again), or NULL.  With a workspace and few output tiles (small M) the tensor-core kernel splits K
  * across SMs and sums the partial tiles in a fixed order (deterministic); without one it never splits.
  * dev_status as for surelock_compact. */
 int surelock_gemm(const void *A, const void *W, void *C, const int32_t *n_active, int max_rows, int n_out, int K,
@@ -310,8 +320,8 @@ int surelock_gemm_fused(const void *A, const void *W, const void *W2, void *C, c
                         int n_out, int K, int dtype, int epilogue, int impl, void *workspace, int32_t *dev_status,
                         void *stream);
 
-/* M x N bidirectional attention of the packed queries against the whole cache (Algorithm 1 line 12; Sec. 2.1:
- * "variable-length attention against the full key/value tables"): for packed row r at flat position
+/* M x N bidirectional attention of the packed queries against the whole cache (Algorithm 1 line 12; Sec. 2.1: the
+ * packed active queries attend to all N cached keys and values of their sequence): for packed row r at flat position
  * active_idx[r] = b*N+i and every head h, o[r][h] = softmax_j(q[r][h] . K[b*N+j][h] / sqrt(d_h)) V[b*N+j][h],
  * j = 0..N-1.  q, o: dev [M][H][d_h]; k_cache, v_cache: dev [B*N][H][d_h]; all of `dtype`. */
 int surelock_attention(const void *q, const void *k_cache, const void *v_cache, const int32_t *active_idx,

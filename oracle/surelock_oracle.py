@@ -251,6 +251,25 @@ def update_mask(tokens: np.ndarray, mask_state: np.ndarray, conf: np.ndarray, ar
     return tokens, mask_state, revealed
 
 
+def selection_skip(lock: np.ndarray, mask_state: np.ndarray, scores: np.ndarray, fraction: float) -> np.ndarray:
+    """The selection surrogate of Experiment 5 ("computes only on a fixed fraction k of active tokens at each step").
+    Which positions a selection method drops is not the paper's subject; the surrogate's rule, given per-position
+    scores as input: per sequence, with U = number of unlocked positions, skip the floor((1 - k) U) eligible positions
+    (unlocked and unmasked: a masked position is always computed, the sampler needs its posterior) that have the
+    lowest scores, ties to the lower position; fewer if there are not that many eligible ones.
+    Returns uint8 [B][N], 1 = not computed in this step."""
+    lock = np.asarray(lock)
+    B, N = lock.shape
+    skip = np.zeros((B, N), np.uint8)
+    for b in range(B):
+        unlocked = [i for i in range(N) if lock[b, i] == 0]
+        eligible = [i for i in unlocked if mask_state[b, i] == 0]
+        n_skip = min(int(np.floor(np.float32(len(unlocked)) * np.float32(1.0 - fraction))), len(eligible))
+        for i in sorted(eligible, key=lambda i: (scores[b, i], i))[:n_skip]:
+            skip[b, i] = 1
+    return skip
+
+
 # --------------------------------------------------------------------------
 # Algorithmic FLOPs (Sec. 2.3)
 # --------------------------------------------------------------------------

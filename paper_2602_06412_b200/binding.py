@@ -61,6 +61,7 @@ def lib() -> C.CDLL:
         "surelock_prev_logits": (i32, [vp, C.POINTER(vp), C.POINTER(vp)]),
         "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
         "surelock_last_launch_count": (i32, [vp]),
+        "surelock_last_fallback_count": (i32, [vp]),
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
         "surelock_conf_gate_lock": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, f32, f32, vp, vp]),
         "surelock_update_mask": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
@@ -276,6 +277,10 @@ def surelock_state_import(ctx: Ctx, state: bytes):
 
 def surelock_last_launch_count(ctx: Ctx) -> int:
     return lib().surelock_last_launch_count(ctx.handle)
+
+
+def surelock_last_fallback_count(ctx: Ctx) -> int:
+    return lib().surelock_last_fallback_count(ctx.handle)
 
 
 KERNEL_CLASSES = ("compact", "gather", "rmsnorm", "gemm_qkv", "rope", "kv_scatter", "attention", "gemm_o",

@@ -30,10 +30,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "--threads", "8", "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
            "-I", os.path.join(HERE, "csrc")]
-    # development aid: extra compiler flags, e.g. SURELOCK_NVCC_FLAGS="-DATT_PROFILE" (cycle counters of the attention
-    # kernel's softmax and MMA threads, printed to stderr at every launch) or "-DGEMM_PROFILE" (per-CTA time stamps of a
-    # GEMM launch); such a build is for looking at one kernel, not for timing a step
-    cmd += os.environ.get("SURELOCK_NVCC_FLAGS", "").split()
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources() + ["-o", LIB]

@@ -35,6 +35,9 @@ struct surelock_ctx {
   bool have_prev = false;
   int launches = 0;
   int gemm_impl = 0;                  // 0 = tensor cores when possible, 1 = CUDA cores
+  bool strict_tc = false;             // refuse (SL_EUNSUPPORTED) instead of falling back to the CUDA-core kernels
+  int fallbacks = 0;                  // launches that fell back since the last reset
+  int32_t* n_prev = nullptr;          // rows of the previous step's logits (copy of n_active taken at the end of a step)
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
   bool timing = false;                // per-kernel-class CUDA-event timing (off by default)
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
@@ -112,7 +115,8 @@ static int attention(surelock_ctx* c, int l) {
   if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_attention_tc(c->q, c->kcache(l), c->vcache(l), c->row_offsets, c->R, c->B, c->N, g.n_heads,
                                        g.head_dim, c->attn, c->status, c->st);
-    if (rc != SL_EUNSUPPORTED) return rc;
+    if (rc != SL_EUNSUPPORTED || c->strict_tc) return rc;
+    ++c->fallbacks;
   }
   return launch_attention_simt(c->q, c->kcache(l), c->vcache(l), c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim,
                                c->attn, g.dtype, c->st);
@@ -123,7 +127,8 @@ static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, v
   if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->split, c->st);
     c->last_gemm_tc = rc == SL_OK;
-    if (rc != SL_EUNSUPPORTED) return rc;
+    if (rc != SL_EUNSUPPORTED || c->strict_tc) return rc;
+    ++c->fallbacks;
   }
   return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
 }
@@ -142,8 +147,10 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
     if (rc == SL_OK) {
       tock(c);
       fused = true;
-    } else if (rc != SL_EUNSUPPORTED) {
+    } else if (rc != SL_EUNSUPPORTED || c->strict_tc) {
       return rc;
+    } else {
+      ++c->fallbacks;
     }
   }
   if (!fused) {
@@ -228,6 +235,7 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
   A_(c->idx, R * 4);
   A_(c->row_offsets, ((size_t)batch + 1) * 4);
   A_(c->n_active, 16);
+  A_(c->n_prev, 16);
   A_(c->status, 16);
   A_(c->argmax, R * 4);
   A_(c->kl, R * 4);
@@ -271,6 +279,12 @@ int surelock_reset(surelock_ctx* c) {
   for (int i = 0; i < 2; ++i) SL_CUDA_TRY(cudaMemsetAsync(c->row_of_pos[i], 0xff, (size_t)c->R * 4, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->status, 0, 16, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->n_active, 0, 16, c->st));
+  SL_CUDA_TRY(cudaMemsetAsync(c->n_prev, 0, 16, c->st));
+  c->fallbacks = 0;
+  // a GEMM that gave up on a bounded wait leaves its tiles' hand-over counters half-way: start from zero again
+  if (c->split.counters)
+    SL_CUDA_TRY(cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * 3 * sizeof(int), c->st));
+  if (c->lse_valid) SL_CUDA_TRY(cudaMemsetAsync(c->lse_valid, 0, 16, c->st));
   if (c->kv_valid) SL_CUDA_TRY(cudaMemsetAsync(c->kv_valid, 0, (size_t)c->R, c->st));   // cache contents are undefined now
   return SL_OK;
 }
@@ -323,6 +337,8 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
     out->conf = c->conf;
     out->argmax = c->argmax;
   }
+  // the row count of the logits the next step reads as "previous" (n_active itself is overwritten by other calls)
+  SL_CUDA_TRY(cudaMemcpyAsync(c->n_prev, c->n_active, 4, cudaMemcpyDeviceToDevice, c->st));
   c->cur = prv;
   c->have_prev = true;
   return SL_OK;
@@ -424,7 +440,8 @@ int surelock_state_export(surelock_ctx* c, void* host_dst, size_t capacity, size
   fill_header(c, &h);
   h.have_prev = c->have_prev ? 1 : 0;
   int32_t m_prev = 0;
-  if (c->have_prev) SL_CUDA_TRY(cudaMemcpy(&m_prev, c->n_active, 4, cudaMemcpyDeviceToHost));
+  if (c->have_prev) SL_CUDA_TRY(cudaMemcpy(&m_prev, c->n_prev, 4, cudaMemcpyDeviceToHost));
+  if (c->have_prev && m_prev == 0) m_prev = c->R;   // previous logits seeded by the caller ("have_prev"): keep every row
   if (m_prev < 0 || m_prev > c->R) return SL_EDEVICE;
   h.rows_prev = m_prev;
   const size_t kvb = 2 * (size_t)c->cfg.n_layers * c->kv_layer_bytes();
@@ -470,6 +487,8 @@ int surelock_state_import(surelock_ctx* c, const void* host_src, size_t bytes) {
   p += lsb;
   SL_CUDA_TRY(cudaMemcpyAsync(c->row_of_pos[prv], p, rpb, cudaMemcpyHostToDevice, c->st));
   c->have_prev = h.have_prev != 0;
+  const int32_t rows_prev = h.rows_prev;
+  SL_CUDA_TRY(cudaMemcpyAsync(c->n_prev, &rows_prev, 4, cudaMemcpyHostToDevice, c->st));
   SL_CUDA_TRY(cudaStreamSynchronize(c->st));
   return SL_OK;
 }
@@ -477,6 +496,7 @@ int surelock_state_import(surelock_ctx* c, const void* host_src, size_t bytes) {
 int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
+  if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
   if (!strcmp(name, "check_cache")) {
     if (value && !c->kv_valid) {
@@ -527,6 +547,8 @@ int surelock_set_confidence_gate(surelock_ctx* c, float m_percent, const float**
 }
 
 int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
+
+int surelock_last_fallback_count(surelock_ctx* c) { return c ? c->fallbacks : SL_EINVAL; }
 
 int surelock_kernel_times(surelock_ctx* c, float* ms, int32_t* launches, int n_classes) {
   if (!c || !ms || n_classes < K_NUM) return SL_EINVAL;

@@ -61,7 +61,7 @@ template <int DH>
 __global__ void __launch_bounds__(PP_THREADS, 1)
 attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                     const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
-                    bf16* __restrict__ o, float scale_log2, int32_t* status, unsigned long long* prof) {
+                    bf16* __restrict__ o, float scale_log2, int32_t* status) {
   constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
   constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
   constexpr int Q_BYTES = SLABS * SLAB_BYTES;          // one Q tile
@@ -381,12 +381,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       }
       tc_wait_st();
     };
-#ifdef ATT_PROFILE
-    unsigned long long tp[8] = {0, 0, 0, 0, 0, 0, 0, 0}, t0 = clock64(), t1;
-#define ATT_T(i) { t1 = clock64(); tp[i] += t1 - t0; t0 = t1; }
-#else
-#define ATT_T(i)
-#endif
     // PAIRS: tile t of every item of this CTA; STREAMS: every item of stream t
     const int w_first = (int)blockIdx.x + (streams ? t * (int)gridDim.x : 0), w_step = streams ? nstream : (int)gridDim.x;
     const int t_off = streams ? 0 : t * PP_BQ;
@@ -400,9 +394,7 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       // common path is free of branches and the compiler can interleave loads, maxima and exponentials)
       auto block = [&](int j, auto masked_tag) -> bool {
         constexpr bool MASKED = decltype(masked_tag)::value;
-        ATT_T(0)
         if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL + t), (g + j) & 1, s_abort))) return false;
-        ATT_T(1)
         tc_fence_after();
         uint32_t s[128];
         tc_ld32(s_addr, s);
@@ -410,7 +402,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc_ld32(s_addr + 64, s + 64);
         tc_ld32(s_addr + 96, s + 96);
         tc_wait_ld();
-        ATT_T(2)
         if (MASKED) {
           const int nvalid = N - j * PP_BKV;             // keys of this block that exist
 #pragma unroll
@@ -441,8 +432,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         }
         // S of this block is complete, so the previous block's P V is too, and this block's has not been issued
         if (j > 0 && __any_sync(0xffffffffu, need)) rescale_o(corr);
-        ATT_T(3)
-        ATT_T(4)
         const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(-m_used, -m_used);
         float2 sum2[4] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #define PP_EXP32(c0)                                                                                                   \
@@ -461,7 +450,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_HALF + t));     // the first half of P V can start
-        ATT_T(5)
         PP_EXP32(96)
         tc_st32(s_addr + 96, s + 32);                    // keys 64..127
         sum2[0] = __fadd2_rn(__fadd2_rn(sum2[0], sum2[1]), __fadd2_rn(sum2[2], sum2[3]));
@@ -470,7 +458,6 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_FULL + t));
-        ATT_T(6)
         return true;
       };
       const int nfast = (N % PP_BKV) ? nblk - 1 : nblk;
@@ -504,12 +491,7 @@ attention_pp_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(O_FREE + t));
-      ATT_T(7)
     }
-#ifdef ATT_PROFILE
-    if (prof && blockIdx.x == 0 && (warp == 2 || warp == 6) && lane == 0)
-      for (int i = 0; i < 8; ++i) prof[(warp == 6 ? 8 : 0) + i] = tp[i];
-#endif
   }
 
   tc_fence_before();
@@ -536,23 +518,8 @@ static int launch_pp_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtens
   if (items < grid) grid = (int)items;
   if (grid < 1) grid = 1;
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  unsigned long long* prof = nullptr;
-#ifdef ATT_PROFILE
-  static unsigned long long* d_prof = nullptr;
-  if (!d_prof) cudaMalloc(&d_prof, 192);
-  prof = d_prof;
-#endif
   SL_CUDA_TRY(launch_pdl(attention_pp_kernel<DH>, dim3(grid), dim3(PP_THREADS), (size_t)smem, st, q, k, v, row_offsets, B, N, H,
-                         (bf16*)o, scale_log2, status, prof));
-#ifdef ATT_PROFILE
-  {
-    unsigned long long h[24];
-    cudaMemcpy(h, d_prof, 192, cudaMemcpyDeviceToHost);
-    for (int t = 0; t < 2; ++t)
-      fprintf(stderr, "ATT_PROFILE tile %d cycles: loop %llu waitS %llu ldS %llu max %llu turn %llu exp-to-half %llu rest %llu waitO+epi %llu\n",
-              t, h[8 * t], h[8 * t + 1], h[8 * t + 2], h[8 * t + 3], h[8 * t + 4], h[8 * t + 5], h[8 * t + 6], h[8 * t + 7]);
-  }
-#endif
+                         (bf16*)o, scale_log2, status));
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

@@ -38,18 +38,6 @@ constexpr int TC_MAX_STAGES = 16;
 constexpr unsigned long long SPLIT_HELP_CYCLES = 200000ull;   // how long a split waits for its siblings before leaving (~0.1 ms)
 constexpr int TC_DATA_BYTES = 216 * 1024;   // operand stages: 4 x 48 KB (128 rows of A + a 256-wide weight tile) ... 16 x 12 KB
 
-#ifdef GEMM_PROFILE
-// development aid: per-CTA time stamps (ns) of the first item of a launch
-__device__ unsigned long long g_gemm_prof[160 * 8];
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define GP(i) { g_gemm_prof[blockIdx.x * 8 + (i)] = gtime(); }
-#else
-#define GP(i) {}
-#endif
 constexpr int EPI_QKV = 3;   // three weight matrices side by side; epilogue = RoPE + packed q + K/V cache scatter
 
 struct QkvArgs {
@@ -546,7 +534,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       return;
     }
   }
-  if (threadIdx.x == 0) GP(0)
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + TC_DATA_BYTES);
   // bars: full[STAGES], empty[STAGES], acc_full[2], acc_empty[2]
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 4);
@@ -577,7 +564,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
-  if (threadIdx.x == 0) GP(1)
 
   const int M = *n_active;
   const int num_kb = (K + TC_BK - 1) / TC_BK;
@@ -701,7 +687,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN_MAX);
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(full_bar(stage), phase, s_abort))) break;
-          if (it == 0 && kb == kb0) GP(2)
           tc_fence_after();
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
           const uint64_t adesc = smem_desc_k_sw128(sa), bdesc = smem_desc_k_sw128(sb);
@@ -712,7 +697,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (++stage == nst) { stage = 0; phase ^= 1; }
         }
         if (ok) tc_commit(accf_bar(acc));
-        if (it == 0) GP(3)
       }
     }
   } else {
@@ -735,7 +719,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      if (it == 0 && warp == 2 && lane == 0) GP(4)
       tc_fence_after();
       const int trow = quarter * 32 + lane;
       const int row = m0 + trow;
@@ -808,7 +791,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
           s_fin[0] = role;
           s_fin[1] = ticket;
-          if (it == 0) GP(5)
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const int role = s_fin[0], ticket = s_fin[1];
@@ -849,7 +831,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             *arrived = 0;                              // every split has arrived and only this CTA is still here
           }
         }
-        if (it == 0 && warp == 2 && lane == 0) GP(6)
       }
     }
     if (EPI == EPI_RESIDUAL) bulk_wait0();      // every reduction of this thread has been performed before the CTA leaves
@@ -857,7 +838,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) GP(7)
   if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_GEMM_TIMEOUT);
   if (warp == 1) {
     tc_fence_after();
@@ -973,29 +953,6 @@ static int launch_cfg(const CUtensorMap* a, const CUtensorMap* b, const CUtensor
   SL_CUDA_TRY(cudaLaunchKernelEx(&cfg, gemm_tc_kernel<EPI, STAGES>, a[0], a[1], a[2], b[0], b[1], b[2], wb[0], wb[1], wb[2], xb[0], xb[1], xb[2], C, n_active,
                                  n_out, K, status, qkv, sw.ws, sw.counters, sw.tiles, force_cfg(0),
                                  force_cfg(1), pair, sw.prefetch_w ? 1 : 0));
-#ifdef GEMM_PROFILE
-  {
-    static unsigned long long h[160 * 8];
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(h, g_gemm_prof, sizeof(h));
-    unsigned long long t0 = ~0ull;
-    for (int c = 0; c < grid; ++c) if (h[c * 8] && h[c * 8] < t0) t0 = h[c * 8];
-    const char* names[8] = {"entry", "prologue", "first-stage", "mma-issued", "acc-ready", "partial+count", "finisher", "exit"};
-    fprintf(stderr, "GEMM_PROFILE epi %d n_out %d K %d (us after the first CTA's entry; min / mean / max over CTAs that report)\n", EPI, n_out, K);
-    for (int i = 0; i < 8; ++i) {
-      double mn = 1e30, mx = 0, sum = 0; int n = 0;
-      for (int c = 0; c < grid; ++c) {
-        const unsigned long long v = h[c * 8 + i];
-        if (v < t0) continue;
-        const double d = (double)(v - t0) * 1e-3;
-        mn = d < mn ? d : mn; mx = d > mx ? d : mx; sum += d; ++n;
-      }
-      if (n) fprintf(stderr, "  %-14s n %3d  %7.2f %7.2f %7.2f\n", names[i], n, mn, sum / n, mx);
-    }
-    static unsigned long long z[160 * 8];
-    cudaMemcpyToSymbol(g_gemm_prof, z, sizeof(z));
-  }
-#endif
   return SL_OK;
 }
 

@@ -152,3 +152,10 @@ def kl_logit_pairs(rows: int, vocab: int, seed: int, dtype=torch.bfloat16, devic
     prev_r[same] = cur_r[same]
     mask_state = (torch.rand(rows, generator=g, device=device) < 0.5).to(torch.uint8)
     return cur_r, prev_r, mask_state
+
+
+def selection_scores(B: int, N: int, step: int, seed: int, device="cpu") -> torch.Tensor:
+    """Seeded uniform scores [B][N] float32 for the selection surrogate of Experiment 5 (which positions a selection
+    method would skip in this step is that method's business; the surrogate ranks positions by these scores).  Drawn
+    on the CPU so that every consumer sees the same numbers, then moved to `device`."""
+    return torch.rand((B, N), generator=_gen(seed * 1000003 + step), dtype=torch.float32).to(device)

@@ -18,6 +18,7 @@ from typing import Dict
 import torch
 
 from . import binding as SL
+from . import inputs
 
 
 def algorithmic_flops_per_step(cfg: Dict, B: int, N: int) -> int:
@@ -28,12 +29,13 @@ def algorithmic_flops_per_step(cfg: Dict, B: int, N: int) -> int:
 
 def selection_skip_mask(lock: torch.Tensor, mask_state: torch.Tensor, fraction: float, step: int, seed: int):
     """Surrogate of a selection-based method (Experiment 5): compute only a fixed `fraction` of the positions that are
-    not locked.  Which ones is the selection method's business; this surrogate draws them with a seeded generator,
-    per sequence, and never skips a masked position (the sampler needs its posterior).  Returns uint8 [B][N], 1 = skip
-    this step.  Device arithmetic on the lock mask only; the step itself is unchanged."""
+    not locked.  Which ones is the selection method's business; this surrogate ranks them by seeded scores
+    (`inputs.selection_scores`), per sequence, and never skips a masked position (the sampler needs its posterior):
+    of the eligible positions (unlocked and unmasked) the floor((1 - fraction) * unlocked) with the lowest scores are
+    skipped, fewer when there are not that many.  Returns uint8 [B][N], 1 = skip this step.  This is harness code
+    (torch operations on the lock mask, outside the library): the step itself is unchanged."""
     B, N = lock.shape
-    g = torch.Generator(device=lock.device).manual_seed(seed * 1000003 + step)
-    score = torch.rand((B, N), generator=g, device=lock.device)
+    score = inputs.selection_scores(B, N, step, seed, device=lock.device)
     eligible = (lock == 0) & (mask_state == 0)                       # may be skipped
     n_unlocked = (lock == 0).sum(dim=1, keepdim=True)
     n_skip = torch.minimum(torch.floor(n_unlocked * (1.0 - fraction)).long(), eligible.sum(dim=1, keepdim=True))
@@ -44,13 +46,17 @@ def selection_skip_mask(lock: torch.Tensor, mask_state: torch.Tensor, fraction: 
 
 def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: int, block_len: int, steps: int,
         kl_eps: float, surelock: bool = True, unmask_per_step: int = 1, select_fraction: float = None,
-        select_seed: int = 0) -> Dict:
+        select_seed: int = 0, observer=None) -> Dict:
     """Run `steps` diffusion steps on device tensors tokens int32 [B][N], mask_state uint8 [B][N] (both updated in
     place).  Generation positions n_prompt.. are decoded block by block (`block_len` positions, `steps_per_block` =
     ceil(block_len / unmask_per_step) steps each).  `select_fraction` (Experiment 5, e.g. 0.8) adds the selection
     surrogate: every step only that fraction of the not-yet-locked positions is computed; with `surelock` this is the
     paper's combination, without it the selection baseline.  A skipped row keeps its cached K/V; it has no posterior in
     that step, so it cannot lock in the step in which it returns (D needs the previous step's posterior).
+    `observer`, when given, is called after every step, before the unmasking of line 16, as
+    observer(t, out, lock_in, lock_out, tokens, mask_state) with lock_in a copy of the lock mask the step was given
+    (skip mask included) and lock_out the mask after the step; it is for tests that look at a step from outside and
+    makes the loop wait for the GPU.
     Returns the trace and the paper's metrics."""
     B, N = tokens.shape
     dev = tokens.device
@@ -66,12 +72,16 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
     ev[0].record()
     for t in range(steps):
         if select_fraction is None:
+            lock_in = lock.clone() if observer is not None else None
             out = SL.surelock_step(ctx, tokens, mask_state, lock, kl_eps)
         else:
             skip = selection_skip_mask(lock, mask_state, select_fraction, t, select_seed)
             step_lock = lock | skip                                          # skipped rows are simply not active
+            lock_in = step_lock.clone() if observer is not None else None
             out = SL.surelock_step(ctx, tokens, mask_state, step_lock, kl_eps)
             lock |= step_lock & (skip ^ 1)                                   # new locks come from computed rows only
+        if observer is not None:
+            observer(t, out, lock_in, lock, tokens, mask_state)
         if not surelock:
             lock.zero_()                                                     # baseline sampler: nothing stays locked
         m_trace[t:t + 1] = out.n_active

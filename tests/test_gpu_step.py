@@ -331,3 +331,31 @@ def test_cache_check_flags_a_locked_position_without_keys_and_values():
     SL.surelock_state_import(other, state)
     SL.surelock_step(other, tok_d, mask_d, lock, eps)
     assert SL.surelock_status_poll(other) == 0
+
+
+def test_cuda_core_fallback_is_counted_and_can_be_refused():
+    """A bf16 shape the tensor-core kernels do not take (d_ff not a multiple of 8 elements is refused at init, so the
+    case here is a head count whose hidden width is not a multiple of 256: the fused QKV launch declines) runs on the
+    CUDA-core kernels and is counted; with "strict_tc" the step reports SL_EUNSUPPORTED instead.  The shapes of the
+    benchmark configurations never fall back."""
+    cfg = inputs.model_shape("tiny", d_model=192, n_heads=3, head_dim=64, d_ff=512, vocab=1024)
+    w = to_dev(inputs.make_weights(cfg, 41, dtype=torch.bfloat16, std=0.05))
+    B, N = 2, 64
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, 32, cfg["vocab"], 41)
+    lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
+    SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, 1e-3)
+    assert SL.surelock_status_poll(ctx) == 0
+    assert SL.surelock_last_fallback_count(ctx) == cfg["n_layers"]            # the fused QKV launch of every layer
+    SL.surelock_reset(ctx)
+    assert SL.surelock_last_fallback_count(ctx) == 0
+    SL.surelock_set_option(ctx, "strict_tc", 1)
+    with pytest.raises(SL.SurelockError, match="not supported"):
+        SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), lock, 1e-3)
+    # a shape every tensor-core kernel takes never falls back
+    cfg2 = inputs.model_shape("tiny")
+    ctx2 = SL.surelock_init(cfg2, to_dev(inputs.make_weights(cfg2, 42, dtype=torch.bfloat16)), N, B)
+    SL.surelock_set_option(ctx2, "strict_tc", 1)
+    tokens2, mask2 = inputs.make_tokens(B, N, 32, cfg2["vocab"], 42)
+    SL.surelock_step(ctx2, tokens2.to(DEV), mask2.to(DEV), lock, 1e-3)
+    assert SL.surelock_status_poll(ctx2) == 0 and SL.surelock_last_fallback_count(ctx2) == 0

@@ -34,8 +34,24 @@ def _np_layer(lw):
     return {k: v.detach().to("cpu", torch.float32).numpy() for k, v in lw.items()}
 
 
+def tile_covering_sample(r0, r1, n_rows, rng):
+    """Rows (relative to r0) of the packed range [r0, r1) of one sequence: one seeded row out of every 128-row tile of
+    the GLOBAL packed order that the range touches (the GEMMs' row tiles; every second one is the peer CTA of a
+    256-row pair tile), one out of every 128-row tile counted from r0 (the attention kernel's query tiles), the first
+    and the last row, and seeded extra rows up to n_rows."""
+    rows = {0, r1 - r0 - 1}
+    for t in range(r0 // 128, (r1 - 1) // 128 + 1):
+        lo, hi = max(t * 128, r0), min((t + 1) * 128, r1)
+        rows.add(int(rng.integers(lo, hi)) - r0)
+    for lo in range(0, r1 - r0, 128):
+        rows.add(int(rng.integers(lo, min(lo + 128, r1 - r0))))
+    while len(rows) < min(n_rows, r1 - r0):
+        rows.add(int(rng.integers(0, r1 - r0)))
+    return np.array(sorted(rows), dtype=np.int64)
+
+
 def _check_step(cfg, w_dev, ctx, out, lock_in, mask, kl_eps, prev_logits_view, prev_row_of_pos, layers, seqs, n_rows,
-                seed, lock_after):
+                seed, lock_after, tokens=None):
     oc = O.ModelCfg(**cfg)
     B, N, L = ctx.B, ctx.N, cfg["n_layers"]
     idx, offs = O.active_set(lock_in.numpy())
@@ -50,7 +66,14 @@ def _check_step(cfg, w_dev, ctx, out, lock_in, mask, kl_eps, prev_logits_view, p
     for b in seqs:
         r0, r1 = int(offs[b]), int(offs[b + 1])
         if r1 > r0:
-            sample_rows[b] = np.sort(rng.choice(r1 - r0, size=min(n_rows, r1 - r0), replace=False))
+            sample_rows[b] = tile_covering_sample(r0, r1, n_rows, rng)
+    if tokens is not None:
+        # the block input of the first layer is the embedding of the active rows' tokens (Algorithm 1 line 7): a copy,
+        # compared bit for bit (the fp32 stream holds the bf16 table entry widened: its bits shifted left by 16)
+        emb_bits = w_dev["tok_emb"].view(torch.int16).cpu().numpy().astype(np.int32)
+        tok = tokens.cpu().numpy().reshape(-1)
+        got = trace[0, :M].view(torch.int32).cpu().numpy()
+        assert np.array_equal(got, emb_bits[tok[idx]] << 16)
     for l in layers:
         lw = _np_layer(w_dev["layers"][l])
         kg, vg = SL.surelock_kv_cache(ctx, l)
@@ -110,7 +133,7 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     l0 = lock0.to(DEV)
     out0 = SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), l0, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
-    w0 = _check_step(cfg, w_dev, ctx, out0, lock0, mask, 1e-3, None, None, layers, seqs, n_rows, seed, l0)
+    w0 = _check_step(cfg, w_dev, ctx, out0, lock0, mask, 1e-3, None, None, layers, seqs, n_rows, seed, l0, tokens=tokens)
     assert not l0.any()                                              # first step: D = inf, nothing locks
     prev_rop = np.arange(B * N, dtype=np.int64)                      # step 0 packed every position in order
     snap = [[t.clone() for t in SL.surelock_kv_cache(ctx, l)] for l in layers]
@@ -125,7 +148,8 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     l1 = lock1.to(DEV)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
-    w1 = _check_step(cfg, w_dev, ctx, out1, lock1, mask2, 1e-3, out0.logits, prev_rop, layers, seqs, n_rows, seed + 7, l1)
+    w1 = _check_step(cfg, w_dev, ctx, out1, lock1, mask2, 1e-3, out0.logits, prev_rop, layers, seqs, n_rows, seed + 7, l1,
+                     tokens=tok2)
     locked = lock1.reshape(-1).bool().to(DEV)
     for i, l in enumerate(layers):                                   # frozen rows: bytes unchanged by the second step
         k, v = SL.surelock_kv_cache(ctx, l)
@@ -152,7 +176,7 @@ def test_llada8b_full_size_sampled():
     cfg = inputs.model_shape("llada8b")
     B, N = 8, 1536
     na = [int(N * 0.5 * f) for f in (1.3, 0.7, 1.0, 0.9, 1.25, 0.75, 1.1, 1.0)]
-    w0, w1 = _two_steps(cfg, B=B, N=N, n_prompt=512, n_active=na, seed=33, layers=[0, 13, 31], seqs=[0, 5], n_rows=10,
+    w0, w1 = _two_steps(cfg, B=B, N=N, n_prompt=512, n_active=na, seed=33, layers=[0, 13, 31], seqs=[0, 5], n_rows=16,
                         w_device=DEV)
     print("worst stage errors, full size:", w0, w1)
 

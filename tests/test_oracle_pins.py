@@ -747,3 +747,20 @@ def test_unlock_cycle_by_hand_cool_down_and_stricter_relock():
     exact0 = r["kl"][rows] <= e_rows[0, freed]
     assert np.array_equal(r["new_lock"][0, freed].astype(bool), exact0)
     assert np.array_equal(O.sure_test(np.array([1e-31, 1e-4]), np.zeros(2), np.array([1e-33, 1e-3])), [False, True])
+
+
+def test_selection_skip_rule_by_hand():
+    """The selection surrogate's rule on a hand case: floor(0.2 * unlocked) eligible positions with the lowest scores,
+    never a locked or a masked one, ties to the lower position, capped by the number of eligible positions."""
+    lock = np.array([[0, 0, 1, 0, 0, 0, 0, 0, 0, 0, 0], [0, 0, 0, 0, 0, 1, 1, 1, 1, 1, 1]], np.uint8)
+    mask = np.array([[0, 0, 0, 1, 0, 0, 0, 0, 0, 0, 0], [1, 1, 1, 1, 0, 0, 0, 0, 0, 0, 0]], np.uint8)
+    sc = np.array([[.5, .1, .0, .0, .3, .1, .9, .8, .7, .6, .4], [.1, .2, .3, .4, .9, .0, .0, .0, .0, .0, .0]], np.float32)
+    skip = O.selection_skip(lock, mask, sc, 0.8)
+    # sequence 0: 10 unlocked -> 2 skipped: scores .1 at positions 1 and 5 (position 2 is locked, 3 masked)
+    # sequence 1: 5 unlocked -> 1 skipped: the only eligible position is 4
+    assert skip.tolist() == [[0, 1, 0, 0, 0, 1, 0, 0, 0, 0, 0], [0, 0, 0, 0, 1, 0, 0, 0, 0, 0, 0]]
+    assert O.selection_skip(lock, mask, sc, 1.0).sum() == 0
+    mask[1, 4] = 1
+    assert O.selection_skip(lock, mask, sc, 0.5)[1].sum() == 0        # nothing eligible
+    # sequence 0 at k = 0.5: 5 of the eligible scores .5 .1 .3 .1 .9 .8 .7 .6 .4 -> .1 .1 .3 .4 .5
+    assert O.selection_skip(lock, mask, sc, 0.5)[0].tolist() == [1, 1, 0, 0, 1, 1, 0, 0, 0, 0, 1]

@@ -58,3 +58,24 @@ def test_noalloc_compaction_rejects_sizes_beyond_its_capacity():
     i32 = torch.zeros(16, dtype=torch.int32, device=DEV)
     with pytest.raises(SL.SurelockError, match="capacity"):
         SL.surelock_compact_noalloc(one, B, N, i32, i32, i32, None, None)
+
+
+def test_noalloc_compaction_takes_no_device_memory():
+    """The property in the name: after a warm-up call (which also fetches the array's address), further calls leave
+    the amount of free device memory exactly where it was."""
+    g = torch.Generator().manual_seed(78)
+    lock = (torch.rand((4, 30000), generator=g) < 0.5).to(torch.uint8).to(DEV)
+    B, N = lock.shape
+    idx = torch.empty(B * N, dtype=torch.int32, device=DEV)
+    offs = torch.empty(B + 1, dtype=torch.int32, device=DEV)
+    n = torch.empty(1, dtype=torch.int32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    SL.surelock_compact_noalloc(lock, B, N, idx, offs, n, None, status)          # warm-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        SL.surelock_compact_noalloc(lock, B, N, idx, offs, n, None, status)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0 and status.item() == 0
+    assert int(n.item()) == int((lock == 0).sum())
