@@ -100,7 +100,10 @@ int surelock_reset(surelock_ctx *ctx);
  *                                  Locking a row whose cache entries were never written is the caller's error.
  *   kl_eps      threshold eps >= 0 (not NaN)
  *   out         host struct filled with dev pointers (may be NULL)
- * Asynchronous; performs no allocation and no host synchronisation. */
+ * Asynchronous; performs no allocation and never waits for the work it enqueues, nor for the previous step's.  (It
+ * does wait for the step BEFORE the previous one to have finished, whose row count M, copied to the host, serves as
+ * the upper bound of this step's M from which launch configurations are chosen: the host can run two steps ahead of
+ * the GPU.  The bound affects speed only: every kernel reads M itself from device memory.) */
 int surelock_step(surelock_ctx *ctx, const int32_t *tokens, const uint8_t *mask_state, uint8_t *lock_mask,
                   float kl_eps, surelock_step_out *out);
 
@@ -178,7 +181,11 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * surelock_kv_cache()); 0 = off (default).  A violation stores device status 5 and the step goes on; one small kernel
  * per step, one flag byte per position (allocated here).  surelock_reset() invalidates all positions,
  * surelock_state_import() validates all.  surelock_layer_step() neither checks nor marks.
- * Unknown names return SL_EINVAL. */
+ *  "row_bound": v > 0 = the caller's
+ * upper bound of the number of active rows of later steps, used instead of the automatic one (the row count two steps
+ * back) when kernels and launch configurations are chosen; a bound that is too small costs time, never correctness
+ * (with at most 128 rows the contractions run on a weight-streaming kernel that then makes several passes); 0 = automatic
+ * (default).  Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
 /* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [2L+1][B*N][d] (rows packed as in
@@ -301,7 +308,8 @@ size_t surelock_gemm_workspace_bytes(void);
 /* Dense contraction on packed rows, C[r][n] = sum_k A[r][k] * W[n][k] for r < *n_active (the projections of
  * Algorithm 1 lines 10, 12, 15; FLOP terms of Sec. 2.3).  A: dev [M][K]; W: dev [n_out][K]; C: dev [M][n_out];
  * A, W, C of `dtype`; fp32 accumulation.  impl: 0 = best available (tcgen05 tensor cores for SL_BF16 when the
- * shape allows), 1 = force the CUDA-core kernel.
+ * shape allows), 1 = force the CUDA-core kernel.  With max_rows <= 128 (few rows: the contraction is bound by reading W
+ * once) impl 0 runs the weight-streaming kernel, which needs no workspace.
  * workspace: dev, surelock_gemm_workspace_bytes() bytes, ZERO-FILLED by the caller before its first use (the kernel
  * leaves it reusable, unless it gave up on a bounded wait: after device status 2 zero-fill it again), or NULL.  With a workspace and few output tiles (small M) the tensor-core kernel splits K
  * across SMs and sums the partial tiles in a fixed order (deterministic); without one it never splits.

@@ -38,6 +38,18 @@ struct surelock_ctx {
   bool strict_tc = false;             // refuse (SL_EUNSUPPORTED) instead of falling back to the CUDA-core kernels
   int fallbacks = 0;                  // launches that fell back since the last reset
   int32_t* n_prev = nullptr;          // rows of the previous step's logits (copy of n_active taken at the end of a step)
+  // Upper bound of M for choosing launch configurations on the host (M itself stays in device memory).  Every step
+  // copies its row count into a page-locked word and records an event; a step first waits for the event of the step
+  // BEFORE THE PREVIOUS ONE (normally long complete: the host may run two steps ahead, not more) and takes that count
+  // as the bound: lock masks normally only grow, so the count two steps ago bounds this step's.  Always the same
+  // step's count, whatever the timing, so that the choice of kernels, and with it every bit of the results, is
+  // reproducible.  A bound that turns out too small only costs time (the kernels stay correct for any M).
+  int32_t* h_m = nullptr;             // page-locked [2]
+  cudaEvent_t ev_m[2] = {nullptr, nullptr};
+  bool ev_m_valid[2] = {false, false};
+  long long calls = 0;                // steps / layer steps since the last reset
+  int row_bound_opt = 0;              // "row_bound" option: > 0 = the caller's bound, used instead
+  int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
   bool timing = false;                // per-kernel-class CUDA-event timing (off by default)
   std::vector<cudaEvent_t> ev;        // event pool, created when timing is switched on
@@ -101,6 +113,12 @@ static inline void tock(surelock_ctx* c) {
   } while (0)
 
 namespace sl {
+int launch_gemm_stream(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
+                       int m_bound, int n_out, int K, int epilogue, int32_t* status, bool prefetch_w, cudaStream_t st);   // gemm_stream.cu
+int launch_gemm_stream_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
+                           void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
+                           int m_bound, int n_seq, int hd, int dh, int K, int32_t* status, bool prefetch_w,
+                           cudaStream_t st);                                                                          // gemm_stream.cu
 int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const int32_t* n_active, int max_rows,
                    int n_out, int K, int epilogue, int32_t* status, const SplitWs& sw, cudaStream_t st);   // gemm_tc.cu; SL_EUNSUPPORTED if the shape does not fit
 int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
@@ -122,8 +140,36 @@ static int attention(surelock_ctx* c, int l) {
                                c->attn, g.dtype, c->st);
 }
 
+// the bound on M for this call (see surelock_ctx::h_m)
+static int begin_call(surelock_ctx* c) {
+  const int slot = (int)(c->calls & 1);
+  c->m_bound = c->R;
+  if (c->ev_m_valid[slot]) {
+    SL_CUDA_TRY(cudaEventSynchronize(c->ev_m[slot]));
+    if (c->h_m[slot] >= 0 && c->h_m[slot] <= c->R) c->m_bound = c->h_m[slot];
+  }
+  if (c->row_bound_opt > 0) c->m_bound = c->row_bound_opt < c->R ? c->row_bound_opt : c->R;
+  return SL_OK;
+}
+static int end_call(surelock_ctx* c) {
+  const int slot = (int)(c->calls & 1);
+  SL_CUDA_TRY(cudaMemcpyAsync(&c->h_m[slot], c->n_active, 4, cudaMemcpyDeviceToHost, c->st));
+  SL_CUDA_TRY(cudaEventRecord(c->ev_m[slot], c->st));
+  c->ev_m_valid[slot] = true;
+  ++c->calls;
+  return SL_OK;
+}
+static inline bool use_stream(const surelock_ctx* c) {
+  return c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 && c->m_bound <= 128;
+}
+
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
   c->last_gemm_tc = false;
+  if (use_stream(c)) {
+    const int rc = launch_gemm_stream(A, W, W2, C, c->n_active, c->R, c->m_bound, n_out, K, epi, c->status,
+                                      c->split.prefetch_w, c->st);
+    if (rc != SL_EUNSUPPORTED) return rc;          // (the weight-streaming kernel leaves no softmax statistics)
+  }
   if (c->cfg.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_gemm_tc(A, W, W2, C, c->n_active, c->R, n_out, K, epi, c->status, c->split, c->st);
     c->last_gemm_tc = rc == SL_OK;
@@ -142,8 +188,14 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
     // one launch: Q, K, V projections + RoPE + K/V written straight into the cache rows of the active positions
     tick(c, K_GEMM_QKV);
-    const int rc = launch_gemm_tc_qkv(c->h, c->wq[l], c->wk[l], c->wv[l], c->q, c->kcache(l), c->vcache(l), c->idx, c->rope,
-                                      c->n_active, c->R, c->N, hd, g.head_dim, d, c->status, c->split, c->st);
+    int rc = SL_EUNSUPPORTED;
+    if (use_stream(c))
+      rc = launch_gemm_stream_qkv(c->h, c->wq[l], c->wk[l], c->wv[l], c->q, c->kcache(l), c->vcache(l), c->idx, c->rope,
+                                  c->n_active, c->R, c->m_bound, c->N, hd, g.head_dim, d, c->status, c->split.prefetch_w,
+                                  c->st);
+    if (rc == SL_EUNSUPPORTED)
+      rc = launch_gemm_tc_qkv(c->h, c->wq[l], c->wk[l], c->wv[l], c->q, c->kcache(l), c->vcache(l), c->idx, c->rope,
+                              c->n_active, c->R, c->N, hd, g.head_dim, d, c->status, c->split, c->st);
     if (rc == SL_OK) {
       tock(c);
       fused = true;
@@ -255,6 +307,9 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     A_(c->lse_valid, 16);
     if (rc == SL_OK && cudaMemsetAsync(c->lse_valid, 0, 16, c->st) != cudaSuccess) rc = SL_ECUDA;
   }
+  if (rc == SL_OK && cudaMallocHost(reinterpret_cast<void**>(&c->h_m), 2 * sizeof(int32_t)) != cudaSuccess) rc = SL_ENOMEM;
+  for (int i = 0; i < 2 && rc == SL_OK; ++i)
+    if (cudaEventCreateWithFlags(&c->ev_m[i], cudaEventDisableTiming) != cudaSuccess) rc = SL_ECUDA;
   A_(c->theta, ((size_t)batch + 1) * 4);
   A_(c->st_tokens, R * 4);
   A_(c->st_mask, R);
@@ -276,6 +331,8 @@ int surelock_reset(surelock_ctx* c) {
   if (!c) return SL_EINVAL;
   c->have_prev = false;
   c->cur = 0;
+  c->calls = 0;
+  c->ev_m_valid[0] = c->ev_m_valid[1] = false;
   for (int i = 0; i < 2; ++i) SL_CUDA_TRY(cudaMemsetAsync(c->row_of_pos[i], 0xff, (size_t)c->R * 4, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->status, 0, 16, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->n_active, 0, 16, c->st));
@@ -298,6 +355,7 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   c->launches = 0;
   const int cur = c->cur, prv = cur ^ 1;
   c->n_ev = 0;
+  SL_TRY(begin_call(c));
   if (c->check_cache) SL_K(K_COMPACT, launch_cache_check(lock_mask, c->kv_valid, c->R, c->status, c->st));
   SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur],
                                  c->scratch, c->status, c->st));
@@ -339,6 +397,7 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   }
   // the row count of the logits the next step reads as "previous" (n_active itself is overwritten by other calls)
   SL_CUDA_TRY(cudaMemcpyAsync(c->n_prev, c->n_active, 4, cudaMemcpyDeviceToDevice, c->st));
+  SL_TRY(end_call(c));
   c->cur = prv;
   c->have_prev = true;
   return SL_OK;
@@ -369,11 +428,13 @@ int surelock_layer_step(surelock_ctx* c, int layer, const void* hidden_in, const
   const surelock_model_cfg& g = c->cfg;
   c->launches = 0;
   c->n_ev = 0;
+  SL_TRY(begin_call(c));
   SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, nullptr, c->scratch,
                                  c->status, c->st));
   SL_K(K_GATHER, launch_gather_rows(hidden_in, nullptr, c->idx, c->n_active, c->R, g.d_model, c->R, hidden_out, g.dtype,
                                     c->status, c->st));
   SL_TRY(run_layer(c, layer, hidden_out));
+  SL_TRY(end_call(c));
   if (out) {
     memset(out, 0, sizeof(*out));
     out->active_idx = c->idx;
@@ -497,6 +558,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
+  if (!strcmp(name, "row_bound")) { c->row_bound_opt = value > 0 ? value : 0; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
   if (!strcmp(name, "check_cache")) {
     if (value && !c->kv_valid) {
@@ -571,6 +633,9 @@ void surelock_destroy(surelock_ctx* c) {
   if (!c) return;
   cudaStreamSynchronize(c->st);
   for (cudaEvent_t e : c->ev) cudaEventDestroy(e);
+  for (int i = 0; i < 2; ++i)
+    if (c->ev_m[i]) cudaEventDestroy(c->ev_m[i]);
+  if (c->h_m) cudaFreeHost(c->h_m);
   for (void* p : c->allocs) cudaFree(p);
   delete c;
 }
@@ -652,6 +717,12 @@ int surelock_gemm_fused(const void* A, const void* W, const void* W2, void* C, c
   if (epilogue != EPI_STORE && epilogue != EPI_RESIDUAL && epilogue != EPI_SWIGLU) return SL_EINVAL;
   if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
   if (epilogue != EPI_SWIGLU) W2 = nullptr;
+  if (dtype == SL_BF16 && impl == 0 && max_rows >= 1 && max_rows <= 128) {
+    // few rows: the weight-streaming kernel (needs no workspace)
+    const int rc = launch_gemm_stream(A, W, W2, C, n_active, max_rows, max_rows, n_out, K, epilogue, dev_status, false,
+                                      (cudaStream_t)stream);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
   if (dtype == SL_BF16 && impl == 0) {
     SplitWs sw;
     if (workspace) {

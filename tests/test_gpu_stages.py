@@ -382,3 +382,42 @@ def test_conf_gate_lock(B, N, m):
     assert np.array_equal(got[~near], want[~near])
     assert np.array_equal(new[lock.numpy() == 1], lock.numpy()[lock.numpy() == 1])   # locked rows stay locked
     assert not got[~cand].any()
+
+
+@pytest.mark.parametrize("epi", [0, 1, 2])
+@pytest.mark.parametrize("M,n_out,K", [(1, 256, 256), (7, 4096, 4096), (23, 4096, 12288), (32, 12288, 4096), (33, 4096, 4096),
+                                       (64, 1024, 8192), (103, 4096, 4096), (128, 4096, 12288), (16, 136, 200), (0, 256, 512)])
+def test_gemm_weight_streaming_few_rows(M, n_out, K, epi):
+    """The weight-streaming (swapped-operand) kernel, taken when the matrix of activations has at most 128 rows: every
+    row padding (16 / 32 / 64 / 128), cluster sizes 1 ... 8 (K split through distributed shared memory), one and several
+    32-row reduction chunks, a ragged feature tile, all three fused epilogues; rows beyond M untouched, two runs give
+    the same bits."""
+    g = torch.Generator().manual_seed(M * 17 + K + epi)
+    cap = max(M, 1)
+    A = torch.randn((cap, K), generator=g).to(torch.bfloat16)
+    W = (torch.randn((n_out, K), generator=g) * 0.05).to(torch.bfloat16)
+    W2 = (torch.randn((n_out, K), generator=g) * 0.05).to(torch.bfloat16) if epi == 2 else None
+    x0 = torch.randn((cap, n_out), generator=g)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    Ad, Wd, n = A.to(DEV), W.to(DEV), torch.tensor([M], dtype=torch.int32, device=DEV)
+    W2d = W2.to(DEV) if W2 is not None else None
+    outs = []
+    for _ in range(2):
+        out = x0.to(DEV) if epi == 1 else torch.full((cap, n_out), 3.0, dtype=torch.bfloat16, device=DEV)
+        SL.surelock_gemm_fused(Ad, Wd, W2d, out, n, epi, impl=0, dev_status=status)
+        torch.cuda.synchronize()
+        outs.append(out)
+    assert status.item() == 0
+    out = outs[0]
+    if M:
+        acc = f64(A[:M]) @ f64(W).T
+        ref = acc if epi == 0 else (f64(x0[:M]) + acc if epi == 1 else O.silu(acc) * (f64(A[:M]) @ f64(W2).T))
+        assert rel_err_rows(f64(out[:M]), ref) < 2e-2
+        if epi == 1:
+            assert np.abs(f64(out[:M]) - ref).max() < 1e-3 * (1 + np.abs(ref).max())
+    if epi == 1:
+        assert torch.equal(out[M:].cpu(), x0[M:])
+        assert torch.equal(outs[0].view(torch.int32), outs[1].view(torch.int32))
+    else:
+        assert (out[M:] == 3.0).all()
+        assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))

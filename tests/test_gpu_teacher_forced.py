@@ -123,7 +123,7 @@ def _check_step(cfg, w_dev, ctx, out, lock_in, mask, kl_eps, prev_logits_view, p
 
 
 def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.02, w_device="cpu",
-               lock_fn=inputs.random_lock):
+               lock_fn=inputs.random_lock, row_bound_after_first=0):
     w = inputs.make_weights(cfg, seed, dtype=torch.bfloat16, std=std, device=w_device)
     w_dev = w if w_device != "cpu" else to_dev(w)
     ctx = SL.surelock_init(cfg, w_dev, N, B)
@@ -146,6 +146,8 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     mask2[:, n_prompt:n_prompt + 8] = 0
     lock1 = lock_fn(B, N, n_active, seed + 1)
     l1 = lock1.to(DEV)
+    if row_bound_after_first:
+        SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
     w1 = _check_step(cfg, w_dev, ctx, out1, lock1, mask2, 1e-3, out0.logits, prev_rop, layers, seqs, n_rows, seed + 7, l1,
@@ -201,3 +203,15 @@ def test_single_sequence_few_active_rows(n_active):
     w0, w1 = _two_steps(cfg, B=1, N=512, n_prompt=128, n_active=n_active, seed=50 + n_active[0], layers=[0, 1], seqs=[0],
                         n_rows=12, w_device=DEV)
     print("worst stage errors, single sequence:", n_active, w0, w1)
+
+
+@pytest.mark.parametrize("n_active,bound", [([23], 23), ([103], 128), ([60], 16), ([9, 1, 14], 32)])
+def test_weight_streaming_step_with_a_row_bound(n_active, bound):
+    """The step with the "row_bound" option set, so that already the second step (M <= 128) runs every contraction
+    (fused QKV with rotary embedding and cache scatter, output projection, SwiGLU, down projection, LM head) on the
+    weight-streaming kernel; bound 16 with 60 active rows makes that kernel take four passes over the weights."""
+    cfg = inputs.model_shape("llada8b", n_layers=2, vocab=8192)
+    B = len(n_active)
+    w0, w1 = _two_steps(cfg, B=B, N=512, n_prompt=128, n_active=n_active, seed=90 + n_active[0], layers=[0, 1],
+                        seqs=list(range(B)), n_rows=12, w_device=DEV, row_bound_after_first=bound)
+    print("worst stage errors, weight streaming:", n_active, bound, w0, w1)
