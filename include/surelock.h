@@ -181,11 +181,12 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * surelock_kv_cache()); 0 = off (default).  A violation stores device status 5 and the step goes on; one small kernel
  * per step, one flag byte per position (allocated here).  surelock_reset() invalidates all positions,
  * surelock_state_import() validates all.  surelock_layer_step() neither checks nor marks.
- *  "row_bound": v > 0 = the caller's
- * upper bound of the number of active rows of later steps, used instead of the automatic one (the row count two steps
- * back) when kernels and launch configurations are chosen; a bound that is too small costs time, never correctness
- * (with at most 128 rows the contractions run on a weight-streaming kernel that then makes several passes); 0 = automatic
- * (default).  Unknown names return SL_EINVAL. */
+ *  "gemm_stream": 1 = steps whose bound on the number of
+ * active rows is at most 128 run their contractions on the weight-streaming kernel (see surelock_gemm, impl 2); 0
+ * (default) = always the general kernel, which measured as fast or faster inside a step.  "row_bound": v > 0 = the
+ * caller's upper bound of the number of active rows of later steps, used instead of the automatic one (the row count
+ * two steps back); a bound that is too small costs time, never correctness (the weight-streaming kernel then makes
+ * several passes over the weights); 0 = automatic (default).  Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
 /* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [2L+1][B*N][d] (rows packed as in
@@ -308,8 +309,9 @@ size_t surelock_gemm_workspace_bytes(void);
 /* Dense contraction on packed rows, C[r][n] = sum_k A[r][k] * W[n][k] for r < *n_active (the projections of
  * Algorithm 1 lines 10, 12, 15; FLOP terms of Sec. 2.3).  A: dev [M][K]; W: dev [n_out][K]; C: dev [M][n_out];
  * A, W, C of `dtype`; fp32 accumulation.  impl: 0 = best available (tcgen05 tensor cores for SL_BF16 when the
- * shape allows), 1 = force the CUDA-core kernel.  With max_rows <= 128 (few rows: the contraction is bound by reading W
- * once) impl 0 runs the weight-streaming kernel, which needs no workspace.
+ * shape allows), 1 = force the CUDA-core kernel, 2 = the weight-streaming tensor-core kernel for few rows (SL_BF16 and
+ * max_rows <= 128 only, else SL_EUNSUPPORTED; weights on the 128-row side of the MMA, K split inside a thread-block
+ * cluster; needs no workspace).
  * workspace: dev, surelock_gemm_workspace_bytes() bytes, ZERO-FILLED by the caller before its first use (the kernel
  * leaves it reusable, unless it gave up on a bounded wait: after device status 2 zero-fill it again), or NULL.  With a workspace and few output tiles (small M) the tensor-core kernel splits K
  * across SMs and sums the partial tiles in a fixed order (deterministic); without one it never splits.

@@ -49,6 +49,7 @@ struct surelock_ctx {
   bool ev_m_valid[2] = {false, false};
   long long calls = 0;                // steps / layer steps since the last reset
   int row_bound_opt = 0;              // "row_bound" option: > 0 = the caller's bound, used instead
+  bool gemm_stream = false;           // "gemm_stream" option: contractions of at most 128 rows on the weight-streaming kernel
   int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
   bool timing = false;                // per-kernel-class CUDA-event timing (off by default)
@@ -160,7 +161,7 @@ static int end_call(surelock_ctx* c) {
   return SL_OK;
 }
 static inline bool use_stream(const surelock_ctx* c) {
-  return c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 && c->m_bound <= 128;
+  return c->gemm_stream && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 && c->m_bound <= 128;
 }
 
 static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, void* C, int n_out, int K, int epi) {
@@ -558,6 +559,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!c || !name) return SL_EINVAL;
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
+  if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
   if (!strcmp(name, "row_bound")) { c->row_bound_opt = value > 0 ? value : 0; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
   if (!strcmp(name, "check_cache")) {
@@ -717,12 +719,10 @@ int surelock_gemm_fused(const void* A, const void* W, const void* W2, void* C, c
   if (epilogue != EPI_STORE && epilogue != EPI_RESIDUAL && epilogue != EPI_SWIGLU) return SL_EINVAL;
   if (epilogue == EPI_SWIGLU && !W2) return SL_EINVAL;
   if (epilogue != EPI_SWIGLU) W2 = nullptr;
-  if (dtype == SL_BF16 && impl == 0 && max_rows >= 1 && max_rows <= 128) {
-    // few rows: the weight-streaming kernel (needs no workspace)
-    const int rc = launch_gemm_stream(A, W, W2, C, n_active, max_rows, max_rows, n_out, K, epilogue, dev_status, false,
-                                      (cudaStream_t)stream);
-    if (rc != SL_EUNSUPPORTED) return rc;
-  }
+  if (impl == 2)                                     // the weight-streaming kernel (bf16, at most 128 rows; no workspace)
+    return dtype == SL_BF16 ? launch_gemm_stream(A, W, W2, C, n_active, max_rows, max_rows, n_out, K, epilogue, dev_status,
+                                                 false, (cudaStream_t)stream)
+                            : SL_EUNSUPPORTED;
   if (dtype == SL_BF16 && impl == 0) {
     SplitWs sw;
     if (workspace) {

@@ -83,13 +83,14 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
 struct WsLayout {
   int stage_bytes, stages, red_off, red_bytes, bar_off, total;
 };
-__host__ __device__ inline WsLayout ws_layout(int nacc, int np, int stages) {
+__host__ __device__ inline WsLayout ws_layout(int nacc, int np, int stages, int S) {
   WsLayout l;
   l.stage_bytes = nacc * WS_W_BYTES + np * WS_BK * 2;
   l.stages = stages;
   l.red_off = stages * l.stage_bytes;
   const int cr = np < 32 ? np : 32;
-  l.red_bytes = nacc * cr * WS_BF * 4;          // [nacc][S][cr / S][128] floats
+  const int rpo = (cr + S - 1) / S;             // rows of a chunk one CTA finishes (the last CTAs may have fewer)
+  l.red_bytes = nacc * S * rpo * WS_BF * 4;     // [nacc][S][rpo][128] floats
   l.bar_off = l.red_off + l.red_bytes;
   l.total = l.bar_off + 512;
   return l;
@@ -104,7 +105,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   constexpr int NACC = EPI == EPI_SWIGLU ? 2 : 1;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  const WsLayout L = ws_layout(NACC, np, stages);
+  const WsLayout L = ws_layout(NACC, np, stages, S);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L.bar_off);
   // bars: full[stages], empty[stages], acc_full, acc_empty, red_full, red_free
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * stages + 4);
@@ -117,10 +118,15 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
                  rede_bar = accf_bar + 24u;
 
   // Inside a step neither the weights nor *n_active were written by the kernel launched just before this one
-  // (prefetch_w): the successor may launch at once and the weight copies start before the predecessor has completed.
-  // Otherwise nothing is read before it has.
+  // (prefetch_w): the weight copies start before the predecessor has completed, and the successor may launch as soon
+  // as every CTA of this kernel has its tensor memory.  Otherwise nothing is read before the predecessor has completed.
+  if (threadIdx.x == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmX) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW0) : "memory");
+    if (EPI == EPI_SWIGLU || EPI == WS_EPI_QKV) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW1) : "memory");
+    if (EPI == WS_EPI_QKV) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW2) : "memory");
+  }
   if (!prefetch_w) griddep_wait();
-  griddep_launch();
 
   const uint32_t rank = S > 1 ? cluster_ctarank() : 0u;
   const int tile = (int)blockIdx.x / S;
@@ -128,7 +134,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   const int num_kb = (K + WS_BK - 1) / WS_BK;
   const int kb0 = (int)rank * num_kb / S, kb1 = ((int)rank + 1) * num_kb / S;
   const int cr = np < 32 ? np : 32;             // rows per reduction chunk
-  const int rpo = cr / S;                       // rows of a chunk this CTA finishes
+  const int rpo = (cr + S - 1) / S;             // rows of a chunk a CTA finishes: CTA j rows [j * rpo, min(cr, (j + 1) * rpo))
   const int n_chunks = np / cr;
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < NACC * np) tmem_cols <<= 1;
@@ -146,7 +152,9 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     fence_mbar_init();
   }
   __syncthreads();
-  if (S > 1) cluster_sync_all();                // the peers' barriers exist before anything arrives on them
+  // the peers' barriers must exist before anything arrives on them: every thread arrives here, and the epilogue warps
+  // wait just before their first access to a peer, by which time the phase has long completed
+  if (S > 1) asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
 
   const int M = *n_active;
   const int n_pass = M > 0 ? (M + np - 1) / np : 0;     // 1 when the host's bound on M holds
@@ -202,6 +210,10 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
   } else if (warp == 1) {
     tc_alloc(smem_u32(s_tmem), tmem_cols);
+    // The successor may launch only now that this CTA holds its tensor memory: a successor CTA that shares the SM can
+    // then never take the columns this CTA still has to ask for (it would keep them until this kernel completes, and
+    // this kernel could not complete).
+    griddep_launch();
     tc_fence_before();
     asm volatile("bar.sync 2, 160;" ::: "memory");      // publishes the tensor-memory address to the epilogue warps
     tc_fence_after();
@@ -247,6 +259,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     const uint32_t red_u32 = smem_u32(red);
     bool ok = true;
     int ci = 0;                                          // chunks reduced so far (barrier phases)
+    if (S > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
     for (int p = 0; p < n_pass && ok; ++p) {
       ok = mbar_wait(accf_bar, (uint32_t)p & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
@@ -270,7 +283,7 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             tc_wait_ld();
 #pragma unroll
             for (int j = 0; j < 16; ++j) {
-              const int r = h + j, owner = r / rpo, rl = r - owner * rpo;
+              const int r = h + j, owner = r / rpo, rl = r - owner * rpo;   // owner < S because rpo = ceil(cr / S)
               const uint32_t off = (uint32_t)((((a * S + (int)rank) * rpo + rl) * WS_BF + f) * 4);
               if (S > 1) st_cluster_f32(mapa_u32(red_u32 + off, (uint32_t)owner), __uint_as_float(v[j]));
               else red[off >> 2] = __uint_as_float(v[j]);
@@ -293,7 +306,8 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           asm volatile("bar.sync 1, 128;" ::: "memory");
         }
         // ---- finish this CTA's rows of the chunk: sum the S contributions in split order, fused epilogue
-        for (int rl = 0; rl < rpo; ++rl) {
+        const int my_rows = min(rpo, cr - (int)rank * rpo);          // <= 0 for a CTA that owns no row of the chunk
+        for (int rl = 0; rl < my_rows; ++rl) {
           const int row = p * np + c * cr + (int)rank * rpo + rl;
           float acc[NACC];
 #pragma unroll
@@ -305,19 +319,20 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           if (EPI == WS_EPI_QKV) {
             const int src = n0 / qkv.hd, ln = n - src * qkv.hd;
             const bool live = row < M;
-            const int pos = live ? qkv.idx[row] : 0;
+            const int pos = live ? __ldg(qkv.idx + row) : 0;
             if (src == 2) {
               if (live) qkv.vc[(long long)pos * qkv.hd + ln] = __float2bfloat16_rn(acc[0]);
             } else {
               // rotary embedding: the partner of feature j of a head is j +- dh/2, a lane of another warp: exchange
               // the sums through this thread's own slot of the buffer
-              red[(0 * rpo + rl) * WS_BF + f] = acc[0];
-              asm volatile("bar.sync 1, 128;" ::: "memory");
               const int half = qkv.dh >> 1, j = f % qkv.dh;
               const bool lo = j < half;
-              const float other = red[(0 * rpo + rl) * WS_BF + (lo ? f + half : f - half)];
+              float2 cs = make_float2(1.f, 0.f);
+              if (live) cs = __ldg(qkv.rope + (long long)(pos % qkv.n_seq) * half + (lo ? j : j - half));
+              red[rl * WS_BF + f] = acc[0];
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+              const float other = red[rl * WS_BF + (lo ? f + half : f - half)];
               if (live) {
-                const float2 cs = __ldg(qkv.rope + (long long)(pos % qkv.n_seq) * half + (lo ? j : j - half));
                 const float o = lo ? acc[0] * cs.x - other * cs.y : acc[0] * cs.x + other * cs.y;
                 bf16* dst = src == 0 ? qkv.q + (long long)row * qkv.hd : qkv.kc + (long long)pos * qkv.hd;
                 dst[ln] = __float2bfloat16_rn(o);
@@ -325,8 +340,8 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
             }
           } else if (row < M && n < n_out) {
             if (EPI == EPI_RESIDUAL) {
-              float* dst = reinterpret_cast<float*>(Cv) + (long long)row * n_out + n;
-              *dst += acc[0];
+              // one add per element and launch, performed by the L2 (no load of x, so no latency chain): deterministic
+              atomicAdd(reinterpret_cast<float*>(Cv) + (long long)row * n_out + n, acc[0]);
             } else if (EPI == EPI_SWIGLU) {
               const float g = acc[0];
               reinterpret_cast<bf16*>(Cv)[(long long)row * n_out + n] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * acc[NACC - 1]);
@@ -346,11 +361,15 @@ gemm_stream_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     }
   }
 
+  __syncwarp();
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *s_abort) set_status(status, SL_DEV_GEMM_TIMEOUT);
   // nobody leaves while a peer may still write into its buffer or arrive on its barriers
-  if (S > 1) cluster_sync_all();
+  if (S > 1) {
+    if (warp < 2) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");   // completes the opening phase
+    cluster_sync_all();
+  }
   if (warp == 1) {                              // the epilogue warps have read the accumulators
     tc_fence_after();
     tc_dealloc(tmem_base, tmem_cols);
@@ -369,17 +388,20 @@ static WsPlan ws_plan(int epi, int m_bound, int n_out, int K) {
   p.np = m_bound <= 16 ? 16 : (m_bound <= 32 ? 32 : (m_bound <= 64 ? 64 : 128));
   const int nacc = epi == EPI_SWIGLU ? 2 : 1;
   const int tiles = (n_out + WS_BF - 1) / WS_BF, num_kb = (K + WS_BK - 1) / WS_BK;
-  const int cap = sm_count() * 13 / 5;
+  // K splits (cluster size): the power of two that brings the launch closest to two CTAs per SM without exceeding the
+  // CTAs that can be resident at once (a second wave of clusters costs more than idle SMs), at least four K blocks
+  // per CTA.  Measured on B200 at 32 rows: 96 feature tiles (Q/K/V, gate/up) S = 2, 32 tiles (output, down) S = 4 or 8.
   p.S = 1;
-  while (p.S < 8 && tiles * p.S * 2 <= cap && num_kb / (p.S * 2) >= 8) p.S *= 2;
-  const WsLayout one = ws_layout(nacc, p.np, 1);
-  int st = p.np <= 64 ? (112 * 1024 - one.red_bytes - 512 - 1024) / one.stage_bytes : 0;
+  while (p.S < 8 && tiles * p.S * 2 <= 2 * sm_count() && num_kb / (p.S * 2) >= 4) p.S *= 2;
+  const WsLayout one = ws_layout(nacc, p.np, 1, p.S);
+  const int small_kb = 112;
+  int st = p.np <= 64 ? (small_kb * 1024 - one.red_bytes - 512 - 1024) / one.stage_bytes : 0;
   if (st < 2) st = (220 * 1024 - one.red_bytes - 512 - 1024) / one.stage_bytes;      // one CTA per SM
   st = st > 12 ? 12 : st;
   const int need = (num_kb + p.S - 1) / p.S;
   if (st > need) st = need < 2 ? 2 : need;
   p.stages = st;
-  p.smem = ws_layout(nacc, p.np, st).total + 1024;
+  p.smem = ws_layout(nacc, p.np, st, p.S).total + 1024;
   return p;
 }
 

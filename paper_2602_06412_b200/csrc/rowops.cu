@@ -69,8 +69,10 @@ __global__ void __launch_bounds__(256)
 rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __restrict__ h,
                const int32_t* __restrict__ n_active, int d, float eps) {
   __shared__ float s_part[8];
-  griddep_wait();
+  // nothing is written and nothing but the gain is read before the wait: the successor (a GEMM that first streams
+  // weights) may launch at once
   griddep_launch();
+  griddep_wait();
   const int M = *n_active;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nv = d >> 2;                                   // float4 per row

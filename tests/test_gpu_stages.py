@@ -388,7 +388,7 @@ def test_conf_gate_lock(B, N, m):
 @pytest.mark.parametrize("M,n_out,K", [(1, 256, 256), (7, 4096, 4096), (23, 4096, 12288), (32, 12288, 4096), (33, 4096, 4096),
                                        (64, 1024, 8192), (103, 4096, 4096), (128, 4096, 12288), (16, 136, 200), (0, 256, 512)])
 def test_gemm_weight_streaming_few_rows(M, n_out, K, epi):
-    """The weight-streaming (swapped-operand) kernel, taken when the matrix of activations has at most 128 rows: every
+    """The weight-streaming (swapped-operand) kernel (impl = 2; at most 128 rows of activations): every
     row padding (16 / 32 / 64 / 128), cluster sizes 1 ... 8 (K split through distributed shared memory), one and several
     32-row reduction chunks, a ragged feature tile, all three fused epilogues; rows beyond M untouched, two runs give
     the same bits."""
@@ -404,7 +404,7 @@ def test_gemm_weight_streaming_few_rows(M, n_out, K, epi):
     outs = []
     for _ in range(2):
         out = x0.to(DEV) if epi == 1 else torch.full((cap, n_out), 3.0, dtype=torch.bfloat16, device=DEV)
-        SL.surelock_gemm_fused(Ad, Wd, W2d, out, n, epi, impl=0, dev_status=status)
+        SL.surelock_gemm_fused(Ad, Wd, W2d, out, n, epi, impl=2, dev_status=status)
         torch.cuda.synchronize()
         outs.append(out)
     assert status.item() == 0
@@ -421,3 +421,14 @@ def test_gemm_weight_streaming_few_rows(M, n_out, K, epi):
     else:
         assert (out[M:] == 3.0).all()
         assert torch.equal(outs[0].view(torch.int16), outs[1].view(torch.int16))
+
+
+def test_gemm_weight_streaming_refuses_what_it_does_not_take():
+    A = torch.zeros((200, 256), dtype=torch.bfloat16, device=DEV)
+    W = torch.zeros((256, 256), dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros((200, 256), dtype=torch.bfloat16, device=DEV)
+    n = torch.tensor([5], dtype=torch.int32, device=DEV)
+    with pytest.raises(SL.SurelockError, match="not supported"):
+        SL.surelock_gemm(A, W, out, n, impl=2)                       # more than 128 rows of capacity
+    with pytest.raises(SL.SurelockError, match="not supported"):
+        SL.surelock_gemm(A[:8].float(), W.float(), out[:8].float(), n, impl=2)   # fp32

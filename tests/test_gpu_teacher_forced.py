@@ -147,6 +147,7 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     lock1 = lock_fn(B, N, n_active, seed + 1)
     l1 = lock1.to(DEV)
     if row_bound_after_first:
+        SL.surelock_set_option(ctx, "gemm_stream", 1)
         SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
@@ -207,7 +208,7 @@ def test_single_sequence_few_active_rows(n_active):
 
 @pytest.mark.parametrize("n_active,bound", [([23], 23), ([103], 128), ([60], 16), ([9, 1, 14], 32)])
 def test_weight_streaming_step_with_a_row_bound(n_active, bound):
-    """The step with the "row_bound" option set, so that already the second step (M <= 128) runs every contraction
+    """The step with the "gemm_stream" and "row_bound" options set, so that the second step (M <= 128) runs every contraction
     (fused QKV with rotary embedding and cache scatter, output projection, SwiGLU, down projection, LM head) on the
     weight-streaming kernel; bound 16 with 60 active rows makes that kernel take four passes over the weights."""
     cfg = inputs.model_shape("llada8b", n_layers=2, vocab=8192)
