@@ -163,6 +163,21 @@ def workload_config(args, cfgname, cfg, B, N, pattern, M=None):
             "multi_gpu": "replicas only (one independent batch per rank, no collective)"}
 
 
+def c2_config(M0, N, wbytes):
+    return {"workload": "c2: ONE LLaDA-8B-shaped layer (d=4096, 32 heads x 128, FFN 12288), batch 1, N=1024, "
+                        f"M={M0} active rows (seeded random subset), through surelock_layer_step", "batch": 1,
+            "seq_len": N, "active_rows": M0,
+            "l2": "inputs larger than L2 (every call streams the layer's weights, %.0f MB)" % (wbytes / 1e6),
+            "multi_gpu": "replicas only (one independent layer per rank, no collective)"}
+
+
+def headline_rows(args, B, N):
+    """M of the headline measurement: the ragged per-sequence active counts of replica 0 (the same seeded draw the
+    GPU arm makes), so that both arms name the same workload."""
+    seed = dist_util.replica_seed(1234, 0)
+    return sum(n_active_per_seq(B, N, args.ratio, seed * 31 + int(args.ratio * 1000)))
+
+
 def run_reference(args, cfgname, B, N, pattern):
     if args.workload == "c2":                                         # the single-layer microbench: the oracle's layer alone
         from oracle import surelock_oracle as O
@@ -188,8 +203,8 @@ def run_reference(args, cfgname, B, N, pattern):
         return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
                 "steps": len(vals), "warmup": max(0, args.warmup), "ms_per_step": 1e3 * secs / len(vals),
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                "config": {"workload": "c2: ONE LLaDA-8B-shaped layer, batch 1, N=1024 (CPU oracle, bounded sample per step)",
-                           "batch": 1, "seq_len": N},
+                "config": c2_config(512, N, 2 * (4 * cfg["n_heads"] * cfg["head_dim"] * cfg["d_model"]
+                                                     + 3 * cfg["d_model"] * cfg["d_ff"])),
                 "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
                 "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     cfg = inputs.model_shape(cfgname)
@@ -203,7 +218,7 @@ def run_reference(args, cfgname, B, N, pattern):
     return {"impl": "reference", "metric": "active_tokens_per_s", "value": v, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": len(vals), "warmup": max(0, args.warmup), "ms_per_step": 1e3 * secs / len(vals), "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": dict(workload_config(args, cfgname, cfg, B, N, pattern), note="CPU oracle, bounded sample per step"),
+            "config": workload_config(args, cfgname, cfg, B, N, pattern, headline_rows(args, B, N)),
             "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": threads, "kind": "oracle", "sample": desc},
             "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
 
@@ -296,11 +311,7 @@ def run_single_layer(args, rank, world, local):
         "metric": "active_tokens_per_s", "value": dist_util.sum_over_ranks(M0, dev) / (ms * 1e-3), "unit": "tokens/s",
         "n_gpus": world, "steps": 50 * steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "c2: ONE LLaDA-8B-shaped layer (d=4096, 32 heads x 128, FFN 12288), batch 1, N=1024, "
-                               f"M={M0} active rows (seeded random subset), through surelock_layer_step", "batch": 1,
-                   "seq_len": N, "active_rows": M0,
-                   "l2": "inputs larger than L2 (every call streams the layer's weights, %.0f MB)" % (wbytes / 1e6),
-                   "multi_gpu": "replicas only (one independent layer per rank, no collective)"},
+        "config": c2_config(M0, N, wbytes),
         "e2e": dict(value=dist_util.sum_over_ranks(M0, dev) / (e2e_ms * 1e-3), unit="tokens/s", ms_per_step=e2e_ms,
                     h2d_bytes_per_step=N * d * 2, d2h_bytes_per_step=M0 * d * 4),
         "gpu_launches": launches, "clocks": clocks, "roofline": roof, "kernels": kernels, "sweep": sweep,
@@ -335,6 +346,25 @@ def run_single_layer(args, rank, world, local):
 
 
 # ----------------------------------------------------------------------------------------------------- GPU leg
+def spawn_ranks(n):
+    """`python bench.py --gpus N` outside a launcher: start the N ranks here, one process per GPU, the way a launcher
+    would (`python -m torch.distributed.run --nnodes=1 --nproc-per-node N --master-addr 127.0.0.1 ...` with the same
+    arguments).  Rank r binds GPU r; rank 0 prints the JSON line, which passes through unchanged.  NCCL's log is
+    switched on and sent to stderr, so the communicator lines show the N ranks without touching stdout."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    env.setdefault("NCCL_DEBUG_FILE", "/dev/stderr")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.run(cmd, env=env).returncode
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -348,13 +378,19 @@ def main():
     ap.add_argument("--sampler-steps", type=int, default=32,
                     help="diffusion steps of the decoding run (SureLock vs the no-locking baseline sampler); 0 = skip")
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        return spawn_ranks(args.gpus)
     rank, world, local = dist_util.env_rank_world()
     cfgname, B, N, n_prompt, pattern = WORKLOADS[args.workload]
 
-    if args.impl == "reference":
+    if args.impl == "reference":                   # the CPU oracle: rank 0 alone works, the others leave at once
         if rank == 0:
+            args.gpus = max(args.gpus, world)
             print(json.dumps(run_reference(args, cfgname, B, N, pattern)), flush=True)
         return 0
+    if world > 1 and torch.cuda.is_available() and local >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} wants GPU {local}, but only {torch.cuda.device_count()} GPU(s) are "
+                         "visible: --gpus N needs N GPUs on this node (one replica per GPU)")
 
     if args.workload == "c2":
         return run_single_layer(args, rank, world, local)

@@ -53,3 +53,38 @@ def test_two_replicas_report_max_time_and_summed_rows():
 def test_single_process_passthrough():
     assert dist_util.max_over_ranks(3.5) == 3.5 and dist_util.sum_over_ranks(2.0) == 2.0
     assert dist_util.job_throughput(100, 50.0) == (2000.0, 50.0)
+
+
+def test_bench_starts_its_own_ranks_when_asked_for_more_than_one_gpu():
+    """`python bench.py --gpus 2` without a launcher starts two ranks itself (torch.distributed.run, rendezvous on
+    127.0.0.1).  Run here on the CPU-only reference arm: rank 0 alone does the work and prints the one JSON line, which
+    names two ranks; the other rank leaves with exit code 0."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--workload",
+                        "tiny", "--steps", "1", "--warmup", "0"], capture_output=True, text=True, cwd=root, timeout=600,
+                       env=env)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.strip().startswith("{")]
+    assert len(lines) == 1, r.stdout
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
+
+
+def test_bench_with_more_ranks_than_gpus_fails_loudly():
+    """The library arm with two ranks on a box that shows fewer than two GPUs ends with a non-zero exit code and says
+    why (here: no CUDA device at all, or a single one)."""
+    import subprocess
+    import sys
+    if torch.cuda.is_available() and torch.cuda.device_count() >= 2:
+        return
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--workload", "tiny", "--steps", "1",
+                        "--warmup", "0", "--no-cpu-baseline", "--sampler-steps", "0", "--ratios", ""], capture_output=True,
+                       text=True, cwd=root, timeout=600, env=env)
+    assert r.returncode != 0
+    assert "CUDA device" in r.stderr or "GPU" in r.stderr
