@@ -228,6 +228,16 @@ size_t surelock_compact_scratch_bytes(int64_t total);
 int surelock_compact(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
                      int32_t *n_active, int32_t *row_of_pos, void *scratch, int32_t *dev_status, void *stream);
 
+/* Diagnostic for the failure-detection path of the compaction (no counterpart in the paper).  Same arguments as
+ * surelock_compact plus `first_ticket`: the launch's chunk tickets start there instead of at 0, as if that many chunks
+ * belonged to CTAs that never publish their counts.  With first_ticket = 1 every chunk that runs waits for chunk 0's
+ * count, which nobody writes: each CTA polls up to its bound (about 70 ms), stores device status 1 in *dev_status
+ * and returns; nothing hangs, faults or traps, outputs are left unspecified.  first_ticket = 0 is surelock_compact.
+ * The mbarrier waits of the tensor-core kernels are bounded the same way (about 2 s; device status 2 / 3). */
+int surelock_compact_from_ticket(const uint8_t *lock_mask, int B, int N, int32_t *active_idx, int32_t *row_offsets,
+                                 int32_t *n_active, int32_t *row_of_pos, void *scratch, uint32_t first_ticket,
+                                 int32_t *dev_status, void *stream);
+
 /* Compaction for callers that must not allocate device memory.  (No counterpart in the paper: this is a
  * packaging variant of surelock_compact, same kernel, same results.)
  *

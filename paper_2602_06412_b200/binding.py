@@ -74,6 +74,7 @@ def lib() -> C.CDLL:
         "surelock_strerror": (C.c_char_p, [i32]),
         "surelock_compact_scratch_bytes": (sz, [C.c_int64]),
         "surelock_compact": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp]),
+        "surelock_compact_from_ticket": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, C.c_uint32, vp, vp]),
         "surelock_compact_noalloc": (i32, [vp, i32, i32, vp, vp, vp, vp, vp, vp]),
         "surelock_compact_noalloc_max_flags": (C.c_int64, []),
         "surelock_kv_scatter": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, i32, vp]),
@@ -305,6 +306,14 @@ def surelock_compact_scratch_bytes(total: int) -> int:
 def surelock_compact(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos, scratch, dev_status=None):
     _check(lib().surelock_compact(_p(lock_mask), B, N, _p(active_idx), _p(row_offsets), _p(n_active), _p(row_of_pos),
                                   _p(scratch), _p(dev_status), _stream()), "surelock_compact")
+
+
+def surelock_compact_from_ticket(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos, scratch,
+                                 first_ticket: int, dev_status=None):
+    """Diagnostic: the compaction with its chunk tickets starting at `first_ticket` (see the header)."""
+    _check(lib().surelock_compact_from_ticket(_p(lock_mask), B, N, _p(active_idx), _p(row_offsets), _p(n_active),
+                                              _p(row_of_pos), _p(scratch), first_ticket, _p(dev_status), _stream()),
+           "surelock_compact_from_ticket")
 
 
 def surelock_compact_noalloc(lock_mask, B: int, N: int, active_idx, row_offsets, n_active, row_of_pos=None,

@@ -667,6 +667,13 @@ int surelock_compact(const uint8_t* lock_mask, int B, int N, int32_t* active_idx
                         (cudaStream_t)stream);
 }
 
+int surelock_compact_from_ticket(const uint8_t* lock_mask, int B, int N, int32_t* active_idx, int32_t* row_offsets,
+                                 int32_t* n_active, int32_t* row_of_pos, void* scratch, uint32_t first_ticket,
+                                 int32_t* dev_status, void* stream) {
+  return launch_compact_from_ticket(lock_mask, B, N, active_idx, row_offsets, n_active, row_of_pos, scratch, first_ticket,
+                                    dev_status, (cudaStream_t)stream);
+}
+
 int surelock_compact_noalloc(const uint8_t* lock_mask, int B, int N, int32_t* active_idx, int32_t* row_offsets,
                              int32_t* n_active, int32_t* row_of_pos, int32_t* dev_status, void* stream) {
   return launch_compact_noalloc(lock_mask, B, N, active_idx, row_offsets, n_active, row_of_pos, dev_status,

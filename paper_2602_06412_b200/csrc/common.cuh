@@ -105,6 +105,8 @@ size_t compact_scratch_bytes(int64_t total);
 int launch_compact(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
                    int32_t* row_of_pos, void* scratch, int32_t* status, cudaStream_t st);
 
+int launch_compact_from_ticket(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
+                               int32_t* row_of_pos, void* scratch, unsigned first_ticket, int32_t* status, cudaStream_t st);
 long long compact_noalloc_max_flags();
 int launch_compact_noalloc(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
                            int32_t* row_of_pos, int32_t* status, cudaStream_t st);

@@ -52,6 +52,7 @@ compact_kernel(const uint8_t* __restrict__ lock, int total, int N, int B, int32_
   }
   __syncthreads();
   const unsigned chunk = s_chunk;
+  if (chunk >= gridDim.x) return;                 // only when the ticket did not start at zero (the diagnostic entry point)
   const long long base = (long long)chunk * CP_CHUNK + (long long)tid * CP_FPT;
 
   unsigned bits = 0;   // bit k set <=> flag base+k is 0 (active)
@@ -176,6 +177,24 @@ int launch_compact(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row
   if (total >= (1ll << 31)) return SL_EINVAL;
   const int chunks = (int)((total + CP_CHUNK - 1) / CP_CHUNK);
   SL_CUDA_TRY(cudaMemsetAsync(scratch, 0, compact_scratch_bytes(total), st));
+  compact_kernel<<<chunks, CP_THREADS, 0, st>>>(lock, (int)total, N, B, idx, row_offsets, n_active, row_of_pos,
+                                                 reinterpret_cast<CompactScratch*>(scratch), status);
+  SL_CUDA_TRY(cudaGetLastError());
+  return SL_OK;
+}
+
+// Diagnostic: the same launch with the ticket counter starting at `first_ticket` instead of 0, as if that many chunks
+// had been taken by CTAs that never publish their counts.  Every CTA that does run finds the words of the chunks
+// before it empty, polls up to its bound (CP_SPIN_LIMIT polls of 64 ns, about 70 ms), records
+// SL_DEV_COMPACT_TIMEOUT and returns: the give-up path of the look-back, reached without hanging or faulting anything.
+int launch_compact_from_ticket(const uint8_t* lock, int B, int N, int32_t* idx, int32_t* row_offsets, int32_t* n_active,
+                               int32_t* row_of_pos, void* scratch, unsigned first_ticket, int32_t* status, cudaStream_t st) {
+  if (!lock || !idx || !row_offsets || !n_active || !scratch || B <= 0 || N <= 0) return SL_EINVAL;
+  const long long total = (long long)B * N;
+  if (total >= (1ll << 31)) return SL_EINVAL;
+  const int chunks = (int)((total + CP_CHUNK - 1) / CP_CHUNK);
+  SL_CUDA_TRY(cudaMemsetAsync(scratch, 0, compact_scratch_bytes(total), st));
+  SL_CUDA_TRY(cudaMemcpyAsync(scratch, &first_ticket, sizeof(unsigned), cudaMemcpyHostToDevice, st));
   compact_kernel<<<chunks, CP_THREADS, 0, st>>>(lock, (int)total, N, B, idx, row_offsets, n_active, row_of_pos,
                                                  reinterpret_cast<CompactScratch*>(scratch), status);
   SL_CUDA_TRY(cudaGetLastError());

@@ -432,3 +432,47 @@ def test_gemm_weight_streaming_refuses_what_it_does_not_take():
         SL.surelock_gemm(A, W, out, n, impl=2)                       # more than 128 rows of capacity
     with pytest.raises(SL.SurelockError, match="not supported"):
         SL.surelock_gemm(A[:8].float(), W.float(), out[:8].float(), n, impl=2)   # fp32
+
+
+def test_compaction_bounded_wait_runs_out_and_is_reported():
+    """Failure detection without a fault: the compaction is launched with its chunk tickets starting at 1, so the
+    count of chunk 0 is never published and every running chunk's look-back polls into its bound (about 70 ms), stores
+    device status 1 and returns.  Nothing hangs or traps; the same buffers then serve a normal call, whose result is
+    right, and a context on the same device still steps."""
+    import time
+    B, N = 1, 3 * 4096 + 100                                         # four chunks: three of them run and wait
+    g = torch.Generator().manual_seed(3)
+    lock = (torch.rand((B, N), generator=g) < 0.5).to(torch.uint8)
+    d = lock.to(DEV)
+    idx = torch.full((B * N,), -7, dtype=torch.int32, device=DEV)
+    offs = torch.full((B + 1,), -7, dtype=torch.int32, device=DEV)
+    n = torch.full((1,), -7, dtype=torch.int32, device=DEV)
+    rop = torch.full((B * N,), -7, dtype=torch.int32, device=DEV)
+    scratch = torch.empty(SL.surelock_compact_scratch_bytes(B * N) + 64, dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    SL.surelock_compact_from_ticket(d, B, N, idx, offs, n, rop, scratch, 1, status)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert status.item() == 1                                        # SL_DEV_COMPACT_TIMEOUT
+    assert 0.02 < waited < 5.0, waited                               # it did wait, and the wait did end
+    # the device is fine: the ordinary call on the same buffers gives the oracle's answer
+    status.zero_()
+    SL.surelock_compact(d, B, N, idx, offs, n, rop, scratch, status)
+    torch.cuda.synchronize()
+    ridx, roffs = O.active_set(lock.numpy())
+    assert status.item() == 0 and int(n.item()) == len(ridx)
+    assert np.array_equal(idx[:len(ridx)].cpu().numpy(), ridx) and np.array_equal(offs.cpu().numpy(), roffs)
+    # first_ticket = 0 is the ordinary compaction
+    idx2 = torch.full_like(idx, -7)
+    SL.surelock_compact_from_ticket(d, B, N, idx2, offs, n, rop, scratch, 0, status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and torch.equal(idx2[:len(ridx)], idx[:len(ridx)])
+    # and a context created afterwards works
+    cfg = inputs.model_shape("tiny")
+    from tests.parity_util import to_dev
+    ctx = SL.surelock_init(cfg, to_dev(inputs.make_weights(cfg, 2, dtype=torch.float32)), 64, 1)
+    tokens, mask = inputs.make_tokens(1, 64, 32, cfg["vocab"], 2)
+    SL.surelock_step(ctx, tokens.to(DEV), mask.to(DEV), torch.zeros((1, 64), dtype=torch.uint8, device=DEV), 1e-3)
+    assert SL.surelock_status_poll(ctx) == 0
