@@ -126,6 +126,53 @@ int surelock_step_host(surelock_ctx *ctx, const int32_t *tokens, const uint8_t *
 int surelock_layer_step(surelock_ctx *ctx, int layer, const void *hidden_in, const uint8_t *lock_mask,
                         float *hidden_out, surelock_step_out *out);
 
+/* ---- optional un-locking (paper App. "Optional Unlocking") ------------------------------------------------------
+ * A locked position whose context has drifted may be returned to the active set.  Readings taken where the appendix
+ * leaves a choice: the "budgeted proxy" is the step's own forward run on the LOCKED rows as queries against the caches
+ * as they stand, without writing their K/V back; a position is un-locked when ALL three conditions of the printed
+ * rule hold:  u~ > theta_t  AND  KL(p^_t || p_{t*}) > eps_unlock  AND  t - t* > d_interval,  where u~ = 1 - max p^_t,
+ * p_{t*} is the posterior the position had in the step t* that locked it, and theta_t is, per sequence, the
+ * m_percent-th percentile (linear interpolation) of u over the rows that were active in step t (a sequence without
+ * active rows un-locks nothing).  An un-locked position is active from the next step on (its K/V are rewritten then),
+ * cannot lock again for d_cool steps, and afterwards only under the threshold rho * kl_eps.  Positions the caller
+ * locked by hand have no t* and are never un-locked. */
+typedef struct {
+  int period;          /* P: surelock_probe_unlock does its work after every P-th step, >= 1 */
+  float eps_unlock;    /* drift threshold, >= 0 */
+  int d_interval;      /* >= 0 */
+  int d_cool;          /* >= 0 */
+  float rho;           /* 0 <= rho <= 1 */
+  float m_percent;     /* 0 ... 100 */
+} surelock_unlock_params;
+
+typedef struct {       /* dev pointers owned by the ctx, valid until the next probe; NULL when probed == 0 */
+  int32_t step;                  /* t: number of the step just taken (1 = first step after a reset) */
+  int32_t probed;                /* 1 if this call ran the probe (t is a multiple of P) */
+  const int32_t *probed_idx;     /* [n] flat positions of the locked rows, ascending */
+  const int32_t *n_probed;       /* [1] n */
+  const float *drift;            /* [n] KL(p^_t || p_{t*}); +inf for a position without t* */
+  const float *conf;             /* [n] max p^_t */
+  const float *theta;            /* [B] theta_t */
+  const int32_t *n_unlocked;     /* [1] */
+  const int32_t *t_star;         /* [B*N] step that locked each position, -1 = none */
+  const int32_t *cool_until;     /* [B*N] last step of the cool-down after an un-lock, -1 = none */
+} surelock_probe_out;
+
+/* Switch un-locking on (params != NULL) or off (NULL).  Switching it on allocates, once, a third logits buffer
+ * [B*N][vocab] (the frozen posteriors p_{t*}, stored as logits; 3.1 GB at batch 8 x 1536 x vocab 126464) and a few
+ * arrays of B*N entries, and calls surelock_reset().  While it is on, every surelock_step applies, per position, the
+ * threshold rho * kl_eps after an earlier un-lock and the cool-down, and copies the logits of every row that locks
+ * (one 2 * vocab byte row copy per lock).  Not part of surelock_state_export(). */
+int surelock_set_unlocking(surelock_ctx *ctx, const surelock_unlock_params *params);
+
+/* The probe, to be called after surelock_step (and after the caller has used that step's outputs: the packed
+ * workspaces, `hidden` and the logits slot of the NEXT step are overwritten; kl / conf / argmax / active_idx of the
+ * step stay valid).  Does nothing unless the number of the step just taken is a multiple of P.
+ *   tokens     dev int32 [B][N]  the current sequence (after the caller's unmasking)
+ *   lock_mask  dev uint8 [B][N]  in: the mask after the step's lock update; out: un-locked positions cleared
+ * Asynchronous.  Costs one forward over the locked rows (queries only) plus two vocabulary sweeps per locked row. */
+int surelock_probe_unlock(surelock_ctx *ctx, const int32_t *tokens, uint8_t *lock_mask, surelock_probe_out *out);
+
 /* Synchronise the ctx stream and report: *device_status = 0, or the first code a kernel stored since the last
  * surelock_reset: 1 = the compaction's bounded look-back wait ran out, 2 = a bounded barrier wait of the tensor-core
  * GEMM ran out, 3 = the same in the attention kernel (in all three the kernel gave up and returned: the step's

@@ -40,6 +40,17 @@ class _StepOut(C.Structure):
                                           "argmax")]
 
 
+class _UnlockParams(C.Structure):
+    _fields_ = [("period", C.c_int), ("eps_unlock", C.c_float), ("d_interval", C.c_int), ("d_cool", C.c_int),
+                ("rho", C.c_float), ("m_percent", C.c_float)]
+
+
+class _ProbeOut(C.Structure):
+    _fields_ = [("step", C.c_int32), ("probed", C.c_int32)] + \
+               [(n, C.c_void_p) for n in ("probed_idx", "n_probed", "drift", "conf", "theta", "n_unlocked", "t_star",
+                                          "cool_until")]
+
+
 def lib() -> C.CDLL:
     """Load libsurelock.so (built in-tree by `paper_2602_06412_b200.build`); raises if it is not there."""
     global _lib
@@ -63,6 +74,8 @@ def lib() -> C.CDLL:
         "surelock_last_launch_count": (i32, [vp]),
         "surelock_last_fallback_count": (i32, [vp]),
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
+        "surelock_set_unlocking": (i32, [vp, C.POINTER(_UnlockParams)]),
+        "surelock_probe_unlock": (i32, [vp, vp, vp, C.POINTER(_ProbeOut)]),
         "surelock_conf_gate_lock": (i32, [vp, vp, vp, vp, i32, i32, vp, vp, f32, f32, vp, vp]),
         "surelock_update_mask": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]),
         "surelock_state_bytes": (sz, [vp]),
@@ -246,6 +259,38 @@ def surelock_set_confidence_gate(ctx: Ctx, m_percent: float) -> torch.Tensor:
     th = C.c_void_p()
     _check(lib().surelock_set_confidence_gate(ctx.handle, m_percent, C.byref(th)), "surelock_set_confidence_gate")
     return device_view(th.value, (ctx.B,), torch.float32)
+
+
+class ProbeOut:
+    """Views of the outputs of surelock_probe_unlock (the first n_probed rows of the packed arrays are valid)."""
+
+    def __init__(self, raw: _ProbeOut, R: int, B: int):
+        self.step, self.probed = int(raw.step), bool(raw.probed)
+        if self.probed:
+            self.probed_idx = device_view(raw.probed_idx, (R,), torch.int32)
+            self.n_probed = device_view(raw.n_probed, (1,), torch.int32)
+            self.drift = device_view(raw.drift, (R,), torch.float32)
+            self.conf = device_view(raw.conf, (R,), torch.float32)
+            self.theta = device_view(raw.theta, (B,), torch.float32)
+            self.n_unlocked = device_view(raw.n_unlocked, (1,), torch.int32)
+            self.t_star = device_view(raw.t_star, (R,), torch.int32)
+            self.cool_until = device_view(raw.cool_until, (R,), torch.int32)
+
+
+def surelock_set_unlocking(ctx: Ctx, period: int = 1, eps_unlock: float = 0.0, d_interval: int = 0, d_cool: int = 0,
+                           rho: float = 1.0, m_percent: float = 20.0, off: bool = False):
+    """Optional un-locking (App. "Optional Unlocking") on with these parameters, or off."""
+    if off:
+        _check(lib().surelock_set_unlocking(ctx.handle, None), "surelock_set_unlocking")
+        return
+    p = _UnlockParams(period, eps_unlock, d_interval, d_cool, rho, m_percent)
+    _check(lib().surelock_set_unlocking(ctx.handle, C.byref(p)), "surelock_set_unlocking")
+
+
+def surelock_probe_unlock(ctx: Ctx, tokens, lock_mask) -> ProbeOut:
+    raw = _ProbeOut()
+    _check(lib().surelock_probe_unlock(ctx.handle, _p(tokens), _p(lock_mask), C.byref(raw)), "surelock_probe_unlock")
+    return ProbeOut(raw, ctx.B * ctx.N, ctx.B)
 
 
 def surelock_conf_gate_lock(conf, kl, active_idx, row_offsets, B: int, N: int, mask_state, lock_mask, kl_eps: float,

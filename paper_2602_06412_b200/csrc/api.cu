@@ -49,6 +49,17 @@ struct surelock_ctx {
   bool ev_m_valid[2] = {false, false};
   long long calls = 0;                // steps / layer steps since the last reset
   int row_bound_opt = 0;              // "row_bound" option: > 0 = the caller's bound, used instead
+  // optional un-locking (App. "Optional Unlocking"); buffers exist once surelock_set_unlocking() switched it on
+  bool unlocking = false;
+  surelock_unlock_params up = {};
+  int t_step = 0;                     // steps since the last reset (the step just taken is number t_step)
+  void* frozen = nullptr;             // [R][V] storage dtype: logits of every position at the step it locked (p_{t*})
+  float* frozen_lse = nullptr;        // [R]
+  int32_t *frozen_rop = nullptr, *t_star = nullptr, *cool_until = nullptr;   // [R]: position (or -1), t*, last cool-down step
+  uint8_t *relock = nullptr, *inv_lock = nullptr;                            // [R]
+  int32_t *p_idx = nullptr, *p_offsets = nullptr, *p_n = nullptr, *p_argmax = nullptr, *n_unlocked = nullptr;
+  float *p_kl = nullptr, *p_conf = nullptr, *p_lse = nullptr, *p_theta = nullptr;
+  bool probe_mode = false;            // run_layer: queries only, nothing is written into the caches
   bool gemm_stream = false;           // "gemm_stream" option: contractions of at most 128 rows on the weight-streaming kernel
   int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
@@ -186,7 +197,12 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   const int d = g.d_model, hd = g.n_heads * g.head_dim;
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
   bool fused = false;
-  if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
+  if (c->probe_mode) {
+    // the probe of un-locking: the rows are queries only; their k, v are not computed and the caches stay as they are
+    SL_K(K_GEMM_QKV, gemm(c, c->h, c->wq[l], nullptr, c->q, hd, d, EPI_STORE));
+    SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
+    fused = true;
+  } else if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
     // one launch: Q, K, V projections + RoPE + K/V written straight into the cache rows of the active positions
     tick(c, K_GEMM_QKV);
     int rc = SL_EUNSUPPORTED;
@@ -334,6 +350,14 @@ int surelock_reset(surelock_ctx* c) {
   c->cur = 0;
   c->calls = 0;
   c->ev_m_valid[0] = c->ev_m_valid[1] = false;
+  c->t_step = 0;
+  if (c->unlocking) {
+    const size_t R = c->R;
+    SL_CUDA_TRY(cudaMemsetAsync(c->frozen_rop, 0xff, R * 4, c->st));
+    SL_CUDA_TRY(cudaMemsetAsync(c->t_star, 0xff, R * 4, c->st));
+    SL_CUDA_TRY(cudaMemsetAsync(c->cool_until, 0xff, R * 4, c->st));
+    SL_CUDA_TRY(cudaMemsetAsync(c->relock, 0, R, c->st));
+  }
   for (int i = 0; i < 2; ++i) SL_CUDA_TRY(cudaMemsetAsync(c->row_of_pos[i], 0xff, (size_t)c->R * 4, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->status, 0, 16, c->st));
   SL_CUDA_TRY(cudaMemsetAsync(c->n_active, 0, 16, c->st));
@@ -357,6 +381,7 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   const int cur = c->cur, prv = cur ^ 1;
   c->n_ev = 0;
   SL_TRY(begin_call(c));
+  ++c->t_step;
   if (c->check_cache) SL_K(K_COMPACT, launch_cache_check(lock_mask, c->kv_valid, c->R, c->status, c->st));
   SL_K(K_COMPACT, launch_compact(lock_mask, c->B, c->N, c->idx, c->row_offsets, c->n_active, c->row_of_pos[cur],
                                  c->scratch, c->status, c->st));
@@ -381,11 +406,16 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
   SL_K(K_SOFTMAX_KL, launch_softmax_kl_sure(c->logits[cur], c->have_prev ? c->logits[prv] : nullptr, c->row_of_pos[prv],
                                             c->lse[prv], c->idx, c->n_active, c->R, g.vocab, g.dtype, mask_state,
                                             lock_mask, kl_eps, c->kl, c->conf, c->argmax, c->lse[cur], c->st,
-                                            c->gate_m < 0.f, head_tc ? c->lse_part : nullptr,
+                                            c->gate_m < 0.f && !c->unlocking, head_tc ? c->lse_part : nullptr,
                                             (g.vocab + 255) / 256, c->R, c->lse_valid));
   if (c->gate_m >= 0.f)
     SL_K(K_CONF_GATE, launch_conf_gate_lock(c->conf, c->kl, c->idx, c->row_offsets, c->B, c->N, mask_state, lock_mask,
-                                            kl_eps, c->gate_m, c->theta, c->st));
+                                            kl_eps, c->gate_m, c->theta, c->st, !c->unlocking));
+  if (c->unlocking)   // per-position threshold and cool-down; rows that lock keep t* and their logits (p_{t*})
+    SL_K(K_CONF_GATE, launch_lock_commit(c->kl, c->conf, c->lse[cur], c->idx, c->n_active, c->R, c->N, mask_state, lock_mask,
+                                         kl_eps, c->up.rho, c->t_step, c->gate_m >= 0.f ? c->theta : nullptr,
+                                         c->cool_until, c->relock, c->t_star, c->frozen_rop, c->frozen_lse,
+                                         c->logits[cur], c->frozen, (size_t)g.vocab * c->esz, c->st));
   if (out) {
     out->active_idx = c->idx;
     out->row_offsets = c->row_offsets;
@@ -442,6 +472,105 @@ int surelock_layer_step(surelock_ctx* c, int layer, const void* hidden_in, const
     out->row_offsets = c->row_offsets;
     out->n_active = c->n_active;
     out->hidden = hidden_out;
+  }
+  return SL_OK;
+}
+
+int surelock_set_unlocking(surelock_ctx* c, const surelock_unlock_params* p) {
+  if (!c) return SL_EINVAL;
+  if (!p) {
+    c->unlocking = false;
+    return SL_OK;
+  }
+  if (p->period < 1 || !(p->eps_unlock >= 0.f) || p->d_interval < 0 || p->d_cool < 0 || !(p->rho >= 0.f) || p->rho > 1.f ||
+      !(p->m_percent >= 0.f) || p->m_percent > 100.f)
+    return SL_EINVAL;
+  if (c->cfg.vocab <= 0) return SL_EUNSUPPORTED;
+  if (!c->frozen) {
+    const size_t R = c->R, V = c->cfg.vocab;
+    int rc = SL_OK;
+#define A_(p_, bytes) if (rc == SL_OK) rc = dev_alloc(c, &(p_), (bytes))
+    A_(c->frozen, R * V * c->esz);
+    A_(c->frozen_lse, R * 4);
+    A_(c->frozen_rop, R * 4);
+    A_(c->t_star, R * 4);
+    A_(c->cool_until, R * 4);
+    A_(c->relock, R);
+    A_(c->inv_lock, R);
+    A_(c->p_idx, R * 4);
+    A_(c->p_offsets, ((size_t)c->B + 1) * 4);
+    A_(c->p_n, 16);
+    A_(c->n_unlocked, 16);
+    A_(c->p_argmax, R * 4);
+    A_(c->p_kl, R * 4);
+    A_(c->p_conf, R * 4);
+    A_(c->p_lse, R * 4);
+    A_(c->p_theta, ((size_t)c->B + 1) * 4);
+#undef A_
+    if (rc != SL_OK) return rc;
+  }
+  c->up = *p;
+  c->unlocking = true;
+  return surelock_reset(c);          // t*, cool-down and the step counter start over
+}
+
+int surelock_probe_unlock(surelock_ctx* c, const int32_t* tokens, uint8_t* lock_mask, surelock_probe_out* out) {
+  if (!c || !tokens || !lock_mask) return SL_EINVAL;
+  if (!c->unlocking) return SL_EINVAL;
+  const surelock_model_cfg& g = c->cfg;
+  if (out) memset(out, 0, sizeof(*out));
+  if (out) out->step = c->t_step;
+  if (c->t_step < 1 || c->t_step % c->up.period != 0) return SL_OK;   // not a probe step
+  const int done = c->cur ^ 1;       // the slot the step just taken wrote; slot c->cur is free until the next step
+  const int scratch_slot = c->cur;
+  // theta_t: per sequence the m-th percentile of u over the rows that were active in the step just taken
+  SL_TRY(launch_conf_gate_lock(c->conf, c->kl, c->idx, c->row_offsets, c->B, c->N, lock_mask, lock_mask, 0.f,
+                               c->up.m_percent, c->p_theta, c->st, false, true, INFINITY));
+  // the locked rows, packed
+  SL_TRY(launch_invert_mask(lock_mask, c->inv_lock, c->R, c->st));
+  SL_TRY(launch_compact(c->inv_lock, c->B, c->N, c->p_idx, c->p_offsets, c->p_n, nullptr, c->scratch, c->status, c->st));
+  // the forward of the step on those rows as queries only (Algorithm 1 lines 7, 10, 12, 15 without line 11)
+  int32_t *s_idx = c->idx, *s_off = c->row_offsets, *s_n = c->n_active;
+  const int s_bound = c->m_bound;
+  c->idx = c->p_idx;
+  c->row_offsets = c->p_offsets;
+  c->n_active = c->p_n;
+  c->m_bound = c->R;
+  c->probe_mode = true;
+  float* keep_trace = c->trace;
+  c->trace = nullptr;
+  int rc = launch_gather_rows(c->tok_emb, tokens, c->idx, c->n_active, c->R, g.d_model, g.vocab, c->x, g.dtype, c->status,
+                              c->st);
+  for (int l = 0; l < g.n_layers && rc == SL_OK; ++l) rc = run_layer(c, l, c->x);
+  if (rc == SL_OK)
+    rc = launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st);
+  if (rc == SL_OK) rc = gemm(c, c->h, c->lm_head, nullptr, c->logits[scratch_slot], g.vocab, g.d_model, EPI_STORE);
+  // drift KL(p^_t || p_{t*}) against the frozen logits of each position, proxy confidence
+  if (rc == SL_OK)
+    rc = launch_softmax_kl_sure(c->logits[scratch_slot], c->frozen, c->frozen_rop, c->frozen_lse, c->idx, c->n_active, c->R,
+                                g.vocab, g.dtype, lock_mask, lock_mask, 0.f, c->p_kl, c->p_conf, c->p_argmax, c->p_lse,
+                                c->st, false);
+  c->idx = s_idx;
+  c->row_offsets = s_off;
+  c->n_active = s_n;
+  c->m_bound = s_bound;
+  c->probe_mode = false;
+  c->trace = keep_trace;
+  (void)done;
+  SL_TRY(rc);
+  SL_CUDA_TRY(cudaMemsetAsync(c->n_unlocked, 0, 4, c->st));
+  SL_TRY(launch_unlock(c->p_kl, c->p_conf, c->p_idx, c->p_n, c->R, c->N, c->p_theta, c->up.eps_unlock, c->up.d_interval,
+                       c->up.d_cool, c->t_step, c->t_star, c->cool_until, c->relock, lock_mask, c->n_unlocked, c->st));
+  if (out) {
+    out->probed = 1;
+    out->probed_idx = c->p_idx;
+    out->n_probed = c->p_n;
+    out->drift = c->p_kl;
+    out->conf = c->p_conf;
+    out->theta = c->p_theta;
+    out->n_unlocked = c->n_unlocked;
+    out->t_star = c->t_star;
+    out->cool_until = c->cool_until;
   }
   return SL_OK;
 }

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <math.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -143,7 +144,18 @@ int launch_softmax_kl_sure(const void* logits, const void* prev_logits, const in
                            const int* lse_valid = nullptr);   // lse_part: per-tile softmax statistics left by the LM head
 int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx, const int32_t* row_offsets, int B, int N,
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
-                          cudaStream_t st);
+                          cudaStream_t st, bool apply_lock = true, bool all_rows = false, float empty_theta = -INFINITY);
+
+// optional un-locking (unlock.cu)
+int launch_invert_mask(const uint8_t* lock, uint8_t* inv, int total, cudaStream_t st);
+int launch_lock_commit(const float* kl, const float* conf, const float* lse, const int32_t* idx, const int32_t* n_active,
+                       int max_rows, int N, const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float rho, int t,
+                       const float* theta, const int32_t* cool_until, const uint8_t* relock, int32_t* t_star,
+                       int32_t* frozen_rop, float* frozen_lse, const void* logits, void* frozen, size_t row_bytes,
+                       cudaStream_t st);
+int launch_unlock(const float* drift, const float* conf, const int32_t* idx, const int32_t* n_probe, int max_rows, int N,
+                  const float* theta, float eps_unlock, int d_interval, int d_cool, int t, const int32_t* t_star,
+                  int32_t* cool_until, uint8_t* relock, uint8_t* lock_mask, int32_t* n_unlocked, cudaStream_t st);
 
 // step precondition check (cache_check.cu): locked positions need kv_valid, active ones become valid
 int launch_cache_check(const uint8_t* lock, uint8_t* kv_valid, int total, int32_t* status, cudaStream_t st);

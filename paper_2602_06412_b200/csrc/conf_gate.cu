@@ -14,7 +14,11 @@ constexpr int CG_MAX_N = 8192;    // rows of one sequence that fit the shared-me
 __global__ void __launch_bounds__(CG_THREADS)
 conf_gate_lock_kernel(const float* __restrict__ conf, const float* __restrict__ kl, const int32_t* __restrict__ idx,
                       const int32_t* __restrict__ row_offsets, const uint8_t* __restrict__ mask_state,
-                      uint8_t* __restrict__ lock_mask, float kl_eps, float m_percent, float* __restrict__ theta_out) {
+                      uint8_t* __restrict__ lock_mask, float kl_eps, float m_percent, float* __restrict__ theta_out,
+                      int apply_lock, int all_rows, float empty_theta) {
+  // apply_lock = 0: only the thresholds are computed (the caller applies them).  all_rows = 1: the percentile is taken
+  // over every active row of the sequence, masked or not (the reference uncertainty of the un-lock rule, App.
+  // "Optional Unlocking"); empty_theta is what a sequence without any such row gets.
   extern __shared__ float s_u[];            // [pow2 >= candidates], padded with +inf
   __shared__ int s_n;
   __shared__ float s_theta;
@@ -26,7 +30,7 @@ conf_gate_lock_kernel(const float* __restrict__ conf, const float* __restrict__ 
   // gather u of the candidates (order is irrelevant: they get sorted)
   for (int i = threadIdx.x; i < rows; i += CG_THREADS) {
     const int r = r0 + i;
-    if (mask_state[idx[r]] == 0) s_u[atomicAdd(&s_n, 1)] = 1.f - conf[r];
+    if (all_rows || mask_state[idx[r]] == 0) s_u[atomicAdd(&s_n, 1)] = 1.f - conf[r];
   }
   __syncthreads();
   const int n = s_n;
@@ -51,7 +55,7 @@ conf_gate_lock_kernel(const float* __restrict__ conf, const float* __restrict__ 
     }
   }
   if (threadIdx.x == 0) {
-    float theta = -INFINITY;                 // no candidates: nothing passes
+    float theta = empty_theta;               // no candidates (gate: -inf, nothing passes)
     if (n > 0) {
       const float h = (float)(n - 1) * (m_percent * 0.01f);
       int lo = (int)floorf(h);
@@ -65,6 +69,7 @@ conf_gate_lock_kernel(const float* __restrict__ conf, const float* __restrict__ 
   }
   __syncthreads();
   const float theta = s_theta;
+  if (!apply_lock) return;
   for (int i = threadIdx.x; i < rows; i += CG_THREADS) {
     const int r = r0 + i, pos = idx[r];
     if (mask_state[pos] == 0 && (1.f - conf[r]) <= theta && kl[r] <= kl_eps) lock_mask[pos] = 1;
@@ -73,12 +78,13 @@ conf_gate_lock_kernel(const float* __restrict__ conf, const float* __restrict__ 
 
 int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx, const int32_t* row_offsets, int B, int N,
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool apply_lock, bool all_rows, float empty_theta) {
   if (N > CG_MAX_N) return SL_EUNSUPPORTED;
   int p2 = 1;
   while (p2 < N) p2 <<= 1;
   conf_gate_lock_kernel<<<B, CG_THREADS, (size_t)p2 * sizeof(float), st>>>(conf, kl, idx, row_offsets, mask_state, lock_mask,
-                                                                          kl_eps, m_percent, theta_out);
+                                                                          kl_eps, m_percent, theta_out, apply_lock ? 1 : 0,
+                                                                          all_rows ? 1 : 0, empty_theta);
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }

@@ -46,13 +46,17 @@ def selection_skip_mask(lock: torch.Tensor, mask_state: torch.Tensor, fraction: 
 
 def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: int, block_len: int, steps: int,
         kl_eps: float, surelock: bool = True, unmask_per_step: int = 1, select_fraction: float = None,
-        select_seed: int = 0, observer=None) -> Dict:
+        select_seed: int = 0, observer=None, unlock: Dict = None) -> Dict:
     """Run `steps` diffusion steps on device tensors tokens int32 [B][N], mask_state uint8 [B][N] (both updated in
     place).  Generation positions n_prompt.. are decoded block by block (`block_len` positions, `steps_per_block` =
     ceil(block_len / unmask_per_step) steps each).  `select_fraction` (Experiment 5, e.g. 0.8) adds the selection
     surrogate: every step only that fraction of the not-yet-locked positions is computed; with `surelock` this is the
     paper's combination, without it the selection baseline.  A skipped row keeps its cached K/V; it has no posterior in
     that step, so it cannot lock in the step in which it returns (D needs the previous step's posterior).
+    `unlock` (App. "Optional Unlocking"): a dict of the parameters of `surelock_set_unlocking` (period, eps_unlock,
+    d_interval, d_cool, rho, m_percent) switches un-locking on for this run: after every step's unmasking the probe is
+    called (it works every `period`-th step) and may return locked positions to the active set; the number of un-locked
+    positions per step is in the result.
     `observer`, when given, is called after every step, before the unmasking of line 16, as
     observer(t, out, lock_in, lock_out, tokens, mask_state) with lock_in a copy of the lock mask the step was given
     (skip mask included) and lock_out the mask after the step; it is for tests that look at a step from outside and
@@ -68,6 +72,9 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
     unmasked_trace = torch.zeros(steps, dtype=torch.int32, device=dev)
     n_rev = torch.zeros(B, dtype=torch.int32, device=dev)
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    if unlock is not None:
+        SL.surelock_set_unlocking(ctx, **unlock)                            # (resets the ctx)
+        unlocked_trace = torch.zeros(steps, dtype=torch.int32, device=dev)
     SL.surelock_reset(ctx)
     ev[0].record()
     for t in range(steps):
@@ -91,9 +98,17 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
         SL.surelock_update_mask(out.conf, out.argmax, out.active_idx, out.row_offsets, B, N, lo, hi, unmask_per_step,
                                 mask_token, tokens, mask_state, n_rev)
         unmasked_trace[t:t + 1] = n_rev.sum(dtype=torch.int32)
+        if unlock is not None and surelock:
+            po = SL.surelock_probe_unlock(ctx, tokens, lock)
+            if po.probed:
+                unlocked_trace[t:t + 1] = po.n_unlocked
         ev[t + 1].record()
     torch.cuda.synchronize()
     ms = [ev[t].elapsed_time(ev[t + 1]) for t in range(steps)]
+    extra = {}
+    if unlock is not None:
+        extra["unlocked_per_step"] = unlocked_trace.cpu().tolist()
+        SL.surelock_set_unlocking(ctx, off=True)
     M = m_trace.cpu().tolist()
     um = unmasked_trace.cpu().tolist()
     total_s = sum(ms) * 1e-3
@@ -104,4 +119,4 @@ def run(ctx: SL.Ctx, tokens: torch.Tensor, mask_state: torch.Tensor, n_prompt: i
                 f_base_per_position=steps * f_base / R, f_prop_per_position=sum(M) * f_base / (R * R),
                 e2e_tps=sum(um) / total_s if total_s > 0 else 0.0,
                 step_tps=[u / (m * 1e-3) if m > 0 else 0.0 for u, m in zip(um, ms)],
-                total_ms=sum(ms), locked_at_end=int(lock.sum().item()), masked_at_end=int(mask_state.sum().item()))
+                total_ms=sum(ms), locked_at_end=int(lock.sum().item()), masked_at_end=int(mask_state.sum().item()), **extra)

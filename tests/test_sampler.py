@@ -119,3 +119,24 @@ def test_selection_skip_mask_properties():
         assert int(skip[b].sum()) == min(int(unlocked * 0.2), eligible)
     assert torch.equal(skip, sampler.selection_skip_mask(lock, mask, 0.8, 5, 7))   # seeded
     assert not torch.equal(skip, sampler.selection_skip_mask(lock, mask, 0.8, 6, 7))
+
+
+@pytest.mark.gpu
+def test_sampler_run_with_unlocking():
+    """The decoding loop with optional un-locking switched on: the run completes, the active-row trace may now grow
+    again after a probe step, and every un-lock the probe reports shows up as that growth."""
+    from paper_2602_06412_b200 import binding as SL
+    from tests.parity_util import to_dev
+    cfg = inputs.model_shape("tiny")
+    w = to_dev(inputs.make_weights(cfg, 13, dtype=torch.float32, std=0.08))
+    B, N, n_prompt, blk, steps = 2, 96, 40, 28, 40
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], 13)
+    res = sampler.run(ctx, tokens.cuda(), mask.cuda(), n_prompt, blk, steps=steps, kl_eps=1e-3,
+                      unlock=dict(period=2, eps_unlock=2e-5, d_interval=1, d_cool=2, rho=0.25, m_percent=50.0))
+    assert SL.surelock_status_poll(ctx) == 0
+    un, M = res["unlocked_per_step"], res["M_trace"]
+    assert sum(un) > 0 and all(u == 0 for u in un[0::2])                # probes after steps 2, 4, ... (indices 1, 3, ...)
+    grew = [t for t in range(1, steps) if M[t] > M[t - 1]]
+    assert grew and all(un[t - 1] > 0 for t in grew)                    # the active set only grows through an un-lock
+    assert res["unmasked_per_step"] == [B] * steps
