@@ -474,23 +474,33 @@ def main():
     gemm_launch = sum(acc[k][1] for k in acc if k.startswith("gemm"))
     flops = M * gemm_flops_per_row(cfg)
     wbytes = weight_bytes(cfg)
-    # DRAM traffic per average GEMM launch, scaled from the ncu capture of a small case (measured / algorithmic
-    # operand bytes = 148.0 MB / 167.8 MB on M=2048 x 12288 x 4096) to this step's algorithmic operand bytes
+    # DRAM traffic per average GEMM launch: measured / algorithmic bytes of each of the step's five GEMM shapes from
+    # one-launch ncu captures at this workload's own row count (M = 6587; profiles/gemm_tc_kernel_M6587_dram_traffic.md),
+    # applied to the algorithmic bytes of the shapes at the M of this run
     d_, F_, V_, L_ = cfg["d_model"], cfg["d_ff"], cfg["vocab"], cfg["n_layers"]
-    act_bytes = M * (L_ * (2 * d_ + 2 * 3 * d_ + 2 * d_ + 8 * d_ + 2 * d_ + 2 * F_ + 2 * F_ + 8 * d_) + 2 * d_ + 2 * V_)
-    traffic = 0.89 * (wbytes + act_bytes) / max(gemm_launch, 1)
+    hd_ = cfg["n_heads"] * cfg["head_dim"]
+    alg = {"qkv": 2 * M * d_ + 2 * 3 * hd_ * d_ + 2 * 3 * M * hd_, "o": 2 * M * hd_ + 2 * hd_ * d_ + 8 * M * d_,
+           "gateup": 2 * M * d_ + 2 * 2 * d_ * F_ + 2 * M * F_, "down": 2 * M * F_ + 2 * F_ * d_ + 8 * M * d_,
+           "head": 2 * M * d_ + 2 * d_ * V_ + 2 * M * V_}
+    measured_over_alg = {"qkv": 1.54, "o": 1.19, "gateup": 2.10, "down": 2.30, "head": 2.53}
+    traffic = (L_ * sum(alg[k] * measured_over_alg[k] for k in ("qkv", "o", "gateup", "down")) +
+               alg["head"] * measured_over_alg["head"]) / max(gemm_launch, 1)
+    traffic_alg = (L_ * sum(alg[k] for k in ("qkv", "o", "gateup", "down")) + alg["head"]) / max(gemm_launch, 1)
     ridge = pk["bf16_tflops_sustained"] * 1e12 / (pk["hbm_gbs"] * 1e9)
     if M >= ridge:
         ach = flops / (gemm_ms * 1e-3) / 1e12
         roof = dict(kernel="gemm_tc (all GEMM launches of the step)", bound="tensor", achieved=ach,
                     peak=pk["bf16_tflops_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_tflops_sustained"],
-                    traffic=traffic, traffic_note="bytes per average launch, scaled from a small-case ncu capture", peak_kind=f"{pk_kind}, sustained", launches_per_step=gemm_launch,
+                    traffic=traffic, traffic_algorithmic=traffic_alg,
+                    traffic_note="DRAM bytes per average GEMM launch: per-shape measured/algorithmic ratios of one-launch ncu captures at M = 6587, applied to this run's algorithmic bytes",
+                    peak_kind=f"{pk_kind}, sustained", launches_per_step=gemm_launch,
                     avg_launch_ms=gemm_ms / max(gemm_launch, 1))
     else:
         ach = wbytes / (gemm_ms * 1e-3) / 1e9
         roof = dict(kernel="gemm_tc (all GEMM launches of the step, weight streaming)", bound="hbm", achieved=ach,
-                    peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=traffic,
-                    traffic_note="bytes per average launch, scaled from a small-case ncu capture", peak_kind=pk_kind,
+                    peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=traffic_alg,
+                    traffic_algorithmic=traffic_alg,
+                    traffic_note="weight-streaming regime: the weights are read once (ncu at M = 32: 102.0 MB read for a 100.7 MB matrix), so algorithmic bytes per average launch", peak_kind=pk_kind,
                     launches_per_step=gemm_launch, avg_launch_ms=gemm_ms / max(gemm_launch, 1))
     total_k = sum(v[0] for v in acc.values())
     kernels = {k: dict(ms=round(v[0], 4), launches=v[1], share=round(v[0] / total_k, 4)) for k, v in acc.items()}

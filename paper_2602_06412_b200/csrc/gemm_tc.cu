@@ -115,13 +115,19 @@ struct WsSrc {
   }
 };
 
+// STREAM: the output is not read again soon (logits, the SwiGLU activations of a large step): stored with the
+// streaming hint so that it does not push the activation tiles, which every column tile re-reads, out of L2
+template <bool STREAM = false>
 __device__ __forceinline__ void store_bf16x32(bf16* dst, const uint32_t* v) {
 #pragma unroll
-  for (int j = 0; j < 32; j += 8)
-    *reinterpret_cast<uint4*>(dst + j) = make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
+  for (int j = 0; j < 32; j += 8) {
+    const uint4 t = make_uint4(pack_bf16(__uint_as_float(v[j]), __uint_as_float(v[j + 1])),
                                                     pack_bf16(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])),
                                                     pack_bf16(__uint_as_float(v[j + 4]), __uint_as_float(v[j + 5])),
                                                     pack_bf16(__uint_as_float(v[j + 6]), __uint_as_float(v[j + 7])));
+    if (STREAM) __stcs(reinterpret_cast<uint4*>(dst + j), t);
+    else *reinterpret_cast<uint4*>(dst + j) = t;
+  }
 }
 
 // One 32-column unit of the LM head: store as bf16 and fold the stored values into the row's running softmax statistics
@@ -161,7 +167,7 @@ __device__ __forceinline__ void store_unit_with_stats(const Src& src, int row, b
   rs.s += acc.x + acc.y;
   bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
   if (col + 32 <= n_out) {
-    store_bf16x32(dst, v);
+    store_bf16x32<true>(dst, v);
   } else {
     for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
   }
@@ -178,7 +184,7 @@ __device__ __forceinline__ int units_per_row(int bn, int n0, const QkvArgs& qkv)
   return bn >> 5;
 }
 
-template <int EPI, typename Src>
+template <int EPI, typename Src, bool STREAM_OUT = false>
 __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, bool live, int u, int n0, int n_out,
                                               void* __restrict__ Cv, const QkvArgs& qkv, uint32_t red_slot = 0) {
   if (EPI == EPI_QKV) {
@@ -250,7 +256,7 @@ __device__ __forceinline__ void epilogue_unit(const Src& src, int bn, int row, b
     } else {
       bf16* dst = reinterpret_cast<bf16*>(Cv) + (long long)row * n_out + col;
       if (col + 32 <= n_out) {
-        store_bf16x32(dst, v);
+        store_bf16x32<STREAM_OUT>(dst, v);
       } else {
         for (int j = 0; j < 32 && col + j < n_out; ++j) dst[j] = __float2bfloat16_rn(__uint_as_float(v[j]));
       }
@@ -321,6 +327,29 @@ __device__ __forceinline__ TileCfg choose_tiles(int M, int n_out, int num_kb, in
   return c;
 }
 
+// Order of the output tiles.  Row tiles are taken in GROUPS whose activation rows (group rows x K x 2 bytes) stay in L2
+// (TILE_GROUP_BYTES, well under the 126 MB); inside a group the row index runs fastest, then the column tile, so a
+// weight tile is fetched from DRAM once per group and the activation rows once in all.  With a single group this is
+// the plain row-fastest order.  (Before: one group; with M x K x 2 bytes beyond the L2 the activation matrix was
+// re-read from DRAM for every few column tiles: 1.28 GB read for the 262 MB of operands of the down projection at
+// M = 6587.)
+#ifndef TILE_GROUP_MB
+#define TILE_GROUP_MB 40
+#endif
+constexpr long long TILE_GROUP_BYTES = (long long)TILE_GROUP_MB << 20;
+__device__ __forceinline__ void tile_of(int w, int m_tiles, int n_tiles, int group, int& mt, int& nt) {
+  const int per_group = group * n_tiles;
+  const int g = w / per_group, r = w - g * per_group;
+  const int m_first = g * group;
+  const int g_rows = m_tiles - m_first < group ? m_tiles - m_first : group;   // the last group may be smaller
+  nt = r / g_rows;
+  mt = m_first + (r - nt * g_rows);
+}
+__device__ __forceinline__ int tile_group(int tile_rows, int K) {
+  const long long g = TILE_GROUP_BYTES / ((long long)tile_rows * K * 2);
+  return g < 1 ? 1 : (g > (1 << 20) ? (1 << 20) : (int)g);
+}
+
 // ---- CTA-pair path (cta_group::2) for the tensor-pipe-bound regime ---------------------------------------------------
 // A cluster of two CTAs owns a 256 x 256 output tile: each CTA loads its own 128 rows of A and HALF of the weight tile
 // (128 of its 256 rows), the leader CTA issues tcgen05.mma.cta_group::2 (M = 256) which reads both CTAs' shared memory,
@@ -378,14 +407,18 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
   const int total = m_pairs * n_tiles;
   const int num_kb = (K + TC_BK - 1) / TC_BK;
   const int cid = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+  const int group = tile_group(2 * TC_BM, K);
 
   if (warp == 0) {
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      const uint64_t keep = l2_policy_evict_last();     // activation tiles: every column tile of the group re-reads them
       for (int w = cid; w < total && ok; w += n_clusters) {
-        const int m0 = (w % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (w / m_pairs) * OUT_BN;
+        int mt, nt;
+        tile_of(w, m_pairs, n_tiles, group, mt, nt);
+        const int m0 = mt * 2 * TC_BM + (int)rank * TC_BM, n0 = nt * OUT_BN;
         // this CTA's half of the weight tile
         const CUtensorMap* mp = tmW0;
         int brow = n0 + (int)rank * 128;
@@ -402,7 +435,7 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
           const uint32_t sa = smem_u32(smem + stage * STAGE_BYTES), sb = sa + A_BYTES;
           const uint32_t fb = mapa_u32(full_bar(stage), 0);
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
-          tma_load_2d_pair(sa, tmA, kb * TC_BK, m0, fb);
+          tma_load_2d_pair_hint(sa, tmA, kb * TC_BK, m0, fb, keep);
           tma_load_2d_pair(sb, mp, kb * TC_BK, brow, fb);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
@@ -447,7 +480,9 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
     for (int w = cid; w < total && ok; w += n_clusters, ++it) {
       const int acc = it & 1;
       const uint32_t use = (uint32_t)(it >> 1);
-      const int m0 = (w % m_pairs) * 2 * TC_BM + (int)rank * TC_BM, n0 = (w / m_pairs) * OUT_BN;
+      int mt, nt;
+      tile_of(w, m_pairs, n_tiles, group, mt, nt);
+      const int m0 = mt * 2 * TC_BM + (int)rank * TC_BM, n0 = nt * OUT_BN;
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -463,7 +498,8 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
           qkv.lse_part[(size_t)(n0 / BN) * qkv.lse_rows + row] = make_float4(rs.m, rs.s, __int_as_float(rs.am), 0.f);
       } else {
 #pragma unroll 1
-        for (int u = 0; u < upr; ++u) epilogue_unit<EPI>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv, red_slot);
+        for (int u = 0; u < upr; ++u)
+          epilogue_unit<EPI, TmemSrc, EPI != EPI_QKV>(TmemSrc{taddr}, BN, row, row < M, u, n0, n_out, Cv, qkv, red_slot);
       }
       tc_fence_before();
       __syncwarp();
@@ -579,6 +615,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     tc.total = tc.tiles * tc.S;
   }
   const int bn = tc.bn, S = tc.S, m_tiles = tc.m_tiles, total = tc.total;
+  const int group = tile_group(TC_BM, K);
   if (EPI == EPI_STORE && qkv.lse_valid && blockIdx.x == 0 && threadIdx.x == 0) *qkv.lse_valid = (S == 1 && bn == 256) ? 1 : 0;
   const int out_bn = EPI == EPI_SWIGLU ? bn >> 1 : bn;
   // Stage layout, chosen from M like the tiles: with a single row tile of few rows only 32 or 64 activation rows are
@@ -628,9 +665,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       };
       bool waited = !prefetch_w;
+      const uint64_t keep = l2_policy_evict_last();     // activation tiles are re-read by every column tile
       for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
         const int t = w / S, sp = w - t * S;
-        const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
+        int mt, nt;
+        tile_of(t, m_tiles, tc.n_tiles, group, mt, nt);
+        const int m0 = mt * TC_BM, n0 = nt * out_bn;
         const int kb0 = sp * num_kb / S, kb1 = (sp + 1) * num_kb / S;
         int kb = kb0;
         if (!waited) {
@@ -645,7 +685,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           griddep_launch();
           waited = true;
           for (int i = 0; i < npre; ++i)
-            tma_load_2d(smem_u32(smem + i * STAGE_BYTES), mapA, (kb0 + i) * TC_BK, m0, full_bar(i));
+            tma_load_2d_hint(smem_u32(smem + i * STAGE_BYTES), mapA, (kb0 + i) * TC_BK, m0, full_bar(i), keep);
           stage = npre;
           if (stage == nst) { stage = 0; phase ^= 1; }
           kb = kb0 + npre;
@@ -653,7 +693,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (; kb < kb1; ++kb) {
           if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1, s_abort))) break;
           mbar_expect_tx(full_bar(stage), stage_tx);
-          tma_load_2d(smem_u32(smem + stage * STAGE_BYTES), mapA, kb * TC_BK, m0, full_bar(stage));
+          tma_load_2d_hint(smem_u32(smem + stage * STAGE_BYTES), mapA, kb * TC_BK, m0, full_bar(stage), keep);
           load_w(stage, kb, n0);
           if (++stage == nst) { stage = 0; phase ^= 1; }
         }
@@ -715,7 +755,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int t = w / S, sp = w - t * S;
       const int acc = it & 1;
       const uint32_t use = (uint32_t)(it >> 1);
-      const int m0 = (t % m_tiles) * TC_BM, n0 = (t / m_tiles) * out_bn;
+      int mt, nt;
+      tile_of(t, m_tiles, tc.n_tiles, group, mt, nt);
+      const int m0 = mt * TC_BM, n0 = nt * out_bn;
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
