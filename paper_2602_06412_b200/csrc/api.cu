@@ -60,6 +60,12 @@ struct surelock_ctx {
   int32_t *p_idx = nullptr, *p_offsets = nullptr, *p_n = nullptr, *p_argmax = nullptr, *n_unlocked = nullptr;
   float *p_kl = nullptr, *p_conf = nullptr, *p_lse = nullptr, *p_theta = nullptr;
   bool probe_mode = false;            // run_layer: queries only, nothing is written into the caches
+  // "layer_chain" option: with at most 64 active rows the four contractions between two attention calls run as one
+  // persistent kernel per layer (gemm_chain.cu)
+  bool layer_chain = false;
+  float *ch_ws = nullptr, *ssq_ffn = nullptr, *ssq_next = nullptr;
+  unsigned* ch_bar = nullptr;
+  unsigned ch_bar_base = 0;           // arrivals on ch_bar by all launches so far (host-side count)
   bool gemm_stream = false;           // "gemm_stream" option: contractions of at most 128 rows on the weight-streaming kernel
   int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
@@ -191,8 +197,9 @@ static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, v
   return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
 }
 
-// Algorithm 1 lines 10-13 for one layer on the packed rows in x (fp32 [M][d], updated in place).
-static int run_layer(surelock_ctx* c, int l, float* x) {
+// Algorithm 1 lines 10-13 for one layer on the packed rows in x (fp32 [M][d], updated in place): layer_front is lines
+// 10-11 (norm, Q/K/V, rotary embedding, cache scatter), layer_back lines 12-13 (attention, output projection, FFN).
+static int layer_front(surelock_ctx* c, int l, float* x) {
   const surelock_model_cfg& g = c->cfg;
   const int d = g.d_model, hd = g.n_heads * g.head_dim;
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
@@ -229,6 +236,43 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
     SL_K(K_ROPE, launch_rope(c->q, c->k, c->idx, c->n_active, c->R, c->N, g.n_heads, g.head_dim, c->rope, g.dtype, c->st));
     SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
   }
+  return SL_OK;
+}
+
+static inline bool use_chain(const surelock_ctx* c) {
+  return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
+         c->m_bound <= 64;
+}
+
+// Attention, then everything up to the next attention as one persistent kernel: output projection, SwiGLU FFN and,
+// when `next` >= 0, the Q/K/V projections of layer `next` (Algorithm 1 lines 12-13, then 10-11 of the next block).
+static int layer_back_chain(surelock_ctx* c, int l, float* x, int next) {
+  const surelock_model_cfg& g = c->cfg;
+  SL_K(K_ATTN, attention(c, l));
+  ChainLaunch L = {};
+  L.attn = c->attn; L.wo = c->wo[l]; L.wg = c->w_gate[l]; L.wu = c->w_up[l]; L.wd = c->w_down[l];
+  if (next >= 0) { L.wq = c->wq[next]; L.wk = c->wk[next]; L.wv = c->wv[next]; }
+  L.x = x; L.xg = c->h; L.act = c->act;
+  L.gain_ffn = c->ffn_norm_g[l];
+  L.gain_next = next >= 0 ? c->attn_norm_g[next] : nullptr;
+  L.ssq_ffn = c->ssq_ffn; L.ssq_next = c->ssq_next;
+  L.q = c->q;
+  if (next >= 0) { L.kc = c->kcache(next); L.vc = c->vcache(next); }
+  L.idx = c->idx; L.rope = c->rope; L.ws = c->ch_ws; L.bar = c->ch_bar; L.bar_base = &c->ch_bar_base;
+  L.n_active = c->n_active; L.status = c->status;
+  if (c->trace && x == c->x) {
+    L.trace_mid = c->trace + (size_t)(2 * l + 1) * c->R * g.d_model;
+    L.trace_out = c->trace + (size_t)(2 * l + 2) * c->R * g.d_model;
+  }
+  L.max_rows = c->R; L.m_bound = c->m_bound; L.d = g.d_model; L.F = g.d_ff; L.hd = g.n_heads * g.head_dim; L.dh = g.head_dim;
+  L.n_seq = c->N; L.rms_eps = g.rms_eps;
+  SL_K(K_GEMM_GATEUP, launch_gemm_chain(L, c->st));
+  return SL_OK;
+}
+
+static int layer_back(surelock_ctx* c, int l, float* x) {
+  const surelock_model_cfg& g = c->cfg;
+  const int d = g.d_model, hd = g.n_heads * g.head_dim;
   SL_K(K_ATTN, attention(c, l));
   SL_K(K_GEMM_O, gemm(c, c->attn, c->wo[l], nullptr, x, d, hd, EPI_RESIDUAL));
   if (c->trace && x == c->x)
@@ -238,6 +282,15 @@ static int run_layer(surelock_ctx* c, int l, float* x) {
   SL_K(K_GEMM_GATEUP, gemm(c, c->h, c->w_gate[l], c->w_up[l], c->act, g.d_ff, d, EPI_SWIGLU));
   SL_K(K_GEMM_DOWN, gemm(c, c->act, c->w_down[l], nullptr, x, d, g.d_ff, EPI_RESIDUAL));
   return SL_OK;
+}
+
+static int run_layer(surelock_ctx* c, int l, float* x) {
+  SL_TRY(layer_front(c, l, x));
+  if (use_chain(c)) {
+    const int rc = layer_back_chain(c, l, x, -1);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
+  return layer_back(c, l, x);
 }
 
 extern "C" {
@@ -350,6 +403,10 @@ int surelock_reset(surelock_ctx* c) {
   c->cur = 0;
   c->calls = 0;
   c->ev_m_valid[0] = c->ev_m_valid[1] = false;
+  if (c->ch_bar) {                      // a chain kernel that gave up leaves the barrier count short: start over
+    SL_CUDA_TRY(cudaMemsetAsync(c->ch_bar, 0, 16, c->st));
+    c->ch_bar_base = 0;
+  }
   c->t_step = 0;
   if (c->unlocking) {
     const size_t R = c->R;
@@ -389,11 +446,22 @@ int surelock_step(surelock_ctx* c, const int32_t* tokens, const uint8_t* mask_st
                                     c->status, c->st));
   const size_t xbytes = (size_t)c->R * g.d_model * sizeof(float);
   if (c->trace) SL_CUDA_TRY(cudaMemcpyAsync(c->trace, c->x, xbytes, cudaMemcpyDeviceToDevice, c->st));
+  bool chained = false;                            // the Q/K/V of layer l were already done by layer l-1's chain kernel
   for (int l = 0; l < g.n_layers; ++l) {
-    SL_TRY(run_layer(c, l, c->x));
-    if (c->trace)
-      SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(2 * l + 2) * c->R * g.d_model, c->x, xbytes, cudaMemcpyDeviceToDevice,
-                                  c->st));
+    if (!chained) SL_TRY(layer_front(c, l, c->x));
+    chained = false;
+    int rc = SL_EUNSUPPORTED;
+    if (use_chain(c)) {
+      rc = layer_back_chain(c, l, c->x, l + 1 < g.n_layers ? l + 1 : -1);
+      if (rc == SL_OK) chained = l + 1 < g.n_layers;
+      else if (rc != SL_EUNSUPPORTED) return rc;
+    }
+    if (rc == SL_EUNSUPPORTED) {
+      SL_TRY(layer_back(c, l, c->x));
+      if (c->trace)
+        SL_CUDA_TRY(cudaMemcpyAsync(c->trace + (size_t)(2 * l + 2) * c->R * g.d_model, c->x, xbytes,
+                                    cudaMemcpyDeviceToDevice, c->st));
+    }
   }
   SL_K(K_RMSNORM, launch_rmsnorm(c->x, c->final_norm_g, c->h, c->n_active, c->R, g.d_model, g.rms_eps, g.dtype, c->st));
   c->split.lse_part = c->lse_part;                 // the LM head leaves the rows' softmax statistics for the next kernel
@@ -689,6 +757,19 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
+  if (!strcmp(name, "layer_chain")) {
+    if (value && !c->ch_ws && c->cfg.dtype == SL_BF16) {
+      int rc = dev_alloc(c, &c->ch_ws, gemm_chain_workspace_bytes(64));
+      if (rc == SL_OK) rc = dev_alloc(c, &c->ssq_ffn, (size_t)c->R * (c->cfg.d_model / 32 + 1) * sizeof(float));
+      if (rc == SL_OK) rc = dev_alloc(c, &c->ssq_next, (size_t)c->R * (c->cfg.d_model / 32 + 1) * sizeof(float));
+      if (rc == SL_OK) rc = dev_alloc(c, &c->ch_bar, 16);
+      if (rc != SL_OK) return rc;
+      SL_CUDA_TRY(cudaMemsetAsync(c->ch_bar, 0, 16, c->st));
+      c->ch_bar_base = 0;
+    }
+    c->layer_chain = value != 0;
+    return SL_OK;
+  }
   if (!strcmp(name, "row_bound")) { c->row_bound_opt = value > 0 ? value : 0; return SL_OK; }
   if (!strcmp(name, "have_prev")) { c->have_prev = value != 0; return SL_OK; }
   if (!strcmp(name, "check_cache")) {

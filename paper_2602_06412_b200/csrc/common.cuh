@@ -146,6 +146,28 @@ int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx
                           const uint8_t* mask_state, uint8_t* lock_mask, float kl_eps, float m_percent, float* theta_out,
                           cudaStream_t st, bool apply_lock = true, bool all_rows = false, float empty_theta = -INFINITY);
 
+// the contractions of a layer between two attention calls as one persistent kernel (gemm_chain.cu), bf16, few rows
+struct ChainLaunch {
+  const void *attn, *wo, *wg, *wu, *wd, *wq, *wk, *wv;   // wq == nullptr: no Q/K/V phase
+  float* x;
+  void *xg, *act;
+  const void *gain_ffn, *gain_next;
+  float *ssq_ffn, *ssq_next;
+  void *q, *kc, *vc;
+  const int32_t* idx;
+  const float2* rope;
+  float* ws;
+  unsigned* bar;
+  unsigned* bar_base;          // host-side count of the arrivals of all earlier launches; advanced by the launch
+  const int32_t* n_active;
+  int32_t* status;
+  float *trace_mid, *trace_out;
+  int max_rows, m_bound, d, F, hd, dh, n_seq;
+  float rms_eps;
+};
+int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st);   // SL_EUNSUPPORTED when the shapes do not fit
+size_t gemm_chain_workspace_bytes(int np_max);
+
 // optional un-locking (unlock.cu)
 int launch_invert_mask(const uint8_t* lock, uint8_t* inv, int total, cudaStream_t st);
 int launch_lock_commit(const float* kl, const float* conf, const float* lse, const int32_t* idx, const int32_t* n_active,

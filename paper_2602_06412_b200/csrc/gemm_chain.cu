@@ -1,0 +1,578 @@
+// The contractions of a transformer block for FEW active rows (M <= 64) as ONE persistent kernel per layer:
+// output projection -> gate / up (+ SwiGLU) -> down projection -> Q/K/V projections of the NEXT layer (with its
+// rotary embedding and K/V cache scatter), i.e. everything of Algorithm 1 lines 10-13 between two attention calls.
+//
+// Why: with few rows a step is bound by reading every weight once from HBM (the regime in which the paper reports no
+// gain, App. "Algorithmic Characteristics on Runtime"), and with one kernel per contraction what is lost is the
+// latency chain at every kernel boundary (launch, first bytes, reduction hand-over, exit).  Here the weight stream
+// never stops: every CTA (one per SM, cooperative launch) owns, for each contraction, a contiguous range of
+// (feature tile, K block) units of equal length, so all SMs stream the same number of bytes; its producer warp walks
+// through the ranges of all four contractions back to back, limited only by the shared-memory ring, while the
+// dependent work (activation loads, MMAs, reductions) follows behind through the phases.
+//
+// Per contraction ("phase"):
+//   * a CTA's range may cross feature tiles; every (tile, K range) segment accumulates in tensor memory
+//     (swapped operands as in gemm_stream.cu: 128 weight rows x 64 K are the 128-row MMA operand, the NP padded
+//     activation rows the N operand) and leaves an fp32 partial tile [NP][128] in a workspace;
+//   * grid barrier (a counter in global memory; bounded spin);
+//   * reduction: the partials of a tile are summed in CTA order (deterministic) and the contraction's epilogue is
+//     applied: += into the fp32 residual stream (O, down), silu(gate) * up (gate/up), RoPE + packed q + K/V cache
+//     scatter (Q/K/V);
+//   * grid barrier; the next phase's activation loads may start.
+// RMSNorm is folded in: the reductions of O and down, which produce the final x of a sub-block, also write
+// xg = bf16(x * gain) of the norm that follows and per-(row, 32-column chunk) sums of squares; the contraction after
+// the norm runs on xg and its reduction scales row r by rsqrt(mean(x_r^2) + eps) (the scale is per row, so it commutes
+// with the contraction).
+//
+// Every wait is bounded (mbarrier waits, grid-barrier spins): on expiry the CTA records SL_DEV_GEMM_TIMEOUT, all
+// roles leave, tensor memory is freed.  The grid barrier needs all CTAs resident: the kernel is launched
+// cooperatively with one CTA per SM.
+#include "tc_common.cuh"
+
+namespace sl {
+
+#ifdef CH_PROFILE
+__device__ unsigned long long g_ch_prof[160 * 24];
+__device__ __forceinline__ unsigned long long chtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) :: "memory");
+  return t;
+}
+#define CP(i) { g_ch_prof[blockIdx.x * 24 + (i)] = chtime(); }
+#else
+#define CP(i) {}
+#endif
+
+constexpr int CH_THREADS = 224;          // warp 0 weight producer, 1 activation loader, 2 MMA issue, 3-6 epilogue / reductions
+constexpr int CH_BF = 128, CH_BK = 64;
+constexpr int CH_W_BYTES = CH_BF * CH_BK * 2;      // 16 KB
+constexpr int CH_W_STAGES = 11, CH_X_STAGES = 4;
+constexpr int CH_MAX_SEG = 4;            // (tile, K range) segments of one CTA in one phase
+constexpr int CH_MAX_PHASES = 4;
+constexpr unsigned long long CH_SPIN_CYCLES = 2000000000ull;   // bound of a grid-barrier wait: ~1 s
+
+enum { CH_O = 0, CH_GATEUP = 1, CH_DOWN = 2, CH_QKV = 3 };
+
+struct ChainPhase {
+  int kind, n_tiles, num_kb, w_map0, tiles_per_map, x_map;
+};
+struct ChainArgs {
+  ChainPhase ph[CH_MAX_PHASES];
+  int n_phases, np, d, F, hd, dh, n_seq;
+  float rms_eps;
+  float* x;                    // fp32 residual stream [M][d]
+  bf16* xg;                    // [M][d]  bf16(x * gain) of the norm that follows
+  bf16* act;                   // [M][F]  SwiGLU output
+  const bf16 *gain_ffn, *gain_next;     // gains of the norm after O and after down (nullptr: nothing follows)
+  float *ssq_ffn, *ssq_next;   // [rows][d / 32] sums of squares of x per 32-column chunk, written by the O / down reductions
+  bf16 *q, *kc, *vc;
+  const int32_t* idx;
+  const float2* rope;
+  float* ws;                   // [grid][CH_MAX_SEG][np][128] partial tiles
+  unsigned* bar;               // ONE grid-barrier counter, never reset: every barrier of every launch adds `grid` to it
+  unsigned bar_base;           // its value before this launch (the host keeps count)
+  const int32_t* n_active;
+  int32_t* status;
+  float *trace_mid, *trace_out;         // optional copies of x after the O / down reductions
+};
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// Unit ranges: unit u = tile * num_kb + kb; CTA c owns [c U / G, (c + 1) U / G).  (U * G < 2^31: checked on the host.)
+struct ChainRange {
+  int begin, end;
+};
+__device__ __forceinline__ ChainRange chain_range(const ChainPhase& p, int c, int G) {
+  const int U = p.n_tiles * p.num_kb;
+  return ChainRange{c * U / G, (c + 1) * U / G};
+}
+
+// Sum of the partial tiles of feature tile t, row r, 8 consecutive features starting at f (inside the tile), in CTA
+// order (deterministic).  The CTAs whose unit ranges meet the tile are consecutive, at most CH_MAX_COVER of them
+// (checked on the host); all their loads are issued before the first sum so that the L2 latencies overlap.
+constexpr int CH_MAX_COVER = 8;
+__device__ __forceinline__ void sum_partials8(const ChainArgs& a, const ChainPhase& p, int G, int t, int r, int f, float* out) {
+  const int U = p.n_tiles * p.num_kb, u0 = t * p.num_kb, u1 = u0 + p.num_kb;
+  int c0 = u0 * G / U;
+  while (c0 > 0 && c0 * U / G > u0) --c0;
+  while ((c0 + 1) * U / G <= u0) ++c0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) out[j] = 0.f;
+  // four tiles' loads in flight at a time
+  for (int k0 = 0; k0 < CH_MAX_COVER; k0 += 4) {
+    float4 v[4][2];
+    bool live[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int c = c0 + k0 + k, b = c * U / G;
+      live[k] = c < G && b < u1;
+      if (live[k]) {
+        const int seg = t - b / p.num_kb;                      // which of CTA c's segments this tile is
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f);
+        v[k][0] = __ldcg(src);
+        v[k][1] = __ldcg(src + 1);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (live[k]) {
+        out[0] += v[k][0].x; out[1] += v[k][0].y; out[2] += v[k][0].z; out[3] += v[k][0].w;
+        out[4] += v[k][1].x; out[5] += v[k][1].y; out[6] += v[k][1].z; out[7] += v[k][1].w;
+      }
+    }
+    if (!live[3]) break;
+  }
+}
+
+__device__ __forceinline__ uint4 pack8(const float* v) {
+  return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+}
+
+// rstd of every row from the chunk sums left by the reduction that produced x: s_rstd[r], r < np
+__device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, int e_tid, int M, float* s_rstd) {
+  // four threads per row, each a strided quarter of the chunk sums (fixed order: deterministic)
+  const int chunks = a.d >> 5;
+  for (int r0 = 0; r0 < a.np; r0 += 32) {
+    const int r = r0 + (e_tid >> 2);
+    float s = 0.f;
+    if (r < M)
+      for (int c = (e_tid & 3) * 4; c < chunks; c += 16) {
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(ssq + (size_t)r * chunks + c));
+        s += (v.x + v.y) + (v.z + v.w);
+      }
+    s += __shfl_xor_sync(0xffffffffu, s, 1);
+    s += __shfl_xor_sync(0xffffffffu, s, 2);
+    if ((e_tid & 3) == 0 && r < a.np) s_rstd[r] = rsqrtf(s / (float)a.d + a.rms_eps);
+  }
+  asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+// The reduction + epilogue of one phase, spread over all epilogue threads of the grid.
+__device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int e_tid, int M,
+                                             float* s_rstd) {
+  const int np = a.np;
+  if (p.kind == CH_O || p.kind == CH_DOWN) {
+    // x += sum; xg = bf16(x * gain); sums of squares per (row, 32-column chunk).  A CTA takes 32-column chunks, four
+    // threads per row.
+    const bf16* gain = p.kind == CH_O ? a.gain_ffn : a.gain_next;
+    float* ssq = p.kind == CH_O ? a.ssq_ffn : a.ssq_next;
+    float* trace = p.kind == CH_O ? a.trace_mid : a.trace_out;
+    const int chunks = a.d >> 5;
+    for (int ch = c; ch < chunks; ch += G) {
+      for (int r0 = 0; r0 < np; r0 += 32) {
+        const int r = r0 + (e_tid >> 2), n = ch * 32 + (e_tid & 3) * 8;
+        float ss = 0.f;
+        if (r < M) {
+          float s[8];
+          sum_partials8(a, p, G, n >> 7, r, n & 127, s);
+          float4* xp = reinterpret_cast<float4*>(a.x + (size_t)r * a.d + n);
+          float4 x0 = xp[0], x1 = xp[1];
+          x0.x += s[0]; x0.y += s[1]; x0.z += s[2]; x0.w += s[3];
+          x1.x += s[4]; x1.y += s[5]; x1.z += s[6]; x1.w += s[7];
+          xp[0] = x0;
+          xp[1] = x1;
+          if (trace) {
+            float4* tp = reinterpret_cast<float4*>(trace + (size_t)r * a.d + n);
+            tp[0] = x0;
+            tp[1] = x1;
+          }
+          const float xv[8] = {x0.x, x0.y, x0.z, x0.w, x1.x, x1.y, x1.z, x1.w};
+#pragma unroll
+          for (int j = 0; j < 8; ++j) ss += xv[j] * xv[j];
+          if (gain) {
+            const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(gain + n));
+            const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&g4);
+            float o[8];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float2 gf = __bfloat1622float2(gp[j]);
+              o[2 * j] = xv[2 * j] * gf.x;
+              o[2 * j + 1] = xv[2 * j + 1] * gf.y;
+            }
+            *reinterpret_cast<uint4*>(a.xg + (size_t)r * a.d + n) = pack8(o);
+          }
+        }
+        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+        if ((e_tid & 3) == 0 && r < M && gain) ssq[(size_t)r * chunks + ch] = ss;
+      }
+    }
+  } else if (p.kind == CH_GATEUP) {
+    // act = silu(rstd * gate) * (rstd * up)
+    row_rstd(a, a.ssq_ffn, e_tid, M, s_rstd);
+    const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
+    for (int it = c * 128 + e_tid; it < np * groups; it += G * 128) {
+      const int r = it / groups, f = (it % groups) * 8;
+      if (r >= M) continue;
+      float g[8], u[8], o[8];
+      sum_partials8(a, p, G, f >> 7, r, f & 127, g);
+      sum_partials8(a, p, G, half_tiles + (f >> 7), r, f & 127, u);
+      const float rs = s_rstd[r];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float gg = g[j] * rs;
+        o[j] = gg / (1.f + __expf(-gg)) * (u[j] * rs);
+      }
+      *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f) = pack8(o);
+    }
+  } else {
+    // Q/K/V: scale by rstd, rotate q and k with the row's ORIGINAL position, q packed, k / v into the cache row
+    row_rstd(a, a.ssq_next, e_tid, M, s_rstd);
+    const int half = a.dh >> 1, per_head = a.dh >> 4;          // 8-feature groups in half a head
+    for (int it = c * 128 + e_tid; it < np * p.n_tiles * 8; it += G * 128) {
+      const int k = it & 7, t = (it >> 3) % p.n_tiles, r = (it >> 3) / p.n_tiles;
+      if (r >= M) continue;
+      const int src = t / p.tiles_per_map;                       // 0 q, 1 k, 2 v
+      int f_lo, f_hi;
+      if (src == 2) {
+        f_lo = 8 * k;
+        f_hi = 64 + 8 * k;
+      } else {
+        f_lo = (k / per_head) * a.dh + (k % per_head) * 8;
+        f_hi = f_lo + half;
+      }
+      float lo[8], hi[8];
+      sum_partials8(a, p, G, t, r, f_lo, lo);
+      sum_partials8(a, p, G, t, r, f_hi, hi);
+      const float rs = s_rstd[r];
+      const int pos = __ldg(a.idx + r);
+      const int ln = (t - src * p.tiles_per_map) * CH_BF;         // first feature of the tile inside its matrix
+      bf16* dst = src == 0 ? a.q + (size_t)r * a.hd : (src == 1 ? a.kc : a.vc) + (size_t)pos * a.hd;
+      float olo[8], ohi[8];
+      if (src == 2) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          olo[j] = lo[j] * rs;
+          ohi[j] = hi[j] * rs;
+        }
+      } else {
+        const float2* tr = a.rope + (size_t)(pos % a.n_seq) * half + (f_lo % a.dh);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float2 cs = __ldg(tr + j);
+          const float x0 = lo[j] * rs, x1 = hi[j] * rs;
+          olo[j] = x0 * cs.x - x1 * cs.y;
+          ohi[j] = x1 * cs.x + x0 * cs.y;
+        }
+      }
+      *reinterpret_cast<uint4*>(dst + ln + f_lo) = pack8(olo);
+      *reinterpret_cast<uint4*>(dst + ln + f_hi) = pack8(ohi);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(CH_THREADS, 1)
+gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constant__ CUtensorMap tmW1,
+                  const __grid_constant__ CUtensorMap tmW2, const __grid_constant__ CUtensorMap tmW3,
+                  const __grid_constant__ CUtensorMap tmW4, const __grid_constant__ CUtensorMap tmW5,
+                  const __grid_constant__ CUtensorMap tmW6, const __grid_constant__ CUtensorMap tmX0,
+                  const __grid_constant__ CUtensorMap tmX1, const __grid_constant__ CUtensorMap tmX2,
+                  const __grid_constant__ ChainArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int np = a.np;
+  const int X_BYTES = np * CH_BK * 2;
+  uint8_t* sW = smem;
+  uint8_t* sX = sW + CH_W_STAGES * CH_W_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sX + CH_X_STAGES * X_BYTES);
+  // bars: wfull[W], wempty[W], xfull[X], xempty[X], accfull[2], accempty[2], xready
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * CH_W_STAGES + 2 * CH_X_STAGES + 5);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+  float* s_rstd = reinterpret_cast<float*>(s_tmem + 4);                 // [np <= 64]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t bar0 = smem_u32(bars);
+  auto wfull = [&](int s) { return bar0 + 8u * s; };
+  auto wempty = [&](int s) { return bar0 + 8u * (CH_W_STAGES + s); };
+  auto xfull = [&](int s) { return bar0 + 8u * (2 * CH_W_STAGES + s); };
+  auto xempty = [&](int s) { return bar0 + 8u * (2 * CH_W_STAGES + CH_X_STAGES + s); };
+  const uint32_t accfull0 = bar0 + 8u * (2 * CH_W_STAGES + 2 * CH_X_STAGES), accempty0 = accfull0 + 16u,
+                 xready = accfull0 + 32u;
+  const int G = (int)gridDim.x, c = (int)blockIdx.x;
+  const CUtensorMap* wmaps[7] = {&tmW0, &tmW1, &tmW2, &tmW3, &tmW4, &tmW5, &tmW6};
+  const CUtensorMap* xmaps[3] = {&tmX0, &tmX1, &tmX2};
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < CH_W_STAGES; ++s) {
+      mbar_init(wfull(s), 1);
+      mbar_init(wempty(s), 1);
+    }
+    for (int s = 0; s < CH_X_STAGES; ++s) {
+      mbar_init(xfull(s), 1);
+      mbar_init(xempty(s), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(accfull0 + 8u * i, 1);
+      mbar_init(accempty0 + 8u * i, 4);
+    }
+    mbar_init(xready, 1);
+    *s_abort = 0;
+    fence_mbar_init();
+  }
+  uint32_t tmem_cols = 32;
+  while ((int)tmem_cols < 2 * np) tmem_cols <<= 1;
+  if (warp == 2) tc_alloc(smem_u32(s_tmem), tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *s_tmem;
+
+  if (warp == 0) {
+    // ---- weight producer: walks through the unit ranges of ALL phases; weights depend on nothing
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
+        const ChainPhase& p = a.ph[pi];
+        const ChainRange rg = chain_range(p, c, G);
+        for (int u = rg.begin; u < rg.end; ++u) {
+          const int t = u / p.num_kb, kb = u % p.num_kb;
+          if (!(ok = mbar_wait(wempty(stage), phase ^ 1, s_abort))) break;
+          mbar_expect_tx(wfull(stage), CH_W_BYTES);
+          tma_load_2d(smem_u32(sW + stage * CH_W_BYTES), wmaps[p.w_map0 + t / p.tiles_per_map], kb * CH_BK,
+                      (t % p.tiles_per_map) * CH_BF, wfull(stage));
+          if (++stage == CH_W_STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---- activation loader: a phase's activations exist once the previous phase's reduction has passed its barrier
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      griddep_wait();
+      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
+        const ChainPhase& p = a.ph[pi];
+        if (pi > 0 && !(ok = mbar_wait(xready, (uint32_t)(pi - 1) & 1, s_abort))) break;
+        const ChainRange rg = chain_range(p, c, G);
+        for (int u = rg.begin; u < rg.end; ++u) {
+          const int kb = u % p.num_kb;
+          if (!(ok = mbar_wait(xempty(stage), phase ^ 1, s_abort))) break;
+          mbar_expect_tx(xfull(stage), (uint32_t)X_BYTES);
+          tma_load_2d(smem_u32(sX + stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, 0, xfull(stage));
+          if (++stage == CH_X_STAGES) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ---- MMA issue
+    if (lane == 0) {
+      const uint32_t idesc = idesc_bf16_m128(np);
+      int ws = 0, xs = 0, seg = 0;
+      uint32_t wph = 0, xph = 0;
+      bool ok = true;
+      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
+        const ChainPhase& p = a.ph[pi];
+        const ChainRange rg = chain_range(p, c, G);
+        int u = rg.begin;
+        while (u < rg.end && ok) {
+          const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
+          const int acc = seg & 1;
+          if (seg >= 2 && !(ok = mbar_wait(accempty0 + 8u * acc, (uint32_t)((seg >> 1) - 1) & 1, s_abort))) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * np);
+          bool first = true;
+          for (; u < seg_end; ++u) {
+            if (!(ok = mbar_wait(wfull(ws), wph, s_abort))) break;
+            if (!(ok = mbar_wait(xfull(xs), xph, s_abort))) break;
+            tc_fence_after();
+            const uint64_t wdesc = smem_desc_k_sw128(smem_u32(sW + ws * CH_W_BYTES));
+            const uint64_t xdesc = smem_desc_k_sw128(smem_u32(sX + xs * X_BYTES));
+#pragma unroll
+            for (int k = 0; k < CH_BK / 16; ++k)
+              tc_mma_bf16(d_tmem, wdesc + (uint64_t)(2 * k), xdesc + (uint64_t)(2 * k), idesc, (!first) | (k != 0));
+            first = false;
+            tc_commit(wempty(ws));
+            tc_commit(xempty(xs));
+            if (++ws == CH_W_STAGES) { ws = 0; wph ^= 1; }
+            if (++xs == CH_X_STAGES) { xs = 0; xph ^= 1; }
+          }
+          if (ok) tc_commit(accfull0 + 8u * acc);
+          ++seg;
+        }
+      }
+    }
+  } else {
+    // ---- epilogue warps: partial tiles, grid barriers, reductions
+    const int quarter = warp & 3;
+    const int f = quarter * 32 + lane;                     // feature inside the tile = tensor-memory lane
+    const int e_tid = (warp - 3) * 32 + lane;
+    griddep_wait();
+    const int M = *a.n_active;
+    bool ok = true;
+    int seg = 0;
+    int n_bar = 0;                                         // grid barriers passed so far in this launch
+    auto grid_barrier = [&]() -> bool {
+      __threadfence();
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      ++n_bar;
+      if (e_tid == 0) {
+        const unsigned target = a.bar_base + (unsigned)G * (unsigned)n_bar;
+        atomicAdd(a.bar, 1u);
+        const unsigned long long t0 = clock64();
+        while ((int)(ld_acquire_u32(a.bar) - target) < 0) {
+          if (*s_abort || clock64() - t0 > CH_SPIN_CYCLES) {
+            *s_abort = 1;
+            break;
+          }
+        }
+      }
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      __threadfence();
+      return *s_abort == 0;
+    };
+    if (e_tid == 0) CP(0)
+    for (int pi = 0; pi < a.n_phases && ok; ++pi) {
+      const ChainPhase& p = a.ph[pi];
+      const ChainRange rg = chain_range(p, c, G);
+      int j = 0;
+      for (int u = rg.begin; u < rg.end && ok; ++j, ++seg) {
+        const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
+        const int acc = seg & 1;
+        ok = mbar_wait(accfull0 + 8u * acc, (uint32_t)(seg >> 1) & 1, s_abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        float* dst = a.ws + ((size_t)c * CH_MAX_SEG + j) * np * CH_BF + f;
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * np);
+        for (int h = 0; h < np; h += 32) {
+          uint32_t v[32];
+          tc_ld32(taddr + h, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int r = 0; r < 32; ++r)
+            if (h + r < np) __stcg(dst + (size_t)(h + r) * CH_BF, __uint_as_float(v[r]));
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(accempty0 + 8u * acc);
+        u = seg_end;
+      }
+      if (!ok) break;
+      if (e_tid == 0) CP(1 + 4 * pi)
+      if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
+      if (e_tid == 0) CP(2 + 4 * pi)
+      chain_reduce(a, p, G, c, e_tid, M, s_rstd);
+      if (e_tid == 0) CP(3 + 4 * pi)
+      if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
+      if (e_tid == 0) CP(4 + 4 * pi)
+      if (e_tid == 0) mbar_arrive(xready);
+    }
+  }
+
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *s_abort) set_status(a.status, SL_DEV_GEMM_TIMEOUT);
+  if (warp == 2) {
+    tc_fence_after();
+    tc_dealloc(tmem_base, tmem_cols);
+  }
+}
+
+// ----------------------------------------------------------------------------------------------- host side
+size_t gemm_chain_workspace_bytes(int np_max) { return (size_t)sm_count() * CH_MAX_SEG * np_max * CH_BF * sizeof(float); }
+
+// SL_EUNSUPPORTED when the shapes do not fit (the caller then takes the one-kernel-per-contraction path).
+int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
+  if (L.m_bound < 1 || L.m_bound > 64 || L.max_rows < 1) return SL_EUNSUPPORTED;
+  if (L.d % 512 || L.F % 128 || L.hd % 128 || (L.dh != 64 && L.dh != 128)) return SL_EUNSUPPORTED;
+  const int np = L.m_bound <= 16 ? 16 : (L.m_bound <= 32 ? 32 : 64);
+  const int G = sm_count();
+  ChainArgs a = {};
+  int n = 0;
+  auto add = [&](int kind, int n_tiles, int K, int w0, int tpm, int xm) {
+    a.ph[n++] = ChainPhase{kind, n_tiles, K / CH_BK, w0, tpm, xm};
+  };
+  add(CH_O, L.d / CH_BF, L.hd, 0, L.d / CH_BF, 0);
+  add(CH_GATEUP, 2 * L.F / CH_BF, L.d, 1, L.F / CH_BF, 1);
+  add(CH_DOWN, L.d / CH_BF, L.F, 3, L.d / CH_BF, 2);
+  if (L.wq) add(CH_QKV, 3 * L.hd / CH_BF, L.d, 4, L.hd / CH_BF, 1);
+  a.n_phases = n;
+  for (int i = 0; i < n; ++i) {
+    // a CTA's range must not span more than CH_MAX_SEG feature tiles
+    const long long U = (long long)a.ph[i].n_tiles * a.ph[i].num_kb;
+    if ((U + G - 1) / G > (long long)(CH_MAX_SEG - 1) * a.ph[i].num_kb || U * (G + 1) >= (1ll << 31) || U < G)
+      return SL_EUNSUPPORTED;
+    if (a.ph[i].num_kb / (U / G) + 2 > 8) return SL_EUNSUPPORTED;       // CTAs that can meet one tile (CH_MAX_COVER)
+  }
+  a.np = np; a.d = L.d; a.F = L.F; a.hd = L.hd; a.dh = L.dh; a.n_seq = L.n_seq; a.rms_eps = L.rms_eps;
+  a.x = L.x; a.xg = (bf16*)L.xg; a.act = (bf16*)L.act;
+  a.gain_ffn = (const bf16*)L.gain_ffn; a.gain_next = (const bf16*)L.gain_next;
+  a.ssq_ffn = L.ssq_ffn; a.ssq_next = L.ssq_next;
+  a.q = (bf16*)L.q; a.kc = (bf16*)L.kc; a.vc = (bf16*)L.vc; a.idx = L.idx; a.rope = L.rope;
+  a.ws = L.ws; a.bar = L.bar; a.bar_base = *L.bar_base; a.n_active = L.n_active; a.status = L.status;
+  a.trace_mid = L.trace_mid; a.trace_out = L.trace_out;
+  CUtensorMap w[7], x[3];
+  const void* wp[7] = {L.wo, L.wg, L.wu, L.wd, L.wq, L.wk, L.wv};
+  const int wrows[7] = {L.d, L.F, L.F, L.d, L.hd, L.hd, L.hd}, wk_[7] = {L.hd, L.d, L.d, L.F, L.d, L.d, L.d};
+  for (int i = 0; i < 7; ++i) {
+    const int src = wp[i] ? i : 0;                     // unused maps repeat the first one
+    const int rc = get_tensor_map_2d(wp[src], wrows[src], wk_[src], CH_BF, &w[i]);
+    if (rc != SL_OK) return rc;
+  }
+  int rc = get_tensor_map_2d(L.attn, L.max_rows, L.hd, np, &x[0]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(L.xg, L.max_rows, L.d, np, &x[1]);
+  if (rc == SL_OK) rc = get_tensor_map_2d(L.act, L.max_rows, L.F, np, &x[2]);
+  if (rc != SL_OK) return rc;
+  const int smem = CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * np * CH_BK * 2 + 1024 + 1024;
+  static bool attr_set = false;
+  if (!attr_set) {
+    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * 64 * CH_BK * 2 + 2048));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(G);
+  cfg.blockDim = dim3(CH_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeCooperative;          // the grid barrier needs every CTA resident
+  at[0].val.cooperative = 1;
+  // programmatic dependent launch: the CTAs that find a free SM stream weights while the attention kernel still runs
+  at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[1].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  static int with_pdl = -1;                           // -1: not tried yet
+  if (with_pdl < 0) with_pdl = pdl_enabled() ? 1 : 0;
+  cfg.numAttrs = with_pdl ? 2 : 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_chain_kernel, w[0], w[1], w[2], w[3], w[4], w[5], w[6], x[0], x[1], x[2], a);
+  if (e != cudaSuccess && with_pdl) {                 // the combination of the two attributes is refused: cooperative only
+    cudaGetLastError();
+    with_pdl = 0;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, gemm_chain_kernel, w[0], w[1], w[2], w[3], w[4], w[5], w[6], x[0], x[1], x[2], a);
+  }
+  SL_CUDA_TRY(e);
+  *L.bar_base += (unsigned)(2 * n * G);               // two grid barriers per phase
+#ifdef CH_PROFILE
+  if (getenv("CH_PROFILE_PRINT")) {
+    static unsigned long long h[160 * 24];
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(h, g_ch_prof, sizeof(h));
+    unsigned long long t0 = ~0ull;
+    for (int c = 0; c < G; ++c) if (h[c * 24] && h[c * 24] < t0) t0 = h[c * 24];
+    fprintf(stderr, "CH_PROFILE phases %d np %d (us after the first CTA's start; min / mean / max over CTAs)\n", n, np);
+    const char* nm[4] = {"gemm-done", "barrier1", "reduced", "barrier2"};
+    for (int i = 0; i <= 4 * n; ++i) {
+      double mn = 1e30, mx = 0, sum = 0; int cnt = 0;
+      for (int c = 0; c < G; ++c) {
+        const unsigned long long v = h[c * 24 + i];
+        if (v < t0) continue;
+        const double d = (double)(v - t0) * 1e-3;
+        mn = d < mn ? d : mn; mx = d > mx ? d : mx; sum += d; ++cnt;
+      }
+      if (cnt) fprintf(stderr, "  %-10s ph %d  %7.2f %7.2f %7.2f\n", i == 0 ? "start" : nm[(i - 1) % 4], i == 0 ? 0 : (i - 1) / 4, mn, sum / cnt, mx);
+    }
+  }
+#endif
+  return SL_OK;
+}
+
+}  // namespace sl

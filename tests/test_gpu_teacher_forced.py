@@ -123,7 +123,7 @@ def _check_step(cfg, w_dev, ctx, out, lock_in, mask, kl_eps, prev_logits_view, p
 
 
 def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.02, w_device="cpu",
-               lock_fn=inputs.random_lock, row_bound_after_first=0):
+               lock_fn=inputs.random_lock, row_bound_after_first=0, option="gemm_stream"):
     w = inputs.make_weights(cfg, seed, dtype=torch.bfloat16, std=std, device=w_device)
     w_dev = w if w_device != "cpu" else to_dev(w)
     ctx = SL.surelock_init(cfg, w_dev, N, B)
@@ -147,7 +147,7 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     lock1 = lock_fn(B, N, n_active, seed + 1)
     l1 = lock1.to(DEV)
     if row_bound_after_first:
-        SL.surelock_set_option(ctx, "gemm_stream", 1)
+        SL.surelock_set_option(ctx, option, 1)
         SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
@@ -216,3 +216,15 @@ def test_weight_streaming_step_with_a_row_bound(n_active, bound):
     w0, w1 = _two_steps(cfg, B=B, N=512, n_prompt=128, n_active=n_active, seed=90 + n_active[0], layers=[0, 1],
                         seqs=list(range(B)), n_rows=12, w_device=DEV, row_bound_after_first=bound)
     print("worst stage errors, weight streaming:", n_active, bound, w0, w1)
+
+
+@pytest.mark.parametrize("n_active,bound", [([23], 23), ([9, 1, 14], 32), ([60], 64), ([5], 16)])
+def test_layer_chain_step_with_a_row_bound(n_active, bound):
+    """The step with the "layer_chain" option: from the second step on (M <= 64) the output projection, the SwiGLU FFN and
+    the next layer's Q/K/V projections (rotary embedding, cache scatter) of every layer run as one persistent kernel with
+    the RMSNorms folded in; stage by stage against the oracle from the traced inputs, like the kernel-per-contraction path."""
+    cfg = inputs.model_shape("llada8b", n_layers=3, vocab=8192)
+    B = len(n_active)
+    w0, w1 = _two_steps(cfg, B=B, N=512, n_prompt=128, n_active=n_active, seed=190 + n_active[0], layers=[0, 1, 2],
+                        seqs=list(range(B)), n_rows=12, w_device=DEV, row_bound_after_first=bound, option="layer_chain")
+    print("worst stage errors, layer chain:", n_active, bound, w0, w1)
