@@ -60,9 +60,9 @@ struct surelock_ctx {
   int32_t *p_idx = nullptr, *p_offsets = nullptr, *p_n = nullptr, *p_argmax = nullptr, *n_unlocked = nullptr;
   float *p_kl = nullptr, *p_conf = nullptr, *p_lse = nullptr, *p_theta = nullptr;
   bool probe_mode = false;            // run_layer: queries only, nothing is written into the caches
-  // "layer_chain" option: with at most 64 active rows the four contractions between two attention calls run as one
-  // persistent kernel per layer (gemm_chain.cu)
-  bool layer_chain = false;
+  // "layer_chain" option: with few active rows the four contractions between two attention calls run as one persistent
+  // kernel per layer (gemm_chain.cu): 1 (default) when the bound on M is at most 32, 2 up to 64, 0 never
+  int layer_chain = 1;
   float *ch_ws = nullptr, *ssq_ffn = nullptr, *ssq_next = nullptr;
   unsigned* ch_bar = nullptr;
   unsigned ch_bar_base = 0;           // arrivals on ch_bar by all launches so far (host-side count)
@@ -241,7 +241,7 @@ static int layer_front(surelock_ctx* c, int l, float* x) {
 
 static inline bool use_chain(const surelock_ctx* c) {
   return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
-         c->m_bound <= 64;
+         c->m_bound <= (c->layer_chain >= 2 ? 64 : 32);
 }
 
 // Attention, then everything up to the next attention as one persistent kernel: output projection, SwiGLU FFN and,
@@ -371,6 +371,13 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     A_(c->split.counters, (size_t)c->split.tiles * 3 * sizeof(int));
     if (rc == SL_OK && cudaMemsetAsync(c->split.counters, 0, (size_t)c->split.tiles * 3 * sizeof(int), c->st) != cudaSuccess)
       rc = SL_ECUDA;
+  }
+  if (cfg->dtype == SL_BF16) {               // workspace of the layer-chain kernel (few active rows)
+    A_(c->ch_ws, gemm_chain_workspace_bytes(64));
+    A_(c->ssq_ffn, R * (d / 32 + 1) * sizeof(float));
+    A_(c->ssq_next, R * (d / 32 + 1) * sizeof(float));
+    A_(c->ch_bar, 16);
+    if (rc == SL_OK && cudaMemsetAsync(c->ch_bar, 0, 16, c->st) != cudaSuccess) rc = SL_ECUDA;
   }
   if (cfg->dtype == SL_BF16 && V > 0) {
     A_(c->lse_part, ((V + 255) / 256) * R * sizeof(float4));
@@ -758,16 +765,8 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
   if (!strcmp(name, "layer_chain")) {
-    if (value && !c->ch_ws && c->cfg.dtype == SL_BF16) {
-      int rc = dev_alloc(c, &c->ch_ws, gemm_chain_workspace_bytes(64));
-      if (rc == SL_OK) rc = dev_alloc(c, &c->ssq_ffn, (size_t)c->R * (c->cfg.d_model / 32 + 1) * sizeof(float));
-      if (rc == SL_OK) rc = dev_alloc(c, &c->ssq_next, (size_t)c->R * (c->cfg.d_model / 32 + 1) * sizeof(float));
-      if (rc == SL_OK) rc = dev_alloc(c, &c->ch_bar, 16);
-      if (rc != SL_OK) return rc;
-      SL_CUDA_TRY(cudaMemsetAsync(c->ch_bar, 0, 16, c->st));
-      c->ch_bar_base = 0;
-    }
-    c->layer_chain = value != 0;
+    if (value < 0 || value > 2) return SL_EINVAL;
+    c->layer_chain = value;
     return SL_OK;
   }
   if (!strcmp(name, "row_bound")) { c->row_bound_opt = value > 0 ? value : 0; return SL_OK; }

@@ -31,18 +31,6 @@
 
 namespace sl {
 
-#ifdef CH_PROFILE
-__device__ unsigned long long g_ch_prof[160 * 24];
-__device__ __forceinline__ unsigned long long chtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t) :: "memory");
-  return t;
-}
-#define CP(i) { g_ch_prof[blockIdx.x * 24 + (i)] = chtime(); }
-#else
-#define CP(i) {}
-#endif
-
 constexpr int CH_THREADS = 224;          // warp 0 weight producer, 1 activation loader, 2 MMA issue, 3-6 epilogue / reductions
 constexpr int CH_BF = 128, CH_BK = 64;
 constexpr int CH_W_BYTES = CH_BF * CH_BK * 2;      // 16 KB
@@ -426,7 +414,6 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       __threadfence();
       return *s_abort == 0;
     };
-    if (e_tid == 0) CP(0)
     for (int pi = 0; pi < a.n_phases && ok; ++pi) {
       const ChainPhase& p = a.ph[pi];
       const ChainRange rg = chain_range(p, c, G);
@@ -454,13 +441,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
         u = seg_end;
       }
       if (!ok) break;
-      if (e_tid == 0) CP(1 + 4 * pi)
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
-      if (e_tid == 0) CP(2 + 4 * pi)
       chain_reduce(a, p, G, c, e_tid, M, s_rstd);
-      if (e_tid == 0) CP(3 + 4 * pi)
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
-      if (e_tid == 0) CP(4 + 4 * pi)
       if (e_tid == 0) mbar_arrive(xready);
     }
   }
@@ -551,27 +534,6 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   }
   SL_CUDA_TRY(e);
   *L.bar_base += (unsigned)(2 * n * G);               // two grid barriers per phase
-#ifdef CH_PROFILE
-  if (getenv("CH_PROFILE_PRINT")) {
-    static unsigned long long h[160 * 24];
-    cudaDeviceSynchronize();
-    cudaMemcpyFromSymbol(h, g_ch_prof, sizeof(h));
-    unsigned long long t0 = ~0ull;
-    for (int c = 0; c < G; ++c) if (h[c * 24] && h[c * 24] < t0) t0 = h[c * 24];
-    fprintf(stderr, "CH_PROFILE phases %d np %d (us after the first CTA's start; min / mean / max over CTAs)\n", n, np);
-    const char* nm[4] = {"gemm-done", "barrier1", "reduced", "barrier2"};
-    for (int i = 0; i <= 4 * n; ++i) {
-      double mn = 1e30, mx = 0, sum = 0; int cnt = 0;
-      for (int c = 0; c < G; ++c) {
-        const unsigned long long v = h[c * 24 + i];
-        if (v < t0) continue;
-        const double d = (double)(v - t0) * 1e-3;
-        mn = d < mn ? d : mn; mx = d > mx ? d : mx; sum += d; ++cnt;
-      }
-      if (cnt) fprintf(stderr, "  %-10s ph %d  %7.2f %7.2f %7.2f\n", i == 0 ? "start" : nm[(i - 1) % 4], i == 0 ? 0 : (i - 1) / 4, mn, sum / cnt, mx);
-    }
-  }
-#endif
   return SL_OK;
 }
 

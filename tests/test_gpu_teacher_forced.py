@@ -147,7 +147,9 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     lock1 = lock_fn(B, N, n_active, seed + 1)
     l1 = lock1.to(DEV)
     if row_bound_after_first:
-        SL.surelock_set_option(ctx, option, 1)
+        SL.surelock_set_option(ctx, option, 2 if option == "layer_chain" else 1)
+        if option != "layer_chain":
+            SL.surelock_set_option(ctx, "layer_chain", 0)          # so that the kernel under test really runs
         SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
@@ -220,7 +222,7 @@ def test_weight_streaming_step_with_a_row_bound(n_active, bound):
 
 @pytest.mark.parametrize("n_active,bound", [([23], 23), ([9, 1, 14], 32), ([60], 64), ([5], 16)])
 def test_layer_chain_step_with_a_row_bound(n_active, bound):
-    """The step with the "layer_chain" option: from the second step on (M <= 64) the output projection, the SwiGLU FFN and
+    """The step with the "layer_chain" option at 2 (up to 64 rows; the default, 1, stops at 32): in the second step the output projection, the SwiGLU FFN and
     the next layer's Q/K/V projections (rotary embedding, cache scatter) of every layer run as one persistent kernel with
     the RMSNorms folded in; stage by stage against the oracle from the traced inputs, like the kernel-per-contraction path."""
     cfg = inputs.model_shape("llada8b", n_layers=3, vocab=8192)
