@@ -158,7 +158,7 @@ struct ChainLaunch {
   const float2* rope;
   float* ws;
   unsigned* bar;
-  unsigned* bar_base;          // host-side count of the arrivals of all earlier launches; advanced by the launch
+  unsigned* bar_base;          // host-side count of launches since the barrier counter was last zeroed
   const int32_t* n_active;
   int32_t* status;
   float *trace_mid, *trace_out;

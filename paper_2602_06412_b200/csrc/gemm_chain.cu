@@ -57,8 +57,8 @@ struct ChainArgs {
   const int32_t* idx;
   const float2* rope;
   float* ws;                   // [grid][CH_MAX_SEG][np][128] partial tiles
-  unsigned* bar;               // ONE grid-barrier counter, never reset: every barrier of every launch adds `grid` to it
-  unsigned bar_base;           // its value before this launch (the host keeps count)
+  unsigned* bar;               // ONE grid-barrier counter: every barrier of every launch adds `grid` to it, so at a kernel's
+                               // start it is a multiple of `grid` (the host zeroes it long before it could wrap)
   const int32_t* n_active;
   int32_t* status;
   float *trace_mid, *trace_out;         // optional copies of x after the O / down reductions
@@ -121,15 +121,15 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
 }
 
 // rstd of every row from the chunk sums left by the reduction that produced x: s_rstd[r], r < np
-__device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, int e_tid, int M, float* s_rstd) {
+__device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, int e_tid, int M, int row0, float* s_rstd) {
   // four threads per row, each a strided quarter of the chunk sums (fixed order: deterministic)
   const int chunks = a.d >> 5;
   for (int r0 = 0; r0 < a.np; r0 += 32) {
     const int r = r0 + (e_tid >> 2);
     float s = 0.f;
-    if (r < M)
+    if (row0 + r < M)
       for (int c = (e_tid & 3) * 4; c < chunks; c += 16) {
-        const float4 v = __ldcg(reinterpret_cast<const float4*>(ssq + (size_t)r * chunks + c));
+        const float4 v = __ldcg(reinterpret_cast<const float4*>(ssq + (size_t)(row0 + r) * chunks + c));
         s += (v.x + v.y) + (v.z + v.w);
       }
     s += __shfl_xor_sync(0xffffffffu, s, 1);
@@ -140,8 +140,9 @@ __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, i
 }
 
 // The reduction + epilogue of one phase, spread over all epilogue threads of the grid.
+// Rows: this pass covers packed rows row0 ... row0 + np - 1 (partials and s_rstd are indexed by the row inside the pass).
 __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int e_tid, int M,
-                                             float* s_rstd) {
+                                             int row0, float* s_rstd) {
   const int np = a.np;
   if (p.kind == CH_O || p.kind == CH_DOWN) {
     // x += sum; xg = bf16(x * gain); sums of squares per (row, 32-column chunk).  A CTA takes 32-column chunks, four
@@ -154,17 +155,18 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
       for (int r0 = 0; r0 < np; r0 += 32) {
         const int r = r0 + (e_tid >> 2), n = ch * 32 + (e_tid & 3) * 8;
         float ss = 0.f;
-        if (r < M) {
+        const int rg = row0 + r;                           // packed row
+        if (r < np && rg < M) {
           float s[8];
           sum_partials8(a, p, G, n >> 7, r, n & 127, s);
-          float4* xp = reinterpret_cast<float4*>(a.x + (size_t)r * a.d + n);
+          float4* xp = reinterpret_cast<float4*>(a.x + (size_t)rg * a.d + n);
           float4 x0 = xp[0], x1 = xp[1];
           x0.x += s[0]; x0.y += s[1]; x0.z += s[2]; x0.w += s[3];
           x1.x += s[4]; x1.y += s[5]; x1.z += s[6]; x1.w += s[7];
           xp[0] = x0;
           xp[1] = x1;
           if (trace) {
-            float4* tp = reinterpret_cast<float4*>(trace + (size_t)r * a.d + n);
+            float4* tp = reinterpret_cast<float4*>(trace + (size_t)rg * a.d + n);
             tp[0] = x0;
             tp[1] = x1;
           }
@@ -181,21 +183,21 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
               o[2 * j] = xv[2 * j] * gf.x;
               o[2 * j + 1] = xv[2 * j + 1] * gf.y;
             }
-            *reinterpret_cast<uint4*>(a.xg + (size_t)r * a.d + n) = pack8(o);
+            *reinterpret_cast<uint4*>(a.xg + (size_t)rg * a.d + n) = pack8(o);
           }
         }
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-        if ((e_tid & 3) == 0 && r < M && gain) ssq[(size_t)r * chunks + ch] = ss;
+        if ((e_tid & 3) == 0 && r < np && rg < M && gain) ssq[(size_t)rg * chunks + ch] = ss;
       }
     }
   } else if (p.kind == CH_GATEUP) {
     // act = silu(rstd * gate) * (rstd * up)
-    row_rstd(a, a.ssq_ffn, e_tid, M, s_rstd);
+    row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
     const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
     for (int it = c * 128 + e_tid; it < np * groups; it += G * 128) {
       const int r = it / groups, f = (it % groups) * 8;
-      if (r >= M) continue;
+      if (row0 + r >= M) continue;
       float g[8], u[8], o[8];
       sum_partials8(a, p, G, f >> 7, r, f & 127, g);
       sum_partials8(a, p, G, half_tiles + (f >> 7), r, f & 127, u);
@@ -205,15 +207,15 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
         const float gg = g[j] * rs;
         o[j] = gg / (1.f + __expf(-gg)) * (u[j] * rs);
       }
-      *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f) = pack8(o);
+      *reinterpret_cast<uint4*>(a.act + (size_t)(row0 + r) * a.F + f) = pack8(o);
     }
   } else {
     // Q/K/V: scale by rstd, rotate q and k with the row's ORIGINAL position, q packed, k / v into the cache row
-    row_rstd(a, a.ssq_next, e_tid, M, s_rstd);
+    row_rstd(a, a.ssq_next, e_tid, M, row0, s_rstd);
     const int half = a.dh >> 1, per_head = a.dh >> 4;          // 8-feature groups in half a head
     for (int it = c * 128 + e_tid; it < np * p.n_tiles * 8; it += G * 128) {
       const int k = it & 7, t = (it >> 3) % p.n_tiles, r = (it >> 3) / p.n_tiles;
-      if (r >= M) continue;
+      if (row0 + r >= M) continue;
       const int src = t / p.tiles_per_map;                       // 0 q, 1 k, 2 v
       int f_lo, f_hi;
       if (src == 2) {
@@ -227,9 +229,9 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
       sum_partials8(a, p, G, t, r, f_lo, lo);
       sum_partials8(a, p, G, t, r, f_hi, hi);
       const float rs = s_rstd[r];
-      const int pos = __ldg(a.idx + r);
+      const int pos = __ldg(a.idx + row0 + r);
       const int ln = (t - src * p.tiles_per_map) * CH_BF;         // first feature of the tile inside its matrix
-      bf16* dst = src == 0 ? a.q + (size_t)r * a.hd : (src == 1 ? a.kc : a.vc) + (size_t)pos * a.hd;
+      bf16* dst = src == 0 ? a.q + (size_t)(row0 + r) * a.hd : (src == 1 ? a.kc : a.vc) + (size_t)pos * a.hd;
       float olo[8], ohi[8];
       if (src == 2) {
 #pragma unroll
@@ -307,6 +309,10 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *s_tmem;
+  // Rows beyond NP (the host's bound on M was too small) are processed in further passes over the same weights: slow,
+  // but every row is computed.  *n_active was written by the compaction at the start of the step.
+  const int M = *a.n_active;
+  const int n_pass = M > 0 ? (M + np - 1) / np : 0;
 
   if (warp == 0) {
     // ---- weight producer: walks through the unit ranges of ALL phases; weights depend on nothing
@@ -314,8 +320,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
-        const ChainPhase& p = a.ph[pi];
+      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+        const ChainPhase& p = a.ph[pp % a.n_phases];
         const ChainRange rg = chain_range(p, c, G);
         for (int u = rg.begin; u < rg.end; ++u) {
           const int t = u / p.num_kb, kb = u % p.num_kb;
@@ -334,15 +340,16 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       uint32_t phase = 0;
       bool ok = true;
       griddep_wait();
-      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
-        const ChainPhase& p = a.ph[pi];
-        if (pi > 0 && !(ok = mbar_wait(xready, (uint32_t)(pi - 1) & 1, s_abort))) break;
+      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+        const ChainPhase& p = a.ph[pp % a.n_phases];
+        const int row0 = (pp / a.n_phases) * np;
+        if (pp > 0 && !(ok = mbar_wait(xready, (uint32_t)(pp - 1) & 1, s_abort))) break;
         const ChainRange rg = chain_range(p, c, G);
         for (int u = rg.begin; u < rg.end; ++u) {
           const int kb = u % p.num_kb;
           if (!(ok = mbar_wait(xempty(stage), phase ^ 1, s_abort))) break;
           mbar_expect_tx(xfull(stage), (uint32_t)X_BYTES);
-          tma_load_2d(smem_u32(sX + stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, 0, xfull(stage));
+          tma_load_2d(smem_u32(sX + stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, row0, xfull(stage));
           if (++stage == CH_X_STAGES) { stage = 0; phase ^= 1; }
         }
       }
@@ -354,8 +361,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       int ws = 0, xs = 0, seg = 0;
       uint32_t wph = 0, xph = 0;
       bool ok = true;
-      for (int pi = 0; pi < a.n_phases && ok; ++pi) {
-        const ChainPhase& p = a.ph[pi];
+      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+        const ChainPhase& p = a.ph[pp % a.n_phases];
         const ChainRange rg = chain_range(p, c, G);
         int u = rg.begin;
         while (u < rg.end && ok) {
@@ -391,16 +398,23 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
     const int f = quarter * 32 + lane;                     // feature inside the tile = tensor-memory lane
     const int e_tid = (warp - 3) * 32 + lane;
     griddep_wait();
-    const int M = *a.n_active;
     bool ok = true;
     int seg = 0;
     int n_bar = 0;                                         // grid barriers passed so far in this launch
+    // The counter's value before this launch: a multiple of the grid size, and no barrier of this launch can complete
+    // before every CTA has read it here (each reads before its own first arrival), so what a CTA reads is the base
+    // plus fewer than `grid` arrivals.
+    unsigned bar_base = 0;
+    if (e_tid == 0) {
+      const unsigned v = ld_acquire_u32(a.bar);
+      bar_base = v - v % (unsigned)G;
+    }
     auto grid_barrier = [&]() -> bool {
       __threadfence();
       asm volatile("bar.sync 1, 128;" ::: "memory");
       ++n_bar;
       if (e_tid == 0) {
-        const unsigned target = a.bar_base + (unsigned)G * (unsigned)n_bar;
+        const unsigned target = bar_base + (unsigned)G * (unsigned)n_bar;
         atomicAdd(a.bar, 1u);
         const unsigned long long t0 = clock64();
         while ((int)(ld_acquire_u32(a.bar) - target) < 0) {
@@ -414,8 +428,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       __threadfence();
       return *s_abort == 0;
     };
-    for (int pi = 0; pi < a.n_phases && ok; ++pi) {
-      const ChainPhase& p = a.ph[pi];
+    for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+      const ChainPhase& p = a.ph[pp % a.n_phases];
+      const int row0 = (pp / a.n_phases) * np;
       const ChainRange rg = chain_range(p, c, G);
       int j = 0;
       for (int u = rg.begin; u < rg.end && ok; ++j, ++seg) {
@@ -442,7 +457,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       }
       if (!ok) break;
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
-      chain_reduce(a, p, G, c, e_tid, M, s_rstd);
+      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd);
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
       if (e_tid == 0) mbar_arrive(xready);
     }
@@ -489,7 +504,7 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   a.gain_ffn = (const bf16*)L.gain_ffn; a.gain_next = (const bf16*)L.gain_next;
   a.ssq_ffn = L.ssq_ffn; a.ssq_next = L.ssq_next;
   a.q = (bf16*)L.q; a.kc = (bf16*)L.kc; a.vc = (bf16*)L.vc; a.idx = L.idx; a.rope = L.rope;
-  a.ws = L.ws; a.bar = L.bar; a.bar_base = *L.bar_base; a.n_active = L.n_active; a.status = L.status;
+  a.ws = L.ws; a.bar = L.bar; a.n_active = L.n_active; a.status = L.status;
   a.trace_mid = L.trace_mid; a.trace_out = L.trace_out;
   CUtensorMap w[7], x[3];
   const void* wp[7] = {L.wo, L.wg, L.wu, L.wd, L.wq, L.wk, L.wv};
@@ -533,7 +548,11 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
     e = cudaLaunchKernelEx(&cfg, gemm_chain_kernel, w[0], w[1], w[2], w[3], w[4], w[5], w[6], x[0], x[1], x[2], a);
   }
   SL_CUDA_TRY(e);
-  *L.bar_base += (unsigned)(2 * n * G);               // two grid barriers per phase
+  // the barrier counter only grows: zero it (in stream order, between two launches) long before it could wrap
+  if (++*L.bar_base >= (1u << 16)) {
+    *L.bar_base = 0;
+    SL_CUDA_TRY(cudaMemsetAsync(L.bar, 0, sizeof(unsigned), st));
+  }
   return SL_OK;
 }
 
