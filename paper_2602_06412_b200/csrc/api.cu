@@ -61,7 +61,7 @@ struct surelock_ctx {
   float *p_kl = nullptr, *p_conf = nullptr, *p_lse = nullptr, *p_theta = nullptr;
   bool probe_mode = false;            // run_layer: queries only, nothing is written into the caches
   // "layer_chain" option: with few active rows the four contractions between two attention calls run as one persistent
-  // kernel per layer (gemm_chain.cu): 1 (default) when the bound on M is at most 32, 2 up to 64, 0 never
+  // kernel per layer (gemm_chain.cu): 1 (default) when the bound on M is at most 64, 0 never
   int layer_chain = 1;
   float *ch_ws = nullptr, *ssq_ffn = nullptr, *ssq_next = nullptr;
   unsigned* ch_bar = nullptr;
@@ -241,7 +241,7 @@ static int layer_front(surelock_ctx* c, int l, float* x) {
 
 static inline bool use_chain(const surelock_ctx* c) {
   return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
-         c->m_bound <= (c->layer_chain >= 2 ? 64 : 32);
+         c->m_bound <= 64;
 }
 
 // Attention, then everything up to the next attention as one persistent kernel: output projection, SwiGLU FFN and,
@@ -765,7 +765,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
   if (!strcmp(name, "layer_chain")) {
-    if (value < 0 || value > 2) return SL_EINVAL;
+    if (value < 0 || value > 1) return SL_EINVAL;
     c->layer_chain = value;
     return SL_OK;
   }

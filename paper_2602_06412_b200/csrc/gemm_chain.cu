@@ -79,27 +79,49 @@ __device__ __forceinline__ ChainRange chain_range(const ChainPhase& p, int c, in
   return ChainRange{c * U / G, (c + 1) * U / G};
 }
 
-// Sum of the partial tiles of feature tile t, row r, 8 consecutive features starting at f (inside the tile), in CTA
-// order (deterministic).  The CTAs whose unit ranges meet the tile are consecutive, at most CH_MAX_COVER of them
-// (checked on the host); all their loads are issued before the first sum so that the L2 latencies overlap.
+// Where a tile's partials lie, looked up instead of derived (the derivation is a dozen integer divisions, which made
+// the reductions ALU-bound): per phase and tile, the first CTA whose unit range meets the tile and how many consecutive
+// CTAs do (at most CH_MAX_COVER, checked on the host); per phase and CTA, the first tile of its range.  Filled once per
+// kernel by all threads.
 constexpr int CH_MAX_COVER = 8;
-__device__ __forceinline__ void sum_partials8(const ChainArgs& a, const ChainPhase& p, int G, int t, int r, int f, float* out) {
-  const int U = p.n_tiles * p.num_kb, u0 = t * p.num_kb, u1 = u0 + p.num_kb;
-  int c0 = u0 * G / U;
-  while (c0 > 0 && c0 * U / G > u0) --c0;
-  while ((c0 + 1) * U / G <= u0) ++c0;
+constexpr int CH_TAB_TILES = 512, CH_TAB_CTAS = 160;
+struct ChainTables {
+  int cover[CH_MAX_PHASES][CH_TAB_TILES];                  // first CTA | count << 16
+  short first_tile[CH_MAX_PHASES][CH_TAB_CTAS];
+};
+__device__ __forceinline__ void chain_fill_tables(const ChainArgs& a, int G, ChainTables* tb) {
+  for (int i = threadIdx.x; i < a.n_phases * CH_TAB_TILES; i += blockDim.x) {
+    const int pi = i / CH_TAB_TILES, t = i % CH_TAB_TILES;
+    const ChainPhase& p = a.ph[pi];
+    if (t >= p.n_tiles) continue;
+    const int U = p.n_tiles * p.num_kb, u0 = t * p.num_kb, u1 = u0 + p.num_kb;
+    int c0 = u0 * G / U;
+    while (c0 > 0 && c0 * U / G > u0) --c0;
+    while ((c0 + 1) * U / G <= u0) ++c0;
+    int n = 0;
+    while (c0 + n < G && (c0 + n) * U / G < u1) ++n;
+    tb->cover[pi][t] = c0 | (n << 16);
+  }
+  for (int i = threadIdx.x; i < a.n_phases * CH_TAB_CTAS; i += blockDim.x) {
+    const int pi = i / CH_TAB_CTAS, cc = i % CH_TAB_CTAS;
+    const ChainPhase& p = a.ph[pi];
+    if (cc < G) tb->first_tile[pi][cc] = (short)((cc * (p.n_tiles * p.num_kb) / G) / p.num_kb);
+  }
+}
+
+// Sum of the partial tiles of feature tile t, row r, 8 consecutive features starting at f (inside the tile), in CTA
+// order (deterministic); four tiles' loads are issued before the first sum so that the L2 latencies overlap.
+__device__ __forceinline__ void sum_partials8(const ChainArgs& a, const int* cover, const short* first_tile, int t, int r,
+                                              int f, float* out) {
+  const int cv = cover[t], c0 = cv & 0xffff, n = cv >> 16;
 #pragma unroll
   for (int j = 0; j < 8; ++j) out[j] = 0.f;
-  // four tiles' loads in flight at a time
-  for (int k0 = 0; k0 < CH_MAX_COVER; k0 += 4) {
+  for (int k0 = 0; k0 < n; k0 += 4) {
     float4 v[4][2];
-    bool live[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      const int c = c0 + k0 + k, b = c * U / G;
-      live[k] = c < G && b < u1;
-      if (live[k]) {
-        const int seg = t - b / p.num_kb;                      // which of CTA c's segments this tile is
+      if (k0 + k < n) {
+        const int c = c0 + k0 + k, seg = t - first_tile[c];    // which of CTA c's segments this tile is
         const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f);
         v[k][0] = __ldcg(src);
         v[k][1] = __ldcg(src + 1);
@@ -107,12 +129,51 @@ __device__ __forceinline__ void sum_partials8(const ChainArgs& a, const ChainPha
     }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-      if (live[k]) {
+      if (k0 + k < n) {
         out[0] += v[k][0].x; out[1] += v[k][0].y; out[2] += v[k][0].z; out[3] += v[k][0].w;
         out[4] += v[k][1].x; out[5] += v[k][1].y; out[6] += v[k][1].z; out[7] += v[k][1].w;
       }
     }
-    if (!live[3]) break;
+  }
+}
+
+// Two such sums at once (same row, two (tile, feature) places): all loads of a round of both are issued before any sum,
+// so an item of the gate/up and Q/K/V reductions costs one L2 round trip per two covering CTAs (the usual number there).
+__device__ __forceinline__ void sum_partials8x2(const ChainArgs& a, const int* cover, const short* first_tile, int r, int t0,
+                                                int f0, int t1, int f1, float* out0, float* out1) {
+  const int cv0 = cover[t0], cv1 = cover[t1];
+  const int c00 = cv0 & 0xffff, n0 = cv0 >> 16, c10 = cv1 & 0xffff, n1 = cv1 >> 16;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) out0[j] = out1[j] = 0.f;
+  const int nmax = n0 > n1 ? n0 : n1;
+  for (int k0 = 0; k0 < nmax; k0 += 2) {
+    float4 v[2][2], w[2][2];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      if (k0 + k < n0) {
+        const int c = c00 + k0 + k, seg = t0 - first_tile[c];
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f0);
+        v[k][0] = __ldcg(src);
+        v[k][1] = __ldcg(src + 1);
+      }
+      if (k0 + k < n1) {
+        const int c = c10 + k0 + k, seg = t1 - first_tile[c];
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f1);
+        w[k][0] = __ldcg(src);
+        w[k][1] = __ldcg(src + 1);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      if (k0 + k < n0) {
+        out0[0] += v[k][0].x; out0[1] += v[k][0].y; out0[2] += v[k][0].z; out0[3] += v[k][0].w;
+        out0[4] += v[k][1].x; out0[5] += v[k][1].y; out0[6] += v[k][1].z; out0[7] += v[k][1].w;
+      }
+      if (k0 + k < n1) {
+        out1[0] += w[k][0].x; out1[1] += w[k][0].y; out1[2] += w[k][0].z; out1[3] += w[k][0].w;
+        out1[4] += w[k][1].x; out1[5] += w[k][1].y; out1[6] += w[k][1].z; out1[7] += w[k][1].w;
+      }
+    }
   }
 }
 
@@ -127,11 +188,16 @@ __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, i
   for (int r0 = 0; r0 < a.np; r0 += 32) {
     const int r = r0 + (e_tid >> 2);
     float s = 0.f;
-    if (row0 + r < M)
-      for (int c = (e_tid & 3) * 4; c < chunks; c += 16) {
-        const float4 v = __ldcg(reinterpret_cast<const float4*>(ssq + (size_t)(row0 + r) * chunks + c));
-        s += (v.x + v.y) + (v.z + v.w);
+    if (row0 + r < M) {
+      const float4* src = reinterpret_cast<const float4*>(ssq + (size_t)(row0 + r) * chunks);
+      for (int c = (e_tid & 3); c < (chunks >> 2); c += 32) {          // eight loads in flight
+        float4 v[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[k] = c + 4 * k < (chunks >> 2) ? __ldcg(src + c + 4 * k) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 8; ++k) s += (v[k].x + v[k].y) + (v[k].z + v[k].w);
       }
+    }
     s += __shfl_xor_sync(0xffffffffu, s, 1);
     s += __shfl_xor_sync(0xffffffffu, s, 2);
     if ((e_tid & 3) == 0 && r < a.np) s_rstd[r] = rsqrtf(s / (float)a.d + a.rms_eps);
@@ -142,7 +208,7 @@ __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, i
 // The reduction + epilogue of one phase, spread over all epilogue threads of the grid.
 // Rows: this pass covers packed rows row0 ... row0 + np - 1 (partials and s_rstd are indexed by the row inside the pass).
 __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int e_tid, int M,
-                                             int row0, float* s_rstd) {
+                                             int row0, float* s_rstd, const int* cover, const short* first_tile) {
   const int np = a.np;
   if (p.kind == CH_O || p.kind == CH_DOWN) {
     // x += sum; xg = bf16(x * gain); sums of squares per (row, 32-column chunk).  A CTA takes 32-column chunks, four
@@ -158,7 +224,7 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
         const int rg = row0 + r;                           // packed row
         if (r < np && rg < M) {
           float s[8];
-          sum_partials8(a, p, G, n >> 7, r, n & 127, s);
+          sum_partials8(a, cover, first_tile, n >> 7, r, n & 127, s);
           float4* xp = reinterpret_cast<float4*>(a.x + (size_t)rg * a.d + n);
           float4 x0 = xp[0], x1 = xp[1];
           x0.x += s[0]; x0.y += s[1]; x0.z += s[2]; x0.w += s[3];
@@ -195,19 +261,38 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     // act = silu(rstd * gate) * (rstd * up)
     row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
     const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
-    for (int it = c * 128 + e_tid; it < np * groups; it += G * 128) {
-      const int r = it / groups, f = (it % groups) * 8;
-      if (row0 + r >= M) continue;
-      float g[8], u[8], o[8];
-      sum_partials8(a, p, G, f >> 7, r, f & 127, g);
-      sum_partials8(a, p, G, half_tiles + (f >> 7), r, f & 127, u);
-      const float rs = s_rstd[r];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float gg = g[j] * rs;
-        o[j] = gg / (1.f + __expf(-gg)) * (u[j] * rs);
+    const int stride = G * 128, dr = stride / groups, dg = stride % groups;
+    int r = (c * 128 + e_tid) / groups, fg = (c * 128 + e_tid) % groups;
+    // two items per round: the partial tiles of both are requested before either is summed
+    while (r < np && row0 + r < M) {
+      int r1 = r + dr, fg1 = fg + dg;
+      if (fg1 >= groups) {
+        fg1 -= groups;
+        ++r1;
       }
-      *reinterpret_cast<uint4*>(a.act + (size_t)(row0 + r) * a.F + f) = pack8(o);
+      const bool two = r1 < np && row0 + r1 < M;
+      const int f = fg * 8, f1 = fg1 * 8;
+      float g[2][8], u[2][8], o[8];
+      sum_partials8x2(a, cover, first_tile, r, f >> 7, f & 127, half_tiles + (f >> 7), f & 127, g[0], u[0]);
+      if (two) sum_partials8x2(a, cover, first_tile, r1, f1 >> 7, f1 & 127, half_tiles + (f1 >> 7), f1 & 127, g[1], u[1]);
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        if (i == 1 && !two) break;
+        const int ri = i ? r1 : r;
+        const float rs = s_rstd[ri];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float gg = g[i][j] * rs;
+          o[j] = gg / (1.f + __expf(-gg)) * (u[i][j] * rs);
+        }
+        *reinterpret_cast<uint4*>(a.act + (size_t)(row0 + ri) * a.F + (i ? f1 : f)) = pack8(o);
+      }
+      r = r1 + dr;
+      fg = fg1 + dg;
+      if (fg >= groups) {
+        fg -= groups;
+        ++r;
+      }
     }
   } else {
     // Q/K/V: scale by rstd, rotate q and k with the row's ORIGINAL position, q packed, k / v into the cache row
@@ -226,8 +311,7 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
         f_hi = f_lo + half;
       }
       float lo[8], hi[8];
-      sum_partials8(a, p, G, t, r, f_lo, lo);
-      sum_partials8(a, p, G, t, r, f_hi, hi);
+      sum_partials8x2(a, cover, first_tile, r, t, f_lo, t, f_hi, lo, hi);
       const float rs = s_rstd[r];
       const int pos = __ldg(a.idx + row0 + r);
       const int ln = (t - src * p.tiles_per_map) * CH_BF;         // first feature of the tile inside its matrix
@@ -273,6 +357,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * CH_W_STAGES + 2 * CH_X_STAGES + 5);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
   float* s_rstd = reinterpret_cast<float*>(s_tmem + 4);                 // [np <= 64]
+  ChainTables* tabs = reinterpret_cast<ChainTables*>(reinterpret_cast<uint8_t*>(bars) + 1024);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
   auto wfull = [&](int s) { return bar0 + 8u * s; };
@@ -302,6 +387,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
     *s_abort = 0;
     fence_mbar_init();
   }
+  chain_fill_tables(a, G, tabs);
   uint32_t tmem_cols = 32;
   while ((int)tmem_cols < 2 * np) tmem_cols <<= 1;
   if (warp == 2) tc_alloc(smem_u32(s_tmem), tmem_cols);
@@ -320,7 +406,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+      const int total_pp = n_pass * a.n_phases;
+      for (int pp = 0; pp < total_pp && ok; ++pp) {
         const ChainPhase& p = a.ph[pp % a.n_phases];
         const ChainRange rg = chain_range(p, c, G);
         for (int u = rg.begin; u < rg.end; ++u) {
@@ -429,7 +516,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       return *s_abort == 0;
     };
     for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
-      const ChainPhase& p = a.ph[pp % a.n_phases];
+      const int pi = pp % a.n_phases;
+      const ChainPhase& p = a.ph[pi];
       const int row0 = (pp / a.n_phases) * np;
       const ChainRange rg = chain_range(p, c, G);
       int j = 0;
@@ -457,7 +545,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       }
       if (!ok) break;
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
-      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd);
+      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi]);
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
       if (e_tid == 0) mbar_arrive(xready);
     }
@@ -497,7 +585,8 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
     const long long U = (long long)a.ph[i].n_tiles * a.ph[i].num_kb;
     if ((U + G - 1) / G > (long long)(CH_MAX_SEG - 1) * a.ph[i].num_kb || U * (G + 1) >= (1ll << 31) || U < G)
       return SL_EUNSUPPORTED;
-    if (a.ph[i].num_kb / (U / G) + 2 > 8) return SL_EUNSUPPORTED;       // CTAs that can meet one tile (CH_MAX_COVER)
+    if (a.ph[i].num_kb / (U / G) + 2 > CH_MAX_COVER) return SL_EUNSUPPORTED;       // CTAs that can meet one tile
+    if (a.ph[i].n_tiles > CH_TAB_TILES || G > CH_TAB_CTAS) return SL_EUNSUPPORTED;   // the lookup tables' extent
   }
   a.np = np; a.d = L.d; a.F = L.F; a.hd = L.hd; a.dh = L.dh; a.n_seq = L.n_seq; a.rms_eps = L.rms_eps;
   a.x = L.x; a.xg = (bf16*)L.xg; a.act = (bf16*)L.act;
@@ -518,11 +607,11 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   if (rc == SL_OK) rc = get_tensor_map_2d(L.xg, L.max_rows, L.d, np, &x[1]);
   if (rc == SL_OK) rc = get_tensor_map_2d(L.act, L.max_rows, L.F, np, &x[2]);
   if (rc != SL_OK) return rc;
-  const int smem = CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * np * CH_BK * 2 + 1024 + 1024;
+  auto smem_for = [](int rows) { return CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * rows * CH_BK * 2 + 1024 + 1024 + (int)sizeof(ChainTables); };
+  const int smem = smem_for(np);
   static bool attr_set = false;
   if (!attr_set) {
-    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * 64 * CH_BK * 2 + 2048));
+    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(64)));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};

@@ -147,7 +147,7 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
     lock1 = lock_fn(B, N, n_active, seed + 1)
     l1 = lock1.to(DEV)
     if row_bound_after_first:
-        SL.surelock_set_option(ctx, option, 2 if option == "layer_chain" else 1)
+        SL.surelock_set_option(ctx, option, 1)
         if option != "layer_chain":
             SL.surelock_set_option(ctx, "layer_chain", 0)          # so that the kernel under test really runs
         SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
@@ -222,7 +222,7 @@ def test_weight_streaming_step_with_a_row_bound(n_active, bound):
 
 @pytest.mark.parametrize("n_active,bound", [([23], 23), ([9, 1, 14], 32), ([60], 64), ([5], 16), ([60], 16)])
 def test_layer_chain_step_with_a_row_bound(n_active, bound):
-    """The step with the "layer_chain" option at 2 (up to 64 rows; the default, 1, stops at 32): in the second step the output projection, the SwiGLU FFN and
+    """The step with the "layer_chain" option (on by default for bounds of at most 64 rows): in the second step the output projection, the SwiGLU FFN and
     the next layer's Q/K/V projections (rotary embedding, cache scatter) of every layer run as one persistent kernel with
     the RMSNorms folded in; stage by stage against the oracle from the traced inputs, like the kernel-per-contraction path.
     Bound 16 with 60 active rows: the bound was too small, the kernel makes four passes and still computes every row."""
