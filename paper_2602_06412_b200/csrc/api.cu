@@ -197,11 +197,39 @@ static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, v
   return launch_gemm_simt(A, W, W2, C, c->n_active, c->R, n_out, K, c->cfg.dtype, epi, c->st);
 }
 
+static inline bool use_chain(const surelock_ctx* c) {
+  return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
+         c->m_bound <= 64;
+}
+
+// Lines 10-11 of Algorithm 1 for few rows: xg = bf16(x * gain) + chunk sums of squares, then the chain kernel's Q/K/V
+// phase (projection, row scale, rotary embedding, packed q, K/V into the cache rows) as its only phase.
+static int layer_front_chain(surelock_ctx* c, int l, float* x) {
+  const surelock_model_cfg& g = c->cfg;
+  ChainLaunch L = {};
+  L.attn = c->attn; L.wq = c->wq[l]; L.wk = c->wk[l]; L.wv = c->wv[l];
+  L.x = x; L.xg = c->h; L.act = c->act;
+  L.ssq_ffn = c->ssq_ffn; L.ssq_next = c->ssq_next;
+  L.q = c->q; L.kc = c->kcache(l); L.vc = c->vcache(l);
+  L.idx = c->idx; L.rope = c->rope; L.ws = c->ch_ws; L.bar = c->ch_bar; L.bar_base = &c->ch_bar_base;
+  L.n_active = c->n_active; L.status = c->status;
+  L.max_rows = c->R; L.m_bound = c->m_bound; L.d = g.d_model; L.F = g.d_ff; L.hd = g.n_heads * g.head_dim; L.dh = g.head_dim;
+  L.n_seq = c->N; L.rms_eps = g.rms_eps;
+  SL_K(K_RMSNORM, launch_norm_prep(x, c->attn_norm_g[l], c->h, c->ssq_next, c->n_active, c->R, g.d_model, c->st));
+  SL_K(K_GEMM_QKV, launch_gemm_chain(L, c->st));
+  return SL_OK;
+}
+
 // Algorithm 1 lines 10-13 for one layer on the packed rows in x (fp32 [M][d], updated in place): layer_front is lines
 // 10-11 (norm, Q/K/V, rotary embedding, cache scatter), layer_back lines 12-13 (attention, output projection, FFN).
 static int layer_front(surelock_ctx* c, int l, float* x) {
   const surelock_model_cfg& g = c->cfg;
   const int d = g.d_model, hd = g.n_heads * g.head_dim;
+  if (use_chain(c)) {
+    // few rows: the layer chain kernel with the Q/K/V phase alone (the norm folded in as in its other phases)
+    const int rc = layer_front_chain(c, l, x);
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
   SL_K(K_RMSNORM, launch_rmsnorm(x, c->attn_norm_g[l], c->h, c->n_active, c->R, d, g.rms_eps, g.dtype, c->st));
   bool fused = false;
   if (c->probe_mode) {
@@ -237,11 +265,6 @@ static int layer_front(surelock_ctx* c, int l, float* x) {
     SL_K(K_SCATTER, launch_kv_scatter(c->k, c->v, c->idx, c->n_active, c->R, hd, c->kcache(l), c->vcache(l), g.dtype, c->st));
   }
   return SL_OK;
-}
-
-static inline bool use_chain(const surelock_ctx* c) {
-  return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
-         c->m_bound <= 64;
 }
 
 // Attention, then everything up to the next attention as one persistent kernel: output projection, SwiGLU FFN and,

@@ -117,6 +117,9 @@ int launch_gather_rows(const void* table, const int32_t* tokens, const int32_t* 
                        int max_rows, int d, int table_rows, float* x, int dtype, int32_t* status, cudaStream_t st);
 int launch_rmsnorm(const float* x, const void* gain, void* h, const int32_t* n_active, int max_rows, int d,
                    float eps, int dtype, cudaStream_t st);
+// xg = bf16(x * gain) and ssq[r][d / 32] = sums of squares of x per 32-column chunk (bf16 models; rowops.cu)
+int launch_norm_prep(const float* x, const void* gain, void* xg, float* ssq, const int32_t* n_active, int max_rows, int d,
+                     cudaStream_t st);
 int build_rope_table(float2* table, int N, int head_dim, float theta, cudaStream_t st);
 // in-place rotation of q and k [M][H][dh] with position idx[r] % N
 int launch_rope(void* q, void* k, const int32_t* idx, const int32_t* n_active, int max_rows, int N, int H,
@@ -148,7 +151,7 @@ int launch_conf_gate_lock(const float* conf, const float* kl, const int32_t* idx
 
 // the contractions of a layer between two attention calls as one persistent kernel (gemm_chain.cu), bf16, few rows
 struct ChainLaunch {
-  const void *attn, *wo, *wg, *wu, *wd, *wq, *wk, *wv;   // wq == nullptr: no Q/K/V phase
+  const void *attn, *wo, *wg, *wu, *wd, *wq, *wk, *wv;   // wq == nullptr: no Q/K/V phase; wo == nullptr: ONLY that phase
   float* x;
   void *xg, *act;
   const void *gain_ffn, *gain_next;

@@ -575,10 +575,13 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   auto add = [&](int kind, int n_tiles, int K, int w0, int tpm, int xm) {
     a.ph[n++] = ChainPhase{kind, n_tiles, K / CH_BK, w0, tpm, xm};
   };
-  add(CH_O, L.d / CH_BF, L.hd, 0, L.d / CH_BF, 0);
-  add(CH_GATEUP, 2 * L.F / CH_BF, L.d, 1, L.F / CH_BF, 1);
-  add(CH_DOWN, L.d / CH_BF, L.F, 3, L.d / CH_BF, 2);
+  if (L.wo) {
+    add(CH_O, L.d / CH_BF, L.hd, 0, L.d / CH_BF, 0);
+    add(CH_GATEUP, 2 * L.F / CH_BF, L.d, 1, L.F / CH_BF, 1);
+    add(CH_DOWN, L.d / CH_BF, L.F, 3, L.d / CH_BF, 2);
+  }
   if (L.wq) add(CH_QKV, 3 * L.hd / CH_BF, L.d, 4, L.hd / CH_BF, 1);
+  if (n == 0) return SL_EINVAL;
   a.n_phases = n;
   for (int i = 0; i < n; ++i) {
     // a CTA's range must not span more than CH_MAX_SEG feature tiles
@@ -599,7 +602,7 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   const void* wp[7] = {L.wo, L.wg, L.wu, L.wd, L.wq, L.wk, L.wv};
   const int wrows[7] = {L.d, L.F, L.F, L.d, L.hd, L.hd, L.hd}, wk_[7] = {L.hd, L.d, L.d, L.F, L.d, L.d, L.d};
   for (int i = 0; i < 7; ++i) {
-    const int src = wp[i] ? i : 0;                     // unused maps repeat the first one
+    const int src = wp[i] ? i : (L.wo ? 0 : 4);        // unused maps repeat one that is in use
     const int rc = get_tensor_map_2d(wp[src], wrows[src], wk_[src], CH_BF, &w[i]);
     if (rc != SL_OK) return rc;
   }

@@ -139,6 +139,48 @@ rmsnorm_kernel(const float* __restrict__ x, const T* __restrict__ gain, T* __res
   }
 }
 
+// Input of a contraction with the RMSNorm folded in (the layer chain kernel): xg = bf16(x * gain) and, per row and
+// 32-column chunk, the sum of squares of x; the contraction's epilogue scales row r by rsqrt(mean x_r^2 + eps).
+// One CTA per row, one thread per chunk.
+__global__ void __launch_bounds__(128)
+norm_prep_kernel(const float* __restrict__ x, const bf16* __restrict__ gain, bf16* __restrict__ xg, float* __restrict__ ssq,
+                 const int32_t* __restrict__ n_active, int d) {
+  griddep_launch();
+  griddep_wait();
+  const int M = *n_active, chunks = d >> 5;
+  for (int r = blockIdx.x; r < M; r += gridDim.x) {
+    for (int ch = threadIdx.x; ch < chunks; ch += 128) {
+      const float4* xr = reinterpret_cast<const float4*>(x + (size_t)r * d + ch * 32);
+      float4 v[8];
+#pragma unroll
+      for (int k = 0; k < 8; ++k) v[k] = xr[k];
+      float ss = 0.f;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+        const uint2 g2 = *reinterpret_cast<const uint2*>(gain + ch * 32 + 4 * k);
+        const float2 g01 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g2.x));
+        const float2 g23 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&g2.y));
+        const __nv_bfloat162 a = __floats2bfloat162_rn(v[k].x * g01.x, v[k].y * g01.y);
+        const __nv_bfloat162 b = __floats2bfloat162_rn(v[k].z * g23.x, v[k].w * g23.y);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const unsigned*>(&a);
+        pk.y = *reinterpret_cast<const unsigned*>(&b);
+        *reinterpret_cast<uint2*>(xg + (size_t)r * d + ch * 32 + 4 * k) = pk;
+      }
+      ssq[(size_t)r * chunks + ch] = ss;
+    }
+  }
+}
+
+int launch_norm_prep(const float* x, const void* gain, void* xg, float* ssq, const int32_t* n_active, int max_rows, int d,
+                     cudaStream_t st) {
+  if (d % 32) return SL_EUNSUPPORTED;
+  const int g = max_rows < 1 ? 1 : (max_rows > 4 * sm_count() ? 4 * sm_count() : max_rows);
+  SL_CUDA_TRY(launch_pdl(norm_prep_kernel, dim3(g), dim3(128), 0, st, x, (const bf16*)gain, (bf16*)xg, ssq, n_active, d));
+  return SL_OK;
+}
+
 template <typename T>
 static int launch_rms_t(const float* x, const void* gain, void* h, const int32_t* n_active, int g, int d, float eps,
                          cudaStream_t st) {
