@@ -497,11 +497,11 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       bar_base = v - v % (unsigned)G;
     }
     auto grid_barrier = [&]() -> bool {
-      __threadfence();
       asm volatile("bar.sync 1, 128;" ::: "memory");
       ++n_bar;
       if (e_tid == 0) {
         const unsigned target = bar_base + (unsigned)G * (unsigned)n_bar;
+        __threadfence();                                  // release: the CTA's stores (ordered before by the bar.sync)
         atomicAdd(a.bar, 1u);
         const unsigned long long t0 = clock64();
         while ((int)(ld_acquire_u32(a.bar) - target) < 0) {
@@ -512,8 +512,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
         }
       }
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      __threadfence();
-      return *s_abort == 0;
+      return *s_abort == 0;                               // (the acquire load + bar.sync order the CTA's later loads)
     };
     for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
       const int pi = pp % a.n_phases;
@@ -547,7 +546,11 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
       chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi]);
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
-      if (e_tid == 0) mbar_arrive(xready);
+      if (e_tid == 0) {
+        // the next phase's activations were written with ordinary stores (by all CTAs) and are read by bulk tensor copies
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        mbar_arrive(xready);
+      }
     }
   }
 
