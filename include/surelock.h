@@ -233,7 +233,7 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * (default) = always the general kernel, which measured as fast or faster inside a step.  "layer_chain": with few active rows a bf16 step runs, per layer, the output projection, the SwiGLU
  * FFN and the next layer's Q/K/V projections as ONE persistent kernel that keeps the weight stream running across them
  * (RMSNorms folded in; cooperative launch, one CTA per SM): 1 (default) = when the bound on the number of active rows is
- * at most 64, 0 = never (one kernel per contraction).  "row_bound": v > 0 = the
+ * at most 128, 0 = never (one kernel per contraction).  "row_bound": v > 0 = the
  * caller's upper bound of the number of active rows of later steps, used instead of the automatic one (the row count
  * two steps back); a bound that is too small costs time, never correctness (the weight-streaming kernel then makes
  * several passes over the weights); 0 = automatic (default).  Unknown names return SL_EINVAL. */

@@ -61,7 +61,7 @@ struct surelock_ctx {
   float *p_kl = nullptr, *p_conf = nullptr, *p_lse = nullptr, *p_theta = nullptr;
   bool probe_mode = false;            // run_layer: queries only, nothing is written into the caches
   // "layer_chain" option: with few active rows the four contractions between two attention calls run as one persistent
-  // kernel per layer (gemm_chain.cu): 1 (default) when the bound on M is at most 64, 0 never
+  // kernel per layer (gemm_chain.cu): 1 (default) when the bound on M is at most 128, 0 never
   int layer_chain = 1;
   float *ch_ws = nullptr, *ssq_ffn = nullptr, *ssq_next = nullptr;
   unsigned* ch_bar = nullptr;
@@ -199,7 +199,7 @@ static int gemm(surelock_ctx* c, const void* A, const void* W, const void* W2, v
 
 static inline bool use_chain(const surelock_ctx* c) {
   return c->layer_chain && c->ch_ws && !c->probe_mode && c->cfg.dtype == SL_BF16 && c->gemm_impl == 0 && c->m_bound >= 1 &&
-         c->m_bound <= 64;
+         c->m_bound <= 128;
 }
 
 // Lines 10-11 of Algorithm 1 for few rows: xg = bf16(x * gain) + chunk sums of squares, then the chain kernel's Q/K/V
@@ -396,7 +396,7 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
       rc = SL_ECUDA;
   }
   if (cfg->dtype == SL_BF16) {               // workspace of the layer-chain kernel (few active rows)
-    A_(c->ch_ws, gemm_chain_workspace_bytes(64));
+    A_(c->ch_ws, gemm_chain_workspace_bytes(128));
     A_(c->ssq_ffn, R * (d / 32 + 1) * sizeof(float));
     A_(c->ssq_next, R * (d / 32 + 1) * sizeof(float));
     A_(c->ch_bar, 16);

@@ -34,7 +34,10 @@ namespace sl {
 constexpr int CH_THREADS = 224;          // warp 0 weight producer, 1 activation loader, 2 MMA issue, 3-6 epilogue / reductions
 constexpr int CH_BF = 128, CH_BK = 64;
 constexpr int CH_W_BYTES = CH_BF * CH_BK * 2;      // 16 KB
-constexpr int CH_W_STAGES = 11, CH_X_STAGES = 4;
+constexpr int CH_W_STAGES = 11, CH_X_STAGES = 4;     // at most; with 128 rows (16 KB per activation stage) 10 and 3
+__host__ __device__ constexpr int ch_w_stages(int np) { return np <= 64 ? CH_W_STAGES : CH_W_STAGES - 1; }
+__host__ __device__ constexpr int ch_x_stages(int np) { return np <= 64 ? CH_X_STAGES : CH_X_STAGES - 1; }
+constexpr int CH_MAX_ROWS = 128;         // rows of one pass (the N of the MMA)
 constexpr int CH_MAX_SEG = 4;            // (tile, K range) segments of one CTA in one phase
 constexpr int CH_MAX_PHASES = 4;
 constexpr unsigned long long CH_SPIN_CYCLES = 2000000000ull;   // bound of a grid-barrier wait: ~1 s
@@ -350,13 +353,14 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const int np = a.np;
   const int X_BYTES = np * CH_BK * 2;
+  const int w_stages = ch_w_stages(np), x_stages = ch_x_stages(np);
   uint8_t* sW = smem;
-  uint8_t* sX = sW + CH_W_STAGES * CH_W_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(sX + CH_X_STAGES * X_BYTES);
+  uint8_t* sX = sW + w_stages * CH_W_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(sX + x_stages * X_BYTES);
   // bars: wfull[W], wempty[W], xfull[X], xempty[X], accfull[2], accempty[2], xready
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * CH_W_STAGES + 2 * CH_X_STAGES + 5);
   volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-  float* s_rstd = reinterpret_cast<float*>(s_tmem + 4);                 // [np <= 64]
+  float* s_rstd = reinterpret_cast<float*>(s_tmem + 4);                 // [np <= 128]
   ChainTables* tabs = reinterpret_cast<ChainTables*>(reinterpret_cast<uint8_t*>(bars) + 1024);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t bar0 = smem_u32(bars);
@@ -416,7 +420,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
           mbar_expect_tx(wfull(stage), CH_W_BYTES);
           tma_load_2d(smem_u32(sW + stage * CH_W_BYTES), wmaps[p.w_map0 + t / p.tiles_per_map], kb * CH_BK,
                       (t % p.tiles_per_map) * CH_BF, wfull(stage));
-          if (++stage == CH_W_STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == w_stages) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -437,7 +441,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
           if (!(ok = mbar_wait(xempty(stage), phase ^ 1, s_abort))) break;
           mbar_expect_tx(xfull(stage), (uint32_t)X_BYTES);
           tma_load_2d(smem_u32(sX + stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, row0, xfull(stage));
-          if (++stage == CH_X_STAGES) { stage = 0; phase ^= 1; }
+          if (++stage == x_stages) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -471,8 +475,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
             first = false;
             tc_commit(wempty(ws));
             tc_commit(xempty(xs));
-            if (++ws == CH_W_STAGES) { ws = 0; wph ^= 1; }
-            if (++xs == CH_X_STAGES) { xs = 0; xph ^= 1; }
+            if (++ws == w_stages) { ws = 0; wph ^= 1; }
+            if (++xs == x_stages) { xs = 0; xph ^= 1; }
           }
           if (ok) tc_commit(accfull0 + 8u * acc);
           ++seg;
@@ -569,9 +573,9 @@ size_t gemm_chain_workspace_bytes(int np_max) { return (size_t)sm_count() * CH_M
 
 // SL_EUNSUPPORTED when the shapes do not fit (the caller then takes the one-kernel-per-contraction path).
 int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
-  if (L.m_bound < 1 || L.m_bound > 64 || L.max_rows < 1) return SL_EUNSUPPORTED;
+  if (L.m_bound < 1 || L.m_bound > CH_MAX_ROWS || L.max_rows < 1) return SL_EUNSUPPORTED;
   if (L.d % 512 || L.F % 128 || L.hd % 128 || (L.dh != 64 && L.dh != 128)) return SL_EUNSUPPORTED;
-  const int np = L.m_bound <= 16 ? 16 : (L.m_bound <= 32 ? 32 : 64);
+  const int np = L.m_bound <= 16 ? 16 : (L.m_bound <= 32 ? 32 : (L.m_bound <= 64 ? 64 : 128));
   const int G = sm_count();
   ChainArgs a = {};
   int n = 0;
@@ -613,11 +617,14 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   if (rc == SL_OK) rc = get_tensor_map_2d(L.xg, L.max_rows, L.d, np, &x[1]);
   if (rc == SL_OK) rc = get_tensor_map_2d(L.act, L.max_rows, L.F, np, &x[2]);
   if (rc != SL_OK) return rc;
-  auto smem_for = [](int rows) { return CH_W_STAGES * CH_W_BYTES + CH_X_STAGES * rows * CH_BK * 2 + 1024 + 1024 + (int)sizeof(ChainTables); };
+  auto smem_for = [](int rows) {
+    return ch_w_stages(rows) * CH_W_BYTES + ch_x_stages(rows) * rows * CH_BK * 2 + 1024 + 1024 + (int)sizeof(ChainTables);
+  };
   const int smem = smem_for(np);
   static bool attr_set = false;
   if (!attr_set) {
-    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_for(64)));
+    SL_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     smem_for(64) > smem_for(128) ? smem_for(64) : smem_for(128)));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg = {};

@@ -220,12 +220,13 @@ def test_weight_streaming_step_with_a_row_bound(n_active, bound):
     print("worst stage errors, weight streaming:", n_active, bound, w0, w1)
 
 
-@pytest.mark.parametrize("n_active,bound", [([23], 23), ([9, 1, 14], 32), ([60], 64), ([5], 16), ([60], 16)])
+@pytest.mark.parametrize("n_active,bound", [([23], 23), ([9, 1, 14], 32), ([60], 64), ([5], 16), ([60], 16), ([101], 128), ([70, 50], 120), ([150], 128)])
 def test_layer_chain_step_with_a_row_bound(n_active, bound):
-    """The step with the "layer_chain" option (on by default for bounds of at most 64 rows): in the second step the output projection, the SwiGLU FFN and
+    """The step with the "layer_chain" option (on by default for bounds of at most 128 rows): in the second step the output projection, the SwiGLU FFN and
     the next layer's Q/K/V projections (rotary embedding, cache scatter) of every layer run as one persistent kernel with
     the RMSNorms folded in; stage by stage against the oracle from the traced inputs, like the kernel-per-contraction path.
-    Bound 16 with 60 active rows: the bound was too small, the kernel makes four passes and still computes every row."""
+    Bound 16 with 60 active rows (128 with 150): the bound was too small, the kernel makes four (two) passes and still
+    computes every row."""
     cfg = inputs.model_shape("llada8b", n_layers=3, vocab=8192)
     B = len(n_active)
     w0, w1 = _two_steps(cfg, B=B, N=512, n_prompt=128, n_active=n_active, seed=190 + n_active[0], layers=[0, 1, 2],
