@@ -233,7 +233,9 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * (default) = always the general kernel, which measured as fast or faster inside a step.  "layer_chain": with few active rows a bf16 step runs, per layer, the output projection, the SwiGLU
  * FFN and the next layer's Q/K/V projections as ONE persistent kernel that keeps the weight stream running across them
  * (RMSNorms folded in; cooperative launch, one CTA per SM): 1 (default) = when the bound on the number of active rows is
- * at most 128, 0 = never (one kernel per contraction).  "row_bound": v > 0 = the
+ * at most 128, 0 = never (one kernel per contraction).  "attn_split": 1 (default) = in a bf16 step whose bound on the
+ * number of active rows is at most 128, and when batch x heads x 2 CTAs fit the GPU at one per SM, attention runs with the
+ * keys of every (sequence, head) split over several CTAs, which meet in a workspace (allocated at init); 0 = never.  "row_bound": v > 0 = the
  * caller's upper bound of the number of active rows of later steps, used instead of the automatic one (the row count
  * two steps back); a bound that is too small costs time, never correctness (the weight-streaming kernel then makes
  * several passes over the weights); 0 = automatic (default).  Unknown names return SL_EINVAL. */
@@ -249,6 +251,11 @@ int surelock_last_launch_count(surelock_ctx *ctx);
 /* Number of launches since the last surelock_reset in which a bf16 ctx with "gemm_impl" 0 ran a CUDA-core kernel
  * because the tensor-core kernel does not take the shape (host-side count; 0 for every benchmark configuration). */
 int surelock_last_fallback_count(surelock_ctx *ctx);
+
+/* Which of the kernels for few active rows the last surelock_step / surelock_layer_step call launched (host-side
+ * flags): bit 0 = the layer chain kernel ("layer_chain"), bit 1 = attention with the keys of a (sequence, head) split
+ * over several CTAs ("attn_split"). */
+int surelock_last_step_paths(surelock_ctx *ctx);
 
 /* Per-kernel-class device time of the LAST step, measured with CUDA events on the ctx stream; needs
  * surelock_set_option(ctx, "time_kernels", 1) before that step (events add a few microseconds per launch, so time

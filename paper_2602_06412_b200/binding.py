@@ -73,6 +73,7 @@ def lib() -> C.CDLL:
         "surelock_set_option": (i32, [vp, C.c_char_p, i32]),
         "surelock_last_launch_count": (i32, [vp]),
         "surelock_last_fallback_count": (i32, [vp]),
+        "surelock_last_step_paths": (i32, [vp]),
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
         "surelock_set_unlocking": (i32, [vp, C.POINTER(_UnlockParams)]),
         "surelock_probe_unlock": (i32, [vp, vp, vp, C.POINTER(_ProbeOut)]),
@@ -327,6 +328,11 @@ def surelock_last_launch_count(ctx: Ctx) -> int:
 
 def surelock_last_fallback_count(ctx: Ctx) -> int:
     return lib().surelock_last_fallback_count(ctx.handle)
+
+
+def surelock_last_step_paths(ctx: Ctx) -> int:
+    """Bit 0: the last call used the layer chain kernel; bit 1: split-key attention."""
+    return lib().surelock_last_step_paths(ctx.handle)
 
 
 KERNEL_CLASSES = ("compact", "gather", "rmsnorm", "gemm_qkv", "rope", "kv_scatter", "attention", "gemm_o",

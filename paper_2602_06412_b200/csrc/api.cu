@@ -66,6 +66,12 @@ struct surelock_ctx {
   float *ch_ws = nullptr, *ssq_ffn = nullptr, *ssq_next = nullptr;
   unsigned* ch_bar = nullptr;
   unsigned ch_bar_base = 0;           // arrivals on ch_bar by all launches so far (host-side count)
+  // "attn_split" option (default 1): with at most 128 active rows and few sequences, attention with the keys of a
+  // (sequence, head) split over several CTAs (attention_split.cu)
+  int attn_split = 1, att_S = 0;
+  int paths = 0;                      // few-row kernels the current call has taken: 1 layer chain, 2 split-key attention
+  float* att_ws = nullptr;
+  unsigned* att_cnt = nullptr;
   bool gemm_stream = false;           // "gemm_stream" option: contractions of at most 128 rows on the weight-streaming kernel
   int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
@@ -142,12 +148,24 @@ int launch_gemm_tc(const void* A, const void* W, const void* W2, void* C, const 
 int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void* Wv, void* q_out, void* k_cache,
                        void* v_cache, const int32_t* idx, const float2* rope, const int32_t* n_active, int max_rows,
                        int n_seq, int hd, int dh, int K, int32_t* status, const SplitWs& sw, cudaStream_t st);   // gemm_tc.cu
+int attention_split_plan(int B, int N, int H);
+size_t attention_split_workspace_bytes(int head_dim);
+int launch_attention_split(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
+                           int N, int H, int head_dim, int S, void* o, float* ws, unsigned* counters, int32_t* status,
+                           cudaStream_t st);
 int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
 }
 
 static int attention(surelock_ctx* c, int l) {
   const surelock_model_cfg& g = c->cfg;
+  if (g.dtype == SL_BF16 && c->gemm_impl == 0 && c->attn_split && c->att_S >= 2 && !c->probe_mode && c->m_bound >= 1 &&
+      c->m_bound <= 128) {
+    const int rc = launch_attention_split(c->q, c->kcache(l), c->vcache(l), c->row_offsets, c->R, c->B, c->N, g.n_heads,
+                                          g.head_dim, c->att_S, c->attn, c->att_ws, c->att_cnt, c->status, c->st);
+    if (rc == SL_OK) c->paths |= 2;
+    if (rc != SL_EUNSUPPORTED) return rc;
+  }
   if (g.dtype == SL_BF16 && c->gemm_impl == 0) {
     const int rc = launch_attention_tc(c->q, c->kcache(l), c->vcache(l), c->row_offsets, c->R, c->B, c->N, g.n_heads,
                                        g.head_dim, c->attn, c->status, c->st);
@@ -162,6 +180,7 @@ static int attention(surelock_ctx* c, int l) {
 static int begin_call(surelock_ctx* c) {
   const int slot = (int)(c->calls & 1);
   c->m_bound = c->R;
+  c->paths = 0;
   if (c->ev_m_valid[slot]) {
     SL_CUDA_TRY(cudaEventSynchronize(c->ev_m[slot]));
     if (c->h_m[slot] >= 0 && c->h_m[slot] <= c->R) c->m_bound = c->h_m[slot];
@@ -217,6 +236,7 @@ static int layer_front_chain(surelock_ctx* c, int l, float* x) {
   L.n_seq = c->N; L.rms_eps = g.rms_eps;
   SL_K(K_RMSNORM, launch_norm_prep(x, c->attn_norm_g[l], c->h, c->ssq_next, c->n_active, c->R, g.d_model, c->st));
   SL_K(K_GEMM_QKV, launch_gemm_chain(L, c->st));
+  c->paths |= 1;
   return SL_OK;
 }
 
@@ -290,6 +310,7 @@ static int layer_back_chain(surelock_ctx* c, int l, float* x, int next) {
   L.max_rows = c->R; L.m_bound = c->m_bound; L.d = g.d_model; L.F = g.d_ff; L.hd = g.n_heads * g.head_dim; L.dh = g.head_dim;
   L.n_seq = c->N; L.rms_eps = g.rms_eps;
   SL_K(K_GEMM_GATEUP, launch_gemm_chain(L, c->st));
+  c->paths |= 1;
   return SL_OK;
 }
 
@@ -401,6 +422,13 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     A_(c->ssq_next, R * (d / 32 + 1) * sizeof(float));
     A_(c->ch_bar, 16);
     if (rc == SL_OK && cudaMemsetAsync(c->ch_bar, 0, 16, c->st) != cudaSuccess) rc = SL_ECUDA;
+    c->att_S = attention_split_plan(batch, N, cfg->n_heads);
+    if (c->att_S >= 2) {                     // few sequences: attention with split keys for steps with few active rows
+      A_(c->att_ws, attention_split_workspace_bytes(cfg->head_dim));
+      A_(c->att_cnt, (size_t)batch * cfg->n_heads * sizeof(unsigned));
+      if (rc == SL_OK && cudaMemsetAsync(c->att_cnt, 0, (size_t)batch * cfg->n_heads * sizeof(unsigned), c->st) != cudaSuccess)
+        rc = SL_ECUDA;
+    }
   }
   if (cfg->dtype == SL_BF16 && V > 0) {
     A_(c->lse_part, ((V + 255) / 256) * R * sizeof(float4));
@@ -433,6 +461,7 @@ int surelock_reset(surelock_ctx* c) {
   c->cur = 0;
   c->calls = 0;
   c->ev_m_valid[0] = c->ev_m_valid[1] = false;
+  if (c->att_cnt) SL_CUDA_TRY(cudaMemsetAsync(c->att_cnt, 0, (size_t)c->B * c->cfg.n_heads * sizeof(unsigned), c->st));
   if (c->ch_bar) {                      // a chain kernel that gave up leaves the barrier count short: start over
     SL_CUDA_TRY(cudaMemsetAsync(c->ch_bar, 0, 16, c->st));
     c->ch_bar_base = 0;
@@ -787,6 +816,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
+  if (!strcmp(name, "attn_split")) { c->attn_split = value != 0; return SL_OK; }
   if (!strcmp(name, "layer_chain")) {
     if (value < 0 || value > 1) return SL_EINVAL;
     c->layer_chain = value;
@@ -845,6 +875,7 @@ int surelock_set_confidence_gate(surelock_ctx* c, float m_percent, const float**
 int surelock_last_launch_count(surelock_ctx* c) { return c ? c->launches : SL_EINVAL; }
 
 int surelock_last_fallback_count(surelock_ctx* c) { return c ? c->fallbacks : SL_EINVAL; }
+int surelock_last_step_paths(surelock_ctx* c) { return c ? c->paths : SL_EINVAL; }
 
 int surelock_kernel_times(surelock_ctx* c, float* ms, int32_t* launches, int n_classes) {
   if (!c || !ms || n_classes < K_NUM) return SL_EINVAL;

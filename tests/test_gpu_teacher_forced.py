@@ -123,7 +123,7 @@ def _check_step(cfg, w_dev, ctx, out, lock_in, mask, kl_eps, prev_logits_view, p
 
 
 def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.02, w_device="cpu",
-               lock_fn=inputs.random_lock, row_bound_after_first=0, option="gemm_stream"):
+               lock_fn=inputs.random_lock, row_bound_after_first=0, option="gemm_stream", expect_paths=None):
     w = inputs.make_weights(cfg, seed, dtype=torch.bfloat16, std=std, device=w_device)
     w_dev = w if w_device != "cpu" else to_dev(w)
     ctx = SL.surelock_init(cfg, w_dev, N, B)
@@ -153,6 +153,8 @@ def _two_steps(cfg, B, N, n_prompt, n_active, seed, layers, seqs, n_rows, std=0.
         SL.surelock_set_option(ctx, "row_bound", row_bound_after_first)
     out1 = SL.surelock_step(ctx, tok2.to(DEV), mask2.to(DEV), l1, 1e-3)
     assert SL.surelock_status_poll(ctx) == 0
+    if expect_paths is not None:                                     # the few-row kernels under test really ran
+        assert SL.surelock_last_step_paths(ctx) == expect_paths
     w1 = _check_step(cfg, w_dev, ctx, out1, lock1, mask2, 1e-3, out0.logits, prev_rop, layers, seqs, n_rows, seed + 7, l1,
                      tokens=tok2)
     locked = lock1.reshape(-1).bool().to(DEV)
@@ -230,5 +232,20 @@ def test_layer_chain_step_with_a_row_bound(n_active, bound):
     cfg = inputs.model_shape("llada8b", n_layers=3, vocab=8192)
     B = len(n_active)
     w0, w1 = _two_steps(cfg, B=B, N=512, n_prompt=128, n_active=n_active, seed=190 + n_active[0], layers=[0, 1, 2],
-                        seqs=list(range(B)), n_rows=12, w_device=DEV, row_bound_after_first=bound, option="layer_chain")
+                        seqs=list(range(B)), n_rows=12, w_device=DEV, row_bound_after_first=bound, option="layer_chain",
+                        expect_paths=3 if B <= 2 else 1)
     print("worst stage errors, layer chain:", n_active, bound, w0, w1)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("N,n_active", [(700, [40]), (1536, [17]), (300, [90, 30])])
+def test_split_key_attention_with_few_rows(N, n_active):
+    """Steps with at most 128 active rows and one or two sequences take the attention kernel that splits the keys of a
+    (sequence, head) over several CTAs (on by default): a key count that is no multiple of 128 (the last block is
+    masked, 6 blocks over 3 splits; 3 blocks over 2), twelve blocks over four splits, two sequences; stage by stage
+    against the oracle like every other path."""
+    cfg = inputs.model_shape("llada8b", n_layers=2, vocab=8192)
+    B = len(n_active)
+    w0, w1 = _two_steps(cfg, B=B, N=N, n_prompt=64, n_active=n_active, seed=300 + N, layers=[0, 1], seqs=list(range(B)),
+                        n_rows=12, w_device=DEV, row_bound_after_first=sum(n_active), option="layer_chain", expect_paths=3)
+    print("worst stage errors, split-key attention:", N, n_active, w0, w1)
