@@ -91,6 +91,7 @@ constexpr int CH_TAB_TILES = 512, CH_TAB_CTAS = 160;
 struct ChainTables {
   int cover[CH_MAX_PHASES][CH_TAB_TILES];                  // first CTA | count << 16
   short first_tile[CH_MAX_PHASES][CH_TAB_CTAS];
+  int2 pos[CH_MAX_ROWS];                                   // per row of the pass: original position, position in its sequence
 };
 __device__ __forceinline__ void chain_fill_tables(const ChainArgs& a, int G, ChainTables* tb) {
   for (int i = threadIdx.x; i < a.n_phases * CH_TAB_TILES; i += blockDim.x) {
@@ -211,7 +212,8 @@ __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, i
 // The reduction + epilogue of one phase, spread over all epilogue threads of the grid.
 // Rows: this pass covers packed rows row0 ... row0 + np - 1 (partials and s_rstd are indexed by the row inside the pass).
 __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int e_tid, int M,
-                                             int row0, float* s_rstd, const int* cover, const short* first_tile) {
+                                             int row0, float* s_rstd, const int* cover, const short* first_tile,
+                                             const int2* s_pos) {
   const int np = a.np;
   if (p.kind == CH_O || p.kind == CH_DOWN) {
     // x += sum; xg = bf16(x * gain); sums of squares per (row, 32-column chunk).  A CTA takes 32-column chunks, four
@@ -221,15 +223,19 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     float* trace = p.kind == CH_O ? a.trace_mid : a.trace_out;
     const int chunks = a.d >> 5;
     for (int ch = c; ch < chunks; ch += G) {
+      const int n = ch * 32 + (e_tid & 3) * 8;
+      uint4 g4 = make_uint4(0u, 0u, 0u, 0u);
+      if (gain) g4 = __ldg(reinterpret_cast<const uint4*>(gain + n));
       for (int r0 = 0; r0 < np; r0 += 32) {
-        const int r = r0 + (e_tid >> 2), n = ch * 32 + (e_tid & 3) * 8;
+        const int r = r0 + (e_tid >> 2);
         float ss = 0.f;
         const int rg = row0 + r;                           // packed row
         if (r < np && rg < M) {
+          // the residual row is requested before the partial tiles (independent loads: one round trip, not two)
+          float4* xp = reinterpret_cast<float4*>(a.x + (size_t)rg * a.d + n);
+          float4 x0 = __ldcg(xp), x1 = __ldcg(xp + 1);
           float s[8];
           sum_partials8(a, cover, first_tile, n >> 7, r, n & 127, s);
-          float4* xp = reinterpret_cast<float4*>(a.x + (size_t)rg * a.d + n);
-          float4 x0 = xp[0], x1 = xp[1];
           x0.x += s[0]; x0.y += s[1]; x0.z += s[2]; x0.w += s[3];
           x1.x += s[4]; x1.y += s[5]; x1.z += s[6]; x1.w += s[7];
           xp[0] = x0;
@@ -243,7 +249,6 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
 #pragma unroll
           for (int j = 0; j < 8; ++j) ss += xv[j] * xv[j];
           if (gain) {
-            const uint4 g4 = __ldg(reinterpret_cast<const uint4*>(gain + n));
             const __nv_bfloat162* gp = reinterpret_cast<const __nv_bfloat162*>(&g4);
             float o[8];
 #pragma unroll
@@ -262,7 +267,6 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     }
   } else if (p.kind == CH_GATEUP) {
     // act = silu(rstd * gate) * (rstd * up)
-    row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
     const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
     const int stride = G * 128, dr = stride / groups, dg = stride % groups;
     int r = (c * 128 + e_tid) / groups, fg = (c * 128 + e_tid) % groups;
@@ -299,7 +303,6 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     }
   } else {
     // Q/K/V: scale by rstd, rotate q and k with the row's ORIGINAL position, q packed, k / v into the cache row
-    row_rstd(a, a.ssq_next, e_tid, M, row0, s_rstd);
     const int half = a.dh >> 1, per_head = a.dh >> 4;          // 8-feature groups in half a head
     for (int it = c * 128 + e_tid; it < np * p.n_tiles * 8; it += G * 128) {
       const int k = it & 7, t = (it >> 3) % p.n_tiles, r = (it >> 3) / p.n_tiles;
@@ -313,12 +316,19 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
         f_lo = (k / per_head) * a.dh + (k % per_head) * 8;
         f_hi = f_lo + half;
       }
+      // position and rotation factors first: independent of the partial tiles, so one round trip for all
+      const int2 ps = s_pos[r];
+      float2 cs[8];
+      if (src != 2) {
+        const float2* tr = a.rope + (size_t)ps.y * half + (f_lo & (a.dh - 1));
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cs[j] = __ldg(tr + j);
+      }
       float lo[8], hi[8];
       sum_partials8x2(a, cover, first_tile, r, t, f_lo, t, f_hi, lo, hi);
       const float rs = s_rstd[r];
-      const int pos = __ldg(a.idx + row0 + r);
       const int ln = (t - src * p.tiles_per_map) * CH_BF;         // first feature of the tile inside its matrix
-      bf16* dst = src == 0 ? a.q + (size_t)(row0 + r) * a.hd : (src == 1 ? a.kc : a.vc) + (size_t)pos * a.hd;
+      bf16* dst = src == 0 ? a.q + (size_t)(row0 + r) * a.hd : (src == 1 ? a.kc : a.vc) + (size_t)ps.x * a.hd;
       float olo[8], ohi[8];
       if (src == 2) {
 #pragma unroll
@@ -327,13 +337,11 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
           ohi[j] = hi[j] * rs;
         }
       } else {
-        const float2* tr = a.rope + (size_t)(pos % a.n_seq) * half + (f_lo % a.dh);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const float2 cs = __ldg(tr + j);
           const float x0 = lo[j] * rs, x1 = hi[j] * rs;
-          olo[j] = x0 * cs.x - x1 * cs.y;
-          ohi[j] = x1 * cs.x + x0 * cs.y;
+          olo[j] = x0 * cs[j].x - x1 * cs[j].y;
+          ohi[j] = x1 * cs[j].x + x0 * cs[j].y;
         }
       }
       *reinterpret_cast<uint4*>(dst + ln + f_lo) = pack8(olo);
@@ -523,6 +531,16 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       const ChainPhase& p = a.ph[pi];
       const int row0 = (pp / a.n_phases) * np;
       const ChainRange rg = chain_range(p, c, G);
+      // the row scales this phase's reduction will need: their inputs are complete (the previous phase's second barrier,
+      // or the kernel before), and these warps have nothing to do until the first accumulator is full
+      if (p.kind == CH_GATEUP) row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
+      else if (p.kind == CH_QKV) {
+        for (int r = e_tid; r < np; r += 128) {            // and the rows' positions (rotary embedding, cache rows)
+          const int pos = row0 + r < M ? __ldg(a.idx + row0 + r) : 0;
+          tabs->pos[r] = make_int2(pos, pos % a.n_seq);
+        }
+        row_rstd(a, a.ssq_next, e_tid, M, row0, s_rstd);   // (ends with a barrier of these warps)
+      }
       int j = 0;
       for (int u = rg.begin; u < rg.end && ok; ++j, ++seg) {
         const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
@@ -548,7 +566,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       }
       if (!ok) break;
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
-      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi]);
+      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi], tabs->pos);
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
       if (e_tid == 0) {
         // the next phase's activations were written with ordinary stores (by all CTAs) and are read by bulk tensor copies
