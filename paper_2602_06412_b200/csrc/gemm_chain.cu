@@ -46,6 +46,7 @@ enum { CH_O = 0, CH_GATEUP = 1, CH_DOWN = 2, CH_QKV = 3 };
 
 struct ChainPhase {
   int kind, n_tiles, num_kb, w_map0, tiles_per_map, x_map;
+  int max_cover;   // bound on the CTAs whose unit ranges meet one tile
 };
 struct ChainArgs {
   ChainPhase ph[CH_MAX_PHASES];
@@ -113,6 +114,18 @@ __device__ __forceinline__ void chain_fill_tables(const ChainArgs& a, int G, Cha
   }
 }
 
+// 32 bytes with one load (L2 only): a thread's eight consecutive features of a partial tile row
+struct F8 {
+  float v[8];
+};
+__device__ __forceinline__ F8 ldcg8(const float* p) {
+  F8 r;
+  asm volatile("ld.global.cg.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]), "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7])
+               : "l"(p));
+  return r;
+}
+
 // Sum of the partial tiles of feature tile t, row r, 8 consecutive features starting at f (inside the tile), in CTA
 // order (deterministic); four tiles' loads are issued before the first sum so that the L2 latencies overlap.
 __device__ __forceinline__ void sum_partials8(const ChainArgs& a, const int* cover, const short* first_tile, int t, int r,
@@ -126,7 +139,7 @@ __device__ __forceinline__ void sum_partials8(const ChainArgs& a, const int* cov
     for (int k = 0; k < 4; ++k) {
       if (k0 + k < n) {
         const int c = c0 + k0 + k, seg = t - first_tile[c];    // which of CTA c's segments this tile is
-        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f);
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (unsigned)(((c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f));
         v[k][0] = __ldcg(src);
         v[k][1] = __ldcg(src + 1);
       }
@@ -156,13 +169,13 @@ __device__ __forceinline__ void sum_partials8x2(const ChainArgs& a, const int* c
     for (int k = 0; k < 2; ++k) {
       if (k0 + k < n0) {
         const int c = c00 + k0 + k, seg = t0 - first_tile[c];
-        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f0);
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (unsigned)(((c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f0));
         v[k][0] = __ldcg(src);
         v[k][1] = __ldcg(src + 1);
       }
       if (k0 + k < n1) {
         const int c = c10 + k0 + k, seg = t1 - first_tile[c];
-        const float4* src = reinterpret_cast<const float4*>(a.ws + (((size_t)c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f1);
+        const float4* src = reinterpret_cast<const float4*>(a.ws + (unsigned)(((c * CH_MAX_SEG + seg) * a.np + r) * CH_BF + f1));
         w[k][0] = __ldcg(src);
         w[k][1] = __ldcg(src + 1);
       }
@@ -270,35 +283,55 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
     const int stride = G * 128, dr = stride / groups, dg = stride % groups;
     int r = (c * 128 + e_tid) / groups, fg = (c * 128 + e_tid) % groups;
-    // two items per round: the partial tiles of both are requested before either is summed
-    while (r < np && row0 + r < M) {
-      int r1 = r + dr, fg1 = fg + dg;
-      if (fg1 >= groups) {
-        fg1 -= groups;
-        ++r1;
-      }
-      const bool two = r1 < np && row0 + r1 < M;
-      const int f = fg * 8, f1 = fg1 * 8;
-      float g[2][8], u[2][8], o[8];
-      sum_partials8x2(a, cover, first_tile, r, f >> 7, f & 127, half_tiles + (f >> 7), f & 127, g[0], u[0]);
-      if (two) sum_partials8x2(a, cover, first_tile, r1, f1 >> 7, f1 & 127, half_tiles + (f1 >> 7), f1 & 127, g[1], u[1]);
+    {
+      // Software pipeline (a tile is met by at most two CTAs here: checked on the host): the partial tiles of the thread's NEXT item are
+      // requested before this item is summed, so the L2 round trips of consecutive items overlap.
+      struct Part {
+        F8 g[2], u[2];
+        int ng, nu;
+      };
+      auto request = [&](int rr, int f, Part& q) {
+        const int tg = f >> 7, tu = half_tiles + tg, cg = cover[tg], cu = cover[tu];
+        q.ng = cg >> 16;
+        q.nu = cu >> 16;
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        if (i == 1 && !two) break;
-        const int ri = i ? r1 : r;
-        const float rs = s_rstd[ri];
+        for (int k = 0; k < 2; ++k) {
+          if (k < q.ng) {
+            const int cc = (cg & 0xffff) + k;
+            q.g[k] = ldcg8(a.ws + (unsigned)(((cc * CH_MAX_SEG + (tg - first_tile[cc])) * np + rr) * CH_BF + (f & 127)));
+          }
+          if (k < q.nu) {
+            const int cc = (cu & 0xffff) + k;
+            q.u[k] = ldcg8(a.ws + (unsigned)(((cc * CH_MAX_SEG + (tu - first_tile[cc])) * np + rr) * CH_BF + (f & 127)));
+          }
+        }
+      };
+      Part cur, nxt;
+      bool live = r < np && row0 + r < M;
+      if (live) request(r, fg * 8, cur);
+      while (live) {
+        int r1 = r + dr, fg1 = fg + dg;
+        if (fg1 >= groups) {
+          fg1 -= groups;
+          ++r1;
+        }
+        const bool live1 = r1 < np && row0 + r1 < M;
+        if (live1) request(r1, fg1 * 8, nxt);
+        const float rs = s_rstd[r];
+        float o[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const float gg = g[i][j] * rs;
-          o[j] = gg / (1.f + __expf(-gg)) * (u[i][j] * rs);
+          float gs = cur.g[0].v[j], us = cur.u[0].v[j];        // CTA order: deterministic
+          if (cur.ng > 1) gs += cur.g[1].v[j];
+          if (cur.nu > 1) us += cur.u[1].v[j];
+          const float gg = gs * rs;
+          o[j] = __fdividef(gg, 1.f + __expf(-gg)) * (us * rs);   // silu(g) * u; approximate division (2 ulp)
         }
-        *reinterpret_cast<uint4*>(a.act + (size_t)(row0 + ri) * a.F + (i ? f1 : f)) = pack8(o);
-      }
-      r = r1 + dr;
-      fg = fg1 + dg;
-      if (fg >= groups) {
-        fg -= groups;
-        ++r;
+        *reinterpret_cast<uint4*>(a.act + (size_t)(row0 + r) * a.F + fg * 8) = pack8(o);
+        r = r1;
+        fg = fg1;
+        live = live1;
+        cur = nxt;
       }
     }
   } else {
@@ -598,7 +631,7 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   ChainArgs a = {};
   int n = 0;
   auto add = [&](int kind, int n_tiles, int K, int w0, int tpm, int xm) {
-    a.ph[n++] = ChainPhase{kind, n_tiles, K / CH_BK, w0, tpm, xm};
+    a.ph[n++] = ChainPhase{kind, n_tiles, K / CH_BK, w0, tpm, xm, 0};
   };
   if (L.wo) {
     add(CH_O, L.d / CH_BF, L.hd, 0, L.d / CH_BF, 0);
@@ -613,7 +646,8 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
     const long long U = (long long)a.ph[i].n_tiles * a.ph[i].num_kb;
     if ((U + G - 1) / G > (long long)(CH_MAX_SEG - 1) * a.ph[i].num_kb || U * (G + 1) >= (1ll << 31) || U < G)
       return SL_EUNSUPPORTED;
-    if (a.ph[i].num_kb / (U / G) + 2 > CH_MAX_COVER) return SL_EUNSUPPORTED;       // CTAs that can meet one tile
+    a.ph[i].max_cover = (int)(a.ph[i].num_kb / (U / G)) + 2;                       // CTAs that can meet one tile
+    if (a.ph[i].max_cover > (a.ph[i].kind == CH_GATEUP ? 2 : CH_MAX_COVER)) return SL_EUNSUPPORTED;
     if (a.ph[i].n_tiles > CH_TAB_TILES || G > CH_TAB_CTAS) return SL_EUNSUPPORTED;   // the lookup tables' extent
   }
   a.np = np; a.d = L.d; a.F = L.F; a.hd = L.hd; a.dh = L.dh; a.n_seq = L.n_seq; a.rms_eps = L.rms_eps;
