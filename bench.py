@@ -497,10 +497,13 @@ def main():
                     avg_launch_ms=gemm_ms / max(gemm_launch, 1))
     else:
         ach = wbytes / (gemm_ms * 1e-3) / 1e9
-        roof = dict(kernel="gemm_tc (all GEMM launches of the step, weight streaming)", bound="hbm", achieved=ach,
+        chained = bool(SL.surelock_last_step_paths(ctx) & 1)        # few rows: the layer chain kernel ran the layers
+        name = ("gemm_chain (one launch per layer: O, gate/up, down, next Q/K/V) + gemm_tc (LM head), weight streaming"
+                if chained else "gemm_tc (all GEMM launches of the step, weight streaming)")
+        roof = dict(kernel=name, bound="hbm", achieved=ach,
                     peak=pk["hbm_gbs"], unit="GB/s", frac=ach / pk["hbm_gbs"], traffic=traffic_alg,
                     traffic_algorithmic=traffic_alg,
-                    traffic_note="weight-streaming regime: the weights are read once (ncu at M = 32: 102.0 MB read for a 100.7 MB matrix), so algorithmic bytes per average launch", peak_kind=pk_kind,
+                    traffic_note="weight-streaming regime: the weights are read once (ncu at M = 32: 102.0 MB read for a 100.7 MB matrix; 341 MB for the 335.5 MB of a chain launch), so algorithmic bytes per average launch", peak_kind=pk_kind,
                     launches_per_step=gemm_launch, avg_launch_ms=gemm_ms / max(gemm_launch, 1))
     total_k = sum(v[0] for v in acc.values())
     kernels = {k: dict(ms=round(v[0], 4), launches=v[1], share=round(v[0] / total_k, 4)) for k, v in acc.items()}
