@@ -405,6 +405,22 @@ int surelock_attention(const void *q, const void *k_cache, const void *v_cache, 
                        const int32_t *row_offsets, const int32_t *n_active, int max_rows, int B, int N, int H,
                        int head_dim, void *o, int dtype, int impl, int32_t *dev_status, void *stream);
 
+/* The same attention for FEW query rows (bf16; every sequence should have at most 128 packed rows, more cost further
+ * passes), with the keys of every (sequence, head) split over `splits` CTAs that leave partial results in `workspace` and
+ * meet there (see "attn_split" of surelock_set_option; this is the kernel a step then runs).  splits = 0 chooses the
+ * number as a step would; B * H * splits must not exceed the number of SMs and splits must not exceed 8 nor the number of
+ * 128-key blocks (SL_EUNSUPPORTED otherwise, also for head_dim other than 64 / 128 or pointers that are not 16-byte
+ * aligned).  workspace: dev, surelock_attention_split_workspace_bytes(B, H, head_dim) bytes, ZEROED by the caller before
+ * its first use (it begins with one counter per (sequence, head) that only grows) and not shared between streams.
+ * diag_skip: -1 in normal use.  >= 0 is a failure-detection diagnostic: CTA number diag_skip (< B * H * splits) does not
+ * arrive at the meeting of its (sequence, head), so the bounded wait (~0.2 s) of its siblings runs out: they store
+ * device status 3 (see surelock_status_poll) in *dev_status and the kernel returns with o of that pair undefined; nothing hangs or traps; zero
+ * the workspace again before the next use.  Asynchronous on `stream`. */
+size_t surelock_attention_split_workspace_bytes(int B, int H, int head_dim);
+int surelock_attention_split(const void *q, const void *k_cache, const void *v_cache, const int32_t *row_offsets,
+                             int max_rows, int B, int N, int H, int head_dim, int splits, void *o, void *workspace,
+                             int diag_skip, int32_t *dev_status, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

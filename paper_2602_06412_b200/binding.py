@@ -74,6 +74,8 @@ def lib() -> C.CDLL:
         "surelock_last_launch_count": (i32, [vp]),
         "surelock_last_fallback_count": (i32, [vp]),
         "surelock_last_step_paths": (i32, [vp]),
+        "surelock_attention_split_workspace_bytes": (C.c_size_t, [i32, i32, i32]),
+        "surelock_attention_split": (i32, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, i32, vp, vp]),
         "surelock_set_confidence_gate": (i32, [vp, f32, C.POINTER(vp)]),
         "surelock_set_unlocking": (i32, [vp, C.POINTER(_UnlockParams)]),
         "surelock_probe_unlock": (i32, [vp, vp, vp, C.POINTER(_ProbeOut)]),
@@ -407,6 +409,18 @@ def surelock_gemm_fused(A, W, W2, Cout, n_active, epilogue: int, impl: int = 0, 
     _check(lib().surelock_gemm_fused(_p(A), _p(W), _p(W2), _p(Cout), _p(n_active), A.shape[0], W.shape[0], A.shape[1],
                                      _dt(A), epilogue, impl, _p(workspace), _p(dev_status), _stream()),
            "surelock_gemm_fused")
+
+
+def surelock_attention_split_workspace_bytes(B: int, H: int, head_dim: int) -> int:
+    return lib().surelock_attention_split_workspace_bytes(B, H, head_dim)
+
+
+def surelock_attention_split(q, k_cache, v_cache, row_offsets, B: int, N: int, o, workspace, splits: int = 0,
+                             diag_skip: int = -1, dev_status=None):
+    H, dh = q.shape[1], q.shape[2]
+    _check(lib().surelock_attention_split(_p(q), _p(k_cache), _p(v_cache), _p(row_offsets), q.shape[0], B, N, H, dh,
+                                          splits, _p(o), _p(workspace), diag_skip, _p(dev_status), _stream()),
+           "surelock_attention_split")
 
 
 def surelock_attention(q, k_cache, v_cache, active_idx, row_offsets, n_active, B: int, N: int, o, impl: int = 0,

@@ -152,7 +152,7 @@ int attention_split_plan(int B, int N, int H);
 size_t attention_split_workspace_bytes(int head_dim);
 int launch_attention_split(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                            int N, int H, int head_dim, int S, void* o, float* ws, unsigned* counters, int32_t* status,
-                           cudaStream_t st);
+                           int diag_skip, cudaStream_t st);
 int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
 }
@@ -162,7 +162,7 @@ static int attention(surelock_ctx* c, int l) {
   if (g.dtype == SL_BF16 && c->gemm_impl == 0 && c->attn_split && c->att_S >= 2 && !c->probe_mode && c->m_bound >= 1 &&
       c->m_bound <= 128) {
     const int rc = launch_attention_split(c->q, c->kcache(l), c->vcache(l), c->row_offsets, c->R, c->B, c->N, g.n_heads,
-                                          g.head_dim, c->att_S, c->attn, c->att_ws, c->att_cnt, c->status, c->st);
+                                          g.head_dim, c->att_S, c->attn, c->att_ws, c->att_cnt, c->status, -1, c->st);
     if (rc == SL_OK) c->paths |= 2;
     if (rc != SL_EUNSUPPORTED) return rc;
   }
@@ -1014,6 +1014,26 @@ int surelock_update_mask(const float* conf, const int32_t* argmax, const int32_t
     return SL_EINVAL;
   return launch_update_mask(conf, argmax, active_idx, row_offsets, B, N, lo, hi, k, mask_token, tokens, mask_state,
                             n_revealed, (cudaStream_t)stream);
+}
+
+size_t surelock_attention_split_workspace_bytes(int B, int H, int head_dim) {
+  if (B <= 0 || H <= 0 || head_dim <= 0) return 0;
+  return (((size_t)B * H * sizeof(unsigned) + 255) & ~(size_t)255) + attention_split_workspace_bytes(head_dim);
+}
+
+int surelock_attention_split(const void* q, const void* k_cache, const void* v_cache, const int32_t* row_offsets,
+                             int max_rows, int B, int N, int H, int head_dim, int splits, void* o, void* workspace,
+                             int diag_skip, int32_t* dev_status, void* stream) {
+  if (!q || !k_cache || !v_cache || !row_offsets || !o || !workspace || max_rows <= 0 || B <= 0 || N <= 0 || H <= 0 ||
+      splits < 0)
+    return SL_EINVAL;
+  const int S = splits ? splits : attention_split_plan(B, N, H);
+  if (S < 1) return SL_EUNSUPPORTED;
+  if (diag_skip >= B * H * S) return SL_EINVAL;
+  unsigned* counters = static_cast<unsigned*>(workspace);
+  float* ws = reinterpret_cast<float*>(static_cast<char*>(workspace) + (((size_t)B * H * sizeof(unsigned) + 255) & ~(size_t)255));
+  return launch_attention_split(q, k_cache, v_cache, row_offsets, max_rows, B, N, H, head_dim, S, o, ws, counters, dev_status,
+                                diag_skip < 0 ? -1 : diag_skip, (cudaStream_t)stream);
 }
 
 int surelock_attention(const void* q, const void* k_cache, const void* v_cache, const int32_t* active_idx,

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(AS_THREADS, 1)
 attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
                        int S, bf16* __restrict__ o, float scale_log2, float* __restrict__ ws_o, float2* __restrict__ ws_ml,
-                       unsigned* __restrict__ counters, int32_t* status) {
+                       unsigned* __restrict__ counters, int32_t* status, int diag_skip) {
   constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
   constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
   constexpr int Q_BYTES = SLABS * SLAB_BYTES;
@@ -191,7 +191,9 @@ attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     // the S splits of this (sequence, head) meet: every barrier adds S arrivals to the pair's counter, which only grows
     auto meet = [&]() -> bool {
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (e_tid == 0) {
+      if (e_tid == 0 && (int)blockIdx.x == diag_skip) {
+        *s_meet = 1;                                     // diagnostic: this CTA does not arrive, so its siblings' wait runs out
+      } else if (e_tid == 0) {
         __threadfence();                                 // release: the CTA's stores (ordered before by the bar.sync)
         const unsigned ticket = atomicAdd(counters + bh, 1u);
         const unsigned target = (ticket / (unsigned)S + 1u) * (unsigned)S;
@@ -392,7 +394,8 @@ size_t attention_split_workspace_bytes(int head_dim) {
 
 template <int DH>
 static int launch_split_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets, int B,
-                           int N, int H, int S, void* o, float* ws, unsigned* counters, int32_t* status, cudaStream_t st) {
+                           int N, int H, int S, void* o, float* ws, unsigned* counters, int32_t* status, int diag_skip,
+                           cudaStream_t st) {
   constexpr int SLABS = DH / 64;
   const int smem = 5 * SLABS * 128 * 128 + 1024 + 512;
   static bool attr_set = false;
@@ -404,16 +407,18 @@ static int launch_split_dh(const CUtensorMap& q, const CUtensorMap& k, const CUt
   float2* ws_ml = reinterpret_cast<float2*>(ws + (size_t)sm_count() * AS_BQ * DH);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
   SL_CUDA_TRY(launch_pdl(attention_split_kernel<DH>, dim3(B * H * S), dim3(AS_THREADS), (size_t)smem, st, q, k, v, row_offsets,
-                         B, N, H, S, (bf16*)o, scale_log2, ws_o, ws_ml, counters, status));
+                         B, N, H, S, (bf16*)o, scale_log2, ws_o, ws_ml, counters, status, diag_skip));
   SL_CUDA_TRY(cudaGetLastError());
   return SL_OK;
 }
 
 // ws: attention_split_workspace_bytes(head_dim) bytes; counters: B x H words, zero before the first launch.
+// diag_skip >= 0: CTA diag_skip does not arrive at the meeting of its (sequence, head) (failure-detection test: the other
+// splits' bounded wait runs out and the kernel reports SL_DEV_ATTN_TIMEOUT); -1 otherwise.
 // SL_EUNSUPPORTED when the problem does not fit (the caller then takes the general kernel).
 int launch_attention_split(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                            int N, int H, int head_dim, int S, void* o, float* ws, unsigned* counters, int32_t* status,
-                           cudaStream_t st) {
+                           int diag_skip, cudaStream_t st) {
   if ((head_dim != 64 && head_dim != 128) || max_rows < 1 || !row_offsets || !ws || !counters) return SL_EUNSUPPORTED;
   if (S < 1 || S > AS_MAX_SPLITS || (long long)B * H * S > sm_count()) return SL_EUNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(kc) | reinterpret_cast<uintptr_t>(vc) |
@@ -427,8 +432,8 @@ int launch_attention_split(const void* q, const void* kc, const void* vc, const 
   if (rc != SL_OK) return rc;
   rc = get_tensor_map_2d(vc, (long long)B * N, cols, 128, &tv);
   if (rc != SL_OK) return rc;
-  return head_dim == 128 ? launch_split_dh<128>(tq, tk, tv, row_offsets, B, N, H, S, o, ws, counters, status, st)
-                         : launch_split_dh<64>(tq, tk, tv, row_offsets, B, N, H, S, o, ws, counters, status, st);
+  return head_dim == 128 ? launch_split_dh<128>(tq, tk, tv, row_offsets, B, N, H, S, o, ws, counters, status, diag_skip, st)
+                         : launch_split_dh<64>(tq, tk, tv, row_offsets, B, N, H, S, o, ws, counters, status, diag_skip, st);
 }
 
 }  // namespace sl

@@ -346,6 +346,84 @@ def test_attention_tensor_cores(B, N, H, dh, n_act, qscale):
     assert (o[M:] == 5.0).all()                                      # rows beyond M untouched
 
 
+def _split_attention_case(B, N, H, dh, n_act, qscale, splits, diag_skip=-1, seed=13):
+    lock = inputs.random_lock(B, N, n_act, seed)
+    idx, offs = O.active_set(lock.numpy())
+    M = len(idx)
+    g = torch.Generator().manual_seed(N + dh + seed)
+    q = (torch.randn((B * N, H, dh), generator=g) * qscale).to(torch.bfloat16)
+    Kc = torch.randn((B * N, H, dh), generator=g).to(torch.bfloat16)
+    Vc = torch.randn((B * N, H, dh), generator=g).to(torch.bfloat16)
+    o = torch.full((B * N, H, dh), 5.0, dtype=torch.bfloat16, device=DEV)
+    ws = torch.zeros(SL.surelock_attention_split_workspace_bytes(B, H, dh), dtype=torch.uint8, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    args = (q.to(DEV), Kc.to(DEV), Vc.to(DEV), torch.from_numpy(offs).to(DEV), B, N, o, ws)
+    return args, dict(splits=splits, diag_skip=diag_skip, dev_status=status), (q, Kc, Vc, offs, M, o, ws, status)
+
+
+@pytest.mark.parametrize("B,N,H,dh,n_act,qscale,splits", [
+    (1, 512, 32, 128, [23], 1.0, 0), (1, 700, 8, 128, [128], 1.0, 3), (2, 300, 4, 64, [90, 1], 1.0, 0),
+    (1, 1024, 2, 128, [64], 8.0, 4), (1, 1536, 4, 128, [150], 6.0, 6), (3, 200, 2, 128, [0, 77, 5], 1.0, 2),
+    (1, 128, 2, 64, [7], 1.0, 1), (1, 1000, 16, 128, [33], 1.0, 8)])
+def test_attention_split_keys(B, N, H, dh, n_act, qscale, splits):
+    """Attention for few query rows with the keys of a (sequence, head) split over several CTAs, alone, against the
+    oracle: the number of splits a step would choose (0) and given ones, a key count that is no multiple of 128 (the last
+    block masked), score ranges that move the running maximum inside a split (rescaling) and between splits (the
+    combination's weights), a sequence without active rows, one with more than 128 (two query tiles, the slots reused
+    after a second meeting), a single split (written directly), and a repeat on the same workspace (the counters only
+    grow)."""
+    args, kw, (q, Kc, Vc, offs, M, o, ws, status) = _split_attention_case(B, N, H, dh, n_act, qscale, splits)
+    for rep in range(2):
+        o.fill_(5.0)
+        SL.surelock_attention_split(*args, **kw)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        for b in range(B):
+            r0, r1 = offs[b], offs[b + 1]
+            if r1 == r0:
+                continue
+            ref = O.attention_rows(f64(q[r0:r1]), f64(Kc[b * N:(b + 1) * N]), f64(Vc[b * N:(b + 1) * N]))
+            assert rel_err_rows(f64(o[r0:r1]).reshape(r1 - r0, -1), ref) < 2e-2, (b, rep)
+        assert (o[M:] == 5.0).all()                                  # rows beyond M untouched
+
+
+def test_attention_split_arguments():
+    args, kw, _ = _split_attention_case(1, 512, 32, 128, [10], 1.0, 5)
+    with pytest.raises(SL.SurelockError):                            # 5 x 32 CTAs do not fit the GPU at one per SM
+        SL.surelock_attention_split(*args, **kw)
+    args, kw, _ = _split_attention_case(1, 256, 2, 128, [10], 1.0, 2, diag_skip=4)
+    with pytest.raises(SL.SurelockError):                            # there is no CTA 4
+        SL.surelock_attention_split(*args, **kw)
+
+
+def test_attention_split_bounded_wait_runs_out_and_is_reported():
+    """Failure detection without a fault: one CTA of a (sequence, head) is told not to arrive at the meeting of the
+    splits, so its siblings' bounded wait (about 0.2 s) runs out: they store device status 3 (attention timeout) and
+    the kernel returns; nothing hangs or traps.  The other heads are computed as usual, and after the workspace has
+    been zeroed again the same call gives the oracle's answer."""
+    import time
+    B, N, H, dh = 1, 512, 4, 128
+    args, kw, (q, Kc, Vc, offs, M, o, ws, status) = _split_attention_case(B, N, H, dh, [20], 1.0, 4, diag_skip=4 * 2 + 1)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    SL.surelock_attention_split(*args, **kw)
+    torch.cuda.synchronize()
+    waited = time.perf_counter() - t0
+    assert status.item() == 3                                        # attention: a bounded wait ran out
+    assert 0.05 < waited < 5.0, waited                               # it did wait, and the wait did end
+    ref = O.attention_rows(f64(q[:M]), f64(Kc[:N]), f64(Vc[:N]))    # [M][H * dh]
+    got = f64(o[:M]).reshape(M, H, dh)
+    for h in (0, 1, 3):                                              # head 2 is the one that was left incomplete
+        assert rel_err_rows(got[:, h], ref.reshape(M, H, dh)[:, h]) < 2e-2
+    status.zero_()
+    ws.zero_()
+    kw["diag_skip"] = -1
+    SL.surelock_attention_split(*args, **kw)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert rel_err_rows(f64(o[:M]).reshape(M, -1), ref) < 2e-2
+
+
 @pytest.mark.parametrize("B,N,m", [(1, 128, 20.0), (3, 200, 50.0), (4, 4096, 20.0), (2, 33, 0.0), (2, 33, 100.0), (5, 8, 37.5)])
 def test_conf_gate_lock(B, N, m):
     """Confidence gate alone: per-sequence percentile threshold and gated lock decisions against the oracle."""
