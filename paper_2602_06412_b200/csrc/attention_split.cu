@@ -267,13 +267,13 @@ attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(P_FULL));
       }
-      if (!ok) break;
       g += nj;
-      if (nj > 0) {
+      if (ok && nj > 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(bar(O_FULL), qt & 1, s_abort));   // last P V of the tile done
-        if (!ok) break;
         tc_fence_after();
       }
+      if (S > 1) ok = epilogue_warps_agree(ok);           // nobody is left alone at the meeting below
+      if (!ok) break;
       if (S == 1) {
         const float inv = 1.f / l;
         bf16* orow = o + ((long long)(row_first + trow) * H + h) * DH;

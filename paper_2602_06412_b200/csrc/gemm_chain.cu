@@ -597,7 +597,7 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
         if (lane == 0) mbar_arrive(accempty0 + 8u * acc);
         u = seg_end;
       }
-      if (!ok) break;
+      if (!epilogue_warps_agree(ok)) break;                // (a warp that gave up must not leave the others at the barrier)
       if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
       chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi], tabs->pos);
       if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete

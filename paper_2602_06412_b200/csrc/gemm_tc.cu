@@ -760,6 +760,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int m0 = mt * TC_BM, n0 = nt * out_bn;
       ok = mbar_wait(accf_bar(acc), use & 1, s_abort);
       ok = __all_sync(0xffffffffu, ok);
+      if (S > 1) ok = epilogue_warps_agree(ok);           // the splits' meeting below has barriers of all four warps
       if (!ok) break;
       tc_fence_after();
       const int trow = quarter * 32 + lane;

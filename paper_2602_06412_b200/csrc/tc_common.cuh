@@ -65,6 +65,18 @@ __device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap
       ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
       : "memory");
 }
+// AND of a flag over the 128 threads of named barrier 1 (the four epilogue warps of these kernels): after a bounded wait
+// that one warp lost and another won, all of them take the same way out, so that none is left alone at a later barrier.
+__device__ __forceinline__ bool epilogue_warps_agree(bool ok) {
+  int r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, 128, q;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"((int)ok) : "memory");
+  return r != 0;
+}
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
