@@ -238,7 +238,11 @@ int surelock_set_confidence_gate(surelock_ctx *ctx, float m_percent, const float
  * keys of every (sequence, head) split over several CTAs, which meet in a workspace (allocated at init); 0 = never.  "row_bound": v > 0 = the
  * caller's upper bound of the number of active rows of later steps, used instead of the automatic one (the row count
  * two steps back); a bound that is too small costs time, never correctness (the weight-streaming kernel then makes
- * several passes over the weights); 0 = automatic (default).  Unknown names return SL_EINVAL. */
+ * several passes over the weights); 0 = automatic (default).  "debug_chain_skip_barrier": v > 0 = failure-detection
+ * diagnostic, consumed by the NEXT launch of the layer chain kernel only: CTA v - 1 does not arrive at that launch's
+ * first grid barrier, so the bounded wait (about 1 s) of all other CTAs runs out, every role of every CTA leaves, the
+ * kernel returns and device status 2 is reported; the step's results are invalid, nothing hangs or traps, and after
+ * surelock_reset() the ctx works as before.  Unknown names return SL_EINVAL. */
 int surelock_set_option(surelock_ctx *ctx, const char *name, int value);
 
 /* The layer trace written by steps run with "trace_layers" on: *buf = dev fp32 [2L+1][B*N][d] (rows packed as in

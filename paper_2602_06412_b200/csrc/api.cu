@@ -69,6 +69,7 @@ struct surelock_ctx {
   // "attn_split" option (default 1): with at most 128 active rows and few sequences, attention with the keys of a
   // (sequence, head) split over several CTAs (attention_split.cu)
   int attn_split = 1, att_S = 0;
+  int chain_diag_skip = -1;           // "debug_chain_skip_barrier": one-shot, consumed by the next chain launch
   int paths = 0;                      // few-row kernels the current call has taken: 1 layer chain, 2 split-key attention
   float* att_ws = nullptr;
   unsigned* att_cnt = nullptr;
@@ -232,6 +233,8 @@ static int layer_front_chain(surelock_ctx* c, int l, float* x) {
   L.q = c->q; L.kc = c->kcache(l); L.vc = c->vcache(l);
   L.idx = c->idx; L.rope = c->rope; L.ws = c->ch_ws; L.bar = c->ch_bar; L.bar_base = &c->ch_bar_base;
   L.n_active = c->n_active; L.status = c->status;
+  L.diag_skip = c->chain_diag_skip;
+  c->chain_diag_skip = -1;
   L.max_rows = c->R; L.m_bound = c->m_bound; L.d = g.d_model; L.F = g.d_ff; L.hd = g.n_heads * g.head_dim; L.dh = g.head_dim;
   L.n_seq = c->N; L.rms_eps = g.rms_eps;
   SL_K(K_RMSNORM, launch_norm_prep(x, c->attn_norm_g[l], c->h, c->ssq_next, c->n_active, c->R, g.d_model, c->st));
@@ -303,6 +306,8 @@ static int layer_back_chain(surelock_ctx* c, int l, float* x, int next) {
   if (next >= 0) { L.kc = c->kcache(next); L.vc = c->vcache(next); }
   L.idx = c->idx; L.rope = c->rope; L.ws = c->ch_ws; L.bar = c->ch_bar; L.bar_base = &c->ch_bar_base;
   L.n_active = c->n_active; L.status = c->status;
+  L.diag_skip = c->chain_diag_skip;
+  c->chain_diag_skip = -1;
   if (c->trace && x == c->x) {
     L.trace_mid = c->trace + (size_t)(2 * l + 1) * c->R * g.d_model;
     L.trace_out = c->trace + (size_t)(2 * l + 2) * c->R * g.d_model;
@@ -816,6 +821,7 @@ int surelock_set_option(surelock_ctx* c, const char* name, int value) {
   if (!strcmp(name, "gemm_impl")) { c->gemm_impl = value; return SL_OK; }
   if (!strcmp(name, "strict_tc")) { c->strict_tc = value != 0; return SL_OK; }
   if (!strcmp(name, "gemm_stream")) { c->gemm_stream = value != 0; return SL_OK; }
+  if (!strcmp(name, "debug_chain_skip_barrier")) { c->chain_diag_skip = value > 0 ? value - 1 : -1; return SL_OK; }
   if (!strcmp(name, "attn_split")) { c->attn_split = value != 0; return SL_OK; }
   if (!strcmp(name, "layer_chain")) {
     if (value < 0 || value > 1) return SL_EINVAL;

@@ -164,6 +164,7 @@ struct ChainLaunch {
   unsigned* bar_base;          // host-side count of launches since the barrier counter was last zeroed
   const int32_t* n_active;
   int32_t* status;
+  int diag_skip;               // -1, or the CTA that skips its first grid barrier (failure-detection test)
   float *trace_mid, *trace_out;
   int max_rows, m_bound, d, F, hd, dh, n_seq;
   float rms_eps;

@@ -65,6 +65,7 @@ struct ChainArgs {
                                // start it is a multiple of `grid` (the host zeroes it long before it could wrap)
   const int32_t* n_active;
   int32_t* status;
+  int diag_skip;                        // failure-detection diagnostic: this CTA skips its first grid barrier (-1: none)
   float *trace_mid, *trace_out;         // optional copies of x after the O / down reductions
 };
 
@@ -544,7 +545,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
     auto grid_barrier = [&]() -> bool {
       asm volatile("bar.sync 1, 128;" ::: "memory");
       ++n_bar;
-      if (e_tid == 0) {
+      if (e_tid == 0 && c == a.diag_skip && n_bar == 1) {
+        // diagnostic: no arrival and no wait, so the other CTAs' bounded wait runs out (and, later, this one's)
+      } else if (e_tid == 0) {
         const unsigned target = bar_base + (unsigned)G * (unsigned)n_bar;
         __threadfence();                                  // release: the CTA's stores (ordered before by the bar.sync)
         atomicAdd(a.bar, 1u);
@@ -656,6 +659,7 @@ int launch_gemm_chain(const ChainLaunch& L, cudaStream_t st) {
   a.ssq_ffn = L.ssq_ffn; a.ssq_next = L.ssq_next;
   a.q = (bf16*)L.q; a.kc = (bf16*)L.kc; a.vc = (bf16*)L.vc; a.idx = L.idx; a.rope = L.rope;
   a.ws = L.ws; a.bar = L.bar; a.n_active = L.n_active; a.status = L.status;
+  a.diag_skip = L.diag_skip;
   a.trace_mid = L.trace_mid; a.trace_out = L.trace_out;
   CUtensorMap w[7], x[3];
   const void* wp[7] = {L.wo, L.wg, L.wu, L.wd, L.wq, L.wk, L.wv};

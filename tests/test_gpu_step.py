@@ -359,3 +359,46 @@ def test_cuda_core_fallback_is_counted_and_can_be_refused():
     tokens2, mask2 = inputs.make_tokens(B, N, 32, cfg2["vocab"], 42)
     SL.surelock_step(ctx2, tokens2.to(DEV), mask2.to(DEV), lock, 1e-3)
     assert SL.surelock_status_poll(ctx2) == 0 and SL.surelock_last_fallback_count(ctx2) == 0
+
+
+@pytest.mark.gpu
+def test_layer_chain_grid_barrier_wait_runs_out_and_is_reported():
+    """Failure detection without a fault, in the persistent layer chain kernel: one CTA is told to skip the first grid
+    barrier of the next launch, so every other CTA's bounded wait (about 1 s) runs out; all roles leave, tensor memory is
+    freed, the kernel returns and the step reports device status 2.  Nothing hangs or traps: after surelock_reset the same
+    context repeats, bit for bit, what a fresh context computes."""
+    import time
+    cfg = inputs.model_shape("llada8b", n_layers=1, vocab=4096)
+    w = inputs.make_weights(cfg, 77, dtype=torch.bfloat16, device=DEV)
+    B, N = 1, 256
+    tokens, mask = inputs.make_tokens(B, N, 64, cfg["vocab"], 77)
+    tokens, mask = tokens.to(DEV), mask.to(DEV)
+    lock = inputs.random_lock(B, N, [20], 78).to(DEV)
+
+    def two_steps(ctx, diag):
+        SL.surelock_step(ctx, tokens, mask, torch.zeros((B, N), dtype=torch.uint8, device=DEV), 1e-3)
+        SL.surelock_set_option(ctx, "row_bound", 20)
+        if diag:
+            SL.surelock_set_option(ctx, "debug_chain_skip_barrier", 5 + 1)
+        l1 = lock.clone()
+        out = SL.surelock_step(ctx, tokens, mask, l1, 1e-3)
+        return out, l1
+
+    ctx = SL.surelock_init(cfg, w, N, B)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    two_steps(ctx, True)
+    st = SL.surelock_status_poll(ctx)                                # synchronises
+    waited = time.perf_counter() - t0
+    assert st == 2                                                   # a bounded wait of a GEMM kernel ran out
+    assert SL.surelock_last_step_paths(ctx) & 1
+    assert 0.3 < waited < 20.0, waited                               # it did wait, and the wait did end
+    SL.surelock_reset(ctx)
+    SL.surelock_set_option(ctx, "row_bound", 0)
+    out_a, lock_a = two_steps(ctx, False)
+    assert SL.surelock_status_poll(ctx) == 0
+    logits_a = out_a.logits[:20].clone()
+    ctx2 = SL.surelock_init(cfg, w, N, B)
+    out_b, lock_b = two_steps(ctx2, False)
+    assert SL.surelock_status_poll(ctx2) == 0
+    assert torch.equal(logits_a.view(torch.int16), out_b.logits[:20].view(torch.int16)) and torch.equal(lock_a, lock_b)
