@@ -199,6 +199,19 @@ __device__ __forceinline__ uint4 pack8(const float* v) {
   return make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
 }
 
+// AND of a flag over the 192 threads of named barrier 2 (warps 1-6)
+constexpr int CH_RED_THREADS = 192;
+__device__ __forceinline__ bool chain_warps_agree(bool ok) {
+  int r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.b32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 2, 192, q;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"((int)ok) : "memory");
+  return r != 0;
+}
+
 // rstd of every row from the chunk sums left by the reduction that produced x: s_rstd[r], r < np
 __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, int e_tid, int M, int row0, float* s_rstd) {
   // four threads per row, each a strided quarter of the chunk sums (fixed order: deterministic)
@@ -225,7 +238,7 @@ __device__ __forceinline__ void row_rstd(const ChainArgs& a, const float* ssq, i
 
 // The reduction + epilogue of one phase, spread over all epilogue threads of the grid.
 // Rows: this pass covers packed rows row0 ... row0 + np - 1 (partials and s_rstd are indexed by the row inside the pass).
-__device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int e_tid, int M,
+__device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhase& p, int G, int c, int r_tid, int M,
                                              int row0, float* s_rstd, const int* cover, const short* first_tile,
                                              const int2* s_pos) {
   const int np = a.np;
@@ -237,11 +250,11 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
     float* trace = p.kind == CH_O ? a.trace_mid : a.trace_out;
     const int chunks = a.d >> 5;
     for (int ch = c; ch < chunks; ch += G) {
-      const int n = ch * 32 + (e_tid & 3) * 8;
+      const int n = ch * 32 + (r_tid & 3) * 8;
       uint4 g4 = make_uint4(0u, 0u, 0u, 0u);
       if (gain) g4 = __ldg(reinterpret_cast<const uint4*>(gain + n));
-      for (int r0 = 0; r0 < np; r0 += 32) {
-        const int r = r0 + (e_tid >> 2);
+      for (int r0 = 0; r0 < np; r0 += CH_RED_THREADS / 4) {
+        const int r = r0 + (r_tid >> 2);
         float ss = 0.f;
         const int rg = row0 + r;                           // packed row
         if (r < np && rg < M) {
@@ -276,14 +289,14 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
         }
         ss += __shfl_xor_sync(0xffffffffu, ss, 1);
         ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-        if ((e_tid & 3) == 0 && r < np && rg < M && gain) ssq[(size_t)rg * chunks + ch] = ss;
+        if ((r_tid & 3) == 0 && r < np && rg < M && gain) ssq[(size_t)rg * chunks + ch] = ss;
       }
     }
   } else if (p.kind == CH_GATEUP) {
     // act = silu(rstd * gate) * (rstd * up)
     const int groups = a.F >> 3, half_tiles = p.n_tiles >> 1;
-    const int stride = G * 128, dr = stride / groups, dg = stride % groups;
-    int r = (c * 128 + e_tid) / groups, fg = (c * 128 + e_tid) % groups;
+    const int stride = G * CH_RED_THREADS, dr = stride / groups, dg = stride % groups;
+    int r = (c * CH_RED_THREADS + r_tid) / groups, fg = (c * CH_RED_THREADS + r_tid) % groups;
     {
       // Software pipeline (a tile is met by at most two CTAs here: checked on the host): the partial tiles of the thread's NEXT item are
       // requested before this item is summed, so the L2 round trips of consecutive items overlap.
@@ -338,7 +351,7 @@ __device__ __forceinline__ void chain_reduce(const ChainArgs& a, const ChainPhas
   } else {
     // Q/K/V: scale by rstd, rotate q and k with the row's ORIGINAL position, q packed, k / v into the cache row
     const int half = a.dh >> 1, per_head = a.dh >> 4;          // 8-feature groups in half a head
-    for (int it = c * 128 + e_tid; it < np * p.n_tiles * 8; it += G * 128) {
+    for (int it = c * CH_RED_THREADS + r_tid; it < np * p.n_tiles * 8; it += G * CH_RED_THREADS) {
       const int k = it & 7, t = (it >> 3) % p.n_tiles, r = (it >> 3) / p.n_tiles;
       if (row0 + r >= M) continue;
       const int src = t / p.tiles_per_map;                       // 0 q, 1 k, 2 v
@@ -466,83 +479,31 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
         }
       }
     }
-  } else if (warp == 1) {
-    // ---- activation loader: a phase's activations exist once the previous phase's reduction has passed its barrier
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      griddep_wait();
-      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
-        const ChainPhase& p = a.ph[pp % a.n_phases];
-        const int row0 = (pp / a.n_phases) * np;
-        if (pp > 0 && !(ok = mbar_wait(xready, (uint32_t)(pp - 1) & 1, s_abort))) break;
-        const ChainRange rg = chain_range(p, c, G);
-        for (int u = rg.begin; u < rg.end; ++u) {
-          const int kb = u % p.num_kb;
-          if (!(ok = mbar_wait(xempty(stage), phase ^ 1, s_abort))) break;
-          mbar_expect_tx(xfull(stage), (uint32_t)X_BYTES);
-          tma_load_2d(smem_u32(sX + stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, row0, xfull(stage));
-          if (++stage == x_stages) { stage = 0; phase ^= 1; }
-        }
-      }
-    }
-  } else if (warp == 2) {
-    // ---- MMA issue
-    if (lane == 0) {
-      const uint32_t idesc = idesc_bf16_m128(np);
-      int ws = 0, xs = 0, seg = 0;
-      uint32_t wph = 0, xph = 0;
-      bool ok = true;
-      for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
-        const ChainPhase& p = a.ph[pp % a.n_phases];
-        const ChainRange rg = chain_range(p, c, G);
-        int u = rg.begin;
-        while (u < rg.end && ok) {
-          const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
-          const int acc = seg & 1;
-          if (seg >= 2 && !(ok = mbar_wait(accempty0 + 8u * acc, (uint32_t)((seg >> 1) - 1) & 1, s_abort))) break;
-          tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(acc * np);
-          bool first = true;
-          for (; u < seg_end; ++u) {
-            if (!(ok = mbar_wait(wfull(ws), wph, s_abort))) break;
-            if (!(ok = mbar_wait(xfull(xs), xph, s_abort))) break;
-            tc_fence_after();
-            const uint64_t wdesc = smem_desc_k_sw128(smem_u32(sW + ws * CH_W_BYTES));
-            const uint64_t xdesc = smem_desc_k_sw128(smem_u32(sX + xs * X_BYTES));
-#pragma unroll
-            for (int k = 0; k < CH_BK / 16; ++k)
-              tc_mma_bf16(d_tmem, wdesc + (uint64_t)(2 * k), xdesc + (uint64_t)(2 * k), idesc, (!first) | (k != 0));
-            first = false;
-            tc_commit(wempty(ws));
-            tc_commit(xempty(xs));
-            if (++ws == w_stages) { ws = 0; wph ^= 1; }
-            if (++xs == x_stages) { xs = 0; xph ^= 1; }
-          }
-          if (ok) tc_commit(accfull0 + 8u * acc);
-          ++seg;
-        }
-      }
-    }
   } else {
-    // ---- epilogue warps: partial tiles, grid barriers, reductions
+    // ---- warps 1-6 walk through the phases together: the activation loader (one thread of warp 1) and the MMA issuer
+    // (one thread of warp 2) do their part of a phase, warps 3-6 store the partial tiles and pass the first grid barrier,
+    // then ALL SIX warps run the phase's reduction (192 threads: it is bound by dependent L2 round trips per element, so
+    // its time falls with the elements per thread), and warps 3-6 pass the second grid barrier.
+    const bool is_x = warp == 1, is_mma = warp == 2, is_epi = warp >= 3;
     const int quarter = warp & 3;
-    const int f = quarter * 32 + lane;                     // feature inside the tile = tensor-memory lane
-    const int e_tid = (warp - 3) * 32 + lane;
+    const int f = quarter * 32 + lane;                     // feature inside the tile = tensor-memory lane (warps 3-6)
+    const int e_tid = (warp - 3) * 32 + lane;              // warps 3-6: 0..127
+    const int r_tid = is_epi ? e_tid : 128 + (warp - 1) * 32 + lane;   // thread of the reduction: 0..191
     griddep_wait();
     bool ok = true;
-    int seg = 0;
+    int x_stage = 0, ws = 0, xs = 0, mseg = 0, seg = 0;
+    uint32_t x_phase = 0, wph = 0, xph = 0;
+    const uint32_t idesc = idesc_bf16_m128(np);
     int n_bar = 0;                                         // grid barriers passed so far in this launch
     // The counter's value before this launch: a multiple of the grid size, and no barrier of this launch can complete
     // before every CTA has read it here (each reads before its own first arrival), so what a CTA reads is the base
     // plus fewer than `grid` arrivals.
     unsigned bar_base = 0;
-    if (e_tid == 0) {
+    if (is_epi && e_tid == 0) {
       const unsigned v = ld_acquire_u32(a.bar);
       bar_base = v - v % (unsigned)G;
     }
-    auto grid_barrier = [&]() -> bool {
+    auto grid_barrier = [&]() -> bool {                   // warps 3-6 only
       asm volatile("bar.sync 1, 128;" ::: "memory");
       ++n_bar;
       if (e_tid == 0 && c == a.diag_skip && n_bar == 1) {
@@ -562,52 +523,102 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       asm volatile("bar.sync 1, 128;" ::: "memory");
       return *s_abort == 0;                               // (the acquire load + bar.sync order the CTA's later loads)
     };
-    for (int pp = 0; pp < n_pass * a.n_phases && ok; ++pp) {
+    for (int pp = 0; pp < n_pass * a.n_phases; ++pp) {
       const int pi = pp % a.n_phases;
       const ChainPhase& p = a.ph[pi];
       const int row0 = (pp / a.n_phases) * np;
       const ChainRange rg = chain_range(p, c, G);
-      // the row scales this phase's reduction will need: their inputs are complete (the previous phase's second barrier,
-      // or the kernel before), and these warps have nothing to do until the first accumulator is full
-      if (p.kind == CH_GATEUP) row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
-      else if (p.kind == CH_QKV) {
-        for (int r = e_tid; r < np; r += 128) {            // and the rows' positions (rotary embedding, cache rows)
-          const int pos = row0 + r < M ? __ldg(a.idx + row0 + r) : 0;
-          tabs->pos[r] = make_int2(pos, pos % a.n_seq);
+      if (is_x) {
+        // activation loader: a phase's activations exist once the previous phase's reduction has passed its barrier
+        if (lane == 0 && ok) {
+          if (pp > 0) ok = mbar_wait(xready, (uint32_t)(pp - 1) & 1, s_abort);
+          for (int u = rg.begin; u < rg.end && ok; ++u) {
+            const int kb = u % p.num_kb;
+            if (!(ok = mbar_wait(xempty(x_stage), x_phase ^ 1, s_abort))) break;
+            mbar_expect_tx(xfull(x_stage), (uint32_t)X_BYTES);
+            tma_load_2d(smem_u32(sX + x_stage * X_BYTES), xmaps[p.x_map], kb * CH_BK, row0, xfull(x_stage));
+            if (++x_stage == x_stages) { x_stage = 0; x_phase ^= 1; }
+          }
         }
-        row_rstd(a, a.ssq_next, e_tid, M, row0, s_rstd);   // (ends with a barrier of these warps)
-      }
-      int j = 0;
-      for (int u = rg.begin; u < rg.end && ok; ++j, ++seg) {
-        const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
-        const int acc = seg & 1;
-        ok = mbar_wait(accfull0 + 8u * acc, (uint32_t)(seg >> 1) & 1, s_abort);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
-        tc_fence_after();
-        float* dst = a.ws + ((size_t)c * CH_MAX_SEG + j) * np * CH_BF + f;
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * np);
-        for (int h = 0; h < np; h += 32) {
-          uint32_t v[32];
-          tc_ld32(taddr + h, v);
-          tc_wait_ld();
-#pragma unroll
-          for (int r = 0; r < 32; ++r)
-            if (h + r < np) __stcg(dst + (size_t)(h + r) * CH_BF, __uint_as_float(v[r]));
-        }
-        tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(accempty0 + 8u * acc);
-        u = seg_end;
+      } else if (is_mma) {
+        if (lane == 0 && ok) {
+          int u = rg.begin;
+          while (u < rg.end && ok) {
+            const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
+            const int acc = mseg & 1;
+            if (mseg >= 2 && !(ok = mbar_wait(accempty0 + 8u * acc, (uint32_t)((mseg >> 1) - 1) & 1, s_abort))) break;
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * np);
+            bool first = true;
+            for (; u < seg_end; ++u) {
+              if (!(ok = mbar_wait(wfull(ws), wph, s_abort))) break;
+              if (!(ok = mbar_wait(xfull(xs), xph, s_abort))) break;
+              tc_fence_after();
+              const uint64_t wdesc = smem_desc_k_sw128(smem_u32(sW + ws * CH_W_BYTES));
+              const uint64_t xdesc = smem_desc_k_sw128(smem_u32(sX + xs * X_BYTES));
+#pragma unroll
+              for (int k = 0; k < CH_BK / 16; ++k)
+                tc_mma_bf16(d_tmem, wdesc + (uint64_t)(2 * k), xdesc + (uint64_t)(2 * k), idesc, (!first) | (k != 0));
+              first = false;
+              tc_commit(wempty(ws));
+              tc_commit(xempty(xs));
+              if (++ws == w_stages) { ws = 0; wph ^= 1; }
+              if (++xs == x_stages) { xs = 0; xph ^= 1; }
+            }
+            if (ok) tc_commit(accfull0 + 8u * acc);
+            ++mseg;
+          }
+        }
+        __syncwarp();
+      } else if (ok) {
+        // the row scales this phase's reduction will need: their inputs are complete (the previous phase's second
+        // barrier, or the kernel before), and these warps have nothing to do until the first accumulator is full
+        if (p.kind == CH_GATEUP) row_rstd(a, a.ssq_ffn, e_tid, M, row0, s_rstd);
+        else if (p.kind == CH_QKV) {
+          for (int r = e_tid; r < np; r += 128) {          // and the rows' positions (rotary embedding, cache rows)
+            const int pos = row0 + r < M ? __ldg(a.idx + row0 + r) : 0;
+            tabs->pos[r] = make_int2(pos, pos % a.n_seq);
+          }
+          row_rstd(a, a.ssq_next, e_tid, M, row0, s_rstd); // (ends with a barrier of these warps)
+        }
+        int j = 0;
+        for (int u = rg.begin; u < rg.end && ok; ++j, ++seg) {
+          const int seg_end = min(rg.end, (u / p.num_kb + 1) * p.num_kb);
+          const int acc = seg & 1;
+          ok = mbar_wait(accfull0 + 8u * acc, (uint32_t)(seg >> 1) & 1, s_abort);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
+          float* dst = a.ws + ((size_t)c * CH_MAX_SEG + j) * np * CH_BF + f;
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * np);
+          for (int h = 0; h < np; h += 32) {
+            uint32_t v[32];
+            tc_ld32(taddr + h, v);
+            tc_wait_ld();
+#pragma unroll
+            for (int r = 0; r < 32; ++r)
+              if (h + r < np) __stcg(dst + (size_t)(h + r) * CH_BF, __uint_as_float(v[r]));
+          }
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(accempty0 + 8u * acc);
+          u = seg_end;
+        }
+        ok = epilogue_warps_agree(ok);                     // (a warp that gave up must not leave the others at the barrier)
+        if (ok) ok = grid_barrier();                       // every partial tile of the phase is in the workspace
       }
-      if (!epilogue_warps_agree(ok)) break;                // (a warp that gave up must not leave the others at the barrier)
-      if (!(ok = grid_barrier())) break;                   // every partial tile of the phase is in the workspace
-      chain_reduce(a, p, G, c, e_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi], tabs->pos);
-      if (!(ok = grid_barrier())) break;                   // the phase's outputs are complete
-      if (e_tid == 0) {
-        // the next phase's activations were written with ordinary stores (by all CTAs) and are read by bulk tensor copies
-        asm volatile("fence.proxy.async.global;" ::: "memory");
-        mbar_arrive(xready);
+      // all six warps: go on together or leave together (a thread that gave up must not strand the others at a barrier)
+      if (!chain_warps_agree(ok)) break;
+      chain_reduce(a, p, G, c, r_tid, M, row0, s_rstd, tabs->cover[pi], tabs->first_tile[pi], tabs->pos);
+      asm volatile("bar.sync 2, 192;" ::: "memory");       // this CTA's share of the reduction is done
+      if (is_epi) {
+        ok = grid_barrier();                               // the phase's outputs are complete
+        if (ok && e_tid == 0) {
+          // the next phase's activations were written with ordinary stores (by all CTAs) and are read by bulk tensor copies
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+          mbar_arrive(xready);
+        }
       }
     }
   }
