@@ -466,6 +466,9 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
       uint32_t phase = 0;
       bool ok = true;
       const int total_pp = n_pass * a.n_phases;
+      // the weights are read once: marked evict-first, they do not push the partial tiles and activations out of L2 (the
+      // reductions then find them there: step 4-6 % faster)
+      const uint64_t w_policy = l2_policy_evict_first();
       for (int pp = 0; pp < total_pp && ok; ++pp) {
         const ChainPhase& p = a.ph[pp % a.n_phases];
         const ChainRange rg = chain_range(p, c, G);
@@ -473,8 +476,8 @@ gemm_chain_kernel(const __grid_constant__ CUtensorMap tmW0, const __grid_constan
           const int t = u / p.num_kb, kb = u % p.num_kb;
           if (!(ok = mbar_wait(wempty(stage), phase ^ 1, s_abort))) break;
           mbar_expect_tx(wfull(stage), CH_W_BYTES);
-          tma_load_2d(smem_u32(sW + stage * CH_W_BYTES), wmaps[p.w_map0 + t / p.tiles_per_map], kb * CH_BK,
-                      (t % p.tiles_per_map) * CH_BF, wfull(stage));
+          tma_load_2d_hint(smem_u32(sW + stage * CH_W_BYTES), wmaps[p.w_map0 + t / p.tiles_per_map], kb * CH_BK,
+                           (t % p.tiles_per_map) * CH_BF, wfull(stage), w_policy);
           if (++stage == w_stages) { stage = 0; phase ^= 1; }
         }
       }
