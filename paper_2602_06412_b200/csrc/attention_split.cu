@@ -101,6 +101,7 @@ attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
     if (lane == 0) {
       uint32_t kcnt = 0;
       bool ok = true;
+      const uint64_t once = l2_policy_evict_first();    // every K / V block is read by exactly one CTA per step
       for (int qt = 0; qt < n_qt && ok && nj > 0; ++qt) {
         if (!(ok = mbar_wait(bar(Q_FREE), (qt & 1) ^ 1, s_abort))) break;
         mbar_expect_tx(bar(Q_FULL), Q_BYTES);
@@ -115,12 +116,12 @@ attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
           mbar_expect_tx(bar(K_FULL + st), KV_BYTES);
 #pragma unroll
           for (int sl = 0; sl < SLABS; ++sl)
-            tma_load_2d(smem_u32(sK + st * KV_BYTES + sl * SLAB_BYTES), &tmK, h * DH + 64 * sl, key0, bar(K_FULL + st));
+            tma_load_2d_hint(smem_u32(sK + st * KV_BYTES + sl * SLAB_BYTES), &tmK, h * DH + 64 * sl, key0, bar(K_FULL + st), once);
           if (!(ok = mbar_wait(bar(V_FREE + st), ph ^ 1, s_abort))) break;
           mbar_expect_tx(bar(V_FULL + st), KV_BYTES);
 #pragma unroll
           for (int sl = 0; sl < SLABS; ++sl)
-            tma_load_2d(smem_u32(sV + st * KV_BYTES + sl * SLAB_BYTES), &tmV, h * DH + 64 * sl, key0, bar(V_FULL + st));
+            tma_load_2d_hint(smem_u32(sV + st * KV_BYTES + sl * SLAB_BYTES), &tmV, h * DH + 64 * sl, key0, bar(V_FULL + st), once);
         }
       }
     }
