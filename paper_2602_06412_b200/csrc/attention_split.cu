@@ -6,8 +6,8 @@
 // B x H CTAs (32 of 148 SMs for one sequence) and walks through all key blocks one after the other.  Here CTA
 // (b, h, s) takes the s-th of S contiguous ranges of 128-key blocks, so that B x H x S CTAs (at most one per SM) share
 // the key loop, and leaves an unnormalised partial result (fp32 O, running maximum m, sum l) in a workspace.  The S
-// CTAs of a pair then meet on a counter (bounded wait; all of them are resident, the grid being no larger than the
-// number of SMs) and each combines its share of the rows: o = sum_i w_i O_i / sum_i w_i l_i, w_i = 2^(m_i - max m), in
+// CTAs of a pair then meet on a counter (bounded wait; all of them are resident: the launch is cooperative and the
+// grid no larger than the number of SMs) and each combines its share of the rows: o = sum_i w_i O_i / sum_i w_i l_i, w_i = 2^(m_i - max m), in
 // split order (deterministic).  With S = 1 the result is written directly.
 //   warp 0     TMA producer: Q once per query tile, then K and V blocks (two stages each), 128-byte swizzle;
 //   warp 1     one thread issues S = Q K^T and O += P V (P read from tensor memory as the A operand, V the MN-major
@@ -407,9 +407,42 @@ static int launch_split_dh(const CUtensorMap& q, const CUtensorMap& k, const CUt
   float* ws_o = ws;
   float2* ws_ml = reinterpret_cast<float2*>(ws + (size_t)sm_count() * AS_BQ * DH);
   const float scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  SL_CUDA_TRY(launch_pdl(attention_split_kernel<DH>, dim3(B * H * S), dim3(AS_THREADS), (size_t)smem, st, q, k, v, row_offsets,
-                         B, N, H, S, (bf16*)o, scale_log2, ws_o, ws_ml, counters, status, diag_skip));
-  SL_CUDA_TRY(cudaGetLastError());
+  // The splits wait for one another, so with S > 1 the launch is cooperative: every CTA of the grid is resident at the
+  // same time whatever else runs on the device (the grid was checked against one CTA per SM).  Programmatic dependent
+  // launch on top of it where the driver takes the combination.
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(B * H * S);
+  cfg.blockDim = dim3(AS_THREADS);
+  cfg.dynamicSmemBytes = (size_t)smem;
+  cfg.stream = st;
+  cudaLaunchAttribute at[2];
+  int n_at = 0;
+  if (S > 1) {
+    at[n_at].id = cudaLaunchAttributeCooperative;
+    at[n_at].val.cooperative = 1;
+    ++n_at;
+  }
+  static int with_pdl = -1;                            // -1: not tried yet
+  if (with_pdl < 0) with_pdl = pdl_enabled() ? 1 : 0;
+  const int n_base = n_at;
+  if (with_pdl) {
+    at[n_at].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n_at].val.programmaticStreamSerializationAllowed = 1;
+    ++n_at;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = n_at;
+  bf16* op = (bf16*)o;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, attention_split_kernel<DH>, q, k, v, row_offsets, B, N, H, S, op, scale_log2, ws_o,
+                                     ws_ml, counters, status, diag_skip);
+  if (e != cudaSuccess && with_pdl && n_base > 0) {    // the combination of the two attributes is refused: cooperative only
+    cudaGetLastError();
+    with_pdl = 0;
+    cfg.numAttrs = n_base;
+    e = cudaLaunchKernelEx(&cfg, attention_split_kernel<DH>, q, k, v, row_offsets, B, N, H, S, op, scale_log2, ws_o, ws_ml,
+                           counters, status, diag_skip);
+  }
+  SL_CUDA_TRY(e);
   return SL_OK;
 }
 
