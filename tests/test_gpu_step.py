@@ -402,3 +402,31 @@ def test_layer_chain_grid_barrier_wait_runs_out_and_is_reported():
     out_b, lock_b = two_steps(ctx2, False)
     assert SL.surelock_status_poll(ctx2) == 0
     assert torch.equal(logits_a.view(torch.int16), out_b.logits[:20].view(torch.int16)) and torch.equal(lock_a, lock_b)
+
+
+@pytest.mark.gpu
+def test_few_row_kernels_with_no_active_row():
+    """A step whose bound on the row count selects the layer chain kernel and the split-key attention, but in which
+    every position is locked (M = 0): the kernels run as empty launches, nothing is written (caches, lock mask), no
+    status is raised; one active row right after works too."""
+    cfg = inputs.model_shape("llada8b", n_layers=2, vocab=4096)
+    w = inputs.make_weights(cfg, 5, dtype=torch.bfloat16, device=DEV)
+    B, N = 1, 256
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, 64, cfg["vocab"], 5)
+    tokens, mask = tokens.to(DEV), mask.to(DEV)
+    SL.surelock_step(ctx, tokens, mask, torch.zeros((B, N), dtype=torch.uint8, device=DEV), 1e-3)
+    SL.surelock_set_option(ctx, "row_bound", 16)
+    snap = [[t.clone() for t in SL.surelock_kv_cache(ctx, l)] for l in range(cfg["n_layers"])]
+    lock = torch.ones((B, N), dtype=torch.uint8, device=DEV)
+    out = SL.surelock_step(ctx, tokens, mask, lock, 1e-3)
+    assert SL.surelock_status_poll(ctx) == 0 and SL.surelock_last_step_paths(ctx) == 3
+    assert int(out.n_active.item()) == 0 and bool(lock.all())
+    for l in range(cfg["n_layers"]):
+        k, v = SL.surelock_kv_cache(ctx, l)
+        assert torch.equal(k.view(torch.int16), snap[l][0].view(torch.int16))
+        assert torch.equal(v.view(torch.int16), snap[l][1].view(torch.int16))
+    lock1 = inputs.random_lock(B, N, [1], 9).to(DEV)
+    out = SL.surelock_step(ctx, tokens, mask, lock1, 1e-3)
+    assert SL.surelock_status_poll(ctx) == 0 and int(out.n_active.item()) == 1
+    assert bool(torch.isfinite(out.logits[:1].float()).all())
