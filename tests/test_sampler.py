@@ -140,3 +140,22 @@ def test_sampler_run_with_unlocking():
     grew = [t for t in range(1, steps) if M[t] > M[t - 1]]
     assert grew and all(un[t - 1] > 0 for t in grew)                    # the active set only grows through an un-lock
     assert res["unmasked_per_step"] == [B] * steps
+
+
+@pytest.mark.gpu
+def test_sampler_run_bf16_through_the_few_row_kernels():
+    """The decoding loop on a bf16 model of the LLaDA-8B layer shape with one short sequence: from the third step on the
+    row bound (<= 128) selects the layer chain kernel for every step (N = 128 is a single key block, so attention stays
+    on the general kernel); the run completes, the active-row trace never grows, no status is raised."""
+    from paper_2602_06412_b200 import binding as SL
+    cfg = inputs.model_shape("llada8b", n_layers=2, vocab=4096)
+    w = inputs.make_weights(cfg, 21, dtype=torch.bfloat16, device="cuda")
+    B, N, n_prompt, blk, steps = 1, 128, 64, 32, 64
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], 21)
+    tokens, mask = tokens.cuda(), mask.cuda()
+    res = sampler.run(ctx, tokens, mask, n_prompt, blk, steps=steps, kl_eps=1e-3)
+    assert SL.surelock_status_poll(ctx) == 0 and SL.surelock_last_step_paths(ctx) == 1
+    assert res["masked_at_end"] == 0 and res["unmasked_per_step"] == [B] * steps
+    M = res["M_trace"]
+    assert M[0] == B * N and all(a >= b for a, b in zip(M, M[1:]))
