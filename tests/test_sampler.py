@@ -159,3 +159,11 @@ def test_sampler_run_bf16_through_the_few_row_kernels():
     assert res["masked_at_end"] == 0 and res["unmasked_per_step"] == [B] * steps
     M = res["M_trace"]
     assert M[0] == B * N and all(a >= b for a, b in zip(M, M[1:]))
+    # the same with optional un-locking switched on (probe steps run on the general kernels, a row that returns to the
+    # active set may make the bound too small for a step: further passes)
+    ctx = SL.surelock_init(cfg, w, N, B)
+    tokens, mask = inputs.make_tokens(B, N, n_prompt, cfg["vocab"], 21)
+    res = sampler.run(ctx, tokens.cuda(), mask.cuda(), n_prompt, blk, steps=steps, kl_eps=1e-3,
+                      unlock=dict(period=2, eps_unlock=2e-5, d_interval=1, d_cool=2, rho=0.25, m_percent=50.0))
+    assert SL.surelock_status_poll(ctx) == 0
+    assert res["masked_at_end"] == 0 and res["unmasked_per_step"] == [B] * steps
