@@ -194,7 +194,8 @@ int surelock_prev_logits(surelock_ctx *ctx, void **buf, int32_t **row_of_pos);
 /* Checkpoint / resume of a decoding run (the paper has no counterpart; the sampler state it lists in Algorithm 1's
  * "Require" and lines 1-3 is the lock mask, the cache C and p_{t-1}; the lock mask, tokens and mask state are the
  * caller's).  surelock_state_export writes what the ctx holds between two steps into a HOST buffer: a header (model
- * shape, N, batch, element type, rows of the last step), the K/V cache of every layer, and the previous step's logits,
+ * shape, N, batch, element type, rows of the last step, and the row counts of the last two steps, from which the next
+ * two steps take the bound that selects their kernels), the K/V cache of every layer, and the previous step's logits,
  * their log-sum-exps and position -> row table.  surelock_state_import loads such a buffer into a ctx created with the
  * same model shape, N, batch and element type (weights are not part of the state); the next surelock_step then
  * continues bit for bit as the exporting ctx would have.  Both calls synchronise the ctx stream.

@@ -738,7 +738,11 @@ struct StateHeader {
   uint64_t magic;                       // "SLKSTAT1"
   int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab, dtype, N, B;
   int32_t have_prev, rows_prev;         // rows of the previous step's logits that are stored
-  int32_t reserved[5];
+  // the row counts of the last two steps, from which the next two steps take their bound on M (so that a ctx that
+  // imports the state chooses the same kernels as the one that went on): flags bit 0 / 1 = count 0 / 1 is there,
+  // bit 2 = parity of the call counter
+  int32_t m_flags, m_hist[2];
+  int32_t reserved[2];
 };
 static const uint64_t STATE_MAGIC = 0x31544154534b4c53ull;
 
@@ -767,6 +771,9 @@ int surelock_state_export(surelock_ctx* c, void* host_dst, size_t capacity, size
   if (c->have_prev && m_prev == 0) m_prev = c->R;   // previous logits seeded by the caller ("have_prev"): keep every row
   if (m_prev < 0 || m_prev > c->R) return SL_EDEVICE;
   h.rows_prev = m_prev;
+  h.m_flags = (c->ev_m_valid[0] ? 1 : 0) | (c->ev_m_valid[1] ? 2 : 0) | ((c->calls & 1) ? 4 : 0);
+  h.m_hist[0] = c->h_m[0];                // (complete: the stream was synchronised above)
+  h.m_hist[1] = c->h_m[1];
   const size_t kvb = 2 * (size_t)c->cfg.n_layers * c->kv_layer_bytes();
   const size_t lgb = (size_t)m_prev * c->cfg.vocab * c->esz, lsb = (size_t)m_prev * 4, rpb = (size_t)c->R * 4;
   const size_t need = sizeof(h) + kvb + lgb + lsb + rpb;
@@ -812,6 +819,13 @@ int surelock_state_import(surelock_ctx* c, const void* host_src, size_t bytes) {
   c->have_prev = h.have_prev != 0;
   const int32_t rows_prev = h.rows_prev;
   SL_CUDA_TRY(cudaMemcpyAsync(c->n_prev, &rows_prev, 4, cudaMemcpyHostToDevice, c->st));
+  c->calls = (h.m_flags & 4) ? 1 : 0;
+  for (int i = 0; i < 2; ++i) {
+    if (!(h.m_flags & (1 << i)) || h.m_hist[i] < 0 || h.m_hist[i] > c->R) continue;
+    c->h_m[i] = h.m_hist[i];
+    SL_CUDA_TRY(cudaEventRecord(c->ev_m[i], c->st));
+    c->ev_m_valid[i] = true;
+  }
   SL_CUDA_TRY(cudaStreamSynchronize(c->st));
   return SL_OK;
 }

@@ -251,10 +251,13 @@ def test_degenerate_active_sets(dtype, tol):
         assert fin.all() and np.all(np.abs(kl - ref["kl"]) <= 1e-3 * ref["kl"] + 1e-6)
 
 
-def test_checkpoint_resume_continues_bit_for_bit():
+@pytest.mark.parametrize("p_lock", [0.3, 0.65])
+def test_checkpoint_resume_continues_bit_for_bit(p_lock):
     """surelock_state_export / _import: a second ctx that imports the state taken after three steps takes the fourth
     step exactly as the first one does (same packing, logits, KL, lock decisions, cache bytes); a state of another
-    shape is refused."""
+    shape is refused.  With the faster lock schedule the fourth step has few active rows and runs on the kernels the
+    row bound selects (the bound is the row count two steps back: the state carries the pending counts, so the
+    importing ctx makes the same choice)."""
     cfg = inputs.model_shape("tiny", d_model=512, n_heads=4, head_dim=128, d_ff=1536, vocab=4096, n_layers=2)
     B, N, eps = 2, 160, 1e-3
     wd = to_dev(inputs.make_weights(cfg, 21, dtype=torch.bfloat16, std=0.04))
@@ -264,7 +267,8 @@ def test_checkpoint_resume_continues_bit_for_bit():
     lock = torch.zeros((B, N), dtype=torch.uint8, device=DEV)
     for t in range(3):
         SL.surelock_step(a, tok_d, mask_d, lock, eps)
-        lock = inputs.bernoulli_lock_schedule(lock.cpu(), mask == 0, 0.3, 500 + t).to(DEV)
+        lockable = (mask == 0) if p_lock < 0.5 else torch.ones_like(mask)   # (a forced pattern may lock masked rows)
+        lock = inputs.bernoulli_lock_schedule(lock.cpu(), lockable, p_lock, 500 + t).to(DEV)
     state = SL.surelock_state_export(a)
     b = SL.surelock_init(cfg, wd, N, B)
     SL.surelock_state_import(b, state)
@@ -274,6 +278,8 @@ def test_checkpoint_resume_continues_bit_for_bit():
     assert SL.surelock_status_poll(a) == 0 and SL.surelock_status_poll(b) == 0
     M = oa.M()
     assert M == ob.M() and 0 < M < B * N
+    assert SL.surelock_last_step_paths(a) == SL.surelock_last_step_paths(b)
+    assert (SL.surelock_last_step_paths(a) != 0) == (p_lock > 0.5)
     assert torch.equal(oa.active_idx[:M], ob.active_idx[:M])
     assert torch.equal(oa.logits[:M].view(torch.int16), ob.logits[:M].view(torch.int16))
     assert torch.equal(oa.kl[:M].view(torch.int32), ob.kl[:M].view(torch.int32)) and torch.isfinite(oa.kl[:M]).any()
