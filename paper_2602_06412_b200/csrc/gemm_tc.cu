@@ -415,6 +415,11 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
       uint32_t phase = 0;
       bool ok = true;
       const uint64_t keep = l2_policy_evict_last();     // activation tiles: every column tile of the group re-reads them
+#ifndef TC2_W_EVICT_FIRST_PAIRS
+#define TC2_W_EVICT_FIRST_PAIRS 2
+#endif
+      // with at most two pair rows a weight tile is read by the pairs that work on it at the same time and never again
+      const uint64_t wpol = m_pairs <= TC2_W_EVICT_FIRST_PAIRS ? l2_policy_evict_first() : l2_policy_evict_normal();
       for (int w = cid; w < total && ok; w += n_clusters) {
         int mt, nt;
         tile_of(w, m_pairs, n_tiles, group, mt, nt);
@@ -436,7 +441,7 @@ __device__ __forceinline__ void run_pair(const CUtensorMap* tmA, const CUtensorM
           const uint32_t fb = mapa_u32(full_bar(stage), 0);
           if (rank == 0) mbar_expect_tx(full_bar(stage), 2 * STAGE_BYTES);
           tma_load_2d_pair_hint(sa, tmA, kb * TC_BK, m0, fb, keep);
-          tma_load_2d_pair(sb, mp, kb * TC_BK, brow, fb);
+          tma_load_2d_pair_hint(sb, mp, kb * TC_BK, brow, fb, wpol);
           if (++stage == STAGES) { stage = 0; phase ^= 1; }
         }
       }
