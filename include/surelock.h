@@ -416,7 +416,8 @@ int surelock_attention(const void *q, const void *k_cache, const void *v_cache, 
  * number as a step would; B * H * splits must not exceed the number of SMs and splits must not exceed 8 nor the number of
  * 128-key blocks (SL_EUNSUPPORTED otherwise, also for head_dim other than 64 / 128 or pointers that are not 16-byte
  * aligned).  workspace: dev, surelock_attention_split_workspace_bytes(B, H, head_dim) bytes, ZEROED by the caller before
- * its first use (it begins with one counter per (sequence, head) that only grows) and not shared between streams.
+ * its first use (it begins with one 64-bit counter per (sequence, head) that only grows; calls with different numbers of
+ * splits may follow one another on it) and not shared between streams.
  * diag_skip: -1 in normal use.  >= 0 is a failure-detection diagnostic: CTA number diag_skip (< B * H * splits) does not
  * arrive at the meeting of its (sequence, head), so the bounded wait (~0.2 s) of its siblings runs out: they store
  * device status 3 (see surelock_status_poll) in *dev_status and the kernel returns with o of that pair undefined; nothing hangs or traps; zero

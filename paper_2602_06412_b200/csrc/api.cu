@@ -72,7 +72,7 @@ struct surelock_ctx {
   int chain_diag_skip = -1;           // "debug_chain_skip_barrier": one-shot, consumed by the next chain launch
   int paths = 0;                      // few-row kernels the current call has taken: 1 layer chain, 2 split-key attention
   float* att_ws = nullptr;
-  unsigned* att_cnt = nullptr;
+  unsigned long long* att_cnt = nullptr;
   bool gemm_stream = false;           // "gemm_stream" option: contractions of at most 128 rows on the weight-streaming kernel
   int m_bound = 0;                    // the bound the launches of the current call use
   bool last_gemm_tc = false;          // the last gemm() call went to the tensor-core kernel
@@ -152,8 +152,8 @@ int launch_gemm_tc_qkv(const void* A, const void* Wq, const void* Wk, const void
 int attention_split_plan(int B, int N, int H);
 size_t attention_split_workspace_bytes(int head_dim);
 int launch_attention_split(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
-                           int N, int H, int head_dim, int S, void* o, float* ws, unsigned* counters, int32_t* status,
-                           int diag_skip, cudaStream_t st);
+                           int N, int H, int head_dim, int S, void* o, float* ws, unsigned long long* counters,
+                           int32_t* status, int diag_skip, cudaStream_t st);
 int launch_attention_tc(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
                         int N, int H, int head_dim, void* o, int32_t* status, cudaStream_t st);   // attention_tc.cu
 }
@@ -430,8 +430,9 @@ int surelock_init(surelock_ctx** out, const surelock_model_cfg* cfg, const surel
     c->att_S = attention_split_plan(batch, N, cfg->n_heads);
     if (c->att_S >= 2) {                     // few sequences: attention with split keys for steps with few active rows
       A_(c->att_ws, attention_split_workspace_bytes(cfg->head_dim));
-      A_(c->att_cnt, (size_t)batch * cfg->n_heads * sizeof(unsigned));
-      if (rc == SL_OK && cudaMemsetAsync(c->att_cnt, 0, (size_t)batch * cfg->n_heads * sizeof(unsigned), c->st) != cudaSuccess)
+      A_(c->att_cnt, (size_t)batch * cfg->n_heads * sizeof(unsigned long long));
+      if (rc == SL_OK &&
+          cudaMemsetAsync(c->att_cnt, 0, (size_t)batch * cfg->n_heads * sizeof(unsigned long long), c->st) != cudaSuccess)
         rc = SL_ECUDA;
     }
   }
@@ -466,7 +467,8 @@ int surelock_reset(surelock_ctx* c) {
   c->cur = 0;
   c->calls = 0;
   c->ev_m_valid[0] = c->ev_m_valid[1] = false;
-  if (c->att_cnt) SL_CUDA_TRY(cudaMemsetAsync(c->att_cnt, 0, (size_t)c->B * c->cfg.n_heads * sizeof(unsigned), c->st));
+  if (c->att_cnt)
+    SL_CUDA_TRY(cudaMemsetAsync(c->att_cnt, 0, (size_t)c->B * c->cfg.n_heads * sizeof(unsigned long long), c->st));
   if (c->ch_bar) {                      // a chain kernel that gave up leaves the barrier count short: start over
     SL_CUDA_TRY(cudaMemsetAsync(c->ch_bar, 0, 16, c->st));
     c->ch_bar_base = 0;
@@ -1038,7 +1040,7 @@ int surelock_update_mask(const float* conf, const int32_t* argmax, const int32_t
 
 size_t surelock_attention_split_workspace_bytes(int B, int H, int head_dim) {
   if (B <= 0 || H <= 0 || head_dim <= 0) return 0;
-  return (((size_t)B * H * sizeof(unsigned) + 255) & ~(size_t)255) + attention_split_workspace_bytes(head_dim);
+  return (((size_t)B * H * sizeof(unsigned long long) + 255) & ~(size_t)255) + attention_split_workspace_bytes(head_dim);
 }
 
 int surelock_attention_split(const void* q, const void* k_cache, const void* v_cache, const int32_t* row_offsets,
@@ -1050,8 +1052,9 @@ int surelock_attention_split(const void* q, const void* k_cache, const void* v_c
   const int S = splits ? splits : attention_split_plan(B, N, H);
   if (S < 1) return SL_EUNSUPPORTED;
   if (diag_skip >= B * H * S) return SL_EINVAL;
-  unsigned* counters = static_cast<unsigned*>(workspace);
-  float* ws = reinterpret_cast<float*>(static_cast<char*>(workspace) + (((size_t)B * H * sizeof(unsigned) + 255) & ~(size_t)255));
+  unsigned long long* counters = static_cast<unsigned long long*>(workspace);
+  float* ws = reinterpret_cast<float*>(static_cast<char*>(workspace) +
+                                       (((size_t)B * H * sizeof(unsigned long long) + 255) & ~(size_t)255));
   return launch_attention_split(q, k_cache, v_cache, row_offsets, max_rows, B, N, H, head_dim, S, o, ws, counters, dev_status,
                                 diag_skip < 0 ? -1 : diag_skip, (cudaStream_t)stream);
 }

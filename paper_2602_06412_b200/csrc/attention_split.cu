@@ -39,11 +39,15 @@ __device__ __forceinline__ void as_mma_ta(uint32_t d_tmem, uint32_t a_tmem, uint
       : "memory");
 }
 
-__device__ __forceinline__ unsigned as_ld_acquire(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+__device__ __forceinline__ unsigned long long as_ld_acquire(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
   return v;
 }
+// One meeting of the S splits of a (sequence, head) adds AS_MEET_QUANTUM to the pair's 64-bit counter whatever S is (each
+// split adds AS_MEET_QUANTUM / S; S <= 8 divides it), so the counter only grows, never wraps in practice, and launches
+// with different numbers of splits can share a workspace.
+constexpr unsigned long long AS_MEET_QUANTUM = 840;
 
 }  // namespace
 
@@ -52,7 +56,7 @@ __global__ void __launch_bounds__(AS_THREADS, 1)
 attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                        const __grid_constant__ CUtensorMap tmV, const int32_t* __restrict__ row_offsets, int B, int N, int H,
                        int S, bf16* __restrict__ o, float scale_log2, float* __restrict__ ws_o, float2* __restrict__ ws_ml,
-                       unsigned* __restrict__ counters, int32_t* status, int diag_skip) {
+                       unsigned long long* __restrict__ counters, int32_t* status, int diag_skip) {
   constexpr int SLABS = DH / 64;                       // 64-element (128-byte) column blocks per row
   constexpr int SLAB_BYTES = 128 * 128;                // 128 rows x 128 bytes
   constexpr int Q_BYTES = SLABS * SLAB_BYTES;
@@ -189,18 +193,18 @@ attention_split_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_con
       }
       tc_wait_st();
     };
-    // the S splits of this (sequence, head) meet: every barrier adds S arrivals to the pair's counter, which only grows
+    // the S splits of this (sequence, head) meet: every meeting adds one quantum to the pair's counter, which only grows
     auto meet = [&]() -> bool {
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (e_tid == 0 && (int)blockIdx.x == diag_skip) {
         *s_meet = 1;                                     // diagnostic: this CTA does not arrive, so its siblings' wait runs out
       } else if (e_tid == 0) {
         __threadfence();                                 // release: the CTA's stores (ordered before by the bar.sync)
-        const unsigned ticket = atomicAdd(counters + bh, 1u);
-        const unsigned target = (ticket / (unsigned)S + 1u) * (unsigned)S;
+        const unsigned long long ticket = atomicAdd(counters + bh, AS_MEET_QUANTUM / (unsigned long long)S);
+        const unsigned long long target = (ticket / AS_MEET_QUANTUM + 1ull) * AS_MEET_QUANTUM;
         const unsigned long long t0 = clock64();
         int good = 1;
-        while ((int)(as_ld_acquire(counters + bh) - target) < 0) {
+        while (as_ld_acquire(counters + bh) < target) {
           if (*s_abort || clock64() - t0 > AS_MEET_CYCLES) {
             *s_abort = 1;
             good = 0;
@@ -395,7 +399,7 @@ size_t attention_split_workspace_bytes(int head_dim) {
 
 template <int DH>
 static int launch_split_dh(const CUtensorMap& q, const CUtensorMap& k, const CUtensorMap& v, const int32_t* row_offsets, int B,
-                           int N, int H, int S, void* o, float* ws, unsigned* counters, int32_t* status, int diag_skip,
+                           int N, int H, int S, void* o, float* ws, unsigned long long* counters, int32_t* status, int diag_skip,
                            cudaStream_t st) {
   constexpr int SLABS = DH / 64;
   const int smem = 5 * SLABS * 128 * 128 + 1024 + 512;
@@ -446,12 +450,12 @@ static int launch_split_dh(const CUtensorMap& q, const CUtensorMap& k, const CUt
   return SL_OK;
 }
 
-// ws: attention_split_workspace_bytes(head_dim) bytes; counters: B x H words, zero before the first launch.
+// ws: attention_split_workspace_bytes(head_dim) bytes; counters: B x H 64-bit words, zero before the first launch.
 // diag_skip >= 0: CTA diag_skip does not arrive at the meeting of its (sequence, head) (failure-detection test: the other
 // splits' bounded wait runs out and the kernel reports SL_DEV_ATTN_TIMEOUT); -1 otherwise.
 // SL_EUNSUPPORTED when the problem does not fit (the caller then takes the general kernel).
 int launch_attention_split(const void* q, const void* kc, const void* vc, const int32_t* row_offsets, int max_rows, int B,
-                           int N, int H, int head_dim, int S, void* o, float* ws, unsigned* counters, int32_t* status,
+                           int N, int H, int head_dim, int S, void* o, float* ws, unsigned long long* counters, int32_t* status,
                            int diag_skip, cudaStream_t st) {
   if ((head_dim != 64 && head_dim != 128) || max_rows < 1 || !row_offsets || !ws || !counters) return SL_EUNSUPPORTED;
   if (S < 1 || S > AS_MAX_SPLITS || (long long)B * H * S > sm_count()) return SL_EUNSUPPORTED;

@@ -387,6 +387,20 @@ def test_attention_split_keys(B, N, H, dh, n_act, qscale, splits):
         assert (o[M:] == 5.0).all()                                  # rows beyond M untouched
 
 
+def test_attention_split_changing_split_count_on_one_workspace():
+    """Calls with different numbers of key splits follow one another on the same workspace (a meeting advances the
+    pair's counter by the same amount whatever the number of splits)."""
+    args, kw, (q, Kc, Vc, offs, M, o, ws, status) = _split_attention_case(1, 1024, 4, 128, [50], 1.0, 2)
+    ref = O.attention_rows(f64(q[:M]), f64(Kc[:1024]), f64(Vc[:1024]))
+    for splits in (2, 3, 4, 8, 1, 3, 2):
+        kw["splits"] = splits
+        o.fill_(5.0)
+        SL.surelock_attention_split(*args, **kw)
+        torch.cuda.synchronize()
+        assert status.item() == 0, splits
+        assert rel_err_rows(f64(o[:M]).reshape(M, -1), ref) < 2e-2, splits
+
+
 def test_attention_split_arguments():
     args, kw, _ = _split_attention_case(1, 512, 32, 128, [10], 1.0, 5)
     with pytest.raises(SL.SurelockError):                            # 5 x 32 CTAs do not fit the GPU at one per SM
